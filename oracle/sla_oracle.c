@@ -1,0 +1,353 @@
+/*
+ * sla_oracle.c — TEST INFRASTRUCTURE, not the product (see sla_oracle.h).
+ *
+ * Token-by-token recurrent form of Softmax Linear Attention in fp64.
+ * One (batch, head) sequence at a time; the only coupling between heads is the
+ * softmax over the H gate logits of a token (Eq. 4), computed first.
+ *
+ * Readings of the paper taken here:
+ *  - the read-out at step t uses the state after the write of step t (Eq. 5-6);
+ *  - GLA's forget gate acts per key dimension: S <- diag(alpha_t) S  (Eq. 12);
+ *  - Gated DeltaNet (Eq. 14-16) is printed without its decay; a scalar decay
+ *    alpha_t = exp(g_t) is applied to S_{t-1} before the delta step, so g = 0
+ *    gives the printed equations.  The key-side gate multiplies v only; the
+ *    erase term uses the ungated key.  beta_t is a scalar per (token, head).
+ *  - no normaliser and no feature map inside: q, k arrive already mapped;
+ *    `scale` multiplies q.
+ */
+#include "sla_oracle.h"
+
+#include <math.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+int sla_oracle_num_threads(void) {
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/* Eq. 4 — softmax across the head axis. */
+void sla_oracle_head_softmax(const double *logits, long n_tok, int H, double *gates) {
+    for (long t = 0; t < n_tok; ++t) {
+        const double *l = logits + t * H;
+        double *g = gates + t * H;
+        double m = l[0];
+        for (int h = 1; h < H; ++h) if (l[h] > m) m = l[h];
+        double z = 0.0;
+        for (int h = 0; h < H; ++h) { g[h] = exp(l[h] - m); z += g[h]; }
+        for (int h = 0; h < H; ++h) g[h] /= z;
+    }
+}
+
+/* Per-step decay factors a[0..d_k) for sequence (b,h) at token t. */
+static void decay_factors(int variant, const double *log_decay, long bt, int H, int h, int d_k,
+                          double *a) {
+    if (variant == SLA_ORACLE_RETNET) {
+        double g = exp(log_decay[h]);
+        for (int d = 0; d < d_k; ++d) a[d] = g;
+    } else if (variant == SLA_ORACLE_GLA) {
+        const double *g = log_decay + (bt * H + h) * (long)d_k;
+        for (int d = 0; d < d_k; ++d) a[d] = exp(g[d]);
+    } else {
+        double g = exp(log_decay[bt * H + h]);
+        for (int d = 0; d < d_k; ++d) a[d] = g;
+    }
+}
+
+/*
+ * One state transition on S [d_k, d_v] (row = key dimension).
+ *   RETNET / GLA (Eq. 10, 12):  S <- diag(a) S + kw^T vw          kw = Gk k, vw = v
+ *   GDN (Eq. 14-15 + decay):    Sbar = a S ; r = vw - kw Sbar ; u = beta r ; S <- Sbar + kw^T u
+ *                                                                  kw = k,   vw = Gk v
+ * r_out (d_v, GDN only, nullable) receives r.
+ */
+static void state_step(int variant, int d_k, int d_v, const double *a, double beta,
+                       const double *kw, const double *vw, double *S, double *r_out) {
+    for (int d = 0; d < d_k; ++d)
+        for (int j = 0; j < d_v; ++j) S[d * d_v + j] *= a[d];
+    if (variant == SLA_ORACLE_GDN) {
+        double *r = (double *)malloc(sizeof(double) * d_v);
+        for (int j = 0; j < d_v; ++j) {
+            double acc = 0.0;
+            for (int d = 0; d < d_k; ++d) acc += kw[d] * S[d * d_v + j];
+            r[j] = vw[j] - acc;
+        }
+        for (int d = 0; d < d_k; ++d)
+            for (int j = 0; j < d_v; ++j) S[d * d_v + j] += kw[d] * (beta * r[j]);
+        if (r_out) memcpy(r_out, r, sizeof(double) * d_v);
+        free(r);
+    } else {
+        for (int d = 0; d < d_k; ++d)
+            for (int j = 0; j < d_v; ++j) S[d * d_v + j] += kw[d] * vw[j];
+    }
+}
+
+/* Gated operands of one token: qw = scale Gq q ; (kw, vw) as state_step wants them. */
+static void gated_operands(int variant, int d_k, int d_v, double scale, double Gq, double Gk,
+                           const double *q, const double *k, const double *v,
+                           double *qw, double *kw, double *vw) {
+    for (int d = 0; d < d_k; ++d) qw[d] = scale * Gq * q[d];
+    if (variant == SLA_ORACLE_GDN) {
+        for (int d = 0; d < d_k; ++d) kw[d] = k[d];
+        for (int j = 0; j < d_v; ++j) vw[j] = Gk * v[j];
+    } else {
+        for (int d = 0; d < d_k; ++d) kw[d] = Gk * k[d];
+        for (int j = 0; j < d_v; ++j) vw[j] = v[j];
+    }
+}
+
+static int bad_shape(int variant, long B, long T, int H, int d_k, int d_v) {
+    return variant < 0 || variant > 2 || B < 0 || T < 0 || H < 1 || d_k < 1 || d_v < 1;
+}
+
+int sla_oracle_forward(int variant, int B, int T, int H, int d_k, int d_v, double scale,
+                       const double *q, const double *k, const double *v,
+                       const double *log_decay, const double *beta,
+                       const double *lq, const double *lk, const double *h0,
+                       double *o, double *ht) {
+    if (bad_shape(variant, B, T, H, d_k, d_v)) return -1;
+    if (variant == SLA_ORACLE_GDN && !beta) return -1;
+    long n_tok = (long)B * T;
+    double *Gq = (double *)malloc(sizeof(double) * (n_tok * H + 1));
+    double *Gk = (double *)malloc(sizeof(double) * (n_tok * H + 1));
+    sla_oracle_head_softmax(lq, n_tok, H, Gq);
+    sla_oracle_head_softmax(lk, n_tok, H, Gk);
+    long sdim = (long)d_k * d_v;
+
+#pragma omp parallel for collapse(2) schedule(dynamic)
+    for (int b = 0; b < B; ++b) {
+        for (int h = 0; h < H; ++h) {
+            double *S = (double *)calloc(sdim, sizeof(double));
+            double *a = (double *)malloc(sizeof(double) * d_k);
+            double *qw = (double *)malloc(sizeof(double) * d_k);
+            double *kw = (double *)malloc(sizeof(double) * d_k);
+            double *vw = (double *)malloc(sizeof(double) * d_v);
+            if (h0) memcpy(S, h0 + ((long)b * H + h) * sdim, sizeof(double) * sdim);
+            for (int t = 0; t < T; ++t) {
+                long bt = (long)b * T + t;
+                long row = bt * H + h;
+                decay_factors(variant, log_decay, bt, H, h, d_k, a);
+                gated_operands(variant, d_k, d_v, scale, Gq[row], Gk[row],
+                               q + row * d_k, k + row * d_k, v + row * d_v, qw, kw, vw);
+                state_step(variant, d_k, d_v, a, beta ? beta[row] : 0.0, kw, vw, S, NULL);
+                double *ot = o + row * d_v;                      /* Eq. 6: read after write */
+                for (int j = 0; j < d_v; ++j) {
+                    double acc = 0.0;
+                    for (int d = 0; d < d_k; ++d) acc += qw[d] * S[d * d_v + j];
+                    ot[j] = acc;
+                }
+            }
+            if (ht) memcpy(ht + ((long)b * H + h) * sdim, S, sizeof(double) * sdim);
+            free(S); free(a); free(qw); free(kw); free(vw);
+        }
+    }
+    free(Gq); free(Gk);
+    return 0;
+}
+
+int sla_oracle_decode_step(int variant, int Bdec, int H, int d_k, int d_v, double scale,
+                           const double *q_t, const double *k_t, const double *v_t,
+                           const double *log_decay_t, const double *beta_t,
+                           const double *lq_t, const double *lk_t,
+                           double *state, double *o_t) {
+    /* A decode step is the T = 1 forward on the caller's state. */
+    if (!state) return -1;
+    return sla_oracle_forward(variant, Bdec, 1, H, d_k, d_v, scale, q_t, k_t, v_t, log_decay_t,
+                              beta_t, lq_t, lk_t, state, o_t, state);
+}
+
+/* Softmax backward over heads: dl_h = G_h (dG_h - sum_h' G_h' dG_h'). */
+static void head_softmax_backward(const double *G, const double *dG, long n_tok, int H, double *dl) {
+    for (long t = 0; t < n_tok; ++t) {
+        double dot = 0.0;
+        for (int h = 0; h < H; ++h) dot += G[t * H + h] * dG[t * H + h];
+        for (int h = 0; h < H; ++h) dl[t * H + h] = G[t * H + h] * (dG[t * H + h] - dot);
+    }
+}
+
+#define SEG 64   /* states are re-derived SEG tokens at a time from a checkpoint */
+
+int sla_oracle_backward(int variant, int B, int T, int H, int d_k, int d_v, double scale,
+                        const double *q, const double *k, const double *v,
+                        const double *log_decay, const double *beta,
+                        const double *lq, const double *lk, const double *h0,
+                        const double *dO, const double *dht,
+                        double *dq, double *dk, double *dv,
+                        double *dlog_decay, double *dbeta,
+                        double *dlq, double *dlk, double *dh0) {
+    if (bad_shape(variant, B, T, H, d_k, d_v)) return -1;
+    if (variant == SLA_ORACLE_GDN && !beta) return -1;
+    long n_tok = (long)B * T;
+    long sdim = (long)d_k * d_v;
+    double *Gq = (double *)malloc(sizeof(double) * (n_tok * H + 1));
+    double *Gk = (double *)malloc(sizeof(double) * (n_tok * H + 1));
+    double *dGq = (double *)calloc(n_tok * H + 1, sizeof(double));
+    double *dGk = (double *)calloc(n_tok * H + 1, sizeof(double));
+    sla_oracle_head_softmax(lq, n_tok, H, Gq);
+    sla_oracle_head_softmax(lk, n_tok, H, Gk);
+    /* RETNET's log gamma_h is shared by every (b,t): per-(b,h) partial sums, added up at the end. */
+    double *dgamma_part = (double *)calloc((long)B * H + 1, sizeof(double));
+    int nseg = (T + SEG - 1) / SEG;
+
+#pragma omp parallel for collapse(2) schedule(dynamic)
+    for (int b = 0; b < B; ++b) {
+        for (int h = 0; h < H; ++h) {
+            double *ck = (double *)malloc(sizeof(double) * sdim * (nseg + 1)); /* S before each segment */
+            double *buf = (double *)malloc(sizeof(double) * sdim * (SEG + 1)); /* S_{t-1}..S_t inside one */
+            double *S = (double *)calloc(sdim, sizeof(double));
+            double *dS = (double *)calloc(sdim, sizeof(double));
+            double *a = (double *)malloc(sizeof(double) * d_k);
+            double *qw = (double *)malloc(sizeof(double) * d_k);
+            double *kw = (double *)malloc(sizeof(double) * d_k);
+            double *vw = (double *)malloc(sizeof(double) * d_v);
+            double *rr = (double *)malloc(sizeof(double) * d_v * SEG);       /* GDN residuals r_t */
+            double *dqw = (double *)malloc(sizeof(double) * d_k);
+            double *dkw = (double *)malloc(sizeof(double) * d_k);
+            double *dvw = (double *)malloc(sizeof(double) * d_v);
+            double *du = (double *)malloc(sizeof(double) * d_v);
+            if (h0) memcpy(S, h0 + ((long)b * H + h) * sdim, sizeof(double) * sdim);
+
+            /* forward sweep: keep the state at every segment boundary */
+            for (int t = 0; t < T; ++t) {
+                if (t % SEG == 0) memcpy(ck + (long)(t / SEG) * sdim, S, sizeof(double) * sdim);
+                long bt = (long)b * T + t, row = bt * H + h;
+                decay_factors(variant, log_decay, bt, H, h, d_k, a);
+                gated_operands(variant, d_k, d_v, scale, Gq[row], Gk[row],
+                               q + row * d_k, k + row * d_k, v + row * d_v, qw, kw, vw);
+                state_step(variant, d_k, d_v, a, beta ? beta[row] : 0.0, kw, vw, S, NULL);
+            }
+            if (dht) memcpy(dS, dht + ((long)b * H + h) * sdim, sizeof(double) * sdim);
+
+            for (int s = nseg - 1; s >= 0; --s) {
+                int t0 = s * SEG, t1 = (t0 + SEG < T) ? t0 + SEG : T;
+                /* re-derive S_{t0-1} .. S_{t1-1}: buf[i] = state before token t0+i */
+                memcpy(buf, ck + (long)s * sdim, sizeof(double) * sdim);
+                for (int t = t0; t < t1; ++t) {
+                    long bt = (long)b * T + t, row = bt * H + h;
+                    double *Sn = buf + (long)(t - t0 + 1) * sdim;
+                    memcpy(Sn, buf + (long)(t - t0) * sdim, sizeof(double) * sdim);
+                    decay_factors(variant, log_decay, bt, H, h, d_k, a);
+                    gated_operands(variant, d_k, d_v, scale, Gq[row], Gk[row],
+                                   q + row * d_k, k + row * d_k, v + row * d_v, qw, kw, vw);
+                    state_step(variant, d_k, d_v, a, beta ? beta[row] : 0.0, kw, vw, Sn,
+                               rr + (long)(t - t0) * d_v);
+                }
+                for (int t = t1 - 1; t >= t0; --t) {
+                    long bt = (long)b * T + t, row = bt * H + h;
+                    const double *Sp = buf + (long)(t - t0) * sdim;       /* S_{t-1} */
+                    const double *St = buf + (long)(t - t0 + 1) * sdim;   /* S_t     */
+                    const double *dOt = dO + row * d_v;
+                    const double *qt = q + row * d_k, *kt = k + row * d_k, *vt = v + row * d_v;
+                    decay_factors(variant, log_decay, bt, H, h, d_k, a);
+                    gated_operands(variant, d_k, d_v, scale, Gq[row], Gk[row], qt, kt, vt, qw, kw, vw);
+
+                    /* o_t = qw S_t */
+                    for (int d = 0; d < d_k; ++d) {
+                        double acc = 0.0;
+                        for (int j = 0; j < d_v; ++j) {
+                            acc += dOt[j] * St[d * d_v + j];
+                            dS[d * d_v + j] += qw[d] * dOt[j];
+                        }
+                        dqw[d] = acc;
+                    }
+                    /* now dS = dL/dS_t in full */
+                    double dg_scalar = 0.0;
+                    if (variant != SLA_ORACLE_GDN) {
+                        /* S_t = diag(a) S_{t-1} + kw^T vw */
+                        for (int j = 0; j < d_v; ++j) dvw[j] = 0.0;
+                        for (int d = 0; d < d_k; ++d) {
+                            double acck = 0.0, acca = 0.0;
+                            for (int j = 0; j < d_v; ++j) {
+                                double g = dS[d * d_v + j];
+                                acck += g * vw[j];
+                                dvw[j] += kw[d] * g;
+                                acca += g * Sp[d * d_v + j];
+                                dS[d * d_v + j] = a[d] * g;               /* -> dL/dS_{t-1} */
+                            }
+                            dkw[d] = acck;
+                            double dg = acca * a[d];                      /* d/d(log a) */
+                            if (variant == SLA_ORACLE_GLA) {
+                                if (dlog_decay) dlog_decay[row * d_k + d] = dg;
+                            } else {
+                                dg_scalar += dg;
+                            }
+                        }
+                        if (variant == SLA_ORACLE_RETNET) dgamma_part[(long)b * H + h] += dg_scalar;
+                        /* kw = Gk k ; vw = v */
+                        double dotk = 0.0;
+                        for (int d = 0; d < d_k; ++d) {
+                            dotk += kt[d] * dkw[d];
+                            if (dk) dk[row * d_k + d] = Gk[row] * dkw[d];
+                        }
+                        dGk[row] = dotk;
+                        if (dv) for (int j = 0; j < d_v; ++j) dv[row * d_v + j] = dvw[j];
+                    } else {
+                        /* Sbar = a S_{t-1}; r = vw - kw Sbar; u = beta r; S_t = Sbar + kw^T u */
+                        const double *r = rr + (long)(t - t0) * d_v;
+                        double bta = beta[row], al = a[0];
+                        double dbt = 0.0;
+                        for (int j = 0; j < d_v; ++j) {
+                            double acc = 0.0;
+                            for (int d = 0; d < d_k; ++d) acc += kw[d] * dS[d * d_v + j];
+                            du[j] = acc;
+                            dbt += acc * r[j];
+                        }
+                        if (dbeta) dbeta[row] = dbt;
+                        for (int d = 0; d < d_k; ++d) {
+                            double acc = 0.0;
+                            for (int j = 0; j < d_v; ++j) {
+                                double dr = bta * du[j];
+                                /* from kw^T u and from -kw Sbar inside r */
+                                acc += dS[d * d_v + j] * (bta * r[j]) - dr * (al * Sp[d * d_v + j]);
+                            }
+                            dkw[d] = acc;
+                        }
+                        for (int d = 0; d < d_k; ++d)
+                            for (int j = 0; j < d_v; ++j) {
+                                double dSbar = dS[d * d_v + j] - kw[d] * (bta * du[j]);
+                                dg_scalar += dSbar * Sp[d * d_v + j];
+                                dS[d * d_v + j] = al * dSbar;             /* -> dL/dS_{t-1} */
+                            }
+                        if (dlog_decay) dlog_decay[row] = dg_scalar * al;
+                        /* kw = k ; vw = Gk v ; dvw = beta du */
+                        double dotv = 0.0;
+                        for (int j = 0; j < d_v; ++j) {
+                            double dvwj = bta * du[j];
+                            dotv += vt[j] * dvwj;
+                            if (dv) dv[row * d_v + j] = Gk[row] * dvwj;
+                        }
+                        dGk[row] = dotv;
+                        if (dk) for (int d = 0; d < d_k; ++d) dk[row * d_k + d] = dkw[d];
+                    }
+                    /* qw = scale Gq q */
+                    double dotq = 0.0;
+                    for (int d = 0; d < d_k; ++d) {
+                        dotq += qt[d] * dqw[d];
+                        if (dq) dq[row * d_k + d] = scale * Gq[row] * dqw[d];
+                    }
+                    dGq[row] = scale * dotq;
+                }
+            }
+            if (dh0) memcpy(dh0 + ((long)b * H + h) * sdim, dS, sizeof(double) * sdim);
+            free(ck); free(buf); free(S); free(dS); free(a); free(qw); free(kw); free(vw);
+            free(rr); free(dqw); free(dkw); free(dvw); free(du);
+        }
+    }
+    if (variant == SLA_ORACLE_RETNET && dlog_decay) {
+        for (int h = 0; h < H; ++h) {
+            double acc = 0.0;
+            for (int b = 0; b < B; ++b) acc += dgamma_part[(long)b * H + h];
+            dlog_decay[h] = acc;
+        }
+    }
+    if (dlq) head_softmax_backward(Gq, dGq, n_tok, H, dlq);
+    if (dlk) head_softmax_backward(Gk, dGk, n_tok, H, dlk);
+    free(Gq); free(Gk); free(dGq); free(dGk); free(dgamma_part);
+    return 0;
+}

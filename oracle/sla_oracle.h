@@ -1,0 +1,72 @@
+/*
+ * sla_oracle.h — TEST INFRASTRUCTURE, not the product.
+ *
+ * A plain, slow, fp64 CPU statement of what the Softmax-Linear-Attention layer
+ * computes, written token by token from the paper's recurrent equations.  Only
+ * the tests, the smoke check and the benchmark's CPU-baseline leg may call it;
+ * it shares no code with the CUDA library and the CUDA library never calls it.
+ *
+ * Tensor layouts (all dense, row-major, fp64):
+ *   q, k        [B, T, H, d_k]        v, o, dO      [B, T, H, d_v]
+ *   lq, lk      [B, T, H]   head-gate logits for the query / key side
+ *   log_decay   RETNET: [H]  (log gamma_h)     GLA: [B, T, H, d_k]     GDN: [B, T, H]
+ *   beta        GDN: [B, T, H]   (ignored otherwise, may be NULL)
+ *   h0, ht      [B, H, d_k, d_v]   initial / final state, NULL = zeros / not wanted
+ *
+ * Pins (tests/test_oracle_*.py): gates against closed forms and the limits of
+ * Thm 3.2 / Thm 3.3; the recurrence against a brute-force quadratic form with
+ * an explicit decay mask (Eq. 3, App. A) and against unrolled transition-matrix
+ * products for the delta rule; the backward sweep against central finite
+ * differences of the forward.  No function here is "parity unpinned".
+ */
+#ifndef SLA_ORACLE_H
+#define SLA_ORACLE_H
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum { SLA_ORACLE_RETNET = 0, SLA_ORACLE_GLA = 1, SLA_ORACLE_GDN = 2 };
+
+/* Threads the (b,h) loops will use. */
+int sla_oracle_num_threads(void);
+
+/* Eq. 4: softmax over the H heads of one token, for n_tok tokens.
+ * logits, gates: [n_tok, H]. */
+void sla_oracle_head_softmax(const double *logits, long n_tok, int H, double *gates);
+
+/* Eq. 5-7 with the decay / delta-rule instantiations of Eq. 10-16.
+ * Returns 0, or -1 on a bad argument. */
+int sla_oracle_forward(int variant, int B, int T, int H, int d_k, int d_v, double scale,
+                       const double *q, const double *k, const double *v,
+                       const double *log_decay, const double *beta,
+                       const double *lq, const double *lk, const double *h0,
+                       double *o, double *ht);
+
+/* Reverse sweep of sla_oracle_forward.  dO [B,T,H,d_v]; dht nullable.
+ * Outputs (each nullable): dq, dk, dv in the shapes of their primals;
+ * dlog_decay in the shape of log_decay (RETNET: [H], summed over b,t);
+ * dbeta [B,T,H] (GDN); dlq, dlk [B,T,H]; dh0 [B,H,d_k,d_v]. */
+int sla_oracle_backward(int variant, int B, int T, int H, int d_k, int d_v, double scale,
+                        const double *q, const double *k, const double *v,
+                        const double *log_decay, const double *beta,
+                        const double *lq, const double *lk, const double *h0,
+                        const double *dO, const double *dht,
+                        double *dq, double *dk, double *dv,
+                        double *dlog_decay, double *dbeta,
+                        double *dlq, double *dlk, double *dh0);
+
+/* One recurrent step for Bdec sequences (the T = 1 case on a caller-held
+ * state).  q_t, k_t [Bdec,H,d_k]; v_t, o_t [Bdec,H,d_v]; log_decay_t RETNET [H],
+ * GLA [Bdec,H,d_k], GDN [Bdec,H]; beta_t [Bdec,H]; lq_t, lk_t [Bdec,H];
+ * state [Bdec,H,d_k,d_v] updated in place. */
+int sla_oracle_decode_step(int variant, int Bdec, int H, int d_k, int d_v, double scale,
+                           const double *q_t, const double *k_t, const double *v_t,
+                           const double *log_decay_t, const double *beta_t,
+                           const double *lq_t, const double *lk_t,
+                           double *state, double *o_t);
+
+#ifdef __cplusplus
+}
+#endif
+#endif
