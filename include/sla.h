@@ -1,0 +1,142 @@
+/*
+ * sla.h — C ABI of the B200 (sm_100a) Softmax-Linear-Attention hot path.
+ *
+ * The layer (paper Sec. 3.2): per token the H head-gate logits are turned into gates by a
+ * softmax over the heads (Eq. 4); every head then runs a gated linear recurrence on a
+ * d_k x d_v state (Eq. 5-6) in one of three instantiations (Eq. 10-16); the per-head
+ * read-outs are concatenated (Eq. 7, without W^O).  Training-time evaluation is chunkwise
+ * ("Chunkwise Parallel Training"): dense products inside a chunk, the state passed between
+ * chunks.  The result does not depend on the chunk size.
+ *
+ * Conventions for every call
+ *  - All tensor pointers are DEVICE pointers owned by the caller, dense, row-major, aligned
+ *    to 16 bytes.  The library allocates no device memory in sla_forward / sla_backward /
+ *    sla_decode_step: scratch comes from the caller's `workspace`
+ *    (size from sla_plan_workspace_bytes); the library keeps nothing in it between calls.
+ *  - Work is enqueued on `cuda_stream` (a cudaStream_t cast to void*, NULL = default stream)
+ *    and the call returns without waiting.
+ *  - Every function returns an sla_status; nothing throws or aborts across the boundary.
+ *    Shapes the kernels do not cover are refused at sla_plan_create (SLA_ERR_UNSUPPORTED);
+ *    a device that is not sm_100 is refused with SLA_ERR_ARCH.  There is no CPU fallback.
+ *  - io dtype (q, k, v, o and their gradients): fp32 or bf16.  Log-decay, beta, gate logits,
+ *    states and their gradients are always fp32.  Accumulation is fp32.
+ *
+ * Shapes:  q, k [B,T,H,d_k]   v, o, dO [B,T,H,d_v]   gate logits [B,T,H]
+ *          log_decay  RETNET [H] (log gamma_h) | GLA [B,T,H,d_k] | GDN [B,T,H]   (all <= 0)
+ *          beta       GDN [B,T,H] in (0,1), else NULL
+ *          h0, ht, dht, dh0 [B,H,d_k,d_v]  (row = key dimension)
+ */
+#ifndef SLA_H
+#define SLA_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct sla_plan sla_plan;          /* opaque host object */
+
+typedef enum {
+    SLA_OK = 0,
+    SLA_ERR_INVALID_ARG = 1,   /* null / misaligned pointer, bad struct_size, bad enum        */
+    SLA_ERR_UNSUPPORTED = 2,   /* a shape or option the kernels do not cover                   */
+    SLA_ERR_WORKSPACE = 3,     /* workspace NULL or smaller than sla_plan_workspace_bytes      */
+    SLA_ERR_ARCH = 4,          /* current device is not compute capability 10.x                */
+    SLA_ERR_CUDA = 5,          /* a CUDA runtime call failed (launch, attribute, allocation)   */
+    SLA_ERR_TIMEOUT = 6        /* a bounded device-side wait expired (reported by sla_plan_poll) */
+} sla_status;
+
+typedef enum { SLA_RETNET = 0, SLA_GLA = 1, SLA_GDN = 2 } sla_variant;
+typedef enum { SLA_FP32 = 0, SLA_BF16 = 1 } sla_dtype;
+
+/* flags */
+#define SLA_FLAG_FORCE_GENERIC 1u  /* use the fp32 CUDA-core chunk kernels even where a tensor-core
+                                      kernel exists for the shape (same function, other rounding) */
+
+typedef struct {
+    uint32_t struct_size;      /* sizeof(sla_desc) */
+    int32_t  variant;          /* sla_variant */
+    int32_t  io_dtype;         /* sla_dtype   */
+    int32_t  B, T, H;          /* batch, tokens, heads (1 <= H <= 32) */
+    int32_t  d_k, d_v;         /* per-head key / value width: multiples of 16, <= 128 */
+    int32_t  chunk;            /* chunk size C: 16, 32 or 64; T need not be a multiple of it */
+    float    scale;            /* multiplies q (the paper's linear forms have none: use 1) */
+    uint32_t flags;
+} sla_desc;
+
+/* Validates the description against the current CUDA device and builds a plan.
+ * The plan is bound to that device; it owns one small device status word and nothing else. */
+sla_status sla_plan_create(sla_plan **out, const sla_desc *desc);
+sla_status sla_plan_destroy(sla_plan *plan);
+
+/* Bytes of caller-provided scratch that sla_forward / sla_backward need for this plan. */
+sla_status sla_plan_workspace_bytes(const sla_plan *plan, size_t *forward_bytes, size_t *backward_bytes);
+
+/* Synchronises with nothing; copies the plan's device status word back (on the legacy default
+ * stream, so call it after synchronising the stream that ran the work).  SLA_ERR_TIMEOUT if a
+ * kernel gave up a bounded wait since the last poll, SLA_OK otherwise. */
+sla_status sla_plan_poll(sla_plan *plan);
+
+/* Number of kernel launches the last sla_forward / sla_backward / sla_decode_step on this plan
+ * enqueued (for launch accounting in benchmarks). */
+int32_t sla_plan_last_launch_count(const sla_plan *plan);
+
+const char *sla_status_string(sla_status s);
+
+/*
+ * Forward (Eq. 4-7 with Eq. 10-16, evaluated chunkwise).
+ *   gates   Gq = softmax_H(gq_logits), Gk = softmax_H(gk_logits)              (Eq. 4)
+ *   RETNET  S_t = gamma_h S_{t-1} + (Gk k_t)^T v_t                            (Eq. 10)
+ *   GLA     S_t = diag(exp(log_decay_t)) S_{t-1} + (Gk k_t)^T v_t             (Eq. 12)
+ *   GDN     Sb = exp(log_decay_t) S_{t-1};  u = beta_t (Gk v_t - k_t Sb);  S_t = Sb + k_t^T u   (Eq. 14-15)
+ *   o_t     = (scale Gq q_t) S_t, heads concatenated along the last axes      (Eq. 6-7, 11, 13, 16)
+ * h0 may be NULL (zero state); ht may be NULL (final state not wanted).
+ * gq_logits and gk_logits may alias.  Outputs must not alias inputs.
+ */
+sla_status sla_forward(sla_plan *plan,
+                       const void *q, const void *k, const void *v,
+                       const float *log_decay, const float *beta,
+                       const float *gq_logits, const float *gk_logits,
+                       const float *h0,
+                       void *o, float *ht,
+                       void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * Backward of sla_forward (the paper states no gradients; these are the chain rule applied to
+ * Eq. 4-7, 10-16, evaluated chunkwise with the chunk states recomputed).
+ * Inputs: the primal inputs of sla_forward, dO (io dtype) and optionally dht (gradient
+ * flowing into the final state).  Outputs, written in full (not accumulated): dq, dk, dv
+ * (io dtype); dlog_decay fp32 in the shape of log_decay (must be NULL for RETNET, whose gamma_h
+ * is a constant); dbeta fp32 [B,T,H] (GDN, else NULL); dgq_logits, dgk_logits fp32 [B,T,H];
+ * dh0 fp32 or NULL.  dgq_logits and dgk_logits must not alias each other.
+ */
+sla_status sla_backward(sla_plan *plan,
+                        const void *q, const void *k, const void *v,
+                        const float *log_decay, const float *beta,
+                        const float *gq_logits, const float *gk_logits,
+                        const float *h0,
+                        const void *dO, const float *dht,
+                        void *dq, void *dk, void *dv,
+                        float *dlog_decay, float *dbeta,
+                        float *dgq_logits, float *dgk_logits, float *dh0,
+                        void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * One recurrent step (Eq. 5-6 / 10-16 at a single t) for Bdec sequences on a caller-held
+ * state, updated in place.  Uses the plan's variant, dtype, H, d_k, d_v and scale; the plan's
+ * B, T and chunk are ignored.  q_t, k_t [Bdec,H,d_k]; v_t, o_t [Bdec,H,d_v];
+ * log_decay_t RETNET [H] | GLA [Bdec,H,d_k] | GDN [Bdec,H]; beta_t [Bdec,H] (GDN);
+ * logits [Bdec,H]; state [Bdec,H,d_k,d_v] fp32.  Needs no workspace.
+ */
+sla_status sla_decode_step(sla_plan *plan, int32_t Bdec,
+                           const void *q_t, const void *k_t, const void *v_t,
+                           const float *log_decay_t, const float *beta_t,
+                           const float *gq_logits_t, const float *gk_logits_t,
+                           float *state, void *o_t, void *cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SLA_H */

@@ -1,0 +1,173 @@
+"""Thin ctypes binding of libsla.so: argument marshalling only, every step runs in the CUDA kernels.
+
+The functions carry the names of the C entry points (include/sla.h).  Tensors are torch CUDA
+tensors used purely as device memory; the current torch stream is passed to the library.
+There is no fallback: if the shared library is missing or a call is refused, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+
+import torch
+
+_PKG = Path(__file__).resolve().parent
+_SO = _PKG / "libsla.so"
+
+SLA_RETNET, SLA_GLA, SLA_GDN = 0, 1, 2
+SLA_FP32, SLA_BF16 = 0, 1
+SLA_FLAG_FORCE_GENERIC = 1
+VARIANTS = {"retnet": SLA_RETNET, "gla": SLA_GLA, "gdn": SLA_GDN}
+DTYPES = {"fp32": SLA_FP32, "bf16": SLA_BF16, torch.float32: SLA_FP32, torch.bfloat16: SLA_BF16}
+EXPORTS = (
+    "sla_plan_create", "sla_plan_destroy", "sla_plan_workspace_bytes", "sla_plan_poll",
+    "sla_plan_last_launch_count", "sla_status_string", "sla_forward", "sla_backward", "sla_decode_step",
+)
+
+
+class SLAError(RuntimeError):
+    def __init__(self, call: str, status: int, text: str):
+        super().__init__(f"{call} failed: status {status} ({text})")
+        self.status = status
+
+
+class sla_desc(ctypes.Structure):
+    _fields_ = [
+        ("struct_size", ctypes.c_uint32), ("variant", ctypes.c_int32), ("io_dtype", ctypes.c_int32),
+        ("B", ctypes.c_int32), ("T", ctypes.c_int32), ("H", ctypes.c_int32),
+        ("d_k", ctypes.c_int32), ("d_v", ctypes.c_int32), ("chunk", ctypes.c_int32),
+        ("scale", ctypes.c_float), ("flags", ctypes.c_uint32),
+    ]
+
+
+_lib = None
+
+
+def lib():
+    """Load libsla.so (built in-tree by paper_2602_01744_b200.build); raises if it is absent."""
+    global _lib
+    if _lib is None:
+        if not _SO.exists():
+            raise FileNotFoundError(
+                f"{_SO} is missing: run `python -m paper_2602_01744_b200.build` (there is no fallback path)")
+        L = ctypes.CDLL(str(_SO))
+        vp, i32, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_size_t
+        L.sla_plan_create.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(sla_desc)]
+        L.sla_plan_destroy.argtypes = [vp]
+        L.sla_plan_workspace_bytes.argtypes = [vp, ctypes.POINTER(sz), ctypes.POINTER(sz)]
+        L.sla_plan_poll.argtypes = [vp]
+        L.sla_plan_last_launch_count.argtypes = [vp]
+        L.sla_plan_last_launch_count.restype = i32
+        L.sla_status_string.argtypes = [ctypes.c_int]
+        L.sla_status_string.restype = ctypes.c_char_p
+        L.sla_forward.argtypes = [vp] * 11 + [vp, sz, vp]
+        L.sla_backward.argtypes = [vp] * 19 + [vp, sz, vp]
+        L.sla_decode_step.argtypes = [vp, i32] + [vp] * 10
+        for name in ("sla_plan_create", "sla_plan_destroy", "sla_plan_workspace_bytes", "sla_plan_poll",
+                     "sla_forward", "sla_backward", "sla_decode_step"):
+            getattr(L, name).restype = ctypes.c_int
+        _lib = L
+    return _lib
+
+
+def _check(call: str, status: int):
+    if status != 0:
+        raise SLAError(call, status, lib().sla_status_string(status).decode())
+
+
+def _ptr(t):
+    if t is None:
+        return None
+    assert t.is_cuda and t.is_contiguous(), "tensors must be contiguous CUDA tensors"
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+class Plan:
+    """Owns an sla_plan* (see sla_plan_create in include/sla.h)."""
+
+    def __init__(self, variant, io_dtype, B, T, H, d_k, d_v, chunk=64, scale=1.0, flags=0):
+        self.desc = sla_desc(ctypes.sizeof(sla_desc), VARIANTS.get(variant, variant),
+                             DTYPES.get(io_dtype, io_dtype), B, T, H, d_k, d_v, chunk, scale, flags)
+        self.handle = ctypes.c_void_p()
+        _check("sla_plan_create", lib().sla_plan_create(ctypes.byref(self.handle), ctypes.byref(self.desc)))
+        f, b = ctypes.c_size_t(), ctypes.c_size_t()
+        _check("sla_plan_workspace_bytes",
+               lib().sla_plan_workspace_bytes(self.handle, ctypes.byref(f), ctypes.byref(b)))
+        self.forward_workspace_bytes, self.backward_workspace_bytes = f.value, b.value
+        self.io_torch = torch.bfloat16 if self.desc.io_dtype == SLA_BF16 else torch.float32
+
+    def close(self):
+        if getattr(self, "handle", None) and self.handle.value:
+            lib().sla_plan_destroy(self.handle)
+            self.handle = ctypes.c_void_p()
+
+    __del__ = close
+
+    def poll(self):
+        _check("sla_plan_poll", lib().sla_plan_poll(self.handle))
+
+    @property
+    def last_launch_count(self) -> int:
+        return int(lib().sla_plan_last_launch_count(self.handle))
+
+    def workspace(self, backward=False, device="cuda"):
+        n = self.backward_workspace_bytes if backward else self.forward_workspace_bytes
+        return torch.empty(max(n, 16), dtype=torch.uint8, device=device)
+
+
+def sla_plan_create(variant, io_dtype, B, T, H, d_k, d_v, chunk=64, scale=1.0, flags=0) -> Plan:
+    return Plan(variant, io_dtype, B, T, H, d_k, d_v, chunk, scale, flags)
+
+
+def sla_forward(plan: Plan, q, k, v, log_decay, gq_logits, gk_logits, beta=None, h0=None, o=None, ht=None,
+                workspace=None):
+    """Enqueue the chunkwise forward on the current stream.  Returns (o, ht)."""
+    d = plan.desc
+    if o is None:
+        o = torch.empty((d.B, d.T, d.H, d.d_v), dtype=plan.io_torch, device=q.device)
+    if workspace is None:
+        workspace = plan.workspace(False, q.device)
+    _check("sla_forward", lib().sla_forward(
+        plan.handle, _ptr(q), _ptr(k), _ptr(v), _ptr(log_decay), _ptr(beta), _ptr(gq_logits),
+        _ptr(gk_logits), _ptr(h0), _ptr(o), _ptr(ht), _ptr(workspace), workspace.numel(), _stream()))
+    return o, ht
+
+
+def sla_backward(plan: Plan, q, k, v, log_decay, gq_logits, gk_logits, dO, beta=None, h0=None, dht=None,
+                 want_dh0=False, workspace=None, out=None):
+    """Enqueue the chunkwise backward on the current stream.  Returns a dict of gradients."""
+    d = plan.desc
+    dev = q.device
+    if out is None:
+        out = dict(
+            dq=torch.empty_like(q), dk=torch.empty_like(k), dv=torch.empty_like(v),
+            dlog_decay=None if d.variant == SLA_RETNET else torch.empty_like(log_decay),
+            dbeta=torch.empty_like(beta) if d.variant == SLA_GDN else None,
+            dgq_logits=torch.empty_like(gq_logits), dgk_logits=torch.empty_like(gk_logits),
+            dh0=torch.empty((d.B, d.H, d.d_k, d.d_v), dtype=torch.float32, device=dev) if want_dh0 else None,
+        )
+    if workspace is None:
+        workspace = plan.workspace(True, dev)
+    _check("sla_backward", lib().sla_backward(
+        plan.handle, _ptr(q), _ptr(k), _ptr(v), _ptr(log_decay), _ptr(beta), _ptr(gq_logits),
+        _ptr(gk_logits), _ptr(h0), _ptr(dO), _ptr(dht), _ptr(out["dq"]), _ptr(out["dk"]), _ptr(out["dv"]),
+        _ptr(out["dlog_decay"]), _ptr(out["dbeta"]), _ptr(out["dgq_logits"]), _ptr(out["dgk_logits"]),
+        _ptr(out["dh0"]), _ptr(workspace), workspace.numel(), _stream()))
+    return out
+
+
+def sla_decode_step(plan: Plan, q_t, k_t, v_t, log_decay_t, gq_logits_t, gk_logits_t, state, beta_t=None,
+                    o_t=None):
+    """One recurrent step on `state` ([Bdec,H,d_k,d_v] fp32, updated in place).  Returns o_t."""
+    d = plan.desc
+    Bdec = q_t.shape[0]
+    if o_t is None:
+        o_t = torch.empty((Bdec, d.H, d.d_v), dtype=plan.io_torch, device=q_t.device)
+    _check("sla_decode_step", lib().sla_decode_step(
+        plan.handle, Bdec, _ptr(q_t), _ptr(k_t), _ptr(v_t), _ptr(log_decay_t), _ptr(beta_t),
+        _ptr(gq_logits_t), _ptr(gk_logits_t), _ptr(state), _ptr(o_t), _stream()))
+    return o_t

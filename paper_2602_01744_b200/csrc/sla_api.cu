@@ -1,0 +1,207 @@
+// Host side of the C ABI: plan validation, workspace carve-up, launch order.
+#include "sla_internal.h"
+
+#include <new>
+#include <string.h>
+
+struct sla_plan {
+    sla::Dims dims;
+    sla::Workspace ws;
+    uint32_t flags;
+    int device;
+    int *d_status;          // device status word (bounded waits report here)
+    int last_launches;
+};
+
+namespace sla {
+
+static size_t align64(size_t x) { return (x + 63) & ~(size_t)63; }
+
+Workspace plan_workspace(const Dims &d) {
+    Workspace w{};
+    size_t bth = (size_t)d.B * d.T * d.H;
+    size_t off = 0;
+    auto take = [&](size_t n) { size_t o = off; off = align64(off + n); return o; };
+    w.Gq = take(bth);
+    w.Gk = take(bth);
+    w.bcum = take(d.variant == SLA_GLA ? bth * d.dk : bth);
+    w.states = take((size_t)d.B * d.H * (d.NT + 1) * d.dk * d.dv);
+    if (d.variant == SLA_GDN) {
+        w.W = take(bth * d.dk);
+        w.U0 = take(bth * d.dv);
+        w.U = take(bth * d.dv);
+    }
+    w.fwd_floats = off;
+    w.dstates = take((size_t)d.B * d.H * d.NT * d.dk * d.dv);
+    if (d.variant == SLA_GDN) w.dU = take(bth * d.dv);
+    w.dGq = take(bth);
+    w.dGk = take(bth);
+    w.bwd_floats = off;
+    return w;
+}
+
+}  // namespace sla
+
+static bool aligned16(const void *p) { return ((uintptr_t)p & 15u) == 0; }
+
+extern "C" {
+
+const char *sla_status_string(sla_status s) {
+    switch (s) {
+        case SLA_OK: return "ok";
+        case SLA_ERR_INVALID_ARG: return "invalid argument";
+        case SLA_ERR_UNSUPPORTED: return "unsupported shape or option";
+        case SLA_ERR_WORKSPACE: return "workspace missing or too small";
+        case SLA_ERR_ARCH: return "device is not sm_100";
+        case SLA_ERR_CUDA: return "CUDA runtime error";
+        case SLA_ERR_TIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown status";
+}
+
+sla_status sla_plan_create(sla_plan **out, const sla_desc *desc) {
+    if (!out) return SLA_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!desc || desc->struct_size != sizeof(sla_desc)) return SLA_ERR_INVALID_ARG;
+    if (desc->variant < SLA_RETNET || desc->variant > SLA_GDN) return SLA_ERR_INVALID_ARG;
+    if (desc->io_dtype != SLA_FP32 && desc->io_dtype != SLA_BF16) return SLA_ERR_INVALID_ARG;
+    if (desc->B < 0 || desc->T < 0 || desc->H < 1) return SLA_ERR_INVALID_ARG;
+    if (desc->H > 32) return SLA_ERR_UNSUPPORTED;
+    if (desc->d_k < 16 || desc->d_k > 128 || desc->d_k % 16) return SLA_ERR_UNSUPPORTED;
+    if (desc->d_v < 16 || desc->d_v > 128 || desc->d_v % 16) return SLA_ERR_UNSUPPORTED;
+    if (desc->chunk != 16 && desc->chunk != 32 && desc->chunk != 64) return SLA_ERR_UNSUPPORTED;
+    if ((uint64_t)desc->B * desc->H > 65535u) return SLA_ERR_UNSUPPORTED;   // grid.y limit
+    if (!(desc->scale == desc->scale)) return SLA_ERR_INVALID_ARG;
+
+    int dev = 0;
+    cudaDeviceProp prop;
+    if (cudaGetDevice(&dev) != cudaSuccess) return SLA_ERR_CUDA;
+    if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return SLA_ERR_CUDA;
+    if (prop.major != 10) return SLA_ERR_ARCH;
+    if (sla::generic_configure() != 0) return SLA_ERR_CUDA;
+
+    sla_plan *p = new (std::nothrow) sla_plan();
+    if (!p) return SLA_ERR_CUDA;
+    sla::Dims &d = p->dims;
+    d.variant = desc->variant;
+    d.io_bf16 = desc->io_dtype == SLA_BF16;
+    d.B = desc->B; d.T = desc->T; d.H = desc->H;
+    d.dk = desc->d_k; d.dv = desc->d_v; d.C = desc->chunk;
+    d.NT = (desc->T + desc->chunk - 1) / desc->chunk;
+    d.scale = desc->scale;
+    p->ws = sla::plan_workspace(d);
+    p->flags = desc->flags;
+    p->device = dev;
+    p->last_launches = 0;
+    p->d_status = nullptr;
+    if (cudaMalloc((void **)&p->d_status, sizeof(int)) != cudaSuccess ||
+        cudaMemset(p->d_status, 0, sizeof(int)) != cudaSuccess) {
+        if (p->d_status) cudaFree(p->d_status);
+        delete p;
+        return SLA_ERR_CUDA;
+    }
+    *out = p;
+    return SLA_OK;
+}
+
+sla_status sla_plan_destroy(sla_plan *plan) {
+    if (!plan) return SLA_OK;
+    if (plan->d_status) cudaFree(plan->d_status);
+    delete plan;
+    return SLA_OK;
+}
+
+sla_status sla_plan_workspace_bytes(const sla_plan *plan, size_t *fwd, size_t *bwd) {
+    if (!plan) return SLA_ERR_INVALID_ARG;
+    if (fwd) *fwd = plan->ws.fwd_floats * sizeof(float);
+    if (bwd) *bwd = plan->ws.bwd_floats * sizeof(float);
+    return SLA_OK;
+}
+
+sla_status sla_plan_poll(sla_plan *plan) {
+    if (!plan) return SLA_ERR_INVALID_ARG;
+    int v = 0;
+    if (cudaMemcpy(&v, plan->d_status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return SLA_ERR_CUDA;
+    if (v != 0) {
+        cudaMemset(plan->d_status, 0, sizeof(int));
+        return SLA_ERR_TIMEOUT;
+    }
+    return SLA_OK;
+}
+
+int32_t sla_plan_last_launch_count(const sla_plan *plan) { return plan ? plan->last_launches : 0; }
+
+sla_status sla_forward(sla_plan *plan, const void *q, const void *k, const void *v,
+                       const float *log_decay, const float *beta, const float *gq_logits,
+                       const float *gk_logits, const float *h0, void *o, float *ht, void *workspace,
+                       size_t workspace_bytes, void *cuda_stream) {
+    if (!plan) return SLA_ERR_INVALID_ARG;
+    const sla::Dims &d = plan->dims;
+    plan->last_launches = 0;
+    if (d.B == 0 || d.T == 0) return SLA_OK;
+    if (!q || !k || !v || !log_decay || !gq_logits || !gk_logits || !o) return SLA_ERR_INVALID_ARG;
+    if (d.variant == SLA_GDN && !beta) return SLA_ERR_INVALID_ARG;
+    const void *ptrs[] = {q, k, v, log_decay, beta, gq_logits, gk_logits, h0, o, ht, workspace};
+    for (const void *p : ptrs)
+        if (!aligned16(p)) return SLA_ERR_INVALID_ARG;
+    if (!workspace || workspace_bytes < plan->ws.fwd_floats * sizeof(float)) return SLA_ERR_WORKSPACE;
+    sla::FwdArgs a{q, k, v, log_decay, beta, gq_logits, gk_logits, h0, o, ht, (float *)workspace};
+    int n = sla::generic_forward(d, plan->ws, a, true, (cudaStream_t)cuda_stream);
+    if (n < 0) return SLA_ERR_CUDA;
+    plan->last_launches = n;
+    return SLA_OK;
+}
+
+sla_status sla_backward(sla_plan *plan, const void *q, const void *k, const void *v,
+                        const float *log_decay, const float *beta, const float *gq_logits,
+                        const float *gk_logits, const float *h0, const void *dO, const float *dht,
+                        void *dq, void *dk, void *dv, float *dlog_decay, float *dbeta,
+                        float *dgq_logits, float *dgk_logits, float *dh0, void *workspace,
+                        size_t workspace_bytes, void *cuda_stream) {
+    if (!plan) return SLA_ERR_INVALID_ARG;
+    const sla::Dims &d = plan->dims;
+    plan->last_launches = 0;
+    if (d.B == 0 || d.T == 0) return SLA_OK;
+    if (!q || !k || !v || !log_decay || !gq_logits || !gk_logits || !dO || !dq || !dk || !dv ||
+        !dgq_logits || !dgk_logits)
+        return SLA_ERR_INVALID_ARG;
+    if (dgq_logits == dgk_logits) return SLA_ERR_INVALID_ARG;
+    if (d.variant == SLA_GDN && (!beta || !dbeta || !dlog_decay)) return SLA_ERR_INVALID_ARG;
+    if (d.variant == SLA_GLA && !dlog_decay) return SLA_ERR_INVALID_ARG;
+    if (d.variant == SLA_RETNET && dlog_decay) return SLA_ERR_INVALID_ARG;
+    const void *ptrs[] = {q, k, v, log_decay, beta, gq_logits, gk_logits, h0, dO, dht, dq, dk, dv,
+                          dlog_decay, dbeta, dgq_logits, dgk_logits, dh0, workspace};
+    for (const void *p : ptrs)
+        if (!aligned16(p)) return SLA_ERR_INVALID_ARG;
+    if (!workspace || workspace_bytes < plan->ws.bwd_floats * sizeof(float)) return SLA_ERR_WORKSPACE;
+    sla::BwdArgs a{q, k, v, log_decay, beta, gq_logits, gk_logits, h0, dO, dht, dq, dk, dv,
+                   dlog_decay, dbeta, dgq_logits, dgk_logits, dh0, (float *)workspace};
+    int n = sla::generic_backward(d, plan->ws, a, (cudaStream_t)cuda_stream);
+    if (n == -2) return SLA_ERR_UNSUPPORTED;
+    if (n < 0) return SLA_ERR_CUDA;
+    plan->last_launches = n;
+    return SLA_OK;
+}
+
+sla_status sla_decode_step(sla_plan *plan, int32_t Bdec, const void *q_t, const void *k_t,
+                           const void *v_t, const float *log_decay_t, const float *beta_t,
+                           const float *gq_logits_t, const float *gk_logits_t, float *state, void *o_t,
+                           void *cuda_stream) {
+    if (!plan || Bdec < 0) return SLA_ERR_INVALID_ARG;
+    const sla::Dims &d = plan->dims;
+    plan->last_launches = 0;
+    if (Bdec == 0) return SLA_OK;
+    if (!q_t || !k_t || !v_t || !log_decay_t || !gq_logits_t || !gk_logits_t || !state || !o_t)
+        return SLA_ERR_INVALID_ARG;
+    if (d.variant == SLA_GDN && !beta_t) return SLA_ERR_INVALID_ARG;
+    const void *ptrs[] = {q_t, k_t, v_t, log_decay_t, beta_t, gq_logits_t, gk_logits_t, state, o_t};
+    for (const void *p : ptrs)
+        if (!aligned16(p)) return SLA_ERR_INVALID_ARG;
+    sla::DecArgs a{q_t, k_t, v_t, log_decay_t, beta_t, gq_logits_t, gk_logits_t, state, o_t, Bdec};
+    int n = sla::decode_step(d, a, (cudaStream_t)cuda_stream);
+    if (n < 0) return SLA_ERR_CUDA;
+    plan->last_launches = n;
+    return SLA_OK;
+}
+
+}  // extern "C"

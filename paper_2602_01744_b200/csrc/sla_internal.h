@@ -1,0 +1,66 @@
+// Internal declarations shared by the host API and the kernel translation units.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "sla.h"
+
+namespace sla {
+
+struct Dims {
+    int variant;      // sla_variant
+    int io_bf16;      // 1: q,k,v,o are bf16, 0: fp32
+    int B, T, H, dk, dv, C, NT;
+    float scale;
+};
+
+// Carve-up of the caller's workspace (all fp32, offsets in floats, each 64-float aligned).
+struct Workspace {
+    size_t Gq, Gk;          // [B,T,H] gates
+    size_t bcum;            // GLA [B,T,H,dk]; RETNET/GDN [B,T,H]: chunk-local inclusive cumulative log-decay
+    size_t states;          // [B,H,NT+1,dk,dv]: state before each chunk, last = final state
+    size_t W, U0, U;        // GDN: W [B,T,H,dk]; U0 and U = U0 - W S [B,T,H,dv]
+    size_t fwd_floats;
+    size_t dstates;         // [B,H,NT,dk,dv]: gradient w.r.t. the state after each chunk
+    size_t dU;              // GDN: [B,T,H,dv]
+    size_t dGq, dGk;        // [B,T,H]
+    size_t bwd_floats;
+};
+
+Workspace plan_workspace(const Dims &d);
+
+// ---- generic (fp32 CUDA-core) chunk kernels: sla_generic.cu ----
+struct FwdArgs {
+    const void *q, *k, *v;
+    const float *log_decay, *beta, *lq, *lk, *h0;
+    void *o;
+    float *ht;
+    float *ws;
+};
+struct BwdArgs {
+    const void *q, *k, *v;
+    const float *log_decay, *beta, *lq, *lk, *h0;
+    const void *dO;
+    const float *dht;
+    void *dq, *dk, *dv;
+    float *dlog_decay, *dbeta, *dlq, *dlk, *dh0;
+    float *ws;
+};
+struct DecArgs {
+    const void *q, *k, *v;
+    const float *log_decay, *beta, *lq, *lk;
+    float *state;
+    void *o;
+    int Bdec;
+};
+
+// Each returns the number of kernels launched (>0) or -1 after a CUDA launch error.
+int generic_forward(const Dims &d, const Workspace &w, const FwdArgs &a, bool write_o, cudaStream_t st);
+int generic_backward(const Dims &d, const Workspace &w, const BwdArgs &a, cudaStream_t st);
+int decode_step(const Dims &d, const DecArgs &a, cudaStream_t st);
+// Opt the kernels into the shared memory they need (once per device).
+int generic_configure();
+
+}  // namespace sla

@@ -1,0 +1,90 @@
+"""Helpers for the GPU parity tests: run the CUDA path through the C-ABI binding and the oracle on
+the same seeded tensors, and compare per tensor by relative L2 error."""
+import numpy as np
+import torch
+
+from oracle import sla_oracle as orc
+from paper_2602_01744_b200 import api
+from paper_2602_01744_b200.inputs import make_inputs
+
+TOL = {"bf16": 1e-2, "fp32": 1e-4}     # max relative L2 error per tensor (bf16 I/O / fp32 I/O)
+
+
+def rel_l2(x, ref):
+    x = x.detach().double().cpu().numpy() if hasattr(x, "detach") else np.asarray(x, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    den = np.linalg.norm(ref)
+    return float(np.linalg.norm(x - ref) / den) if den > 0 else float(np.abs(x).max())
+
+
+def to_dev(x):
+    return {n: (None if t is None else t.cuda()) for n, t in x.items()}
+
+
+def gpu_forward(cfg, x, h0=None, want_ht=True, flags=0):
+    plan = api.sla_plan_create(cfg.variant, cfg.dtype, cfg.B, cfg.T, cfg.H, cfg.d_k, cfg.d_v, cfg.chunk,
+                               cfg.scale, flags)
+    ht = torch.empty((cfg.B, cfg.H, cfg.d_k, cfg.d_v), dtype=torch.float32, device="cuda") if want_ht else None
+    o, ht = api.sla_forward(plan, x["q"], x["k"], x["v"], x["log_decay"], x["gq_logits"], x["gk_logits"],
+                            beta=x["beta"], h0=h0, ht=ht)
+    torch.cuda.synchronize()
+    plan.poll()
+    return o, ht, plan
+
+
+def gpu_backward(cfg, x, h0=None, dht=None, want_dh0=False, flags=0):
+    plan = api.sla_plan_create(cfg.variant, cfg.dtype, cfg.B, cfg.T, cfg.H, cfg.d_k, cfg.d_v, cfg.chunk,
+                               cfg.scale, flags)
+    g = api.sla_backward(plan, x["q"], x["k"], x["v"], x["log_decay"], x["gq_logits"], x["gk_logits"], x["dO"],
+                         beta=x["beta"], h0=h0, dht=dht, want_dh0=want_dh0)
+    torch.cuda.synchronize()
+    plan.poll()
+    return g, plan
+
+
+def oracle_forward(cfg, x, h0=None, bsel=None):
+    """Oracle on the same bits (optionally on a subset of batch rows: sequences are independent)."""
+    s = (lambda t: t) if bsel is None else (lambda t: None if t is None else (t if t.dim() == 1 else t[bsel]))
+    return orc.forward(cfg.variant, s(x["q"]), s(x["k"]), s(x["v"]), s(x["log_decay"]), s(x["gq_logits"]),
+                       s(x["gk_logits"]), beta=s(x["beta"]), h0=s(h0) if h0 is not None else None,
+                       scale=cfg.scale)
+
+
+def oracle_backward(cfg, x, h0=None, dht=None, bsel=None):
+    s = (lambda t: t) if bsel is None else (lambda t: None if t is None else (t if t.dim() == 1 else t[bsel]))
+    return orc.backward(cfg.variant, s(x["q"]), s(x["k"]), s(x["v"]), s(x["log_decay"]), s(x["gq_logits"]),
+                        s(x["gk_logits"]), s(x["dO"]), beta=s(x["beta"]),
+                        h0=s(h0) if h0 is not None else None, dht=s(dht) if dht is not None else None,
+                        scale=cfg.scale)
+
+
+GRAD_NAMES = {"dq": "dq", "dk": "dk", "dv": "dv", "dlog_decay": "dlog_decay", "dbeta": "dbeta",
+              "dgq_logits": "dlq", "dgk_logits": "dlk", "dh0": "dh0"}
+
+
+def check_forward(cfg, with_h0=False, flags=0, bsel=None):
+    x = make_inputs(cfg, with_dO=False, with_h0=with_h0)
+    xd = to_dev(x)
+    o, ht, _ = gpu_forward(cfg, xd, h0=xd.get("h0"), flags=flags)
+    oref, htref = oracle_forward(cfg, x, h0=x.get("h0"), bsel=bsel)
+    sel = slice(None) if bsel is None else bsel
+    tol = TOL[cfg.dtype]
+    errs = {"o": rel_l2(o[sel], oref), "ht": rel_l2(ht[sel], htref)}
+    assert all(np.isfinite(e) and e <= tol for e in errs.values()), (cfg, errs)
+    return errs
+
+
+def check_backward(cfg, with_h0=False, flags=0, bsel=None):
+    x = make_inputs(cfg, with_dO=True, with_h0=with_h0)
+    xd = to_dev(x)
+    g, _ = gpu_backward(cfg, xd, h0=xd.get("h0"), dht=xd.get("dht"), want_dh0=with_h0, flags=flags)
+    ref = oracle_backward(cfg, x, h0=x.get("h0"), dht=x.get("dht"), bsel=bsel)
+    sel = slice(None) if bsel is None else bsel
+    tol = TOL[cfg.dtype]
+    errs = {}
+    for gname, rname in GRAD_NAMES.items():
+        if g.get(gname) is None:
+            continue
+        errs[gname] = rel_l2(g[gname][sel] if g[gname].dim() > 1 else g[gname], ref[rname])
+    assert all(np.isfinite(e) and e <= tol for e in errs.values()), (cfg, errs)
+    return errs

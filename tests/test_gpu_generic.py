@@ -1,0 +1,112 @@
+"""GPU parity of the fp32 CUDA-core chunk kernels against the fp64 oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2602_01744_b200 import api
+from paper_2602_01744_b200.inputs import CONFIGS, make_inputs, small
+from tests import gpu_util as gu
+
+pytestmark = pytest.mark.gpu
+GEN = api.SLA_FLAG_FORCE_GENERIC
+
+
+def test_c0_retnet_fp32_full_config():
+    errs = gu.check_forward(CONFIGS["C0"], flags=GEN)
+    assert max(errs.values()) <= 1e-4
+
+
+@pytest.mark.parametrize("variant", ["retnet", "gla", "gdn"])
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_forward_small_ragged_tail_with_initial_state(variant, dtype):
+    base = {"retnet": CONFIGS["C0"], "gla": CONFIGS["C1"], "gdn": CONFIGS["C4"]}[variant]
+    cfg = small(base, B=2, T=200, H=3, dtype=dtype, seed=100)      # 200 = 3 chunks + a tail of 8
+    gu.check_forward(cfg, with_h0=True, flags=GEN)
+
+
+@pytest.mark.parametrize("chunk,dk,dv,H", [(16, 64, 128, 4), (32, 16, 48, 1), (64, 128, 64, 16), (64, 32, 32, 5)])
+@pytest.mark.parametrize("variant", ["retnet", "gla", "gdn"])
+def test_forward_shapes(variant, chunk, dk, dv, H):
+    base = {"retnet": CONFIGS["C0"], "gla": CONFIGS["C1"], "gdn": CONFIGS["C4"]}[variant]
+    cfg = small(base, B=1, T=150, H=H, d_k=dk, d_v=dv, chunk=chunk, dtype="fp32", seed=101, scale=0.5)
+    gu.check_forward(cfg, flags=GEN)
+
+
+@pytest.mark.parametrize("variant", ["retnet", "gla"])
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_backward_small_ragged_tail_with_state_gradients(variant, dtype):
+    base = {"retnet": CONFIGS["C0"], "gla": CONFIGS["C2"]}[variant]
+    cfg = small(base, B=2, T=200, H=3, dtype=dtype, seed=102, backward=True)
+    gu.check_backward(cfg, with_h0=True, flags=GEN)
+
+
+@pytest.mark.parametrize("variant", ["retnet", "gla"])
+def test_backward_shapes(variant):
+    base = {"retnet": CONFIGS["C0"], "gla": CONFIGS["C2"]}[variant]
+    cfg = small(base, B=1, T=130, H=4, d_k=64, d_v=32, chunk=32, dtype="fp32", seed=103, scale=0.7)
+    gu.check_backward(cfg, flags=GEN)
+
+
+def test_single_token_and_single_chunk():
+    for T in (1, 64):
+        cfg = small(CONFIGS["C1"], B=1, T=T, H=2, dtype="fp32", seed=104)
+        gu.check_forward(cfg, flags=GEN)
+        gu.check_backward(small(cfg, backward=True), flags=GEN)
+
+
+@pytest.mark.parametrize("variant", ["retnet", "gla", "gdn"])
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_decode_steps_match_oracle_and_chunkwise(variant, dtype):
+    from oracle import sla_oracle as orc
+    from paper_2602_01744_b200.inputs import make_decode_inputs
+    base = {"retnet": CONFIGS["C0"], "gla": CONFIGS["C1"], "gdn": CONFIGS["C4"]}[variant]
+    cfg = small(base, B=3, T=20, H=4, dtype=dtype, seed=105)
+    steps = cfg.T
+    dec = make_decode_inputs(cfg, cfg.B, steps, seed=106)
+    h0 = torch.randn(cfg.B, cfg.H, cfg.d_k, cfg.d_v, generator=torch.Generator().manual_seed(7)) * 0.1
+    plan = api.sla_plan_create(cfg.variant, cfg.dtype, cfg.B, cfg.T, cfg.H, cfg.d_k, cfg.d_v, cfg.chunk)
+    state = h0.clone().cuda()
+    ref_state = np.ascontiguousarray(h0.double().numpy().copy())
+    outs, refs = [], []
+    for t in range(steps):
+        ld = dec["log_decay"] if variant == "retnet" else dec["log_decay"][t]
+        bt = None if dec["beta"] is None else dec["beta"][t]
+        o = api.sla_decode_step(plan, dec["q"][t].cuda(), dec["k"][t].cuda(), dec["v"][t].cuda(), ld.cuda(),
+                                dec["gq_logits"][t].cuda(), dec["gk_logits"][t].cuda(), state,
+                                beta_t=None if bt is None else bt.cuda())
+        outs.append(o)
+        refs.append(orc.decode_step(variant, dec["q"][t], dec["k"][t], dec["v"][t], ld, dec["gq_logits"][t],
+                                    dec["gk_logits"][t], ref_state, beta_t=bt))
+    torch.cuda.synchronize()
+    tol = gu.TOL[dtype]
+    assert gu.rel_l2(torch.stack(outs), np.stack(refs)) <= tol
+    assert gu.rel_l2(state, ref_state) <= tol
+    # the same tokens through the chunkwise forward with the same initial state
+    x = dict(q=dec["q"].transpose(0, 1).contiguous(), k=dec["k"].transpose(0, 1).contiguous(),
+             v=dec["v"].transpose(0, 1).contiguous(),
+             log_decay=dec["log_decay"] if variant == "retnet" else dec["log_decay"].transpose(0, 1).contiguous(),
+             beta=None if dec["beta"] is None else dec["beta"].transpose(0, 1).contiguous(),
+             gq_logits=dec["gq_logits"].transpose(0, 1).contiguous(),
+             gk_logits=dec["gk_logits"].transpose(0, 1).contiguous())
+    o2, ht2, _ = gu.gpu_forward(cfg, gu.to_dev(x), h0=h0.cuda(), flags=GEN)
+    assert gu.rel_l2(o2, torch.stack(outs, 1).double().cpu().numpy()) <= 2 * tol
+    assert gu.rel_l2(ht2, state.double().cpu().numpy()) <= 2 * tol
+
+
+def test_rejections():
+    with pytest.raises(api.SLAError) as e:
+        api.sla_plan_create("gla", "bf16", 1, 64, 33, 128, 128)
+    assert e.value.status == 2
+    with pytest.raises(api.SLAError):
+        api.sla_plan_create("gla", "bf16", 1, 64, 4, 100, 128)
+    plan = api.sla_plan_create("gla", "fp32", 1, 64, 2, 16, 16)
+    x = gu.to_dev(make_inputs(small(CONFIGS["C1"], B=1, T=64, H=2, d_k=16, d_v=16, dtype="fp32")))
+    tiny = torch.empty(16, dtype=torch.uint8, device="cuda")
+    with pytest.raises(api.SLAError) as e:
+        api.sla_forward(plan, x["q"], x["k"], x["v"], x["log_decay"], x["gq_logits"], x["gk_logits"], workspace=tiny)
+    assert e.value.status == 3
+    # empty problem: nothing to do, no error
+    p0 = api.sla_plan_create("gla", "fp32", 0, 64, 2, 16, 16)
+    z = torch.empty(0, device="cuda")
+    api.sla_forward(p0, z, z, z, z, z, z, o=z)
+    assert p0.last_launch_count == 0
