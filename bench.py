@@ -1,0 +1,315 @@
+#!/usr/bin/env python
+"""Benchmark of the SLA hot path: SLA-GLA forward + backward tokens/s at B=8, T=4096, H=16, d=128, bf16.
+
+One step = sla_forward followed by sla_backward over one batch of seeded synthetic input, through the
+C-ABI binding.  Prints ONE JSON line (rank 0).  `--impl reference` times the fp64 CPU oracle on a
+bounded sample of the same workload instead.  With --gpus N > 1 (under torchrun) every rank runs an
+independent replica of the workload on its own GPU (the path has no exchange step): weak scaling.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+from pathlib import Path
+
+ROOT = Path(__file__).resolve().parent
+sys.path.insert(0, str(ROOT))
+
+METRIC = "SLA-GLA fwd+bwd tokens/s (T=4K,H=16,d=128,bf16)"
+UNIT = "tokens/s"
+WORKLOAD = "C2"
+CPU_ROWS = 2          # batch rows of the workload the CPU oracle is timed on (about 20 core-seconds)
+# Algorithmic HBM bytes per (token, head) at d_k=d_v=128: bf16 q,k,v,o (+dO,dq,dk,dv), fp32 log-decay
+# (+ its gradient), fp32 gate logits (+ their gradients).
+FWD_BYTES_PER_TOKEN_HEAD = 4 * 256 + 512 + 8            # 1544
+BWD_BYTES_PER_TOKEN_HEAD = 4 * 256 + 512 + 3 * 256 + 512 + 16   # 2832
+KERNEL_BYTES = {  # which share of the compulsory traffic each kernel is accountable for
+    "output": FWD_BYTES_PER_TOKEN_HEAD, "grads_lin": BWD_BYTES_PER_TOKEN_HEAD,
+    "gla_fwd_tc": FWD_BYTES_PER_TOKEN_HEAD, "gla_bwd_tc": BWD_BYTES_PER_TOKEN_HEAD,
+}
+
+
+def measured_peaks():
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        try:
+            d = json.loads(p.read_text())
+            return float(d["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return 6650.0, "fallback"
+
+
+def recorded_traffic(kernel: str):
+    """DRAM bytes per launch from the committed ncu summary, if one covers this kernel."""
+    p = ROOT / "profiles" / "dram_traffic.json"
+    if not p.exists():
+        return None
+    try:
+        e = json.loads(p.read_text()).get(kernel)
+        return None if e is None else e.get("bytes_per_launch_full_size")
+    except Exception:
+        return None
+
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+        self.index = index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=self.tmp, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.tmp.flush()
+        rows = [r.split(",") for r in Path(self.tmp.name).read_text().strip().splitlines() if r.count(",") >= 6]
+        os.unlink(self.tmp.name)
+        if not rows:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        sm = [float(r[0]) for r in rows]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for i, n in enumerate(names) if any(r[3 + i].strip().lower() == "active" for r in rows)]
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": float(rows[0][1]), "samples": len(rows),
+                "power_w_max": max(float(r[2]) for r in rows), "reasons": reasons}
+
+
+def cpu_oracle_sample(cfg, x, steps=1, warmup=0):
+    """fp64 oracle, forward + backward, on the first CPU_ROWS batch rows of the workload (all T tokens, all heads)."""
+    from oracle import sla_oracle as orc
+    s = lambda t: t[0:CPU_ROWS]
+    args = (s(x["q"]), s(x["k"]), s(x["v"]), s(x["log_decay"]), s(x["gq_logits"]), s(x["gk_logits"]))
+    # widen once outside the timed region, as the GPU arm holds its inputs resident
+    args = tuple(a.double().numpy() for a in args)
+    dO = s(x["dO"]).double().numpy()
+    times = []
+    for i in range(warmup + steps):
+        t0 = time.perf_counter()
+        orc.forward(cfg.variant, *args, scale=cfg.scale)
+        orc.backward(cfg.variant, *args, dO, scale=cfg.scale)
+        dt = time.perf_counter() - t0
+        if i >= warmup:
+            times.append(dt)
+    tokens = cfg.T * CPU_ROWS
+    return tokens, times, orc.num_threads()
+
+
+def run_reference(args, cfg, rank):
+    if rank != 0:
+        return
+    from paper_2602_01744_b200.inputs import make_inputs, small
+    x = make_inputs(small(cfg, B=CPU_ROWS))
+    tokens, times, cores = cpu_oracle_sample(cfg, x, steps=args.steps, warmup=min(args.warmup, 1))
+    total = sum(times)
+    value = tokens * len(times) / total
+    sample = f"first {CPU_ROWS} batch rows of {WORKLOAD}: T={cfg.T}, H={cfg.H}, d={cfg.d_k}, forward+backward, fp64 recurrent oracle"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / len(times),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "variant": cfg.variant, "B": CPU_ROWS, "T": cfg.T, "H": cfg.H,
+                   "d_k": cfg.d_k, "d_v": cfg.d_v, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--generic", action="store_true", help="force the fp32 CUDA-core kernels")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "b200" else args.warmup
+
+    from paper_2602_01744_b200.inputs import CONFIGS, make_inputs
+    cfg = CONFIGS[WORKLOAD]
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        run_reference(args, cfg, rank)
+        return
+
+    import torch
+    from paper_2602_01744_b200 import api
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the SLA library has no CPU path")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    x = make_inputs(cfg)                        # every replica draws the same seeded batch
+    names = ["q", "k", "v", "log_decay", "gq_logits", "gk_logits", "dO"]
+    host = {n: x[n].pin_memory() for n in names}
+    dev = {n: host[n].cuda() for n in names}
+    flags = api.SLA_FLAG_FORCE_GENERIC if args.generic else 0
+    plan = api.sla_plan_create(cfg.variant, cfg.dtype, cfg.B, cfg.T, cfg.H, cfg.d_k, cfg.d_v, cfg.chunk,
+                               cfg.scale, flags)
+    ws = plan.workspace(backward=True)
+    o = torch.empty_like(dev["v"])
+    grads = dict(dq=torch.empty_like(dev["q"]), dk=torch.empty_like(dev["k"]), dv=torch.empty_like(dev["v"]),
+                 dlog_decay=torch.empty_like(dev["log_decay"]), dbeta=None,
+                 dgq_logits=torch.empty_like(dev["gq_logits"]), dgk_logits=torch.empty_like(dev["gk_logits"]),
+                 dh0=None)
+    launches = [0]
+
+    def step(d):
+        api.sla_forward(plan, d["q"], d["k"], d["v"], d["log_decay"], d["gq_logits"], d["gk_logits"], o=o,
+                        workspace=ws)
+        launches[0] += plan.last_launch_count
+        api.sla_backward(plan, d["q"], d["k"], d["v"], d["log_decay"], d["gq_logits"], d["gk_logits"], d["dO"],
+                         workspace=ws, out=grads)
+        launches[0] += plan.last_launch_count
+
+    for _ in range(args.warmup):
+        step(dev)
+    barrier()
+    plan.poll()
+
+    # ---- device-resident timing (inputs in HBM; 0.77 GB of inputs per step, far beyond the 126 MB L2) ----
+    launches[0] = 0
+    plan.set_kernel_timing(True)
+    sampler = ClockSampler(local)
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    for _ in range(args.steps):
+        step(dev)
+    e1.record()
+    barrier()
+    ms = e0.elapsed_time(e1)
+    clocks = sampler.stop()
+    ktimes = plan.kernel_times()
+    plan.set_kernel_timing(False)
+    plan.poll()
+    n_launch = launches[0]
+    if dist is not None:
+        t = torch.tensor([ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    tokens_step = cfg.B * cfg.T
+    value = world * tokens_step * args.steps / (ms * 1e-3)
+
+    # ---- end to end: pinned host inputs -> device, run, results -> pinned host, every step ----
+    outs = [o, grads["dq"], grads["dk"], grads["dv"], grads["dlog_decay"], grads["dgq_logits"], grads["dgk_logits"]]
+    host_out = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in outs]
+    stage = {n: torch.empty_like(dev[n]) for n in names}
+    h2d = sum(host[n].numel() * host[n].element_size() for n in names)
+    d2h = sum(t.numel() * t.element_size() for t in outs)
+    e2e_steps = max(3, min(args.steps, 10))
+
+    def e2e_step():
+        for n in names:
+            stage[n].copy_(host[n], non_blocking=True)
+        step(stage)
+        for src, dst in zip(outs, host_out):
+            dst.copy_(src, non_blocking=True)
+
+    e2e_step()
+    barrier()
+    e0.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record()
+    barrier()
+    ms_e2e = e0.elapsed_time(e1)
+    if dist is not None:
+        t = torch.tensor([ms_e2e], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_e2e = float(t.item())
+    e2e_value = world * tokens_step * e2e_steps / (ms_e2e * 1e-3)
+
+    # ---- roofline of the dominant kernel, from the per-kernel CUDA events of the timed region ----
+    peak, peak_kind = measured_peaks()
+    roof = None
+    if ktimes:
+        top = max(ktimes, key=lambda k: ktimes[k][1])
+        cnt, tot = ktimes[top]
+        avg_ms = tot / cnt
+        per_unit = KERNEL_BYTES.get(top)
+        share = {k: round(v[1] / sum(t[1] for t in ktimes.values()), 4) for k, v in ktimes.items()}
+        if per_unit is not None:
+            alg = per_unit * cfg.B * cfg.T * cfg.H
+            achieved = alg / (avg_ms * 1e-3) / 1e9
+            roof = {"bound": "hbm", "kernel": top, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                    "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": recorded_traffic(top),
+                    "algorithmic_bytes_per_launch": alg, "avg_launch_ms": avg_ms, "kernel_time_share": share}
+        else:
+            roof = {"bound": "hbm", "kernel": top, "achieved": None, "peak": peak, "unit": "GB/s", "frac": None,
+                    "peak_kind": f"of {peak_kind}", "traffic": None, "avg_launch_ms": avg_ms,
+                    "kernel_time_share": share}
+    # whole-step figure against the same peak: all compulsory bytes of forward + backward / step time
+    step_bytes = (FWD_BYTES_PER_TOKEN_HEAD + BWD_BYTES_PER_TOKEN_HEAD) * cfg.B * cfg.T * cfg.H
+    step_gbs = step_bytes / (ms / args.steps * 1e-3) / 1e9
+
+    if rank == 0:
+        cpu = None
+        if world == 1 and not args.no_cpu_baseline:
+            tokens, times, cores = cpu_oracle_sample(cfg, x, steps=1)
+            cpu = {"value": tokens / times[0], "unit": UNIT, "cores": cores, "kind": "oracle",
+                   "sample": f"first {CPU_ROWS} batch rows of {WORKLOAD} (T={cfg.T}, H={cfg.H}), forward+backward, "
+                             f"{times[0]:.1f} s of fp64 recurrent oracle"}
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "variant": cfg.variant, "B": cfg.B, "T": cfg.T, "H": cfg.H,
+                       "d_k": cfg.d_k, "d_v": cfg.d_v, "chunk": cfg.chunk, "pass": "forward+backward",
+                       "io": "bf16 q,k,v,o and gradients; fp32 decay, logits, state; fp32 accumulation",
+                       "l2": "inputs (0.77 GB per step) exceed the 126 MB L2; no flush needed",
+                       "parallelism": "replicas only" if world > 1 else "single GPU",
+                       "kernels": "generic fp32 CUDA-core" if args.generic else "default"},
+            "clocks": clocks,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "steps": e2e_steps, "ms_per_step": ms_e2e / e2e_steps},
+            "gpu_launches": n_launch,
+            "roofline": roof,
+            "step_hbm": {"algorithmic_bytes_per_step": step_bytes, "achieved_gbs": step_gbs, "frac": step_gbs / peak},
+            "cpu_baseline": cpu,
+        }
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -83,6 +83,19 @@ sla_status sla_plan_poll(sla_plan *plan);
  * enqueued (for launch accounting in benchmarks). */
 int32_t sla_plan_last_launch_count(const sla_plan *plan);
 
+/*
+ * Optional per-kernel timing (measurement aid; the paper has no counterpart).  While enabled, every
+ * entry point records one CUDA event before its first kernel and one after each kernel on the
+ * launch stream.  sla_plan_kernel_timing_collect waits for the last recorded event, folds the
+ * elapsed times into per-kernel totals (by kernel name) and returns how many names there are;
+ * sla_plan_kernel_timing_get reads one total.  `name` points at a string literal owned by the library.
+ * Enabling (or disabling) clears the totals.  Events are created on first use and reused.
+ */
+sla_status sla_plan_set_kernel_timing(sla_plan *plan, int32_t enable);
+sla_status sla_plan_kernel_timing_collect(sla_plan *plan, int32_t *n_kernels);
+sla_status sla_plan_kernel_timing_get(const sla_plan *plan, int32_t index, const char **name,
+                                      int32_t *launches, float *total_ms);
+
 const char *sla_status_string(sla_status s);
 
 /*

@@ -21,7 +21,8 @@ VARIANTS = {"retnet": SLA_RETNET, "gla": SLA_GLA, "gdn": SLA_GDN}
 DTYPES = {"fp32": SLA_FP32, "bf16": SLA_BF16, torch.float32: SLA_FP32, torch.bfloat16: SLA_BF16}
 EXPORTS = (
     "sla_plan_create", "sla_plan_destroy", "sla_plan_workspace_bytes", "sla_plan_poll",
-    "sla_plan_last_launch_count", "sla_status_string", "sla_forward", "sla_backward", "sla_decode_step",
+    "sla_plan_last_launch_count", "sla_plan_set_kernel_timing", "sla_plan_kernel_timing_collect",
+    "sla_plan_kernel_timing_get", "sla_status_string", "sla_forward", "sla_backward", "sla_decode_step",
 )
 
 
@@ -58,13 +59,18 @@ def lib():
         L.sla_plan_poll.argtypes = [vp]
         L.sla_plan_last_launch_count.argtypes = [vp]
         L.sla_plan_last_launch_count.restype = i32
+        L.sla_plan_set_kernel_timing.argtypes = [vp, i32]
+        L.sla_plan_kernel_timing_collect.argtypes = [vp, ctypes.POINTER(i32)]
+        L.sla_plan_kernel_timing_get.argtypes = [vp, i32, ctypes.POINTER(ctypes.c_char_p), ctypes.POINTER(i32),
+                                                 ctypes.POINTER(ctypes.c_float)]
         L.sla_status_string.argtypes = [ctypes.c_int]
         L.sla_status_string.restype = ctypes.c_char_p
         L.sla_forward.argtypes = [vp] * 11 + [vp, sz, vp]
         L.sla_backward.argtypes = [vp] * 19 + [vp, sz, vp]
         L.sla_decode_step.argtypes = [vp, i32] + [vp] * 10
         for name in ("sla_plan_create", "sla_plan_destroy", "sla_plan_workspace_bytes", "sla_plan_poll",
-                     "sla_forward", "sla_backward", "sla_decode_step"):
+                     "sla_plan_set_kernel_timing", "sla_plan_kernel_timing_collect",
+                     "sla_plan_kernel_timing_get", "sla_forward", "sla_backward", "sla_decode_step"):
             getattr(L, name).restype = ctypes.c_int
         _lib = L
     return _lib
@@ -113,6 +119,21 @@ class Plan:
     @property
     def last_launch_count(self) -> int:
         return int(lib().sla_plan_last_launch_count(self.handle))
+
+    def set_kernel_timing(self, enable: bool):
+        _check("sla_plan_set_kernel_timing", lib().sla_plan_set_kernel_timing(self.handle, int(enable)))
+
+    def kernel_times(self) -> dict:
+        """{kernel name: (launches, total ms)} accumulated since timing was enabled."""
+        n = ctypes.c_int32()
+        _check("sla_plan_kernel_timing_collect", lib().sla_plan_kernel_timing_collect(self.handle, ctypes.byref(n)))
+        out = {}
+        for i in range(n.value):
+            name, cnt, ms = ctypes.c_char_p(), ctypes.c_int32(), ctypes.c_float()
+            _check("sla_plan_kernel_timing_get", lib().sla_plan_kernel_timing_get(
+                self.handle, i, ctypes.byref(name), ctypes.byref(cnt), ctypes.byref(ms)))
+            out[name.value.decode()] = (cnt.value, ms.value)
+        return out
 
     def workspace(self, backward=False, device="cuda"):
         n = self.backward_workspace_bytes if backward else self.forward_workspace_bytes

@@ -3,6 +3,8 @@
 
 #include <new>
 #include <string.h>
+#include <utility>
+#include <vector>
 
 struct sla_plan {
     sla::Dims dims;
@@ -11,6 +13,8 @@ struct sla_plan {
     int device;
     int *d_status;          // device status word (bounded waits report here)
     int last_launches;
+    sla::Tracer tracer;
+    std::vector<std::pair<const char *, std::pair<int, float>>> agg;   // name -> (launches, total ms)
 };
 
 namespace sla {
@@ -107,6 +111,7 @@ sla_status sla_plan_create(sla_plan **out, const sla_desc *desc) {
 sla_status sla_plan_destroy(sla_plan *plan) {
     if (!plan) return SLA_OK;
     if (plan->d_status) cudaFree(plan->d_status);
+    plan->tracer.destroy();
     delete plan;
     return SLA_OK;
 }
@@ -131,6 +136,40 @@ sla_status sla_plan_poll(sla_plan *plan) {
 
 int32_t sla_plan_last_launch_count(const sla_plan *plan) { return plan ? plan->last_launches : 0; }
 
+sla_status sla_plan_set_kernel_timing(sla_plan *plan, int32_t enable) {
+    if (!plan) return SLA_ERR_INVALID_ARG;
+    plan->tracer.clear();
+    plan->agg.clear();
+    plan->tracer.on = enable != 0;
+    return SLA_OK;
+}
+
+sla_status sla_plan_kernel_timing_collect(sla_plan *plan, int32_t *n_kernels) {
+    if (!plan || !n_kernels) return SLA_ERR_INVALID_ARG;
+    sla::Tracer &t = plan->tracer;
+    if (t.used && cudaEventSynchronize(t.pool[t.used - 1]) != cudaSuccess) return SLA_ERR_CUDA;
+    for (const auto &r : t.recs) {
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, t.pool[r.e0], t.pool[r.e1]) != cudaSuccess) return SLA_ERR_CUDA;
+        bool found = false;
+        for (auto &a : plan->agg)
+            if (!strcmp(a.first, r.name)) { a.second.first += 1; a.second.second += ms; found = true; break; }
+        if (!found) plan->agg.push_back({r.name, {1, ms}});
+    }
+    t.clear();
+    *n_kernels = (int32_t)plan->agg.size();
+    return SLA_OK;
+}
+
+sla_status sla_plan_kernel_timing_get(const sla_plan *plan, int32_t index, const char **name,
+                                      int32_t *launches, float *total_ms) {
+    if (!plan || index < 0 || (size_t)index >= plan->agg.size()) return SLA_ERR_INVALID_ARG;
+    if (name) *name = plan->agg[index].first;
+    if (launches) *launches = plan->agg[index].second.first;
+    if (total_ms) *total_ms = plan->agg[index].second.second;
+    return SLA_OK;
+}
+
 sla_status sla_forward(sla_plan *plan, const void *q, const void *k, const void *v,
                        const float *log_decay, const float *beta, const float *gq_logits,
                        const float *gk_logits, const float *h0, void *o, float *ht, void *workspace,
@@ -146,7 +185,8 @@ sla_status sla_forward(sla_plan *plan, const void *q, const void *k, const void 
         if (!aligned16(p)) return SLA_ERR_INVALID_ARG;
     if (!workspace || workspace_bytes < plan->ws.fwd_floats * sizeof(float)) return SLA_ERR_WORKSPACE;
     sla::FwdArgs a{q, k, v, log_decay, beta, gq_logits, gk_logits, h0, o, ht, (float *)workspace};
-    int n = sla::generic_forward(d, plan->ws, a, true, (cudaStream_t)cuda_stream);
+    plan->tracer.start((cudaStream_t)cuda_stream);
+    int n = sla::generic_forward(d, plan->ws, a, true, (cudaStream_t)cuda_stream, plan->tracer);
     if (n < 0) return SLA_ERR_CUDA;
     plan->last_launches = n;
     return SLA_OK;
@@ -176,7 +216,8 @@ sla_status sla_backward(sla_plan *plan, const void *q, const void *k, const void
     if (!workspace || workspace_bytes < plan->ws.bwd_floats * sizeof(float)) return SLA_ERR_WORKSPACE;
     sla::BwdArgs a{q, k, v, log_decay, beta, gq_logits, gk_logits, h0, dO, dht, dq, dk, dv,
                    dlog_decay, dbeta, dgq_logits, dgk_logits, dh0, (float *)workspace};
-    int n = sla::generic_backward(d, plan->ws, a, (cudaStream_t)cuda_stream);
+    plan->tracer.start((cudaStream_t)cuda_stream);
+    int n = sla::generic_backward(d, plan->ws, a, (cudaStream_t)cuda_stream, plan->tracer);
     if (n == -2) return SLA_ERR_UNSUPPORTED;
     if (n < 0) return SLA_ERR_CUDA;
     plan->last_launches = n;
@@ -198,7 +239,8 @@ sla_status sla_decode_step(sla_plan *plan, int32_t Bdec, const void *q_t, const 
     for (const void *p : ptrs)
         if (!aligned16(p)) return SLA_ERR_INVALID_ARG;
     sla::DecArgs a{q_t, k_t, v_t, log_decay_t, beta_t, gq_logits_t, gk_logits_t, state, o_t, Bdec};
-    int n = sla::decode_step(d, a, (cudaStream_t)cuda_stream);
+    plan->tracer.start((cudaStream_t)cuda_stream);
+    int n = sla::decode_step(d, a, (cudaStream_t)cuda_stream, plan->tracer);
     if (n < 0) return SLA_ERR_CUDA;
     plan->last_launches = n;
     return SLA_OK;

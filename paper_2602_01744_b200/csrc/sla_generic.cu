@@ -785,7 +785,7 @@ void launch_gate_bwd(const float *Gq, const float *Gk, const float *dGq, const f
 }
 
 template <typename TIO>
-int forward_t(const Dims &d, const Workspace &w, const FwdArgs &a, bool write_o, cudaStream_t st) {
+int forward_t(const Dims &d, const Workspace &w, const FwdArgs &a, bool write_o, cudaStream_t st, Tracer &tr) {
     float *ws = a.ws;
     float *Gq = ws + w.Gq, *Gk = ws + w.Gk, *bcum = ws + w.bcum, *states = ws + w.states;
     float *Wws = ws + w.W, *U0ws = ws + w.U0, *Uws = ws + w.U;
@@ -801,27 +801,32 @@ int forward_t(const Dims &d, const Workspace &w, const FwdArgs &a, bool write_o,
         case 16: launch_gate_fwd<16>(a.lq, a.lk, Gq, Gk, n_tok, d.H, st); break;
         default: launch_gate_fwd<32>(a.lq, a.lk, Gq, Gk, n_tok, d.H, st); break;
     }
+    tr.mark("gate_fwd");
     ++launches;
     dim3 tiles(d.NT, d.B * d.H);
     k_cumdecay<<<tiles, d.variant == SLA_GLA ? 128 : 32, 0, st>>>(d, a.log_decay, bcum);
+    tr.mark("cumdecay");
     ++launches;
     const TIO *q = (const TIO *)a.q, *k = (const TIO *)a.k, *v = (const TIO *)a.v;
     if (d.variant == SLA_GDN) {
         k_gdn_prepare<TIO><<<tiles, 256, smem_prepare(d), st>>>(d, k, v, a.beta, Gk, bcum, Wws, U0ws);
+        tr.mark("gdn_prepare");
         ++launches;
     }
     dim3 slices(d.dv / VS, d.B * d.H);
     k_state_scan<TIO><<<slices, 128, smem_scan(d), st>>>(d, k, v, Gk, bcum, a.h0, states, a.ht, Wws, U0ws, Uws);
+    tr.mark("state_scan");
     ++launches;
     if (write_o) {
         k_output<TIO><<<tiles, 256, smem_output(d), st>>>(d, q, k, v, Gq, Gk, bcum, states, Uws, (TIO *)a.o);
+        tr.mark("output");
         ++launches;
     }
     return cudaGetLastError() == cudaSuccess ? launches : -1;
 }
 
 template <typename TIO>
-int backward_lin_t(const Dims &d, const Workspace &w, const BwdArgs &a, cudaStream_t st) {
+int backward_lin_t(const Dims &d, const Workspace &w, const BwdArgs &a, cudaStream_t st, Tracer &tr) {
     float *ws = a.ws;
     float *Gq = ws + w.Gq, *Gk = ws + w.Gk, *bcum = ws + w.bcum, *states = ws + w.states;
     float *dstates = ws + w.dstates, *dGq = ws + w.dGq, *dGk = ws + w.dGk;
@@ -830,10 +835,12 @@ int backward_lin_t(const Dims &d, const Workspace &w, const BwdArgs &a, cudaStre
     dim3 tiles(d.NT, d.B * d.H), slices(d.dv / VS, d.B * d.H);
     k_dstate_scan<TIO><<<slices, 128, smem_dscan(d), st>>>(d, q, k, dO, Gq, bcum, a.dht, dstates, a.dh0,
                                                            nullptr, nullptr);
+    tr.mark("dstate_scan");
     ++launches;
     k_grads_lin<TIO><<<tiles, 256, smem_grads_lin(d), st>>>(d, q, k, v, dO, Gq, Gk, bcum, states, dstates,
                                                             (TIO *)a.dq, (TIO *)a.dk, (TIO *)a.dv,
                                                             a.dlog_decay, dGq, dGk);
+    tr.mark("grads_lin");
     ++launches;
     return cudaGetLastError() == cudaSuccess ? launches : -1;
 }
@@ -857,18 +864,18 @@ int generic_configure() {
     return ok ? 0 : -1;
 }
 
-int generic_forward(const Dims &d, const Workspace &w, const FwdArgs &a, bool write_o, cudaStream_t st) {
-    return d.io_bf16 ? forward_t<__nv_bfloat16>(d, w, a, write_o, st) : forward_t<float>(d, w, a, write_o, st);
+int generic_forward(const Dims &d, const Workspace &w, const FwdArgs &a, bool write_o, cudaStream_t st, Tracer &tr) {
+    return d.io_bf16 ? forward_t<__nv_bfloat16>(d, w, a, write_o, st, tr) : forward_t<float>(d, w, a, write_o, st, tr);
 }
 
-int generic_backward(const Dims &d, const Workspace &w, const BwdArgs &a, cudaStream_t st) {
+int generic_backward(const Dims &d, const Workspace &w, const BwdArgs &a, cudaStream_t st, Tracer &tr) {
     // recompute gates, cumulative decays and the per-chunk states (no output store)
     FwdArgs f{a.q, a.k, a.v, a.log_decay, a.beta, a.lq, a.lk, a.h0, nullptr, nullptr, a.ws};
-    int n1 = generic_forward(d, w, f, false, st);
+    int n1 = generic_forward(d, w, f, false, st, tr);
     if (n1 < 0) return -1;
     int n2;
     if (d.variant == SLA_GDN) return -2;   // delta-rule gradients live in sla_generic_gdn.cu (not built yet)
-    n2 = d.io_bf16 ? backward_lin_t<__nv_bfloat16>(d, w, a, st) : backward_lin_t<float>(d, w, a, st);
+    n2 = d.io_bf16 ? backward_lin_t<__nv_bfloat16>(d, w, a, st, tr) : backward_lin_t<float>(d, w, a, st, tr);
     if (n2 < 0) return -1;
     float *ws = a.ws;
     long n_tok = (long)d.B * d.T;
@@ -883,11 +890,12 @@ int generic_backward(const Dims &d, const Workspace &w, const BwdArgs &a, cudaSt
         case 16: launch_gate_bwd<16>(Gq, Gk, dGq, dGk, a.dlq, a.dlk, n_tok, d.H, st); break;
         default: launch_gate_bwd<32>(Gq, Gk, dGq, dGk, a.dlq, a.dlk, n_tok, d.H, st); break;
     }
+    tr.mark("gate_bwd");
     if (cudaGetLastError() != cudaSuccess) return -1;
     return n1 + n2 + 1;
 }
 
-int decode_step(const Dims &d, const DecArgs &a, cudaStream_t st) {
+int decode_step(const Dims &d, const DecArgs &a, cudaStream_t st, Tracer &tr) {
     dim3 grid(a.Bdec * d.H);
     if (d.io_bf16)
         k_decode<__nv_bfloat16><<<grid, 256, 0, st>>>(d, a.Bdec, (const __nv_bfloat16 *)a.q,
@@ -898,6 +906,7 @@ int decode_step(const Dims &d, const DecArgs &a, cudaStream_t st) {
         k_decode<float><<<grid, 256, 0, st>>>(d, a.Bdec, (const float *)a.q, (const float *)a.k,
                                               (const float *)a.v, a.log_decay, a.beta, a.lq, a.lk, a.state,
                                               (float *)a.o);
+    tr.mark("decode");
     return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 

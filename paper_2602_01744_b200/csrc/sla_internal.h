@@ -4,6 +4,7 @@
 #include <cuda_bf16.h>
 #include <stdint.h>
 #include <stddef.h>
+#include <vector>
 
 #include "sla.h"
 
@@ -56,10 +57,35 @@ struct DecArgs {
     int Bdec;
 };
 
+// Optional per-kernel timing: one CUDA event before the first kernel of a call and one after every
+// kernel, all on the launch stream.  Off by default (mark() is then a no-op).
+struct Tracer {
+    bool on = false;
+    cudaStream_t st = nullptr;
+    std::vector<cudaEvent_t> pool;
+    size_t used = 0;
+    struct Rec { const char *name; size_t e0, e1; };
+    std::vector<Rec> recs;
+    size_t last = 0;
+    size_t record() {
+        if (used == pool.size()) {
+            cudaEvent_t e;
+            cudaEventCreate(&e);
+            pool.push_back(e);
+        }
+        cudaEventRecord(pool[used], st);
+        return used++;
+    }
+    void start(cudaStream_t s) { if (on) { st = s; last = record(); } }
+    void mark(const char *name) { if (on) { size_t e = record(); recs.push_back({name, last, e}); last = e; } }
+    void clear() { used = 0; recs.clear(); }
+    void destroy() { for (auto e : pool) cudaEventDestroy(e); pool.clear(); clear(); }
+};
+
 // Each returns the number of kernels launched (>0) or -1 after a CUDA launch error.
-int generic_forward(const Dims &d, const Workspace &w, const FwdArgs &a, bool write_o, cudaStream_t st);
-int generic_backward(const Dims &d, const Workspace &w, const BwdArgs &a, cudaStream_t st);
-int decode_step(const Dims &d, const DecArgs &a, cudaStream_t st);
+int generic_forward(const Dims &d, const Workspace &w, const FwdArgs &a, bool write_o, cudaStream_t st, Tracer &tr);
+int generic_backward(const Dims &d, const Workspace &w, const BwdArgs &a, cudaStream_t st, Tracer &tr);
+int decode_step(const Dims &d, const DecArgs &a, cudaStream_t st, Tracer &tr);
 // Opt the kernels into the shared memory they need (once per device).
 int generic_configure();
 
