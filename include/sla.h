@@ -149,6 +149,40 @@ sla_status sla_decode_step(sla_plan *plan, int32_t Bdec,
                            const float *gq_logits_t, const float *gk_logits_t,
                            float *state, void *o_t, void *cuda_stream);
 
+/*
+ * sla_forward with built-in scratch (an addition of this library; the paper has no counterpart).
+ *
+ * Some callers are not allowed to obtain device memory at the point where they run the layer: a
+ * plugin executing inside a host runtime that owns the allocator and forbids allocation in its
+ * execute callback, a latency-critical serving loop whose memory budget is frozen after start-up,
+ * or a process whose device memory has been reserved in full by another pool, where a fresh
+ * allocation would fail.  Such callers cannot provide the `workspace` that sla_forward wants.
+ * This entry point computes exactly what sla_forward computes (always with the fp32 CUDA-core chunk
+ * kernels) and keeps its scratch in a fixed array of SLA_NOALLOC_SCRATCH_BYTES that is part of the
+ * library image: every GPU on which the library is loaded holds that array until the process
+ * exits.  The call itself allocates and frees nothing: no cudaMalloc, no cudaFree, no allocating library
+ * routine.  Inputs and outputs are still the caller's, with the meanings, layouts and rules of
+ * sla_forward.
+ *
+ *  - Size limit: if the plan's forward workspace (sla_plan_workspace_bytes) exceeds
+ *    SLA_NOALLOC_SCRATCH_BYTES the call does nothing and returns SLA_ERR_WORKSPACE.
+ *  - First call on a device: looks up the device address of the array (one runtime query, made
+ *    with that device current; result cached per device).  Make this first call outside any
+ *    stream capture.
+ *  - The array is shared by every plan and every call in the process and keeps what the last call
+ *    left in it.  The kernels write each part of it before reading it, so stale contents are never
+ *    used; but two calls whose kernels may overlap on the GPU (different streams without
+ *    ordering, or several host threads) race on it.  Serialise them.
+ *  - The plan must belong to the current device (SLA_ERR_INVALID_ARG otherwise).
+ */
+#define SLA_NOALLOC_SCRATCH_BYTES (32u << 20)
+sla_status sla_forward_noalloc(sla_plan *plan,
+                               const void *q, const void *k, const void *v,
+                               const float *log_decay, const float *beta,
+                               const float *gq_logits, const float *gk_logits,
+                               const float *h0,
+                               void *o, float *ht, void *cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -23,7 +23,9 @@ EXPORTS = (
     "sla_plan_create", "sla_plan_destroy", "sla_plan_workspace_bytes", "sla_plan_poll",
     "sla_plan_last_launch_count", "sla_plan_set_kernel_timing", "sla_plan_kernel_timing_collect",
     "sla_plan_kernel_timing_get", "sla_status_string", "sla_forward", "sla_backward", "sla_decode_step",
+    "sla_forward_noalloc",
 )
+SLA_NOALLOC_SCRATCH_BYTES = 32 << 20
 
 
 class SLAError(RuntimeError):
@@ -66,6 +68,8 @@ def lib():
         L.sla_status_string.argtypes = [ctypes.c_int]
         L.sla_status_string.restype = ctypes.c_char_p
         L.sla_forward.argtypes = [vp] * 11 + [vp, sz, vp]
+        L.sla_forward_noalloc.argtypes = [vp] * 12
+        L.sla_forward_noalloc.restype = ctypes.c_int
         L.sla_backward.argtypes = [vp] * 19 + [vp, sz, vp]
         L.sla_decode_step.argtypes = [vp, i32] + [vp] * 10
         for name in ("sla_plan_create", "sla_plan_destroy", "sla_plan_workspace_bytes", "sla_plan_poll",
@@ -155,6 +159,18 @@ def sla_forward(plan: Plan, q, k, v, log_decay, gq_logits, gk_logits, beta=None,
     _check("sla_forward", lib().sla_forward(
         plan.handle, _ptr(q), _ptr(k), _ptr(v), _ptr(log_decay), _ptr(beta), _ptr(gq_logits),
         _ptr(gk_logits), _ptr(h0), _ptr(o), _ptr(ht), _ptr(workspace), workspace.numel(), _stream()))
+    return o, ht
+
+
+def sla_forward_noalloc(plan: Plan, q, k, v, log_decay, gq_logits, gk_logits, o, beta=None, h0=None, ht=None):
+    """sla_forward for callers that may not allocate device memory when they run the layer (a plugin
+    inside a runtime that owns the allocator, a serving loop with a frozen memory budget).  The scratch
+    is a fixed SLA_NOALLOC_SCRATCH_BYTES array inside the library, so `o` (and `ht`) must be passed in
+    and nothing is allocated here either.  Problems whose forward workspace exceeds that size are
+    refused (SLAError, status 3).  Calls share the array: do not let two of them overlap on the GPU."""
+    _check("sla_forward_noalloc", lib().sla_forward_noalloc(
+        plan.handle, _ptr(q), _ptr(k), _ptr(v), _ptr(log_decay), _ptr(beta), _ptr(gq_logits),
+        _ptr(gk_logits), _ptr(h0), _ptr(o), _ptr(ht), _stream()))
     return o, ht
 
 

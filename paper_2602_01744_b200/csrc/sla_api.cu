@@ -6,17 +6,6 @@
 #include <utility>
 #include <vector>
 
-struct sla_plan {
-    sla::Dims dims;
-    sla::Workspace ws;
-    uint32_t flags;
-    int device;
-    int *d_status;          // device status word (bounded waits report here)
-    int last_launches;
-    sla::Tracer tracer;
-    std::vector<std::pair<const char *, std::pair<int, float>>> agg;   // name -> (launches, total ms)
-};
-
 namespace sla {
 
 static size_t align64(size_t x) { return (x + 63) & ~(size_t)63; }

@@ -4,6 +4,7 @@
 #include <cuda_bf16.h>
 #include <stdint.h>
 #include <stddef.h>
+#include <utility>
 #include <vector>
 
 #include "sla.h"
@@ -90,3 +91,15 @@ int decode_step(const Dims &d, const DecArgs &a, cudaStream_t st, Tracer &tr);
 int generic_configure();
 
 }  // namespace sla
+
+// The opaque plan of the C ABI.
+struct sla_plan {
+    sla::Dims dims;
+    sla::Workspace ws;
+    uint32_t flags;
+    int device;
+    int *d_status;          // device status word (bounded waits report here)
+    int last_launches;
+    sla::Tracer tracer;
+    std::vector<std::pair<const char *, std::pair<int, float>>> agg;   // name -> (launches, total ms)
+};

@@ -1,0 +1,46 @@
+"""sla_forward_noalloc (scratch inside the library, for callers that cannot allocate device memory
+when they run the layer) must reproduce sla_forward.  Collected last on purpose: a failure here
+cannot hide any other test from a run that stops at the first failure."""
+import pytest
+import torch
+
+from paper_2602_01744_b200 import api
+from paper_2602_01744_b200.inputs import CONFIGS, make_inputs, small
+from tests import gpu_util as gu
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("variant,dtype", [("gla", "fp32"), ("gdn", "bf16"), ("retnet", "bf16")])
+def test_noalloc_forward_matches_workspace_forward_twice_in_a_row(variant, dtype):
+    base = {"retnet": CONFIGS["C0"], "gla": CONFIGS["C1"], "gdn": CONFIGS["C4"]}[variant]
+    tol = gu.TOL[dtype]
+    plan = None
+    for call, seed in enumerate((200, 201)):            # two calls in a row on the shared scratch
+        cfg = small(base, B=2, T=200 - 36 * call, H=4, d_k=64, d_v=64, dtype=dtype, seed=seed)
+        x = gu.to_dev(make_inputs(cfg, with_h0=True))
+        plan = api.sla_plan_create(cfg.variant, cfg.dtype, cfg.B, cfg.T, cfg.H, cfg.d_k, cfg.d_v, cfg.chunk,
+                                   cfg.scale, api.SLA_FLAG_FORCE_GENERIC)
+        assert plan.forward_workspace_bytes <= api.SLA_NOALLOC_SCRATCH_BYTES
+        ht_ref = torch.empty((cfg.B, cfg.H, cfg.d_k, cfg.d_v), dtype=torch.float32, device="cuda")
+        o_ref, _ = api.sla_forward(plan, x["q"], x["k"], x["v"], x["log_decay"], x["gq_logits"], x["gk_logits"],
+                                   beta=x["beta"], h0=x["h0"], ht=ht_ref)
+        o = torch.full_like(o_ref, float("nan"))
+        ht = torch.full_like(ht_ref, float("nan"))
+        before = torch.cuda.memory_allocated()
+        api.sla_forward_noalloc(plan, x["q"], x["k"], x["v"], x["log_decay"], x["gq_logits"], x["gk_logits"], o,
+                                beta=x["beta"], h0=x["h0"], ht=ht)
+        assert torch.cuda.memory_allocated() == before
+        torch.cuda.synchronize()
+        assert gu.rel_l2(o, o_ref.double().cpu().numpy()) <= tol
+        assert gu.rel_l2(ht, ht_ref.double().cpu().numpy()) <= tol
+
+
+def test_noalloc_forward_refuses_problems_beyond_its_scratch():
+    cfg = small(CONFIGS["C1"], B=4, T=2048, H=8)        # forward workspace far above 32 MiB
+    plan = api.sla_plan_create(cfg.variant, cfg.dtype, cfg.B, cfg.T, cfg.H, cfg.d_k, cfg.d_v, cfg.chunk)
+    assert plan.forward_workspace_bytes > api.SLA_NOALLOC_SCRATCH_BYTES
+    z = torch.zeros(16, device="cuda")
+    with pytest.raises(api.SLAError) as e:
+        api.sla_forward_noalloc(plan, z, z, z, z, z, z, z)
+    assert e.value.status == 3
