@@ -26,7 +26,12 @@ Workspace plan_workspace(const Dims &d) {
     }
     w.fwd_floats = off;
     w.dstates = take((size_t)d.B * d.H * d.NT * d.dk * d.dv);
-    if (d.variant == SLA_GDN) w.dU = take(bth * d.dv);
+    if (d.variant == SLA_GDN) {
+        w.dU = take(bth * d.dv);
+        w.dKbg = take(bth * d.dk);
+        w.dVb = take(bth * d.dv);
+        w.dbpart = take(bth);
+    }
     w.dGq = take(bth);
     w.dGk = take(bth);
     w.bwd_floats = off;
@@ -71,7 +76,7 @@ sla_status sla_plan_create(sla_plan **out, const sla_desc *desc) {
     if (cudaGetDevice(&dev) != cudaSuccess) return SLA_ERR_CUDA;
     if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return SLA_ERR_CUDA;
     if (prop.major != 10) return SLA_ERR_ARCH;
-    if (sla::generic_configure() != 0) return SLA_ERR_CUDA;
+    if (sla::generic_configure() != 0 || sla::gdn_configure() != 0) return SLA_ERR_CUDA;
 
     sla_plan *p = new (std::nothrow) sla_plan();
     if (!p) return SLA_ERR_CUDA;

@@ -27,6 +27,7 @@ struct Workspace {
     size_t fwd_floats;
     size_t dstates;         // [B,H,NT,dk,dv]: gradient w.r.t. the state after each chunk
     size_t dU;              // GDN: [B,T,H,dv]
+    size_t dKbg, dVb, dbpart;  // GDN: [B,T,H,dk], [B,T,H,dv], [B,T,H]
     size_t dGq, dGk;        // [B,T,H]
     size_t bwd_floats;
 };
@@ -89,6 +90,9 @@ int generic_backward(const Dims &d, const Workspace &w, const BwdArgs &a, cudaSt
 int decode_step(const Dims &d, const DecArgs &a, cudaStream_t st, Tracer &tr);
 // Opt the kernels into the shared memory they need (once per device).
 int generic_configure();
+int gdn_configure();
+// GDN per-tile gradient kernels (after the recompute pass and the state-gradient scan).
+int gdn_backward_tiles(const Dims &d, const Workspace &w, const BwdArgs &a, cudaStream_t st, Tracer &tr);
 
 }  // namespace sla
 

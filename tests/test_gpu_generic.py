@@ -32,26 +32,27 @@ def test_forward_shapes(variant, chunk, dk, dv, H):
     gu.check_forward(cfg, flags=GEN)
 
 
-@pytest.mark.parametrize("variant", ["retnet", "gla"])
+@pytest.mark.parametrize("variant", ["retnet", "gla", "gdn"])
 @pytest.mark.parametrize("dtype", ["fp32", "bf16"])
 def test_backward_small_ragged_tail_with_state_gradients(variant, dtype):
-    base = {"retnet": CONFIGS["C0"], "gla": CONFIGS["C2"]}[variant]
+    base = {"retnet": CONFIGS["C0"], "gla": CONFIGS["C2"], "gdn": CONFIGS["C4"]}[variant]
     cfg = small(base, B=2, T=200, H=3, dtype=dtype, seed=102, backward=True)
     gu.check_backward(cfg, with_h0=True, flags=GEN)
 
 
-@pytest.mark.parametrize("variant", ["retnet", "gla"])
+@pytest.mark.parametrize("variant", ["retnet", "gla", "gdn"])
 def test_backward_shapes(variant):
-    base = {"retnet": CONFIGS["C0"], "gla": CONFIGS["C2"]}[variant]
+    base = {"retnet": CONFIGS["C0"], "gla": CONFIGS["C2"], "gdn": CONFIGS["C4"]}[variant]
     cfg = small(base, B=1, T=130, H=4, d_k=64, d_v=32, chunk=32, dtype="fp32", seed=103, scale=0.7)
     gu.check_backward(cfg, flags=GEN)
 
 
 def test_single_token_and_single_chunk():
     for T in (1, 64):
-        cfg = small(CONFIGS["C1"], B=1, T=T, H=2, dtype="fp32", seed=104)
-        gu.check_forward(cfg, flags=GEN)
-        gu.check_backward(small(cfg, backward=True), flags=GEN)
+        for base in (CONFIGS["C1"], CONFIGS["C4"]):
+            cfg = small(base, B=1, T=T, H=2, dtype="fp32", seed=104)
+            gu.check_forward(cfg, flags=GEN)
+            gu.check_backward(small(cfg, backward=True), flags=GEN)
 
 
 @pytest.mark.parametrize("variant", ["retnet", "gla", "gdn"])
