@@ -111,9 +111,13 @@ class Plan:
         self.io_torch = torch.bfloat16 if self.desc.io_dtype == SLA_BF16 else torch.float32
 
     def close(self):
-        if getattr(self, "handle", None) and self.handle.value:
-            lib().sla_plan_destroy(self.handle)
-            self.handle = ctypes.c_void_p()
+        h = getattr(self, "handle", None)
+        if h is not None and h.value and _lib is not None:     # (at interpreter shutdown the module may be gone)
+            try:
+                _lib.sla_plan_destroy(h)
+            except Exception:
+                pass
+            self.handle.value = None
 
     __del__ = close
 

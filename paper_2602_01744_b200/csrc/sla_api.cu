@@ -44,6 +44,12 @@ static bool aligned16(const void *p) { return ((uintptr_t)p & 15u) == 0; }
 
 extern "C" {
 
+// Profiling aid (not declared in sla.h): device buffer of >= 16 uint64 that block 0 of the tensor-core
+// kernels fills with %globaltimer stamps at the phase boundaries of one chunk; NULL switches it off.
+void sla_debug_set_phase_timestamps(void *device_buffer) {
+    sla::gla_tc_set_phase_ts((unsigned long long *)device_buffer);
+}
+
 const char *sla_status_string(sla_status s) {
     switch (s) {
         case SLA_OK: return "ok";
@@ -76,7 +82,7 @@ sla_status sla_plan_create(sla_plan **out, const sla_desc *desc) {
     if (cudaGetDevice(&dev) != cudaSuccess) return SLA_ERR_CUDA;
     if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return SLA_ERR_CUDA;
     if (prop.major != 10) return SLA_ERR_ARCH;
-    if (sla::generic_configure() != 0 || sla::gdn_configure() != 0) return SLA_ERR_CUDA;
+    if (sla::generic_configure() != 0 || sla::gdn_configure() != 0 || sla::gla_tc_configure() != 0) return SLA_ERR_CUDA;
 
     sla_plan *p = new (std::nothrow) sla_plan();
     if (!p) return SLA_ERR_CUDA;
@@ -180,7 +186,9 @@ sla_status sla_forward(sla_plan *plan, const void *q, const void *k, const void 
     if (!workspace || workspace_bytes < plan->ws.fwd_floats * sizeof(float)) return SLA_ERR_WORKSPACE;
     sla::FwdArgs a{q, k, v, log_decay, beta, gq_logits, gk_logits, h0, o, ht, (float *)workspace};
     plan->tracer.start((cudaStream_t)cuda_stream);
-    int n = sla::generic_forward(d, plan->ws, a, true, (cudaStream_t)cuda_stream, plan->tracer);
+    const bool tc = sla::gla_tc_supported(d) && !(plan->flags & SLA_FLAG_FORCE_GENERIC);
+    int n = tc ? sla::gla_tc_forward(d, a, plan->d_status, (cudaStream_t)cuda_stream, plan->tracer)
+               : sla::generic_forward(d, plan->ws, a, true, (cudaStream_t)cuda_stream, plan->tracer);
     if (n < 0) return SLA_ERR_CUDA;
     plan->last_launches = n;
     return SLA_OK;

@@ -91,6 +91,13 @@ int decode_step(const Dims &d, const DecArgs &a, cudaStream_t st, Tracer &tr);
 // Opt the kernels into the shared memory they need (once per device).
 int generic_configure();
 int gdn_configure();
+
+// ---- tensor-core (tcgen05 / TMEM / TMA) Softmax-GLA kernels: sla_gla_tc.cu ----
+bool gla_tc_supported(const Dims &d);
+int gla_tc_configure();
+void gla_tc_set_phase_ts(unsigned long long *device_buffer);
+int gla_tc_forward(const Dims &d, const FwdArgs &a, int *status, cudaStream_t st, Tracer &tr);
+
 // GDN per-tile gradient kernels (after the recompute pass and the state-gradient scan).
 int gdn_backward_tiles(const Dims &d, const Workspace &w, const BwdArgs &a, cudaStream_t st, Tracer &tr);
 
