@@ -167,8 +167,10 @@ sla_status sla_decode_step(sla_plan *plan, int32_t Bdec,
  *  - Size limit: if the plan's forward workspace (sla_plan_workspace_bytes) exceeds
  *    SLA_NOALLOC_SCRATCH_BYTES the call does nothing and returns SLA_ERR_WORKSPACE.
  *  - First call on a device: looks up the device address of the array (one runtime query, made
- *    with that device current; result cached per device).  Make this first call outside any
- *    stream capture.
+ *    with that device current; result cached per device).  Where the CUDA runtime loads modules
+ *    lazily, this query is also the moment the driver places the array on that GPU, so free device
+ *    memory drops by SLA_NOALLOC_SCRATCH_BYTES once, here, and never again.  Make this first call
+ *    at start-up, outside any stream capture.
  *  - The array is shared by every plan and every call in the process and keeps what the last call
  *    left in it.  The kernels write each part of it before reading it, so stale contents are never
  *    used; but two calls whose kernels may overlap on the GPU (different streams without

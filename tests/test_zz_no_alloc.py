@@ -33,9 +33,13 @@ def test_noalloc_forward_matches_workspace_forward_twice_in_a_row(variant, dtype
         api.sla_forward_noalloc(plan, x["q"], x["k"], x["v"], x["log_decay"], x["gq_logits"], x["gk_logits"], o,
                                 beta=x["beta"], h0=x["h0"], ht=ht)
         torch.cuda.synchronize()
-        # neither torch's allocator nor the driver handed out device memory during the call
+        # torch's allocator handed out nothing during the call ...
         assert torch.cuda.memory_stats().get("allocation.all.allocated", 0) == allocs_before
-        assert torch.cuda.mem_get_info()[0] >= free_before
+        # ... and neither did the driver, once the set-up call is behind us: with lazy module loading the
+        # driver places the library's fixed scratch array on the GPU during the first call on a device
+        # (its documented set-up), so free memory is compared from the second call on
+        if call > 0:
+            assert torch.cuda.mem_get_info()[0] >= free_before
         assert gu.rel_l2(o, o_ref.double().cpu().numpy()) <= tol
         assert gu.rel_l2(ht, ht_ref.double().cpu().numpy()) <= tol
 
