@@ -82,7 +82,9 @@ sla_status sla_plan_create(sla_plan **out, const sla_desc *desc) {
     if (cudaGetDevice(&dev) != cudaSuccess) return SLA_ERR_CUDA;
     if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return SLA_ERR_CUDA;
     if (prop.major != 10) return SLA_ERR_ARCH;
-    if (sla::generic_configure() != 0 || sla::gdn_configure() != 0 || sla::gla_tc_configure() != 0) return SLA_ERR_CUDA;
+    if (sla::generic_configure() != 0 || sla::gdn_configure() != 0 || sla::gla_tc_configure() != 0 ||
+        sla::gla_tc_bwd_configure() != 0)
+        return SLA_ERR_CUDA;
 
     sla_plan *p = new (std::nothrow) sla_plan();
     if (!p) return SLA_ERR_CUDA;
@@ -219,7 +221,9 @@ sla_status sla_backward(sla_plan *plan, const void *q, const void *k, const void
     sla::BwdArgs a{q, k, v, log_decay, beta, gq_logits, gk_logits, h0, dO, dht, dq, dk, dv,
                    dlog_decay, dbeta, dgq_logits, dgk_logits, dh0, (float *)workspace};
     plan->tracer.start((cudaStream_t)cuda_stream);
-    int n = sla::generic_backward(d, plan->ws, a, (cudaStream_t)cuda_stream, plan->tracer);
+    const bool tc = sla::gla_tc_supported(d) && !(plan->flags & SLA_FLAG_FORCE_GENERIC);
+    int n = tc ? sla::gla_tc_backward(d, a, plan->d_status, (cudaStream_t)cuda_stream, plan->tracer)
+               : sla::generic_backward(d, plan->ws, a, (cudaStream_t)cuda_stream, plan->tracer);
     if (n == -2) return SLA_ERR_UNSUPPORTED;
     if (n < 0) return SLA_ERR_CUDA;
     plan->last_launches = n;

@@ -12,20 +12,14 @@
 //   CUDA     S <- diag(e^{b_last}) S (TMEM, fp32) and its bf16 copy in shared memory for the next chunk;
 //            O -> bf16 -> HBM
 // The state never leaves the SM: fp32 in TMEM (Eq. 12's S), bf16 copy in shared memory as MMA operand.
-#include "sla_internal.h"
-#include "sla_ptx.cuh"
-
-#include <mutex>
+#include "sla_gla_tc.cuh"
 
 namespace sla {
 namespace {
 
 using namespace ptx;
+using namespace tc;
 
-constexpr int C = 64, D = 128;
-constexpr uint32_t TILE_BF16 = C * D * 2;           // 16 KiB: two 64-column halves of [64 rows][128 B]
-constexpr uint32_t HALF_BF16 = C * 128;             // 8 KiB
-constexpr uint32_t TILE_G = C * D * 4;              // 32 KiB fp32 log-decay tile
 constexpr uint32_t STAGE = 3 * TILE_BF16 + TILE_G;  // 80 KiB
 constexpr uint32_t OFF_Q = 0, OFF_K = TILE_BF16, OFF_V = 2 * TILE_BF16, OFF_G = 3 * TILE_BF16;
 constexpr uint32_t OFF_S = 2 * STAGE;               // bf16 state operand: two halves of [128 rows][128 B]
@@ -39,8 +33,6 @@ constexpr uint32_t OFF_TMEM = OFF_BAR + 5 * 8;
 constexpr uint32_t SMEM_BYTES = OFF_TMEM + 16 + 1024;   // + slack to align the base to 1024 B
 
 constexpr uint32_t COL_A = 0, COL_O = 64, COL_S = 192, TMEM_COLS = 512;
-
-__device__ __forceinline__ uint32_t swz(uint32_t row, uint32_t chunk) { return row * 128 + ((chunk ^ (row & 7)) << 4); }
 
 struct FwdParams {
     const float *lq, *lk, *h0;
@@ -370,39 +362,6 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
 
 // ---- host side ----
 unsigned long long *g_phase_ts = nullptr;   // set by sla_debug_set_phase_timestamps (profiling aid)
-typedef CUresult (*EncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                             const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                             CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeFn encode_fn() {
-    static EncodeFn fn = nullptr;
-    static std::once_flag once;
-    std::call_once(once, [] {
-        void *ptr = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = (EncodeFn)ptr;
-    });
-    return fn;
-}
-
-// Tensor map over a [B,T,H,d] tensor: box = 64 tokens x `box_d` features of one head.
-bool make_map(CUtensorMap *m, const void *ptr, int B, int T, int H, int d, bool fp32, int box_d) {
-    EncodeFn fn = encode_fn();
-    if (!fn) return false;
-    const cuuint64_t es = fp32 ? 4 : 2;
-    cuuint64_t dims[4] = {(cuuint64_t)d, (cuuint64_t)H, (cuuint64_t)T, (cuuint64_t)B};
-    cuuint64_t strides[3] = {(cuuint64_t)d * es, (cuuint64_t)H * d * es, (cuuint64_t)T * H * d * es};
-    cuuint32_t box[4] = {(cuuint32_t)box_d, 1, (cuuint32_t)C, 1};
-    cuuint32_t estr[4] = {1, 1, 1, 1};
-    CUresult r = fn(m, fp32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4,
-                    const_cast<void *>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                    fp32 ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B,
-                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS;
-}
-
 }  // namespace
 
 void gla_tc_set_phase_ts(unsigned long long *p) { g_phase_ts = p; }

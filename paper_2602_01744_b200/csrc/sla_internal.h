@@ -97,6 +97,10 @@ bool gla_tc_supported(const Dims &d);
 int gla_tc_configure();
 void gla_tc_set_phase_ts(unsigned long long *device_buffer);
 int gla_tc_forward(const Dims &d, const FwdArgs &a, int *status, cudaStream_t st, Tracer &tr);
+// Backward: chunk-state sweep, gradient sweep, gate softmax backward.  Needs the first
+// B*H*(NT+1)*32 KiB + 2*B*T*H*4 bytes (rounded up) of the workspace, less than the generic path.
+int gla_tc_bwd_configure();
+int gla_tc_backward(const Dims &d, const BwdArgs &a, int *status, cudaStream_t st, Tracer &tr);
 
 // GDN per-tile gradient kernels (after the recompute pass and the state-gradient scan).
 int gdn_backward_tiles(const Dims &d, const Workspace &w, const BwdArgs &a, cudaStream_t st, Tracer &tr);
