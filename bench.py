@@ -147,11 +147,17 @@ def main():
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--generic", action="store_true", help="force the fp32 CUDA-core kernels")
+    ap.add_argument("--batch", type=int, default=0,
+                    help="profiling aid: shrink the batch of the workload (0 = the full configuration; "
+                         "a reduced batch is not the benchmark and is labelled in config)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "b200" else args.warmup
 
     from paper_2602_01744_b200.inputs import CONFIGS, make_inputs
     cfg = CONFIGS[WORKLOAD]
+    if args.batch > 0:
+        from paper_2602_01744_b200.inputs import small
+        cfg = small(cfg, B=args.batch)
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
@@ -292,7 +298,8 @@ def main():
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": WORKLOAD, "variant": cfg.variant, "B": cfg.B, "T": cfg.T, "H": cfg.H,
+            "config": {"workload": WORKLOAD if args.batch <= 0 else f"{WORKLOAD} reduced to batch {cfg.B} (profiling only)",
+                       "variant": cfg.variant, "B": cfg.B, "T": cfg.T, "H": cfg.H,
                        "d_k": cfg.d_k, "d_v": cfg.d_v, "chunk": cfg.chunk, "pass": "forward+backward",
                        "io": "bf16 q,k,v,o and gradients; fp32 decay, logits, state; fp32 accumulation",
                        "l2": "inputs (0.77 GB per step) exceed the 126 MB L2; no flush needed",

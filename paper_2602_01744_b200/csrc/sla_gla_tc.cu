@@ -20,19 +20,29 @@ namespace {
 using namespace ptx;
 using namespace tc;
 
-constexpr uint32_t STAGE = 3 * TILE_BF16 + TILE_G;  // 80 KiB
-constexpr uint32_t OFF_Q = 0, OFF_K = TILE_BF16, OFF_V = 2 * TILE_BF16, OFF_G = 3 * TILE_BF16;
-constexpr uint32_t OFF_S = 2 * STAGE;               // bf16 state operand: two halves of [128 rows][128 B]
-constexpr uint32_t OFF_A = OFF_S + 2 * D * 128;     // masked A, [64 rows][128 B]
-constexpr uint32_t OFF_TOT = OFF_A + C * 128;       // [16][128] fp32 partial column sums
-constexpr uint32_t OFF_EB = OFF_TOT + 16 * D * 4;   // [128] exp(b_last)
-constexpr uint32_t OFF_GQ = OFF_EB + D * 4;         // [64] scale*Gq
-constexpr uint32_t OFF_GK = OFF_GQ + C * 4;         // [64] Gk
-constexpr uint32_t OFF_BAR = OFF_GK + C * 4;        // mbarriers: full[2], a, z, o
-constexpr uint32_t OFF_TMEM = OFF_BAR + 5 * 8;
-constexpr uint32_t SMEM_BYTES = OFF_TMEM + 16 + 1024;   // + slack to align the base to 1024 B
+// shared memory: one log-decay buffer (dead right after the prologue), three q/k operand buffers (chunk n in the
+// tensor core, n+1 in the prologue, n+2 in flight), two v buffers, the bf16 state operand, the masked A tile
+constexpr uint32_t OFF_G = 0;                                   // 32 KiB fp32 log-decay tile
+constexpr uint32_t QK_BYTES = 2 * TILE_BF16;                    // q then k
+constexpr uint32_t OFF_QK = OFF_G + TILE_G;                     // [3]
+constexpr uint32_t OFF_V = OFF_QK + 3 * QK_BYTES;               // [2]
+constexpr uint32_t OFF_S = OFF_V + 2 * TILE_BF16;               // bf16 state operand: two halves of [128 rows][128 B]
+constexpr uint32_t OFF_A = OFF_S + STATE_BF16;                  // masked A, [64 rows][128 B]
+constexpr uint32_t OFF_OST = OFF_A + HALF_BF16;                 // bf16 output tile staged for the TMA store
+constexpr uint32_t OFF_TOT = OFF_OST + TILE_BF16;               // prologue scratch
+constexpr uint32_t OFF_EB = OFF_TOT + TOT_BYTES;                // [2][128] 2^{b_last}
+constexpr uint32_t OFF_GATE = OFF_EB + 2 * D * 4;               // [4][2][64]: scale*Gq, Gk of four chunks
+constexpr uint32_t OFF_BAR = OFF_GATE + 4 * 2 * C * 4;          // mbarriers, see Bar
+constexpr uint32_t OFF_TMEM = OFF_BAR + 32 * 8;                 // TMEM base address, then the abort flag
+constexpr uint32_t SMEM_BYTES = OFF_TMEM + 16 + 1024;           // + slack to align the base to 1024 B
+static_assert(SMEM_BYTES <= 232448, "shared memory budget");
 
-constexpr uint32_t COL_A = 0, COL_O = 64, COL_S = 192, TMEM_COLS = 512;
+constexpr uint32_t COL_A = 0, COL_O = 64, COL_S = 320, TMEM_COLS = 512;   // O: two buffers of 128 columns
+constexpr int NTHREADS = NCOMPUTE + 32 + NGATE + 32;   // warps 0..7 compute, 8 MMA issue, 9..12 gates, 13 TMA
+
+// mbarrier slots (8 bytes each)
+enum Bar { FULL_G = 0, FULL_QK = 1, FULL_V = 4, OPR = 6, GREADY = 9, GFREE = 13, SREADY = 17, OFREE, AREADY, BAR_A, BAR_Z,
+           BAR_O /* [2], one per O accumulator */, OSTAGED = BAR_O + 2, OSFREE, DRAIN, QKFREE /* [3] */, NBAR = QKFREE + 3 };
 
 struct FwdParams {
     const float *lq, *lk, *h0;
@@ -45,206 +55,264 @@ struct FwdParams {
 };
 #define SLA_TS(k) do { if (p.phase_ts && bh == 0 && tid == 0 && n == 8) p.phase_ts[k] = globaltimer_ns(); } while (0)
 
-__global__ void __launch_bounds__(256, 1)
+// One CTA per (batch, head) sequence, four roles:
+//   warp 8 (one lane)  every tcgen05.mma
+//   warp 13 (one lane) TMA: loads (log-decay one chunk ahead, q/k three, v two) and the output store
+//   warps 9..12        head-softmax gates (Eq. 4) up to four chunks ahead, one thread per (token, gate)
+//   warps 0..7         prologue (cumulative decay, qh, kh), causal mask of A, state rescale, output staging
+// While the tensor core works on chunk n the compute warps already run the prologue of chunk n+1, so per chunk
+// the critical path is prologue -> mask -> rescale -> store.
+__global__ void __launch_bounds__(NTHREADS, 1)
 k_gla_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-             const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_g, FwdParams p) {
+             const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_g,
+             const __grid_constant__ CUtensorMap tm_o, FwdParams p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t *sm = smem_raw + (base - raw);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int bh = blockIdx.x, b = bh / p.H, h = bh % p.H;
-    const uint32_t bar_full0 = base + OFF_BAR, bar_a = bar_full0 + 16, bar_z = bar_full0 + 24, bar_o = bar_full0 + 32;
+    auto bar = [&](int i) { return base + OFF_BAR + 8u * i; };
     float *tot = reinterpret_cast<float *>(sm + OFF_TOT);
     float *eblast = reinterpret_cast<float *>(sm + OFF_EB);
-    float *gq_s = reinterpret_cast<float *>(sm + OFF_GQ);
-    float *gk_s = reinterpret_cast<float *>(sm + OFF_GK);
+    float *gate_s = reinterpret_cast<float *>(sm + OFF_GATE);
+    // Every wait is bounded.  The first thread whose wait expires raises the CTA's abort flag; from then on nobody
+    // waits any more, the control lane stops issuing and drains what is in flight, and the kernel reports the failure.
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(sm + OFF_TMEM + 8);
     bool failed = false;
+    auto wait = [&](int i, uint32_t parity) {
+        if (!failed && !mbar_wait_bounded(bar(i), parity, abort_flag)) { failed = true; *abort_flag = 1; }
+    };
+    auto wait_relaxed = [&](int i, uint32_t parity) {     // for the warps that run ahead: poll with a back-off
+        if (!failed && !mbar_wait_bounded<128>(bar(i), parity, abort_flag)) { failed = true; *abort_flag = 1; }
+    };
 
     if (tid == 0) {
-        for (int i = 0; i < 5; ++i) mbar_init(bar_full0 + 8 * i, 1);
+        *abort_flag = 0;
+        for (int i = 0; i < NBAR; ++i) {
+            const bool all = (i >= OPR && i < GREADY) || (i >= GFREE && i <= AREADY) || i == OSTAGED;
+            mbar_init(bar(i), all ? NCOMPUTE : (i >= GREADY && i < GFREE) ? NGATE / 32 : 1);
+        }
         fence_mbar_init();
         tma_prefetch_desc(&tm_q);
         tma_prefetch_desc(&tm_k);
         tma_prefetch_desc(&tm_v);
         tma_prefetch_desc(&tm_g);
+        tma_prefetch_desc(&tm_o);
     }
     if (warp == 0) tmem_alloc(base + OFF_TMEM, TMEM_COLS);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *reinterpret_cast<volatile uint32_t *>(sm + OFF_TMEM);
-    const uint32_t lane_base = (uint32_t)(32 * (warp & 3)) << 16;   // this warp's TMEM lane quarter
-    const int colhalf = warp >> 2;                                   // which 64 state / output columns
+    const size_t tokb = (size_t)b * p.T;
 
-    auto issue_tma = [&](int n, int s) {
-        const uint32_t bar = bar_full0 + 8 * s, st = base + s * STAGE;
-        mbar_expect_tx(bar, STAGE);
-        const int t0 = n * C;
-        tma_load_4d(st + OFF_Q, &tm_q, 0, h, t0, b, bar);
-        tma_load_4d(st + OFF_Q + HALF_BF16, &tm_q, 64, h, t0, b, bar);
-        tma_load_4d(st + OFF_K, &tm_k, 0, h, t0, b, bar);
-        tma_load_4d(st + OFF_K + HALF_BF16, &tm_k, 64, h, t0, b, bar);
-        tma_load_4d(st + OFF_V, &tm_v, 0, h, t0, b, bar);
-        tma_load_4d(st + OFF_V + HALF_BF16, &tm_v, 64, h, t0, b, bar);
-        tma_load_4d(st + OFF_G, &tm_g, 0, h, t0, b, bar);
-    };
-    if (tid == 0) issue_tma(0, 0);
-
-    {   // initial state: fp32 into TMEM, bf16 copy into shared memory (row = key dimension)
-        const int row = 32 * (warp & 3) + lane;
-        const float *src = p.h0 ? p.h0 + ((size_t)bh * D + row) * D + 64 * colhalf : nullptr;
+    if (warp == 8) {
+        // ---------------- MMA issue (one lane) ----------------
+        if (lane == 0) {
+            constexpr uint32_t ID_A = idesc_bf16(64, 64, 0, 0);      // qh (K-major) x kh (K-major)
+            constexpr uint32_t ID_O = idesc_bf16(64, 128, 0, 1);     // qh x S, A x V (B operand MN-major)
+            constexpr uint32_t ID_Z = idesc_bf16(128, 128, 1, 1);    // kh^T (MN-major) x V (MN-major)
+            for (int n = 0; n < p.NT; ++n) {
+                const uint32_t par = n & 1;
+                const uint32_t sQ = base + OFF_QK + (n % 3) * QK_BYTES, sK = sQ + TILE_BF16;
+                const uint32_t sV = base + OFF_V + (n & 1) * TILE_BF16;
+                const uint32_t tO = tmem + COL_O + (n & 1) * D;
+                wait(OPR + n % 3, (n / 3) & 1);        // qh, kh of chunk n are in place
+                wait(SREADY, par);                     // S_n: fp32 in TMEM, bf16 in shared memory
+                if (n > 1) wait(OFREE, n & 1);         // O of chunk n-2 (same TMEM buffer) has been read out
+                wait(FULL_V + (n & 1), (n >> 1) & 1);
+                if (failed) break;
+                tc_fence_after();
 #pragma unroll
-        for (int part = 0; part < 2; ++part) {
-            float v[32];
+                for (int kk = 0; kk < 8; ++kk)         // A = qh kh^T
+                    tc_mma_bf16(tmem + COL_A, desc_kmajor(sQ, kk, HALF_BF16), desc_kmajor(sK, kk, HALF_BF16), ID_A, kk > 0);
+                tc_commit(bar(BAR_A));
 #pragma unroll
-            for (int j = 0; j < 32; ++j) v[j] = src ? src[32 * part + j] : 0.f;
-            tmem_st32(tmem + lane_base + COL_S + 64 * colhalf + 32 * part, v);
+                for (int kk = 0; kk < 8; ++kk)         // O = qh S_n
+                    tc_mma_bf16(tO, desc_kmajor(sQ, kk, HALF_BF16), desc_mnmajor(base + OFF_S, kk, STATE_HALF), ID_O, kk > 0);
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint4 w;
-                w.x = pack_bf16(v[8 * c + 0], v[8 * c + 1]);
-                w.y = pack_bf16(v[8 * c + 2], v[8 * c + 3]);
-                w.z = pack_bf16(v[8 * c + 4], v[8 * c + 5]);
-                w.w = pack_bf16(v[8 * c + 6], v[8 * c + 7]);
-                *reinterpret_cast<uint4 *>(sm + OFF_S + colhalf * (D * 128) + swz(row, 4 * part + c)) = w;
+                for (int kk = 0; kk < 4; ++kk)         // S += kh^T V
+                    tc_mma_bf16(tmem + COL_S, desc_mnmajor(sK, kk, HALF_BF16), desc_mnmajor(sV, kk, HALF_BF16), ID_Z, 1);
+                tc_commit(bar(BAR_Z));
+                tc_commit(bar(QKFREE + n % 3));        // (same event, own barrier: the TMA lane may look at it much later)
+                wait(AREADY, par);                     // masked A is in shared memory
+                if (failed) break;
+                tc_fence_after();
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)         // O += A V
+                    tc_mma_bf16(tO, desc_kmajor(base + OFF_A, kk, 0), desc_mnmajor(sV, kk, HALF_BF16), ID_O, 1);
+                tc_commit(bar(BAR_O + (n & 1)));
             }
+            // let the tensor core finish before TMEM goes away (after an abort some of its work may still be queued)
+            tc_commit(bar(DRAIN));
+            mbar_wait_bounded(bar(DRAIN), 0, nullptr, 20000000ull);
         }
-        tmem_wait_st();
-    }
-    fence_proxy_async();
-    tc_fence_before();
-    __syncthreads();
-
-    constexpr uint32_t ID_A = idesc_bf16(64, 64, 0, 0);      // qh (K-major) x kh (K-major)
-    constexpr uint32_t ID_O1 = idesc_bf16(64, 128, 0, 1);    // qh (K-major) x S (MN-major)
-    constexpr uint32_t ID_O2 = idesc_bf16(64, 128, 0, 1);    // A (K-major) x V (MN-major)
-    constexpr uint32_t ID_Z = idesc_bf16(128, 128, 1, 1);    // kh^T (MN-major) x V (MN-major)
-    uint32_t ph_full[2] = {0, 0}, ph_a = 0, ph_z = 0, ph_o = 0;
-    const int rg = tid >> 4, cj = tid & 15;                   // prologue: rows 4rg..4rg+3, columns 8cj..8cj+7
-
-    for (int n = 0; n < p.NT; ++n) {
-        const int s = n & 1;
-        const uint32_t st = base + s * STAGE;
-        uint8_t *stp = sm + s * STAGE;
-        const int t0 = n * C, cn = min(C, p.T - t0);
-        if (tid == 0 && n + 1 < p.NT) issue_tma(n + 1, s ^ 1);
-        SLA_TS(0);
-
-        if (tid < C) {   // a1: head-softmax gates of this chunk's tokens (Eq. 4)
-            float gq = 0.f, gk = 0.f;
-            if (tid < cn) {
-                const float *l1 = p.lq + ((size_t)b * p.T + t0 + tid) * p.H;
-                const float *l2 = p.lk + ((size_t)b * p.T + t0 + tid) * p.H;
-                float m1 = -INFINITY, m2 = -INFINITY;
-                for (int j = 0; j < p.H; ++j) { m1 = fmaxf(m1, l1[j]); m2 = fmaxf(m2, l2[j]); }
-                float s1 = 0.f, s2 = 0.f;
-                for (int j = 0; j < p.H; ++j) { s1 += expf(l1[j] - m1); s2 += expf(l2[j] - m2); }
-                gq = p.scale * expf(l1[h] - m1) / s1;
-                gk = expf(l2[h] - m2) / s2;
-            }
-            gq_s[tid] = gq;
-            gk_s[tid] = gk;
-        }
-        if (!failed && !mbar_wait_bounded(bar_full0 + 8 * s, ph_full[s])) failed = true;
-        ph_full[s] ^= 1;
-        SLA_TS(1);
-
-        // a2: chunk-local cumulative log-decay, two-level: per-4-row partial sums, then a running sum
-        const float *gs = reinterpret_cast<const float *>(stp + OFF_G);
-        {
-            float acc[8];
-#pragma unroll
-            for (int e = 0; e < 8; ++e) acc[e] = 0.f;
-#pragma unroll
-            for (int rr = 0; rr < 4; ++rr) {
-                const float4 g0 = *reinterpret_cast<const float4 *>(gs + (4 * rg + rr) * D + 8 * cj);
-                const float4 g1 = *reinterpret_cast<const float4 *>(gs + (4 * rg + rr) * D + 8 * cj + 4);
-                acc[0] += g0.x; acc[1] += g0.y; acc[2] += g0.z; acc[3] += g0.w;
-                acc[4] += g1.x; acc[5] += g1.y; acc[6] += g1.z; acc[7] += g1.w;
-            }
-            *reinterpret_cast<float4 *>(tot + rg * D + 8 * cj) = make_float4(acc[0], acc[1], acc[2], acc[3]);
-            *reinterpret_cast<float4 *>(tot + rg * D + 8 * cj + 4) = make_float4(acc[4], acc[5], acc[6], acc[7]);
-        }
-        __syncthreads();
-        {
-            float bsum[8];
-#pragma unroll
-            for (int e = 0; e < 8; ++e) bsum[e] = 0.f;
-            for (int g = 0; g < rg; ++g) {
-                const float4 a0 = *reinterpret_cast<const float4 *>(tot + g * D + 8 * cj);
-                const float4 a1 = *reinterpret_cast<const float4 *>(tot + g * D + 8 * cj + 4);
-                bsum[0] += a0.x; bsum[1] += a0.y; bsum[2] += a0.z; bsum[3] += a0.w;
-                bsum[4] += a1.x; bsum[5] += a1.y; bsum[6] += a1.z; bsum[7] += a1.w;
-            }
-            const uint32_t half = cj >> 3, chunk = cj & 7;
-#pragma unroll
-            for (int rr = 0; rr < 4; ++rr) {
-                const int r = 4 * rg + rr;
-                const float4 g0 = *reinterpret_cast<const float4 *>(gs + r * D + 8 * cj);
-                const float4 g1 = *reinterpret_cast<const float4 *>(gs + r * D + 8 * cj + 4);
-                bsum[0] += g0.x; bsum[1] += g0.y; bsum[2] += g0.z; bsum[3] += g0.w;
-                bsum[4] += g1.x; bsum[5] += g1.y; bsum[6] += g1.z; bsum[7] += g1.w;
-                const float gq = gq_s[r], gk = gk_s[r];
-                uint4 *qp = reinterpret_cast<uint4 *>(stp + OFF_Q + half * HALF_BF16 + swz(r, chunk));
-                uint4 *kp = reinterpret_cast<uint4 *>(stp + OFF_K + half * HALF_BF16 + swz(r, chunk));
-                uint4 qv = *qp, kv = *kp;
-                uint32_t *qw = reinterpret_cast<uint32_t *>(&qv), *kw = reinterpret_cast<uint32_t *>(&kv);
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const float e0 = __expf(bsum[2 * e]), e1 = __expf(bsum[2 * e + 1]);
-                    const float i0 = __expf(-bsum[2 * e]), i1 = __expf(-bsum[2 * e + 1]);
-                    float2 qf = unpack_bf16(qw[e]), kf = unpack_bf16(kw[e]);
-                    qw[e] = pack_bf16(qf.x * gq * e0, qf.y * gq * e1);
-                    kw[e] = pack_bf16(kf.x * gk * i0, kf.y * gk * i1);
+    } else if (warp == 13) {
+        // ---------------- TMA (one lane): loads ahead of the compute warps, output stores behind them ----------------
+        if (lane == 0) {
+            auto load_g = [&](int n) {
+                mbar_expect_tx(bar(FULL_G), TILE_G);
+                tma_load_4d(base + OFF_G, &tm_g, 0, h, n * C, b, bar(FULL_G));
+            };
+            auto load_qk = [&](int n) {
+                const uint32_t bf = bar(FULL_QK + n % 3), dst = base + OFF_QK + (n % 3) * QK_BYTES;
+                mbar_expect_tx(bf, QK_BYTES);
+                tma_load_4d(dst, &tm_q, 0, h, n * C, b, bf);
+                tma_load_4d(dst + HALF_BF16, &tm_q, 64, h, n * C, b, bf);
+                tma_load_4d(dst + TILE_BF16, &tm_k, 0, h, n * C, b, bf);
+                tma_load_4d(dst + TILE_BF16 + HALF_BF16, &tm_k, 64, h, n * C, b, bf);
+            };
+            auto load_v = [&](int n) {
+                const uint32_t bf = bar(FULL_V + (n & 1)), dst = base + OFF_V + (n & 1) * TILE_BF16;
+                mbar_expect_tx(bf, TILE_BF16);
+                tma_load_4d(dst, &tm_v, 0, h, n * C, b, bf);
+                tma_load_4d(dst + HALF_BF16, &tm_v, 64, h, n * C, b, bf);
+            };
+            auto store_o = [&](int m) {                // staged by the compute warps; rows past T are clipped
+                wait_relaxed(OSTAGED, m & 1);
+                if (failed) return;
+                tma_store_4d(&tm_o, base + OFF_OST, 0, h, m * C, b);
+                tma_store_4d(&tm_o, base + OFF_OST + HALF_BF16, 64, h, m * C, b);
+                bulk_commit();
+                bulk_wait_read0();
+                mbar_arrive(bar(OSFREE));
+            };
+            load_g(0);
+            for (int n = 0; n < 3 && n < p.NT; ++n) load_qk(n);
+            for (int n = 0; n < 2 && n < p.NT; ++n) load_v(n);
+            wait(OPR + 0, 0);                          // prologue of chunk 0 done: the log-decay buffer is free
+            if (p.NT > 1 && !failed) load_g(1);
+            for (int n = 0; n < p.NT && !failed; ++n) {
+                if (n + 3 < p.NT) {                    // q/k buffer: free once A, qh S and kh^T V have read it
+                    wait(QKFREE + n % 3, (n / 3) & 1);
+                    if (failed) break;
+                    load_qk(n + 3);
                 }
-                *qp = qv;
-                *kp = kv;
+                if (n + 2 < p.NT) {                    // log-decay buffer: free once the prologue of chunk n+1 is done
+                    wait(OPR + (n + 1) % 3, ((n + 1) / 3) & 1);
+                    if (failed) break;
+                    load_g(n + 2);
+                }
+                if (n + 2 < p.NT) {                    // v buffer: free once A V has read it
+                    wait(BAR_O + (n & 1), (n >> 1) & 1);
+                    if (failed) break;
+                    load_v(n + 2);
+                }
+                if (n > 0) store_o(n - 1);
             }
-            if (rg == 15) {
+            if (!failed) store_o(p.NT - 1);
+            bulk_wait0();
+            if (failed) {   // give loads that are still in flight time to land before shared memory goes away
+                const uint64_t t0 = globaltimer_ns();
+                while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
+            }
+        }
+    } else if (warp >= 9) {
+        // ---------------- gates: softmax over the heads, up to four chunks ahead ----------------
+        const int g = tid - (NCOMPUTE + 32), t = g & (C - 1);
+        const float *l = g < C ? p.lq : p.lk;
+        const float mult = g < C ? p.scale : 1.f;
+        for (int n = 0; n < p.NT; ++n) {
+            if (n >= 4) wait_relaxed(GFREE + (n & 3), ((n >> 2) - 1) & 1);
+            if (failed) break;
+            const int cn = min(C, p.T - n * C);
+            gate_s[(n & 3) * 2 * C + g] = t < cn ? mult * token_gate_any(l + (tokb + (size_t)n * C + t) * p.H, p.H, h) : 0.f;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(GREADY + (n & 3)));
+        }
+    } else {
+        // ---------------- compute warps ----------------
+        const uint32_t lane_base = (uint32_t)(32 * (warp & 3)) << 16;   // this warp's TMEM lane quarter
+        const int colhalf = warp >> 2;                                   // which 64 state / output columns
+        const int row = 32 * (warp & 3) + lane;
+
+        {   // initial state: fp32 into TMEM, bf16 copy into shared memory (row = key dimension)
+            const float *src = p.h0 ? p.h0 + ((size_t)bh * D + row) * D + 64 * colhalf : nullptr;
 #pragma unroll
-                for (int e = 0; e < 8; ++e) eblast[8 * cj + e] = __expf(bsum[e]);
+            for (int part = 0; part < 2; ++part) {
+                float v[32];
+#pragma unroll
+                for (int j = 0; j < 32; ++j) v[j] = src ? src[32 * part + j] : 0.f;
+                tmem_st32(tmem + lane_base + COL_S + 64 * colhalf + 32 * part, v);
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    uint4 w;
+                    w.x = pack_bf16(v[8 * c + 0], v[8 * c + 1]);
+                    w.y = pack_bf16(v[8 * c + 2], v[8 * c + 3]);
+                    w.z = pack_bf16(v[8 * c + 4], v[8 * c + 5]);
+                    w.w = pack_bf16(v[8 * c + 6], v[8 * c + 7]);
+                    *reinterpret_cast<uint4 *>(sm + OFF_S + colhalf * STATE_HALF + swz(row, 4 * part + c)) = w;
+                }
             }
+            tmem_wait_st();
         }
         fence_proxy_async();
         tc_fence_before();
-        __syncthreads();
-        SLA_TS(2);
+        mbar_arrive(bar(SREADY));
 
-        if (tid == 0) {
+        auto prologue = [&](int n) {
+#define SLA_TSP(k) do { if (p.phase_ts && bh == 0 && tid == 0 && n == 9) p.phase_ts[k] = globaltimer_ns(); } while (0)
+            SLA_TSP(16);
+            wait(GREADY + (n & 3), (n >> 2) & 1);
+            SLA_TSP(17);
+            wait(FULL_G, n & 1);
+            SLA_TSP(18);
+            wait(FULL_QK + n % 3, (n / 3) & 1);
+            SLA_TSP(19);
+            uint8_t *qk = sm + OFF_QK + (n % 3) * QK_BYTES;
+            const float *g = gate_s + (n & 3) * 2 * C;
+            chunk_prologue<true, false>(qk, qk + TILE_BF16, reinterpret_cast<const float *>(sm + OFF_G), tot, g, g + C,
+                                        eblast + (n & 1) * D, nullptr, nullptr, tid);
+            fence_proxy_async();
+            mbar_arrive(bar(OPR + n % 3));
+            mbar_arrive(bar(GFREE + (n & 3)));
+        };
+        // O of chunk m: TMEM -> bf16 -> staging tile (the TMA warp stores it)
+        auto stage_o = [&](int m) {
+            wait(BAR_O + (m & 1), (m >> 1) & 1);
             tc_fence_after();
-            // A = qh kh^T
+            const int i = 16 * (warp & 3) + lane;
+            float v0[32], v1[32];
+            tmem_ld32(tmem + lane_base + COL_O + (m & 1) * D + 64 * colhalf, v0);
+            tmem_ld32(tmem + lane_base + COL_O + (m & 1) * D + 64 * colhalf + 32, v1);
+            tmem_wait_ld();
+            tc_fence_before();
+            mbar_arrive(bar(OFREE));
+            if (m > 0) wait(OSFREE, (m - 1) & 1);      // the previous store has left the staging tile
+            if (lane < 16) {
 #pragma unroll
-            for (int kk = 0; kk < 8; ++kk) {
-                const uint32_t off = (kk >> 2) * HALF_BF16 + (kk & 3) * 32;
-                tc_mma_bf16(tmem + COL_A, smem_desc_sw128(st + OFF_Q + off, 16, 1024),
-                            smem_desc_sw128(st + OFF_K + off, 16, 1024), ID_A, kk > 0);
+                for (int c = 0; c < 4; ++c) {
+                    uint4 w;
+                    w.x = pack_bf16(v0[8 * c + 0], v0[8 * c + 1]);
+                    w.y = pack_bf16(v0[8 * c + 2], v0[8 * c + 3]);
+                    w.z = pack_bf16(v0[8 * c + 4], v0[8 * c + 5]);
+                    w.w = pack_bf16(v0[8 * c + 6], v0[8 * c + 7]);
+                    *reinterpret_cast<uint4 *>(sm + OFF_OST + colhalf * HALF_BF16 + swz(i, c)) = w;
+                    w.x = pack_bf16(v1[8 * c + 0], v1[8 * c + 1]);
+                    w.y = pack_bf16(v1[8 * c + 2], v1[8 * c + 3]);
+                    w.z = pack_bf16(v1[8 * c + 4], v1[8 * c + 5]);
+                    w.w = pack_bf16(v1[8 * c + 6], v1[8 * c + 7]);
+                    *reinterpret_cast<uint4 *>(sm + OFF_OST + colhalf * HALF_BF16 + swz(i, 4 + c)) = w;
+                }
             }
-            tc_commit(bar_a);
-            // O = qh S_prev   (S operand: [K = d_k rows][N = d_v], two 64-column halves 16 KiB apart)
-#pragma unroll
-            for (int kk = 0; kk < 8; ++kk) {
-                const uint32_t off = (kk >> 2) * HALF_BF16 + (kk & 3) * 32;
-                tc_mma_bf16(tmem + COL_O, smem_desc_sw128(st + OFF_Q + off, 16, 1024),
-                            smem_desc_sw128(base + OFF_S + kk * 2048, D * 128, 1024), ID_O1, kk > 0);
-            }
-            // S += kh^T V   (both operands token-major: MN-major descriptors, halves 8 KiB apart)
-#pragma unroll
-            for (int kk = 0; kk < 4; ++kk)
-                tc_mma_bf16(tmem + COL_S, smem_desc_sw128(st + OFF_K + kk * 2048, HALF_BF16, 1024),
-                            smem_desc_sw128(st + OFF_V + kk * 2048, HALF_BF16, 1024), ID_Z, 1);
-            tc_commit(bar_z);
-        }
+            fence_proxy_async();
+            mbar_arrive(bar(OSTAGED));
+        };
+        prologue(0);
 
-        // A: TMEM -> causal mask -> bf16 -> shared memory (row i of the M=64 tile sits in lane 32*(i/16) + i%16)
-        if (!failed && !mbar_wait_bounded(bar_a, ph_a)) failed = true;
-        ph_a ^= 1;
-        tc_fence_after();
-        SLA_TS(3);
-        if (warp < 4) {
-            const int i = 16 * warp + lane;
-#pragma unroll
-            for (int part = 0; part < 2; ++part) {
+        for (int n = 0; n < p.NT; ++n) {
+            const uint32_t par = n & 1;
+            SLA_TS(0);
+            if (n + 1 < p.NT) prologue(n + 1);         // overlaps the MMAs of chunk n
+            SLA_TS(1);
+
+            // A: TMEM -> causal mask -> bf16 -> shared memory (row i of the M=64 tile sits in lane 32*(i/16) + i%16)
+            wait(BAR_A, par);
+            tc_fence_after();
+            SLA_TS(2);
+            {
+                const int i = 16 * (warp & 3) + lane, part = colhalf;
                 float v[32];
                 tmem_ld32(tmem + lane_base + COL_A + 32 * part, v);
                 tmem_wait_ld();
@@ -261,66 +329,26 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
                     }
                 }
             }
-        }
-        fence_proxy_async();
-        tc_fence_before();
-        __syncthreads();
-        SLA_TS(4);
-        if (tid == 0) {
+            fence_proxy_async();
+            tc_fence_before();
+            mbar_arrive(bar(AREADY));
+            SLA_TS(3);
+
+            // S_{n+1} = diag(2^{b_last}) (S_n + kh^T V): fp32 back into TMEM, bf16 copy for the next chunk's qh S
+            wait(BAR_Z, par);
             tc_fence_after();
-            // O += A V
+            SLA_TS(4);
+            {
+                const float e = eblast[(n & 1) * D + row];
 #pragma unroll
-            for (int kk = 0; kk < 4; ++kk)
-                tc_mma_bf16(tmem + COL_O, smem_desc_sw128(base + OFF_A + kk * 32, 16, 1024),
-                            smem_desc_sw128(st + OFF_V + kk * 2048, HALF_BF16, 1024), ID_O2, 1);
-            tc_commit(bar_o);
-        }
-
-        // S <- diag(e^{b_last}) S : fp32 back into TMEM, bf16 copy for the next chunk's qh S product
-        if (!failed && !mbar_wait_bounded(bar_z, ph_z)) failed = true;
-        ph_z ^= 1;
-        tc_fence_after();
-        SLA_TS(5);
-        {
-            const int row = 32 * (warp & 3) + lane;
-            const float e = eblast[row];
+                for (int part = 0; part < 2; ++part) {
+                    float v[32];
+                    const uint32_t ta = tmem + lane_base + COL_S + 64 * colhalf + 32 * part;
+                    tmem_ld32(ta, v);
+                    tmem_wait_ld();
 #pragma unroll
-            for (int part = 0; part < 2; ++part) {
-                float v[32];
-                const uint32_t ta = tmem + lane_base + COL_S + 64 * colhalf + 32 * part;
-                tmem_ld32(ta, v);
-                tmem_wait_ld();
-#pragma unroll
-                for (int j = 0; j < 32; ++j) v[j] *= e;
-                tmem_st32(ta, v);
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint4 w;
-                    w.x = pack_bf16(v[8 * c + 0], v[8 * c + 1]);
-                    w.y = pack_bf16(v[8 * c + 2], v[8 * c + 3]);
-                    w.z = pack_bf16(v[8 * c + 4], v[8 * c + 5]);
-                    w.w = pack_bf16(v[8 * c + 6], v[8 * c + 7]);
-                    *reinterpret_cast<uint4 *>(sm + OFF_S + colhalf * (D * 128) + swz(row, 4 * part + c)) = w;
-                }
-            }
-            tmem_wait_st();
-        }
-
-        // O: TMEM -> bf16 -> HBM (heads concatenated: row stride H*d_v)
-        if (!failed && !mbar_wait_bounded(bar_o, ph_o)) failed = true;
-        SLA_TS(6);
-        ph_o ^= 1;
-        tc_fence_after();
-        SLA_TS(7);
-        {
-            const int i = 16 * (warp & 3) + lane;
-#pragma unroll
-            for (int part = 0; part < 2; ++part) {
-                float v[32];
-                tmem_ld32(tmem + lane_base + COL_O + 64 * colhalf + 32 * part, v);
-                tmem_wait_ld();
-                if (lane < 16 && i < cn) {
-                    __nv_bfloat16 *dst = p.o + (((size_t)b * p.T + t0 + i) * p.H + h) * D + 64 * colhalf + 32 * part;
+                    for (int j = 0; j < 32; ++j) v[j] *= e;
+                    tmem_st32(ta, v);
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
                         uint4 w;
@@ -328,30 +356,32 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
                         w.y = pack_bf16(v[8 * c + 2], v[8 * c + 3]);
                         w.z = pack_bf16(v[8 * c + 4], v[8 * c + 5]);
                         w.w = pack_bf16(v[8 * c + 6], v[8 * c + 7]);
-                        reinterpret_cast<uint4 *>(dst)[c] = w;
+                        *reinterpret_cast<uint4 *>(sm + OFF_S + colhalf * STATE_HALF + swz(row, 4 * part + c)) = w;
                     }
                 }
+                tmem_wait_st();
             }
-        }
-        SLA_TS(8);
-        fence_proxy_async();
-        tc_fence_before();
-        __syncthreads();
-        tc_fence_after();
-        SLA_TS(9);
-    }
+            fence_proxy_async();
+            tc_fence_before();
+            mbar_arrive(bar(SREADY));
+            SLA_TS(5);
 
-    if (p.ht) {   // final state, fp32
-        const int row = 32 * (warp & 3) + lane;
-        float *dst = p.ht + ((size_t)bh * D + row) * D + 64 * colhalf;
+            if (n > 0) stage_o(n - 1);                 // chunk n-1's output: its MMAs finished long ago
+            SLA_TS(6);
+        }
+        stage_o(p.NT - 1);
+
+        if (p.ht) {   // final state, fp32 (each thread reads back what it wrote in the last rescale)
+            float *dst = p.ht + ((size_t)bh * D + row) * D + 64 * colhalf;
 #pragma unroll
-        for (int part = 0; part < 2; ++part) {
-            float v[32];
-            tmem_ld32(tmem + lane_base + COL_S + 64 * colhalf + 32 * part, v);
-            tmem_wait_ld();
+            for (int part = 0; part < 2; ++part) {
+                float v[32];
+                tmem_ld32(tmem + lane_base + COL_S + 64 * colhalf + 32 * part, v);
+                tmem_wait_ld();
 #pragma unroll
-            for (int j = 0; j < 32; j += 4)
-                *reinterpret_cast<float4 *>(dst + 32 * part + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                for (int j = 0; j < 32; j += 4)
+                    *reinterpret_cast<float4 *>(dst + 32 * part + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+            }
         }
     }
     if (failed) atomicExch(p.status, 1);
@@ -365,6 +395,7 @@ unsigned long long *g_phase_ts = nullptr;   // set by sla_debug_set_phase_timest
 }  // namespace
 
 void gla_tc_set_phase_ts(unsigned long long *p) { g_phase_ts = p; }
+unsigned long long *gla_tc_phase_ts() { return g_phase_ts; }
 
 bool gla_tc_supported(const Dims &d) {
     return d.variant == SLA_GLA && d.io_bf16 && d.dk == 128 && d.dv == 128 && d.C == 64;
@@ -377,12 +408,13 @@ int gla_tc_configure() {
 }
 
 int gla_tc_forward(const Dims &d, const FwdArgs &a, int *status, cudaStream_t st, Tracer &tr) {
-    CUtensorMap mq, mk, mv, mg;
+    CUtensorMap mq, mk, mv, mg, mo;
     if (!make_map(&mq, a.q, d.B, d.T, d.H, d.dk, false, 64) || !make_map(&mk, a.k, d.B, d.T, d.H, d.dk, false, 64) ||
-        !make_map(&mv, a.v, d.B, d.T, d.H, d.dv, false, 64) || !make_map(&mg, a.log_decay, d.B, d.T, d.H, d.dk, true, 128))
+        !make_map(&mv, a.v, d.B, d.T, d.H, d.dv, false, 64) || !make_map(&mg, a.log_decay, d.B, d.T, d.H, d.dk, true, 128) ||
+        !make_map(&mo, a.o, d.B, d.T, d.H, d.dv, false, 64))
         return -1;
     FwdParams p{a.lq, a.lk, a.h0, (__nv_bfloat16 *)a.o, a.ht, status, d.T, d.H, d.NT, d.scale, g_phase_ts};
-    k_gla_fwd_tc<<<d.B * d.H, 256, SMEM_BYTES, st>>>(mq, mk, mv, mg, p);
+    k_gla_fwd_tc<<<d.B * d.H, NTHREADS, SMEM_BYTES, st>>>(mq, mk, mv, mg, mo, p);
     tr.mark("gla_fwd_tc");
     return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }

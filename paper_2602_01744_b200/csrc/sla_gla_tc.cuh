@@ -72,5 +72,112 @@ __device__ __forceinline__ float2 head_gates(const float *lq, const float *lk, i
     return make_float2(expf(lq[h] - m1) / s1, expf(lk[h] - m2) / s2);
 }
 
+__device__ __forceinline__ float ex2f(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+constexpr uint32_t NCOMPUTE = 256;      // compute threads (warps 0..7); they meet on named barrier 1
+constexpr float LOG2E = 1.4426950408889634f;
+
+// Chunk prologue, run by the 256 compute threads on one landed stage (Eq. 12's decay made chunk-local):
+//   b_i = inclusive cumulative log-decay (kept in log2 units), two-level: per-8-row sums, then a running sum
+//   qh_i = gq_i * q_i * 2^{b_i}   (gq_i = scale*Gq_i)      kh_i = gk_i * k_i * 2^{-b_i}
+// written over q and k in place (the swizzled tiles are the MMA operands); eblast[d] = 2^{b_last,d}.
+// With WITH_E also leaves bf16 tiles e_tile = gq_i 2^{b_i}, ei_tile = gk_i 2^{-b_i} (the factors that turn dqh, dkh
+// into dq, dk), laid out like the q tile.  Thread (rg = warp, cj = lane) owns rows 8rg..8rg+7, columns 4cj..4cj+3.
+// tot: [8][128] floats of scratch.
+constexpr uint32_t TOT_BYTES = 8 * D * 4;
+template <bool WITH_Q, bool WITH_E>
+__device__ __forceinline__ void chunk_prologue(uint8_t *q_tile, uint8_t *k_tile, const float *gs, float *tot,
+                                               const float *gq_s, const float *gk_s, float *eblast,
+                                               uint8_t *e_tile, uint8_t *ei_tile, int tid) {
+    using namespace ptx;
+    const int rg = tid >> 5, cj = tid & 31;
+    {
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int rr = 0; rr < 8; ++rr) {
+            const float4 g = *reinterpret_cast<const float4 *>(gs + (8 * rg + rr) * D + 4 * cj);
+            acc.x += g.x; acc.y += g.y; acc.z += g.z; acc.w += g.w;
+        }
+        *reinterpret_cast<float4 *>(tot + rg * D + 4 * cj) = acc;
+    }
+    named_bar_sync(1, NCOMPUTE);
+    float bsum[4] = {0.f, 0.f, 0.f, 0.f};
+    for (int g = 0; g < rg; ++g) {
+        const float4 a = *reinterpret_cast<const float4 *>(tot + g * D + 4 * cj);
+        bsum[0] += a.x; bsum[1] += a.y; bsum[2] += a.z; bsum[3] += a.w;
+    }
+#pragma unroll
+    for (int e = 0; e < 4; ++e) bsum[e] *= LOG2E;
+    // columns 4cj..4cj+3 = 8 bytes of a bf16 row: half cj>>4, 16-byte chunk (cj&15)>>1, upper or lower 8 bytes
+    const uint32_t half = cj >> 4, chunk = (cj & 15) >> 1, sub = (cj & 1) * 8;
+#pragma unroll
+    for (int rr = 0; rr < 8; ++rr) {
+        const int r = 8 * rg + rr;
+        const float4 g = *reinterpret_cast<const float4 *>(gs + r * D + 4 * cj);
+        bsum[0] = fmaf(g.x, LOG2E, bsum[0]); bsum[1] = fmaf(g.y, LOG2E, bsum[1]);
+        bsum[2] = fmaf(g.z, LOG2E, bsum[2]); bsum[3] = fmaf(g.w, LOG2E, bsum[3]);
+        const float gq = WITH_Q ? gq_s[r] : 0.f, gk = gk_s[r];
+        const uint32_t off = half * HALF_BF16 + swz(r, chunk) + sub;
+        uint2 qv, kv = *reinterpret_cast<uint2 *>(k_tile + off), ev, iv;
+        if (WITH_Q) qv = *reinterpret_cast<uint2 *>(q_tile + off);
+        uint32_t *qw = reinterpret_cast<uint32_t *>(&qv), *kw = reinterpret_cast<uint32_t *>(&kv);
+        uint32_t *ew = reinterpret_cast<uint32_t *>(&ev), *iw = reinterpret_cast<uint32_t *>(&iv);
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+            const float i0 = gk * ex2f(-bsum[2 * e]), i1 = gk * ex2f(-bsum[2 * e + 1]);
+            const float2 kf = unpack_bf16(kw[e]);
+            kw[e] = pack_bf16(kf.x * i0, kf.y * i1);
+            if (WITH_E) iw[e] = pack_bf16(i0, i1);
+            if (WITH_Q) {
+                const float e0 = gq * ex2f(bsum[2 * e]), e1 = gq * ex2f(bsum[2 * e + 1]);
+                const float2 qf = unpack_bf16(qw[e]);
+                qw[e] = pack_bf16(qf.x * e0, qf.y * e1);
+                if (WITH_E) ew[e] = pack_bf16(e0, e1);
+            }
+        }
+        *reinterpret_cast<uint2 *>(k_tile + off) = kv;
+        if (WITH_Q) *reinterpret_cast<uint2 *>(q_tile + off) = qv;
+        if (WITH_E) {
+            *reinterpret_cast<uint2 *>(e_tile + off) = ev;
+            *reinterpret_cast<uint2 *>(ei_tile + off) = iv;
+        }
+    }
+    if (rg == 7) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) eblast[4 * cj + e] = ex2f(bsum[e]);
+    }
+}
+
+// Head-softmax gate (Eq. 4) of ONE token for head h: the H <= HP logits are fetched before the first use (one memory
+// round trip), then max, exp and sum run over registers.  Returns softmax(row[0..H))[h].
+template <int HP>
+__device__ __forceinline__ float token_gate(const float *__restrict__ row, int H, int h) {
+    float x[HP];
+#pragma unroll
+    for (int j = 0; j < HP; ++j) x[j] = j < H ? row[j] : -INFINITY;
+    float m = x[0];
+#pragma unroll
+    for (int j = 1; j < HP; ++j) m = fmaxf(m, x[j]);
+    float sum = 0.f, eh = 0.f;
+#pragma unroll
+    for (int j = 0; j < HP; ++j) {
+        const float e = __expf(x[j] - m);      // exp(-inf) = 0 for the padding lanes
+        sum += e;
+        eh = j == h ? e : eh;
+    }
+    return eh / sum;
+}
+__device__ __forceinline__ float token_gate_any(const float *row, int H, int h) {
+    if (H <= 4) return token_gate<4>(row, H, h);
+    if (H <= 8) return token_gate<8>(row, H, h);
+    if (H <= 16) return token_gate<16>(row, H, h);
+    return token_gate<32>(row, H, h);
+}
+constexpr int NGATE = 128;   // gate threads: g < 64 -> scale*Gq of token g, g >= 64 -> Gk of token g-64
+
 }  // namespace tc
 }  // namespace sla

@@ -264,7 +264,9 @@ struct BwdParams {
     int *status;
     int T, H, NT;
     float scale;
+    unsigned long long *phase_ts;   // optional: block 0 / thread 0 stamps the phases of one chunk
 };
+#define SLA_TS(k) do { if (p.phase_ts && bh == 0 && tid == 0 && n == 8) p.phase_ts[k] = globaltimer_ns(); } while (0)
 
 // Sum v[j] over the 32 lanes for every j: afterwards lane l holds the total of v[l] in v[0].
 __device__ __forceinline__ float warp_transpose_sum(float (&v)[32], int lane) {
@@ -395,6 +397,7 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
 
     for (int n = nlast; n >= 0; --n) {
         const int t0 = n * C, cn = min(C, p.T - t0);
+        SLA_TS(0);
         if (tid < C) {   // head-softmax gates of this chunk's tokens (Eq. 4)
             float gq = 0.f, gk = 0.f;
             if (tid < cn) {
@@ -410,6 +413,7 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
         ph_g ^= 1;
         if (!failed && !mbar_wait_bounded(bar_qk, ph_qk)) failed = true;
         ph_qk ^= 1;
+        SLA_TS(1);
 
         // cumulative log-decay; qh, kh in place; e^b kept as bf16 for the epilogue
         const float *gs = reinterpret_cast<const float *>(sm + OFF_G);
@@ -474,6 +478,7 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
         fence_proxy_async();
         tc_fence_before();
         __syncthreads();
+        SLA_TS(2);
 
         if (tid == 0) {
             if (n > 0) issue_g(n - 1);       // the log-decay tile is consumed: fetch the next one early
@@ -506,11 +511,13 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             }
             tmem_wait_st();
         }
+        SLA_TS(3);
 
         // A, dA: TMEM -> causal mask -> bf16 -> shared memory (row i of an M=64 tile sits in lane 32*(i/16) + i%16)
         if (!failed && !mbar_wait_bounded(bar_a, ph_a)) failed = true;
         ph_a ^= 1;
         tc_fence_after();
+        SLA_TS(4);
         {
             const int i = 16 * (warp & 3) + lane;
             const uint32_t col = wh ? COL_DA : COL_A;
@@ -537,6 +544,7 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
         fence_proxy_async();
         tc_fence_before();
         __syncthreads();
+        SLA_TS(5);
 
         if (tid == 0) {
             if (!failed && !mbar_wait_bounded(bar_s, ph_s)) failed = true;
@@ -582,6 +590,7 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
         if (!failed && !mbar_wait_bounded(bar_m, ph_m)) failed = true;
         ph_m ^= 1;
         tc_fence_after();
+        SLA_TS(6);
 
         const float *Rcur = Rs + (n & 1) * 2 * D;
         {   // R_{n-1} = rowsum(dS_n * S_n), this thread's 64 columns
@@ -596,6 +605,7 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             Rs[((n & 1) ^ 1) * 2 * D + wh * D + row] = rpart;
         }
 
+        SLA_TS(7);
         // gradient tiles: this thread owns key dimension `row` and tokens 32*wh .. 32*wh+31
         const size_t tok0 = (size_t)b * p.T + t0;
         float sfx[32];
@@ -630,6 +640,7 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             red[warp * 32 + lane] = sq;
             red[8 * 32 + warp * 32 + lane] = sk;
         }
+        SLA_TS(8);
         {   // dV^T -> dv
             float dvt[32];
             tmem_ld32(tmem + lane_base + COL_DV + 32 * wh, dvt);
@@ -640,9 +651,11 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
                 if (i < cn) p.dv[((tok0 + i) * p.H + h) * D + row] = __float2bfloat16_rn(dvt[ii]);
             }
         }
+        SLA_TS(9);
         fence_proxy_async();
         tc_fence_before();
         __syncthreads();
+        SLA_TS(10);
         if (tid == 0 && n > 0) issue_rest(n - 1);      // every operand buffer is free again
         tc_fence_after();
         {   // log-decay gradient: in-chunk suffix sum + what flows in from the right of the chunk
@@ -665,6 +678,7 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             p.pk[(tok0 + tid) * p.H + h] = sk;
         }
         __syncthreads();     // red, up, Rs are rewritten by the next chunk
+        SLA_TS(11);
     }
 
     if (p.dh0) {   // dS_0, fp32
@@ -747,7 +761,7 @@ int gla_tc_backward(const Dims &d, const BwdArgs &a, int *status, cudaStream_t s
     k_gla_states_tc<<<d.B * d.H, 256, st1::SMEM_BYTES, st>>>(mk, mv, mg, sp);
     tr.mark("gla_states_tc");
     BwdParams bp{a.lq, a.lk, a.dht, simg, (__nv_bfloat16 *)a.dq, (__nv_bfloat16 *)a.dk, (__nv_bfloat16 *)a.dv,
-                 a.dlog_decay, pq, pk, a.dh0, status, d.T, d.H, d.NT, d.scale};
+                 a.dlog_decay, pq, pk, a.dh0, status, d.T, d.H, d.NT, d.scale, gla_tc_phase_ts()};
     k_gla_bwd_tc<<<d.B * d.H, 256, st2::SMEM_BYTES, st>>>(mq, mk, mv, mdo, mg, bp);
     tr.mark("gla_bwd_tc");
     const long n_tok = (long)d.B * d.T;

@@ -96,6 +96,7 @@ int gdn_configure();
 bool gla_tc_supported(const Dims &d);
 int gla_tc_configure();
 void gla_tc_set_phase_ts(unsigned long long *device_buffer);
+unsigned long long *gla_tc_phase_ts();
 int gla_tc_forward(const Dims &d, const FwdArgs &a, int *status, cudaStream_t st, Tracer &tr);
 // Backward: chunk-state sweep, gradient sweep, gate softmax backward.  Needs the first
 // B*H*(NT+1)*32 KiB + 2*B*T*H*4 bytes (rounded up) of the workspace, less than the generic path.
