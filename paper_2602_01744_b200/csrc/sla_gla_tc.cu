@@ -126,14 +126,14 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
                 tc_fence_after();
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk)         // A = qh kh^T
-                    tc_mma_bf16(tmem + COL_A, desc_kmajor(sQ, kk, HALF_BF16), desc_kmajor(sK, kk, HALF_BF16), ID_A, kk > 0);
+                    tc_mma_bf16(tmem + COL_A, (desc_kmajor(sQ) + kstep_kmajor(kk, HALF_BF16)), (desc_kmajor(sK) + kstep_kmajor(kk, HALF_BF16)), ID_A, kk > 0);
                 tc_commit(bar(BAR_A));
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk)         // O = qh S_n
-                    tc_mma_bf16(tO, desc_kmajor(sQ, kk, HALF_BF16), desc_mnmajor(base + OFF_S, kk, STATE_HALF), ID_O, kk > 0);
+                    tc_mma_bf16(tO, (desc_kmajor(sQ) + kstep_kmajor(kk, HALF_BF16)), (desc_mnmajor(base + OFF_S, STATE_HALF) + kstep_mnmajor(kk)), ID_O, kk > 0);
 #pragma unroll
                 for (int kk = 0; kk < 4; ++kk)         // S += kh^T V
-                    tc_mma_bf16(tmem + COL_S, desc_mnmajor(sK, kk, HALF_BF16), desc_mnmajor(sV, kk, HALF_BF16), ID_Z, 1);
+                    tc_mma_bf16(tmem + COL_S, (desc_mnmajor(sK, HALF_BF16) + kstep_mnmajor(kk)), (desc_mnmajor(sV, HALF_BF16) + kstep_mnmajor(kk)), ID_Z, 1);
                 tc_commit(bar(BAR_Z));
                 tc_commit(bar(QKFREE + n % 3));        // (same event, own barrier: the TMA lane may look at it much later)
                 wait(AREADY, par);                     // masked A is in shared memory
@@ -141,7 +141,7 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
                 tc_fence_after();
 #pragma unroll
                 for (int kk = 0; kk < 4; ++kk)         // O += A V
-                    tc_mma_bf16(tO, desc_kmajor(base + OFF_A, kk, 0), desc_mnmajor(sV, kk, HALF_BF16), ID_O, 1);
+                    tc_mma_bf16(tO, (desc_kmajor(base + OFF_A) + kstep_kmajor(kk, 0)), (desc_mnmajor(sV, HALF_BF16) + kstep_mnmajor(kk)), ID_O, 1);
                 tc_commit(bar(BAR_O + (n & 1)));
             }
             // let the tensor core finish before TMEM goes away (after an abort some of its work may still be queued)
@@ -158,22 +158,18 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             auto load_qk = [&](int n) {
                 const uint32_t bf = bar(FULL_QK + n % 3), dst = base + OFF_QK + (n % 3) * QK_BYTES;
                 mbar_expect_tx(bf, QK_BYTES);
-                tma_load_4d(dst, &tm_q, 0, h, n * C, b, bf);
-                tma_load_4d(dst + HALF_BF16, &tm_q, 64, h, n * C, b, bf);
-                tma_load_4d(dst + TILE_BF16, &tm_k, 0, h, n * C, b, bf);
-                tma_load_4d(dst + TILE_BF16 + HALF_BF16, &tm_k, 64, h, n * C, b, bf);
+                tma_load_5d(dst, &tm_q, 0, n * C, 0, h, b, bf);
+                tma_load_5d(dst + TILE_BF16, &tm_k, 0, n * C, 0, h, b, bf);
             };
             auto load_v = [&](int n) {
                 const uint32_t bf = bar(FULL_V + (n & 1)), dst = base + OFF_V + (n & 1) * TILE_BF16;
                 mbar_expect_tx(bf, TILE_BF16);
-                tma_load_4d(dst, &tm_v, 0, h, n * C, b, bf);
-                tma_load_4d(dst + HALF_BF16, &tm_v, 64, h, n * C, b, bf);
+                tma_load_5d(dst, &tm_v, 0, n * C, 0, h, b, bf);
             };
             auto store_o = [&](int m) {                // staged by the compute warps; rows past T are clipped
                 wait_relaxed(OSTAGED, m & 1);
                 if (failed) return;
-                tma_store_4d(&tm_o, base + OFF_OST, 0, h, m * C, b);
-                tma_store_4d(&tm_o, base + OFF_OST + HALF_BF16, 64, h, m * C, b);
+                tma_store_5d(&tm_o, base + OFF_OST, 0, m * C, 0, h, b);
                 bulk_commit();
                 bulk_wait_read0();
                 mbar_arrive(bar(OSFREE));
@@ -263,7 +259,7 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             uint8_t *qk = sm + OFF_QK + (n % 3) * QK_BYTES;
             const float *g = gate_s + (n & 3) * 2 * C;
             chunk_prologue<true, false>(qk, qk + TILE_BF16, reinterpret_cast<const float *>(sm + OFF_G), tot, g, g + C,
-                                        eblast + (n & 1) * D, nullptr, nullptr, tid);
+                                        eblast + (n & 1) * D, nullptr, tid);
             fence_proxy_async();
             mbar_arrive(bar(OPR + n % 3));
             mbar_arrive(bar(GFREE + (n & 3)));
@@ -409,9 +405,9 @@ int gla_tc_configure() {
 
 int gla_tc_forward(const Dims &d, const FwdArgs &a, int *status, cudaStream_t st, Tracer &tr) {
     CUtensorMap mq, mk, mv, mg, mo;
-    if (!make_map(&mq, a.q, d.B, d.T, d.H, d.dk, false, 64) || !make_map(&mk, a.k, d.B, d.T, d.H, d.dk, false, 64) ||
-        !make_map(&mv, a.v, d.B, d.T, d.H, d.dv, false, 64) || !make_map(&mg, a.log_decay, d.B, d.T, d.H, d.dk, true, 128) ||
-        !make_map(&mo, a.o, d.B, d.T, d.H, d.dv, false, 64))
+    if (!make_tile_map(&mq, a.q, d.B, d.T, d.H) || !make_tile_map(&mk, a.k, d.B, d.T, d.H) ||
+        !make_tile_map(&mv, a.v, d.B, d.T, d.H) || !make_map(&mg, a.log_decay, d.B, d.T, d.H, d.dk, true, 128) ||
+        !make_tile_map(&mo, a.o, d.B, d.T, d.H))
         return -1;
     FwdParams p{a.lq, a.lk, a.h0, (__nv_bfloat16 *)a.o, a.ht, status, d.T, d.H, d.NT, d.scale, g_phase_ts};
     k_gla_fwd_tc<<<d.B * d.H, NTHREADS, SMEM_BYTES, st>>>(mq, mk, mv, mg, mo, p);

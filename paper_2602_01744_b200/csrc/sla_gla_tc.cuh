@@ -20,14 +20,18 @@ constexpr uint32_t STATE_BF16 = 2 * STATE_HALF;     // 32 KiB bf16 state as an M
 // byte offset of 16-byte chunk `chunk` (0..7) of row `row` inside a 128-byte-swizzled tile
 __device__ __forceinline__ uint32_t swz(uint32_t row, uint32_t chunk) { return row * 128 + ((chunk ^ (row & 7)) << 4); }
 
-// K-major operand whose 128-wide K extent is split in two halves `half_stride` bytes apart; k-step kk = 16 elements
-__device__ __forceinline__ uint64_t desc_kmajor(uint32_t tile, uint32_t kk, uint32_t half_stride) {
-    return ptx::smem_desc_sw128(tile + (kk >> 2) * half_stride + (kk & 3) * 32, 16, 1024);
+// Shared-memory matrix descriptors are built once per tile (k-step 0); a k-step only moves the start-address field,
+// i.e. adds a small constant to the descriptor, so the issuing lane spends one add per operand per MMA.
+// K-major operand whose 128-wide K extent is split in two halves `half_stride` bytes apart; k-step kk = 16 elements.
+__device__ __forceinline__ uint64_t desc_kmajor(uint32_t tile) { return ptx::smem_desc_sw128(tile, 16, 1024); }
+__device__ __forceinline__ constexpr uint64_t kstep_kmajor(uint32_t kk, uint32_t half_stride) {
+    return ((kk >> 2) * half_stride + (kk & 3) * 32) >> 4;
 }
-// MN-major operand ([K rows][MN contiguous]); 64-element MN blocks `mn_stride` bytes apart; k-step kk = 16 rows
-__device__ __forceinline__ uint64_t desc_mnmajor(uint32_t tile, uint32_t kk, uint32_t mn_stride) {
-    return ptx::smem_desc_sw128(tile + kk * 2048, mn_stride, 1024);
+// MN-major operand ([K rows][MN contiguous]); 64-element MN blocks `mn_stride` bytes apart; k-step kk = 16 rows.
+__device__ __forceinline__ uint64_t desc_mnmajor(uint32_t tile, uint32_t mn_stride) {
+    return ptx::smem_desc_sw128(tile, mn_stride, 1024);
 }
+__device__ __forceinline__ constexpr uint64_t kstep_mnmajor(uint32_t kk) { return (kk * 2048) >> 4; }
 
 typedef CUresult (*EncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                              const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
@@ -63,6 +67,23 @@ inline bool make_map(CUtensorMap *m, const void *ptr, int B, int T, int H, int d
     return r == CUDA_SUCCESS;
 }
 
+// Tensor map over a bf16 [B,T,H,128] tensor that moves a whole 64-token x 128-feature tile of one head in ONE copy:
+// the feature axis is split as (64 within a half, 2 halves) and the halves are made the slowest box dimension, so the
+// tile lands as two 128-byte-swizzled [64 rows][128 B] halves, 8 KiB apart - the layout the MMA descriptors expect.
+// Coordinates: (0, token, 0, head, batch).
+inline bool make_tile_map(CUtensorMap *m, const void *ptr, int B, int T, int H) {
+    EncodeFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[5] = {64, (cuuint64_t)T, 2, (cuuint64_t)H, (cuuint64_t)B};
+    cuuint64_t strides[4] = {(cuuint64_t)H * D * 2, 128, (cuuint64_t)D * 2, (cuuint64_t)T * H * D * 2};
+    cuuint32_t box[5] = {64, (cuuint32_t)C, 2, 1, 1};
+    cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void *>(ptr), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
 // Head-softmax gates (Eq. 4) of one token for head h: returns (Gq_h, Gk_h).
 __device__ __forceinline__ float2 head_gates(const float *lq, const float *lk, int H, int h) {
     float m1 = -INFINITY, m2 = -INFINITY;
@@ -85,14 +106,15 @@ constexpr float LOG2E = 1.4426950408889634f;
 //   b_i = inclusive cumulative log-decay (kept in log2 units), two-level: per-8-row sums, then a running sum
 //   qh_i = gq_i * q_i * 2^{b_i}   (gq_i = scale*Gq_i)      kh_i = gk_i * k_i * 2^{-b_i}
 // written over q and k in place (the swizzled tiles are the MMA operands); eblast[d] = 2^{b_last,d}.
-// With WITH_E also leaves bf16 tiles e_tile = gq_i 2^{b_i}, ei_tile = gk_i 2^{-b_i} (the factors that turn dqh, dkh
-// into dq, dk), laid out like the q tile.  Thread (rg = warp, cj = lane) owns rows 8rg..8rg+7, columns 4cj..4cj+3.
+// With WITH_E also leaves the tile e2[i][d] = (bf16 gq_i 2^{b_i}, bf16 gk_i 2^{-b_i}), 4 bytes per element, rows of 512 B,
+// unswizzled: the factors that turn dqh, dkh into dq, dk.  Thread (rg = warp, cj = lane) owns rows 8rg..8rg+7,
+// columns 4cj..4cj+3.
 // tot: [8][128] floats of scratch.
 constexpr uint32_t TOT_BYTES = 8 * D * 4;
 template <bool WITH_Q, bool WITH_E>
 __device__ __forceinline__ void chunk_prologue(uint8_t *q_tile, uint8_t *k_tile, const float *gs, float *tot,
                                                const float *gq_s, const float *gk_s, float *eblast,
-                                               uint8_t *e_tile, uint8_t *ei_tile, int tid) {
+                                               uint8_t *e2_tile, int tid) {
     using namespace ptx;
     const int rg = tid >> 5, cj = tid & 31;
     {
@@ -122,29 +144,29 @@ __device__ __forceinline__ void chunk_prologue(uint8_t *q_tile, uint8_t *k_tile,
         bsum[2] = fmaf(g.z, LOG2E, bsum[2]); bsum[3] = fmaf(g.w, LOG2E, bsum[3]);
         const float gq = WITH_Q ? gq_s[r] : 0.f, gk = gk_s[r];
         const uint32_t off = half * HALF_BF16 + swz(r, chunk) + sub;
-        uint2 qv, kv = *reinterpret_cast<uint2 *>(k_tile + off), ev, iv;
+        uint2 qv, kv = *reinterpret_cast<uint2 *>(k_tile + off);
+        uint4 e2v;
         if (WITH_Q) qv = *reinterpret_cast<uint2 *>(q_tile + off);
         uint32_t *qw = reinterpret_cast<uint32_t *>(&qv), *kw = reinterpret_cast<uint32_t *>(&kv);
-        uint32_t *ew = reinterpret_cast<uint32_t *>(&ev), *iw = reinterpret_cast<uint32_t *>(&iv);
+        uint32_t *e2w = reinterpret_cast<uint32_t *>(&e2v);
 #pragma unroll
         for (int e = 0; e < 2; ++e) {
             const float i0 = gk * ex2f(-bsum[2 * e]), i1 = gk * ex2f(-bsum[2 * e + 1]);
             const float2 kf = unpack_bf16(kw[e]);
             kw[e] = pack_bf16(kf.x * i0, kf.y * i1);
-            if (WITH_E) iw[e] = pack_bf16(i0, i1);
             if (WITH_Q) {
                 const float e0 = gq * ex2f(bsum[2 * e]), e1 = gq * ex2f(bsum[2 * e + 1]);
                 const float2 qf = unpack_bf16(qw[e]);
                 qw[e] = pack_bf16(qf.x * e0, qf.y * e1);
-                if (WITH_E) ew[e] = pack_bf16(e0, e1);
+                if (WITH_E) {
+                    e2w[2 * e] = pack_bf16(e0, i0);
+                    e2w[2 * e + 1] = pack_bf16(e1, i1);
+                }
             }
         }
         *reinterpret_cast<uint2 *>(k_tile + off) = kv;
         if (WITH_Q) *reinterpret_cast<uint2 *>(q_tile + off) = qv;
-        if (WITH_E) {
-            *reinterpret_cast<uint2 *>(e_tile + off) = ev;
-            *reinterpret_cast<uint2 *>(ei_tile + off) = iv;
-        }
+        if (WITH_E) *reinterpret_cast<uint4 *>(e2_tile + r * (D * 4) + cj * 16) = e2v;
     }
     if (rg == 7) {
 #pragma unroll

@@ -18,6 +18,8 @@
 //                     qh*dqh - kh*dkh plus rowsum(dS_{n+1} * S_{n+1}) carried from the chunk to the right.
 //                     Gate gradients leave as the products Gq*dGq = sum_d qh*dqh, Gk*dGk = sum_d kh*dkh per
 //                     (token, head); the softmax backward over heads runs afterwards on [B,T,H].
+// Both kernels use the forward kernel's roles: one MMA-issuing lane, one TMA lane, gate warps running ahead and
+// eight compute warps; every wait is bounded and abortable.
 #include "sla_gla_tc.cuh"
 
 namespace sla {
@@ -29,15 +31,22 @@ using namespace tc;
 // ------------------------------------------------------------------------------------------------
 // sweep 1: chunk states
 namespace st1 {
-constexpr uint32_t STAGE = 2 * TILE_BF16 + TILE_G;      // k, v, log-decay: 64 KiB
-constexpr uint32_t OFF_K = 0, OFF_V = TILE_BF16, OFF_G = 2 * TILE_BF16;
-constexpr uint32_t OFF_TOT = 2 * STAGE;                 // [16][128] fp32 partial column sums
-constexpr uint32_t OFF_EB = OFF_TOT + 16 * D * 4;       // [128] exp(b_last)
-constexpr uint32_t OFF_GK = OFF_EB + D * 4;             // [64] Gk
-constexpr uint32_t OFF_BAR = OFF_GK + C * 4;            // full[2], z
-constexpr uint32_t OFF_TMEM = OFF_BAR + 3 * 8;
+constexpr uint32_t OFF_G = 0;                               // [2] fp32 log-decay tiles
+constexpr uint32_t OFF_K = OFF_G + 2 * TILE_G;              // [3] k tiles (kh after the prologue)
+constexpr uint32_t OFF_V = OFF_K + 3 * TILE_BF16;           // [2] v tiles
+constexpr uint32_t OFF_IMG = OFF_V + 2 * TILE_BF16;         // bf16 state image staged for the bulk store
+constexpr uint32_t OFF_TOT = OFF_IMG + STATE_BF16;          // prologue scratch
+constexpr uint32_t OFF_EB = OFF_TOT + TOT_BYTES;            // [2][128] 2^{b_last}
+constexpr uint32_t OFF_GATE = OFF_EB + 2 * D * 4;           // [4][64] Gk of four chunks
+constexpr uint32_t OFF_BAR = OFF_GATE + 4 * C * 4;
+constexpr uint32_t OFF_TMEM = OFF_BAR + 32 * 8;             // TMEM base address, then the abort flag
 constexpr uint32_t SMEM_BYTES = OFF_TMEM + 16 + 1024;
 constexpr uint32_t TMEM_COLS = 128;
+constexpr int NGATE1 = 64;                                  // gate threads (Gk only)
+constexpr int NTHREADS = NCOMPUTE + 32 + NGATE1 + 32;       // warps 0..7 compute, 8 MMA issue, 9..10 gates, 11 TMA
+enum Bar { FULL_G = 0 /*[2]*/, FULL_K = 2 /*[3]*/, FULL_V = 5 /*[2]*/, OPR = 7 /*[3]*/, GREADY = 10 /*[4]*/, GFREE = 14 /*[4]*/,
+           SREADY = 18, STAGED, STFREE, BAR_Z, KFREE /*[3]*/, VFREE = KFREE + 3 /*[2]*/, DRAIN = VFREE + 2, NBAR };
+static_assert(NBAR <= 32, "barrier slots");
 }  // namespace st1
 
 struct StatesParams {
@@ -60,7 +69,9 @@ __device__ __forceinline__ void store_state_part(uint8_t *img, int row, int colh
     }
 }
 
-__global__ void __launch_bounds__(256, 1)
+// Per chunk: prologue of chunk n+1 (kh only) while the tensor core adds kh^T V of chunk n to S; then S is rescaled in
+// TMEM and its bf16 image goes to global memory through a staged bulk store.
+__global__ void __launch_bounds__(st1::NTHREADS, 1)
 k_gla_states_tc(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                 const __grid_constant__ CUtensorMap tm_g, StatesParams p) {
     using namespace st1;
@@ -70,14 +81,25 @@ k_gla_states_tc(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
     uint8_t *sm = smem_raw + (base - raw);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int bh = blockIdx.x, b = bh / p.H, h = bh % p.H;
-    const uint32_t bar_full0 = base + OFF_BAR, bar_z = bar_full0 + 16;
+    auto bar = [&](int i) { return base + OFF_BAR + 8u * i; };
     float *tot = reinterpret_cast<float *>(sm + OFF_TOT);
     float *eblast = reinterpret_cast<float *>(sm + OFF_EB);
-    float *gk_s = reinterpret_cast<float *>(sm + OFF_GK);
+    float *gate_s = reinterpret_cast<float *>(sm + OFF_GATE);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(sm + OFF_TMEM + 8);
     bool failed = false;
+    auto wait = [&](int i, uint32_t parity) {
+        if (!failed && !mbar_wait_bounded(bar(i), parity, abort_flag)) { failed = true; *abort_flag = 1; }
+    };
+    auto wait_relaxed = [&](int i, uint32_t parity) {
+        if (!failed && !mbar_wait_bounded<128>(bar(i), parity, abort_flag)) { failed = true; *abort_flag = 1; }
+    };
 
     if (tid == 0) {
-        for (int i = 0; i < 3; ++i) mbar_init(bar_full0 + 8 * i, 1);
+        *abort_flag = 0;
+        for (int i = 0; i < NBAR; ++i) {
+            const bool all = (i >= OPR && i < GREADY) || (i >= GFREE && i <= STAGED);
+            mbar_init(bar(i), all ? NCOMPUTE : (i >= GREADY && i < GFREE) ? NGATE1 / 32 : 1);
+        }
         fence_mbar_init();
         tma_prefetch_desc(&tm_k);
         tma_prefetch_desc(&tm_v);
@@ -88,143 +110,149 @@ k_gla_states_tc(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *reinterpret_cast<volatile uint32_t *>(sm + OFF_TMEM);
-    const uint32_t lane_base = (uint32_t)(32 * (warp & 3)) << 16;
-    const int colhalf = warp >> 2;
-    const int row = 32 * (warp & 3) + lane;
+    const size_t tokb = (size_t)b * p.T;
     uint8_t *img0 = p.simg + (size_t)bh * (p.NT + 1) * STATE_BF16;
 
-    auto issue_tma = [&](int n, int s) {
-        const uint32_t bar = bar_full0 + 8 * s, st = base + s * STAGE;
-        mbar_expect_tx(bar, STAGE);
-        const int t0 = n * C;
-        tma_load_4d(st + OFF_K, &tm_k, 0, h, t0, b, bar);
-        tma_load_4d(st + OFF_K + HALF_BF16, &tm_k, 64, h, t0, b, bar);
-        tma_load_4d(st + OFF_V, &tm_v, 0, h, t0, b, bar);
-        tma_load_4d(st + OFF_V + HALF_BF16, &tm_v, 64, h, t0, b, bar);
-        tma_load_4d(st + OFF_G, &tm_g, 0, h, t0, b, bar);
-    };
-    if (tid == 0) issue_tma(0, 0);
-
-    {   // S_0: fp32 into TMEM, bf16 image into slot 0
-        const float *src = p.h0 ? p.h0 + ((size_t)bh * D + row) * D + 64 * colhalf : nullptr;
+    if (warp == 8) {
+        // ---------------- MMA issue (one lane) ----------------
+        if (lane == 0) {
+            constexpr uint32_t ID_Z = idesc_bf16(128, 128, 1, 1);    // kh^T (MN-major) x V (MN-major)
+            for (int n = 0; n < p.NT; ++n) {
+                const uint32_t sK = base + OFF_K + (n % 3) * TILE_BF16, sV = base + OFF_V + (n & 1) * TILE_BF16;
+                wait(OPR + n % 3, (n / 3) & 1);        // kh of chunk n is in place
+                wait(SREADY, n & 1);                   // S_n is in TMEM
+                wait(FULL_V + (n & 1), (n >> 1) & 1);
+                if (failed) break;
+                tc_fence_after();
+                const uint64_t dK = desc_mnmajor(sK, HALF_BF16), dV = desc_mnmajor(sV, HALF_BF16);
 #pragma unroll
-        for (int part = 0; part < 2; ++part) {
-            float v[32];
-#pragma unroll
-            for (int j = 0; j < 32; ++j) v[j] = src ? src[32 * part + j] : 0.f;
-            tmem_st32(tmem + lane_base + 64 * colhalf + 32 * part, v);
-            store_state_part(img0, row, colhalf, part, v);
-        }
-        tmem_wait_st();
-    }
-    tc_fence_before();
-    __syncthreads();
-
-    constexpr uint32_t ID_Z = idesc_bf16(128, 128, 1, 1);
-    uint32_t ph_full[2] = {0, 0}, ph_z = 0;
-    const int rg = tid >> 4, cj = tid & 15;
-
-    for (int n = 0; n < p.NT; ++n) {
-        const int s = n & 1;
-        const uint32_t st = base + s * STAGE;
-        uint8_t *stp = sm + s * STAGE;
-        const int t0 = n * C, cn = min(C, p.T - t0);
-        if (tid == 0 && n + 1 < p.NT) issue_tma(n + 1, s ^ 1);
-        if (tid < C) {
-            float gk = 0.f;
-            if (tid < cn) {
-                const size_t tok = (size_t)b * p.T + t0 + tid;
-                gk = head_gates(p.lq + tok * p.H, p.lk + tok * p.H, p.H, h).y;
+                for (int kk = 0; kk < 4; ++kk)         // S += kh^T V
+                    tc_mma_bf16(tmem, dK + kstep_mnmajor(kk), dV + kstep_mnmajor(kk), ID_Z, 1);
+                tc_commit(bar(BAR_Z));
+                tc_commit(bar(KFREE + n % 3));         // (same event on per-buffer barriers for the TMA lane)
+                tc_commit(bar(VFREE + (n & 1)));
             }
-            gk_s[tid] = gk;
+            tc_commit(bar(DRAIN));
+            mbar_wait_bounded(bar(DRAIN), 0, nullptr, 20000000ull);
         }
-        if (!failed && !mbar_wait_bounded(bar_full0 + 8 * s, ph_full[s])) failed = true;
-        ph_full[s] ^= 1;
-
-        const float *gs = reinterpret_cast<const float *>(stp + OFF_G);
-        {
-            float acc[8];
-#pragma unroll
-            for (int e = 0; e < 8; ++e) acc[e] = 0.f;
-#pragma unroll
-            for (int rr = 0; rr < 4; ++rr) {
-                const float4 g0 = *reinterpret_cast<const float4 *>(gs + (4 * rg + rr) * D + 8 * cj);
-                const float4 g1 = *reinterpret_cast<const float4 *>(gs + (4 * rg + rr) * D + 8 * cj + 4);
-                acc[0] += g0.x; acc[1] += g0.y; acc[2] += g0.z; acc[3] += g0.w;
-                acc[4] += g1.x; acc[5] += g1.y; acc[6] += g1.z; acc[7] += g1.w;
-            }
-            *reinterpret_cast<float4 *>(tot + rg * D + 8 * cj) = make_float4(acc[0], acc[1], acc[2], acc[3]);
-            *reinterpret_cast<float4 *>(tot + rg * D + 8 * cj + 4) = make_float4(acc[4], acc[5], acc[6], acc[7]);
-        }
-        __syncthreads();
-        {
-            float bsum[8];
-#pragma unroll
-            for (int e = 0; e < 8; ++e) bsum[e] = 0.f;
-            for (int g = 0; g < rg; ++g) {
-                const float4 a0 = *reinterpret_cast<const float4 *>(tot + g * D + 8 * cj);
-                const float4 a1 = *reinterpret_cast<const float4 *>(tot + g * D + 8 * cj + 4);
-                bsum[0] += a0.x; bsum[1] += a0.y; bsum[2] += a0.z; bsum[3] += a0.w;
-                bsum[4] += a1.x; bsum[5] += a1.y; bsum[6] += a1.z; bsum[7] += a1.w;
-            }
-            const uint32_t half = cj >> 3, chunk = cj & 7;
-#pragma unroll
-            for (int rr = 0; rr < 4; ++rr) {
-                const int r = 4 * rg + rr;
-                const float4 g0 = *reinterpret_cast<const float4 *>(gs + r * D + 8 * cj);
-                const float4 g1 = *reinterpret_cast<const float4 *>(gs + r * D + 8 * cj + 4);
-                bsum[0] += g0.x; bsum[1] += g0.y; bsum[2] += g0.z; bsum[3] += g0.w;
-                bsum[4] += g1.x; bsum[5] += g1.y; bsum[6] += g1.z; bsum[7] += g1.w;
-                const float gk = gk_s[r];
-                uint4 *kp = reinterpret_cast<uint4 *>(stp + OFF_K + half * HALF_BF16 + swz(r, chunk));
-                uint4 kv = *kp;
-                uint32_t *kw = reinterpret_cast<uint32_t *>(&kv);
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const float i0 = __expf(-bsum[2 * e]), i1 = __expf(-bsum[2 * e + 1]);
-                    float2 kf = unpack_bf16(kw[e]);
-                    kw[e] = pack_bf16(kf.x * gk * i0, kf.y * gk * i1);
+    } else if (warp == 11) {
+        // ---------------- TMA (one lane) ----------------
+        if (lane == 0) {
+            auto load_g = [&](int n) {
+                mbar_expect_tx(bar(FULL_G + (n & 1)), TILE_G);
+                tma_load_4d(base + OFF_G + (n & 1) * TILE_G, &tm_g, 0, h, n * C, b, bar(FULL_G + (n & 1)));
+            };
+            auto load_k = [&](int n) {
+                const uint32_t bf = bar(FULL_K + n % 3);
+                mbar_expect_tx(bf, TILE_BF16);
+                tma_load_5d(base + OFF_K + (n % 3) * TILE_BF16, &tm_k, 0, n * C, 0, h, b, bf);
+            };
+            auto load_v = [&](int n) {
+                const uint32_t bf = bar(FULL_V + (n & 1));
+                mbar_expect_tx(bf, TILE_BF16);
+                tma_load_5d(base + OFF_V + (n & 1) * TILE_BF16, &tm_v, 0, n * C, 0, h, b, bf);
+            };
+            for (int n = 0; n < 2 && n < p.NT; ++n) load_g(n);
+            for (int n = 0; n < 3 && n < p.NT; ++n) load_k(n);
+            for (int n = 0; n < 2 && n < p.NT; ++n) load_v(n);
+            for (int n = 0; n < p.NT && !failed; ++n) {
+                if (n + 2 < p.NT) {                    // log-decay buffer: free once the prologue of chunk n is done
+                    wait(OPR + n % 3, (n / 3) & 1);
+                    if (failed) break;
+                    load_g(n + 2);
                 }
-                *kp = kv;
+                if (n + 3 < p.NT) {
+                    wait(KFREE + n % 3, (n / 3) & 1);
+                    if (failed) break;
+                    load_k(n + 3);
+                }
+                if (n + 2 < p.NT) {
+                    wait(VFREE + (n & 1), (n >> 1) & 1);
+                    if (failed) break;
+                    load_v(n + 2);
+                }
+                wait_relaxed(STAGED, n & 1);           // image of S_{n+1} is staged
+                if (failed) break;
+                asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                             ::"l"((uint64_t)(img0 + (size_t)(n + 1) * STATE_BF16)), "r"(base + OFF_IMG), "r"(STATE_BF16) : "memory");
+                bulk_commit();
+                bulk_wait_read0();
+                mbar_arrive(bar(STFREE));
             }
-            if (rg == 15) {
-#pragma unroll
-                for (int e = 0; e < 8; ++e) eblast[8 * cj + e] = __expf(bsum[e]);
+            bulk_wait0();
+            if (failed) {   // give loads that are still in flight time to land before shared memory goes away
+                const uint64_t t0 = globaltimer_ns();
+                while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
             }
         }
-        fence_proxy_async();
-        tc_fence_before();
-        __syncthreads();
-
-        if (tid == 0) {
-            tc_fence_after();
-#pragma unroll
-            for (int kk = 0; kk < 4; ++kk)
-                tc_mma_bf16(tmem, desc_mnmajor(st + OFF_K, kk, HALF_BF16), desc_mnmajor(st + OFF_V, kk, HALF_BF16), ID_Z, 1);
-            tc_commit(bar_z);
+    } else if (warp >= 9) {
+        // ---------------- gates (Gk only), up to four chunks ahead ----------------
+        const int t = tid - (NCOMPUTE + 32);
+        for (int n = 0; n < p.NT; ++n) {
+            if (n >= 4) wait_relaxed(GFREE + (n & 3), ((n >> 2) - 1) & 1);
+            if (failed) break;
+            const int cn = min(C, p.T - n * C);
+            gate_s[(n & 3) * C + t] = t < cn ? token_gate_any(p.lk + (tokb + (size_t)n * C + t) * p.H, p.H, h) : 0.f;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(GREADY + (n & 3)));
         }
-        if (!failed && !mbar_wait_bounded(bar_z, ph_z)) failed = true;
-        ph_z ^= 1;
-        tc_fence_after();
-        {   // S_{n+1} = diag(e^{b_last}) (S_n + kh^T V): fp32 back into TMEM, bf16 image into slot n+1
-            const float e = eblast[row];
-            uint8_t *img = img0 + (size_t)(n + 1) * STATE_BF16;
+    } else {
+        // ---------------- compute warps ----------------
+        const uint32_t lane_base = (uint32_t)(32 * (warp & 3)) << 16;
+        const int colhalf = warp >> 2;
+        const int row = 32 * (warp & 3) + lane;
+        {   // S_0: fp32 into TMEM, bf16 image into slot 0
+            const float *src = p.h0 ? p.h0 + ((size_t)bh * D + row) * D + 64 * colhalf : nullptr;
 #pragma unroll
             for (int part = 0; part < 2; ++part) {
                 float v[32];
-                const uint32_t ta = tmem + lane_base + 64 * colhalf + 32 * part;
-                tmem_ld32(ta, v);
-                tmem_wait_ld();
 #pragma unroll
-                for (int j = 0; j < 32; ++j) v[j] *= e;
-                tmem_st32(ta, v);
-                store_state_part(img, row, colhalf, part, v);
+                for (int j = 0; j < 32; ++j) v[j] = src ? src[32 * part + j] : 0.f;
+                tmem_st32(tmem + lane_base + 64 * colhalf + 32 * part, v);
+                store_state_part(img0, row, colhalf, part, v);
             }
             tmem_wait_st();
         }
         tc_fence_before();
-        __syncthreads();
-        tc_fence_after();
+        mbar_arrive(bar(SREADY));
+
+        auto prologue = [&](int n) {
+            wait(GREADY + (n & 3), (n >> 2) & 1);
+            wait(FULL_G + (n & 1), (n >> 1) & 1);
+            wait(FULL_K + n % 3, (n / 3) & 1);
+            chunk_prologue<false, false>(nullptr, sm + OFF_K + (n % 3) * TILE_BF16,
+                                         reinterpret_cast<const float *>(sm + OFF_G + (n & 1) * TILE_G), tot, nullptr,
+                                         gate_s + (n & 3) * C, eblast + (n & 1) * D, nullptr, tid);
+            fence_proxy_async();
+            mbar_arrive(bar(OPR + n % 3));
+            mbar_arrive(bar(GFREE + (n & 3)));
+        };
+        prologue(0);
+        for (int n = 0; n < p.NT; ++n) {
+            if (n + 1 < p.NT) prologue(n + 1);         // overlaps the MMA of chunk n
+            wait(BAR_Z, n & 1);
+            tc_fence_after();
+            {   // S_{n+1} = diag(2^{b_last}) (S_n + kh^T V): fp32 back into TMEM, bf16 image staged for slot n+1
+                const float e = eblast[(n & 1) * D + row];
+                float v0[32], v1[32];
+                const uint32_t ta = tmem + lane_base + 64 * colhalf;
+                tmem_ld32(ta, v0);
+                tmem_ld32(ta + 32, v1);
+                tmem_wait_ld();
+#pragma unroll
+                for (int j = 0; j < 32; ++j) { v0[j] *= e; v1[j] *= e; }
+                tmem_st32(ta, v0);
+                tmem_st32(ta + 32, v1);
+                if (n > 0) wait(STFREE, (n - 1) & 1);  // the previous image has left the staging buffer
+                store_state_part(sm + OFF_IMG, row, colhalf, 0, v0);
+                store_state_part(sm + OFF_IMG, row, colhalf, 1, v1);
+                tmem_wait_st();
+            }
+            fence_proxy_async();
+            tc_fence_before();
+            mbar_arrive(bar(SREADY));
+            mbar_arrive(bar(STAGED));
+        }
     }
     if (failed) atomicExch(p.status, 1);
     tc_fence_before();
@@ -235,32 +263,36 @@ k_gla_states_tc(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
 // ------------------------------------------------------------------------------------------------
 // sweep 2: gradients
 namespace st2 {
-constexpr uint32_t OFF_Q = 0, OFF_K = TILE_BF16, OFF_V = 2 * TILE_BF16, OFF_DO = 3 * TILE_BF16;
-constexpr uint32_t OFF_G = 4 * TILE_BF16;               // fp32 log-decay tile
-constexpr uint32_t OFF_E = OFF_G + TILE_G;              // bf16 e^b, laid out like the q tile
-constexpr uint32_t OFF_S = OFF_E + TILE_BF16;           // bf16 S_n image
-constexpr uint32_t OFF_DZ = OFF_S + STATE_BF16;         // bf16 dZ, same layout
+// two 32 KiB operand buffers that swap roles every chunk: one holds (q, k) -> (qh, kh) -> (dq, dk staged for the
+// store), the other (v, dO); the next chunk's q, k land in the (v, dO) buffer as soon as the MMAs have read it
+constexpr uint32_t OFF_X = 0, OFF_Y = 2 * TILE_BF16;
+constexpr uint32_t OFF_G = 4 * TILE_BF16;               // fp32 log-decay tile (dead after the prologue)
+constexpr uint32_t OFF_E2 = OFF_G + TILE_G;             // [64][128] x (bf16 gq 2^b, bf16 gk 2^-b)
+constexpr uint32_t OFF_S = OFF_E2 + TILE_G;             // bf16 S_n image
+constexpr uint32_t OFF_DZ = OFF_S + STATE_BF16;         // bf16 dZ operand; afterwards the fp32 dlog_decay tile staged for the store
 constexpr uint32_t OFF_A = OFF_DZ + STATE_BF16;         // masked A, [64 rows][128 B]
-constexpr uint32_t OFF_DA = OFF_A + HALF_BF16;          // masked dA
-constexpr uint32_t OFF_TOT = OFF_DA + HALF_BF16;        // [16][128] fp32 partial column sums
-constexpr uint32_t OFF_EB = OFF_TOT + 16 * D * 4;       // [128] exp(b_last)
-constexpr uint32_t OFF_GQ = OFF_EB + D * 4;             // [64] scale*Gq
-constexpr uint32_t OFF_GK = OFF_GQ + C * 4;             // [64] Gk
-constexpr uint32_t OFF_R = OFF_GK + C * 4;              // [2 buffers][2 column halves][128] rowsum(dS*S) partials
+constexpr uint32_t OFF_DA = OFF_A + HALF_BF16;          // masked dA; afterwards A|dA hold the dv tile staged for the store
+constexpr uint32_t OFF_TOT = OFF_DA + HALF_BF16;        // prologue scratch
+constexpr uint32_t OFF_EB = OFF_TOT + TOT_BYTES;        // [128] 2^{b_last}
+constexpr uint32_t OFF_GATE = OFF_EB + D * 4;           // [4][2][64]: scale*Gq, Gk of four chunks
+constexpr uint32_t OFF_R = OFF_GATE + 4 * 2 * C * 4;    // [2 buffers][2 column halves][128] rowsum(dS*S) partials
 constexpr uint32_t OFF_UP = OFF_R + 4 * D * 4;          // [128] suffix total of the upper 32 tokens
 constexpr uint32_t OFF_RED = OFF_UP + D * 4;            // [2][8 warps][32] gate partial sums
-constexpr uint32_t OFF_BAR = OFF_RED + 2 * 8 * 32 * 4;  // g, qk, vdo, s, a, m
-constexpr uint32_t OFF_TMEM = OFF_BAR + 6 * 8;
+constexpr uint32_t OFF_BAR = OFF_RED + 2 * 8 * 32 * 4;
+constexpr uint32_t OFF_TMEM = OFF_BAR + 32 * 8;         // TMEM base address, then the abort flag
 constexpr uint32_t SMEM_BYTES = OFF_TMEM + 16 + 1024;
 constexpr uint32_t COL_DS = 0, COL_A = 128, COL_DA = 192, COL_DQ = 256, COL_DK = 320, COL_DV = 384, TMEM_COLS = 512;
+constexpr int NTHREADS = NCOMPUTE + 32 + NGATE + 32;    // warps 0..7 compute, 8 MMA issue, 9..12 gates, 13 TMA
+enum Bar { FULL_G = 0, FULL_QK, FULL_V, FULL_DO, FULL_S, OPR, GREADY /*[4]*/, GFREE = GREADY + 4 /*[4]*/, ZREADY = GFREE + 4,
+           AREADY, OUT1, OUT2, INIT_DONE, DGFREE, BAR_A, BAR_M1, BAR_M2, DOFREE, INIT_FULL, DRAIN, NBAR };
 static_assert(SMEM_BYTES <= 232448, "shared memory budget");
+static_assert(NBAR <= 32, "barrier slots");
 }  // namespace st2
 
 struct BwdParams {
     const float *lq, *lk, *dht;
     const uint8_t *simg;
-    __nv_bfloat16 *dq, *dk, *dv;
-    float *dg, *pq, *pk, *dh0;     // pq = Gq*dGq, pk = Gk*dGk per (token, head)
+    float *pq, *pk, *dh0;          // pq = Gq*dGq, pk = Gk*dGk per (token, head)
     int *status;
     int T, H, NT;
     float scale;
@@ -283,10 +315,17 @@ __device__ __forceinline__ float warp_transpose_sum(float (&v)[32], int lane) {
     return v[0];
 }
 
-__global__ void __launch_bounds__(256, 1)
+// Chunks in reverse order.  Per chunk n the compute warps run: prologue -> dZ = diag(2^{b_last}) dS_{n+1} -> causal
+// mask of A and dA -> gradient tiles out of TMEM.  The MMA lane issues each product as soon as its operands exist:
+// A, dA and S_n dO^T after the prologue; dZ V^T, dZ^T kh^T and qh^T dO after the dZ pass; only the three products
+// with the masked tiles wait for the mask.  All four gradient tensors leave through staged TMA stores (rows past T
+// are clipped by the tensor map).
+__global__ void __launch_bounds__(st2::NTHREADS, 1)
 k_gla_bwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
              const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
-             const __grid_constant__ CUtensorMap tm_g, BwdParams p) {
+             const __grid_constant__ CUtensorMap tm_g, const __grid_constant__ CUtensorMap tm_dq,
+             const __grid_constant__ CUtensorMap tm_dk, const __grid_constant__ CUtensorMap tm_dv,
+             const __grid_constant__ CUtensorMap tm_dg, BwdParams p) {
     using namespace st2;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -294,403 +333,416 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
     uint8_t *sm = smem_raw + (base - raw);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int bh = blockIdx.x, b = bh / p.H, h = bh % p.H;
-    const uint32_t bar_g = base + OFF_BAR, bar_qk = bar_g + 8, bar_vdo = bar_g + 16, bar_s = bar_g + 24,
-                   bar_a = bar_g + 32, bar_m = bar_g + 40;
+    auto bar = [&](int i) { return base + OFF_BAR + 8u * i; };
     float *tot = reinterpret_cast<float *>(sm + OFF_TOT);
     float *eblast = reinterpret_cast<float *>(sm + OFF_EB);
-    float *gq_s = reinterpret_cast<float *>(sm + OFF_GQ);
-    float *gk_s = reinterpret_cast<float *>(sm + OFF_GK);
+    float *gate_s = reinterpret_cast<float *>(sm + OFF_GATE);
     float *Rs = reinterpret_cast<float *>(sm + OFF_R);
     float *up = reinterpret_cast<float *>(sm + OFF_UP);
     float *red = reinterpret_cast<float *>(sm + OFF_RED);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(sm + OFF_TMEM + 8);
     bool failed = false;
+    auto wait = [&](int i, uint32_t parity) {
+        if (!failed && !mbar_wait_bounded(bar(i), parity, abort_flag)) { failed = true; *abort_flag = 1; }
+    };
+    auto wait_relaxed = [&](int i, uint32_t parity) {
+        if (!failed && !mbar_wait_bounded<128>(bar(i), parity, abort_flag)) { failed = true; *abort_flag = 1; }
+    };
 
     if (tid == 0) {
-        for (int i = 0; i < 6; ++i) mbar_init(bar_g + 8 * i, 1);
+        *abort_flag = 0;
+        for (int i = 0; i < NBAR; ++i) {
+            const bool all = i == OPR || (i >= GFREE && i <= INIT_DONE);
+            mbar_init(bar(i), all ? NCOMPUTE : (i >= GREADY && i < GFREE) ? NGATE / 32 : 1);
+        }
         fence_mbar_init();
         tma_prefetch_desc(&tm_q);
         tma_prefetch_desc(&tm_k);
         tma_prefetch_desc(&tm_v);
         tma_prefetch_desc(&tm_do);
         tma_prefetch_desc(&tm_g);
+        tma_prefetch_desc(&tm_dq);
+        tma_prefetch_desc(&tm_dk);
+        tma_prefetch_desc(&tm_dv);
+        tma_prefetch_desc(&tm_dg);
     }
     if (warp == 0) tmem_alloc(base + OFF_TMEM, TMEM_COLS);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *reinterpret_cast<volatile uint32_t *>(sm + OFF_TMEM);
-    const uint32_t lane_base = (uint32_t)(32 * (warp & 3)) << 16;
-    const int wh = warp >> 2;                       // column half (state passes) / token half (gradient tiles)
-    const int row = 32 * (warp & 3) + lane;         // TMEM lane = key (value) dimension owned by this thread
+    const size_t tokb = (size_t)b * p.T;
     const uint8_t *img0 = p.simg + (size_t)bh * (p.NT + 1) * STATE_BF16;
-    uint32_t ph_g = 0, ph_qk = 0, ph_vdo = 0, ph_s = 0, ph_a = 0, ph_m = 0;
+    const int NT = p.NT;
+    // chunks are visited in the order n = NT-1 ... 0; k = NT-1-n is the visit number that drives every barrier parity
 
-    auto issue_g = [&](int n) {
-        mbar_expect_tx(bar_g, TILE_G);
-        tma_load_4d(base + OFF_G, &tm_g, 0, h, n * C, b, bar_g);
-    };
-    auto issue_rest = [&](int n) {
-        const int t0 = n * C;
-        mbar_expect_tx(bar_qk, 2 * TILE_BF16);
-        tma_load_4d(base + OFF_Q, &tm_q, 0, h, t0, b, bar_qk);
-        tma_load_4d(base + OFF_Q + HALF_BF16, &tm_q, 64, h, t0, b, bar_qk);
-        tma_load_4d(base + OFF_K, &tm_k, 0, h, t0, b, bar_qk);
-        tma_load_4d(base + OFF_K + HALF_BF16, &tm_k, 64, h, t0, b, bar_qk);
-        mbar_expect_tx(bar_vdo, 2 * TILE_BF16);
-        tma_load_4d(base + OFF_V, &tm_v, 0, h, t0, b, bar_vdo);
-        tma_load_4d(base + OFF_V + HALF_BF16, &tm_v, 64, h, t0, b, bar_vdo);
-        tma_load_4d(base + OFF_DO, &tm_do, 0, h, t0, b, bar_vdo);
-        tma_load_4d(base + OFF_DO + HALF_BF16, &tm_do, 64, h, t0, b, bar_vdo);
-        mbar_expect_tx(bar_s, STATE_BF16);
-        bulk_load(base + OFF_S, img0 + (size_t)n * STATE_BF16, STATE_HALF, bar_s);
-        bulk_load(base + OFF_S + STATE_HALF, img0 + (size_t)n * STATE_BF16 + STATE_HALF, STATE_HALF, bar_s);
-    };
-
-    // rowsum(dS * S) over this thread's 64 columns, with dS in registers part by part
-    auto rowdot_part = [&](const float (&v)[32], int part) {
-        float acc = 0.f;
+    if (warp == 8) {
+        // ---------------- MMA issue (one lane) ----------------
+        if (lane == 0) {
+            constexpr uint32_t ID_A = idesc_bf16(64, 64, 0, 0);
+            constexpr uint32_t ID_KK = idesc_bf16(128, 64, 0, 0), ID_MK = idesc_bf16(128, 64, 1, 0),
+                               ID_MM = idesc_bf16(128, 64, 1, 1), ID_S = idesc_bf16(128, 128, 1, 1);
+            const uint64_t kS = desc_kmajor(base + OFF_S), kDZ = desc_kmajor(base + OFF_DZ),
+                           mDZ = desc_mnmajor(base + OFF_DZ, STATE_HALF), mA = desc_mnmajor(base + OFF_A, HALF_BF16),
+                           kDA = desc_kmajor(base + OFF_DA), mDA = desc_mnmajor(base + OFF_DA, HALF_BF16);
+            for (int k = 0; k < NT; ++k) {
+                const uint32_t par = k & 1;
+                const uint32_t sQ = base + ((k & 1) ? OFF_Y : OFF_X), sK = sQ + TILE_BF16;
+                const uint32_t sV = base + ((k & 1) ? OFF_X : OFF_Y), sDO = sV + TILE_BF16;
+                const uint64_t kQ = desc_kmajor(sQ), kK = desc_kmajor(sK), kV = desc_kmajor(sV), kDO = desc_kmajor(sDO),
+                               mQ = desc_mnmajor(sQ, HALF_BF16), mK = desc_mnmajor(sK, HALF_BF16),
+                               mDO = desc_mnmajor(sDO, HALF_BF16);
+                wait(OPR, par);                        // qh, kh in place
+                wait(FULL_V, par);
+                wait(FULL_DO, par);
+                if (failed) break;
+                tc_fence_after();
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            const uint4 w = *reinterpret_cast<const uint4 *>(sm + OFF_S + wh * STATE_HALF + swz(row, 4 * part + c));
-            const uint32_t *ww = reinterpret_cast<const uint32_t *>(&w);
+                for (int kk = 0; kk < 8; ++kk)         // A = qh kh^T
+                    tc_mma_bf16(tmem + COL_A, kQ + kstep_kmajor(kk, HALF_BF16), kK + kstep_kmajor(kk, HALF_BF16), ID_A, kk > 0);
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const float2 sf = unpack_bf16(ww[e]);
-                acc = fmaf(v[8 * c + 2 * e], sf.x, acc);
-                acc = fmaf(v[8 * c + 2 * e + 1], sf.y, acc);
+                for (int kk = 0; kk < 8; ++kk)         // dA = dO V^T
+                    tc_mma_bf16(tmem + COL_DA, kDO + kstep_kmajor(kk, HALF_BF16), kV + kstep_kmajor(kk, HALF_BF16), ID_A, kk > 0);
+                tc_commit(bar(BAR_A));
+                if (k > 0) wait(OUT1, (k - 1) & 1);    // dqh^T, dkh^T of the previous chunk have been read out
+                wait(FULL_S, par);
+                if (failed) break;
+                tc_fence_after();
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk)         // dqh^T = S_n dO^T ...
+                    tc_mma_bf16(tmem + COL_DQ, kS + kstep_kmajor(kk, STATE_HALF), kDO + kstep_kmajor(kk, HALF_BF16), ID_KK, kk > 0);
+                if (k > 0) wait(OUT2, (k - 1) & 1);    // dV^T and dS of the previous chunk have been read out
+                wait(ZREADY, par);                     // dZ: fp32 in TMEM, bf16 in shared memory
+                if (failed) break;
+                tc_fence_after();
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk)         // dkh^T = dZ V^T ...
+                    tc_mma_bf16(tmem + COL_DK, kDZ + kstep_kmajor(kk, STATE_HALF), kV + kstep_kmajor(kk, HALF_BF16), ID_KK, kk > 0);
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk)         // dV^T = dZ^T kh^T ...
+                    tc_mma_bf16(tmem + COL_DV, mDZ + kstep_mnmajor(kk), kK + kstep_kmajor(kk, HALF_BF16), ID_MK, kk > 0);
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)         // dS_n = dZ + qh^T dO
+                    tc_mma_bf16(tmem + COL_DS, mQ + kstep_mnmajor(kk), mDO + kstep_mnmajor(kk), ID_S, 1);
+                wait(AREADY, par);                     // masked A, dA in shared memory
+                if (failed) break;
+                tc_fence_after();
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)         // ... + kh^T dA^T
+                    tc_mma_bf16(tmem + COL_DQ, mK + kstep_mnmajor(kk), kDA + kstep_kmajor(kk, 0), ID_MK, 1);
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)         // ... + qh^T dA
+                    tc_mma_bf16(tmem + COL_DK, mQ + kstep_mnmajor(kk), mDA + kstep_mnmajor(kk), ID_MM, 1);
+                tc_commit(bar(BAR_M1));
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)         // ... + dO^T A
+                    tc_mma_bf16(tmem + COL_DV, mDO + kstep_mnmajor(kk), mA + kstep_mnmajor(kk), ID_MM, 1);
+                tc_commit(bar(BAR_M2));
+                tc_commit(bar(DOFREE));                // (same event, for the TMA lane)
+            }
+            tc_commit(bar(DRAIN));
+            mbar_wait_bounded(bar(DRAIN), 0, nullptr, 20000000ull);
+        }
+    } else if (warp == 13) {
+        // ---------------- TMA (one lane) ----------------
+        if (lane == 0) {
+            auto load_g = [&](int n) {
+                mbar_expect_tx(bar(FULL_G), TILE_G);
+                tma_load_4d(base + OFF_G, &tm_g, 0, h, n * C, b, bar(FULL_G));
+            };
+            // visit k keeps (q, k) in buffer k&1 and (v, dO) in the other one
+            auto load_qk = [&](int n, int k) {
+                const uint32_t dst = base + ((k & 1) ? OFF_Y : OFF_X);
+                mbar_expect_tx(bar(FULL_QK), 2 * TILE_BF16);
+                tma_load_5d(dst, &tm_q, 0, n * C, 0, h, b, bar(FULL_QK));
+                tma_load_5d(dst + TILE_BF16, &tm_k, 0, n * C, 0, h, b, bar(FULL_QK));
+            };
+            auto load_vdo = [&](int n, int k) {
+                const uint32_t dst = base + ((k & 1) ? OFF_X : OFF_Y);
+                mbar_expect_tx(bar(FULL_V), TILE_BF16);
+                tma_load_5d(dst, &tm_v, 0, n * C, 0, h, b, bar(FULL_V));
+                mbar_expect_tx(bar(FULL_DO), TILE_BF16);
+                tma_load_5d(dst + TILE_BF16, &tm_do, 0, n * C, 0, h, b, bar(FULL_DO));
+            };
+            auto load_s = [&](int n) {
+                mbar_expect_tx(bar(FULL_S), STATE_BF16);
+                bulk_load(base + OFF_S, img0 + (size_t)n * STATE_BF16, STATE_BF16, bar(FULL_S));
+            };
+            if (p.dht) {                               // S_NT, for rowsum(dht * S_NT)
+                mbar_expect_tx(bar(INIT_FULL), STATE_BF16);
+                bulk_load(base + OFF_S, img0 + (size_t)NT * STATE_BF16, STATE_BF16, bar(INIT_FULL));
+            }
+            load_g(NT - 1);
+            load_qk(NT - 1, 0);
+            load_vdo(NT - 1, 0);
+            if (p.dht) wait(INIT_DONE, 0);             // the compute warps are done with S_NT
+            if (!failed) load_s(NT - 1);
+            for (int k = 0; k < NT && !failed; ++k) {
+                const int n = NT - 1 - k;
+                const uint32_t par = k & 1;
+                const uint32_t sQK = base + ((k & 1) ? OFF_Y : OFF_X);
+                if (n > 0) {
+                    wait(OPR, par);                    // prologue done: the log-decay buffer is free
+                    if (failed) break;
+                    load_g(n - 1);
+                    wait(DOFREE, par);                 // every MMA of the chunk is done: its (v, dO) buffer takes the next q, k
+                    if (failed) break;
+                    load_qk(n - 1, k + 1);
+                }
+                wait_relaxed(OUT1, par);               // dq, dk staged over qh, kh
+                if (failed) break;
+                tma_store_5d(&tm_dq, sQK, 0, n * C, 0, h, b);
+                tma_store_5d(&tm_dk, sQK + TILE_BF16, 0, n * C, 0, h, b);
+                bulk_commit();
+                bulk_wait_read0();
+                if (n > 0) load_vdo(n - 1, k + 1);     // ... and this buffer takes the next v, dO
+                wait_relaxed(OUT2, par);               // dv, dlog_decay staged; S_n no longer needed
+                if (failed) break;
+                tma_store_5d(&tm_dv, base + OFF_A, 0, n * C, 0, h, b);
+                tma_store_4d(&tm_dg, base + OFF_DZ, 0, h, n * C, b);
+                bulk_commit();
+                if (n > 0) load_s(n - 1);
+                bulk_wait_read0();
+                mbar_arrive(bar(DGFREE));
+            }
+            bulk_wait0();
+            if (failed) {
+                const uint64_t t0 = globaltimer_ns();
+                while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
             }
         }
-        return acc;
-    };
-
-    const int nlast = p.NT - 1;
-    if (tid == 0) issue_g(nlast);
-    {   // dS_NT = dht (or zero) into TMEM; R_{NT-1} = rowsum(dht * S_NT)
-        float rpart = 0.f;
-        if (p.dht) {
-            if (tid == 0) {
-                mbar_expect_tx(bar_s, STATE_BF16);
-                bulk_load(base + OFF_S, img0 + (size_t)p.NT * STATE_BF16, STATE_HALF, bar_s);
-                bulk_load(base + OFF_S + STATE_HALF, img0 + (size_t)p.NT * STATE_BF16 + STATE_HALF, STATE_HALF, bar_s);
-            }
-            if (!mbar_wait_bounded(bar_s, ph_s)) failed = true;
-            ph_s ^= 1;
+    } else if (warp >= 9) {
+        // ---------------- gates, up to four chunks ahead ----------------
+        const int g = tid - (NCOMPUTE + 32), t = g & (C - 1);
+        const float *l = g < C ? p.lq : p.lk;
+        const float mult = g < C ? p.scale : 1.f;
+        for (int k = 0; k < NT; ++k) {
+            const int n = NT - 1 - k;
+            if (k >= 4) wait_relaxed(GFREE + (k & 3), ((k >> 2) - 1) & 1);
+            if (failed) break;
+            const int cn = min(C, p.T - n * C);
+            gate_s[(k & 3) * 2 * C + g] = t < cn ? mult * token_gate_any(l + (tokb + (size_t)n * C + t) * p.H, p.H, h) : 0.f;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(GREADY + (k & 3)));
         }
-        const float *src = p.dht ? p.dht + ((size_t)bh * D + row) * D + 64 * wh : nullptr;
-#pragma unroll
-        for (int part = 0; part < 2; ++part) {
-            float v[32];
-#pragma unroll
-            for (int j = 0; j < 32; ++j) v[j] = src ? src[32 * part + j] : 0.f;
-            tmem_st32(tmem + lane_base + COL_DS + 64 * wh + 32 * part, v);
-            if (p.dht) rpart += rowdot_part(v, part);
-        }
-        tmem_wait_st();
-        Rs[(nlast & 1) * 2 * D + wh * D + row] = rpart;
-    }
-    tc_fence_before();
-    __syncthreads();
-    if (tid == 0) issue_rest(nlast);
+    } else {
+        // ---------------- compute warps ----------------
+        const uint32_t lane_base = (uint32_t)(32 * (warp & 3)) << 16;
+        const int wh = warp >> 2;                       // column half (state passes) / token half (gradient tiles)
+        const int row = 32 * (warp & 3) + lane;         // TMEM lane = key (value) dimension owned by this thread
 
-    constexpr uint32_t ID_A = idesc_bf16(64, 64, 0, 0);
-    const int rg = tid >> 4, cj = tid & 15;
-
-    for (int n = nlast; n >= 0; --n) {
-        const int t0 = n * C, cn = min(C, p.T - t0);
-        SLA_TS(0);
-        if (tid < C) {   // head-softmax gates of this chunk's tokens (Eq. 4)
-            float gq = 0.f, gk = 0.f;
-            if (tid < cn) {
-                const size_t tok = (size_t)b * p.T + t0 + tid;
-                const float2 g = head_gates(p.lq + tok * p.H, p.lk + tok * p.H, p.H, h);
-                gq = p.scale * g.x;
-                gk = g.y;
-            }
-            gq_s[tid] = gq;
-            gk_s[tid] = gk;
-        }
-        if (!failed && !mbar_wait_bounded(bar_g, ph_g)) failed = true;
-        ph_g ^= 1;
-        if (!failed && !mbar_wait_bounded(bar_qk, ph_qk)) failed = true;
-        ph_qk ^= 1;
-        SLA_TS(1);
-
-        // cumulative log-decay; qh, kh in place; e^b kept as bf16 for the epilogue
-        const float *gs = reinterpret_cast<const float *>(sm + OFF_G);
-        {
-            float acc[8];
+        // rowsum(dS * S) over this thread's 64 columns, with dS in registers part by part
+        auto rowdot_part = [&](const float (&v)[32], int part) {
+            float acc = 0.f;
 #pragma unroll
-            for (int e = 0; e < 8; ++e) acc[e] = 0.f;
-#pragma unroll
-            for (int rr = 0; rr < 4; ++rr) {
-                const float4 g0 = *reinterpret_cast<const float4 *>(gs + (4 * rg + rr) * D + 8 * cj);
-                const float4 g1 = *reinterpret_cast<const float4 *>(gs + (4 * rg + rr) * D + 8 * cj + 4);
-                acc[0] += g0.x; acc[1] += g0.y; acc[2] += g0.z; acc[3] += g0.w;
-                acc[4] += g1.x; acc[5] += g1.y; acc[6] += g1.z; acc[7] += g1.w;
-            }
-            *reinterpret_cast<float4 *>(tot + rg * D + 8 * cj) = make_float4(acc[0], acc[1], acc[2], acc[3]);
-            *reinterpret_cast<float4 *>(tot + rg * D + 8 * cj + 4) = make_float4(acc[4], acc[5], acc[6], acc[7]);
-        }
-        __syncthreads();
-        {
-            float bsum[8];
-#pragma unroll
-            for (int e = 0; e < 8; ++e) bsum[e] = 0.f;
-            for (int g = 0; g < rg; ++g) {
-                const float4 a0 = *reinterpret_cast<const float4 *>(tot + g * D + 8 * cj);
-                const float4 a1 = *reinterpret_cast<const float4 *>(tot + g * D + 8 * cj + 4);
-                bsum[0] += a0.x; bsum[1] += a0.y; bsum[2] += a0.z; bsum[3] += a0.w;
-                bsum[4] += a1.x; bsum[5] += a1.y; bsum[6] += a1.z; bsum[7] += a1.w;
-            }
-            const uint32_t half = cj >> 3, chunk = cj & 7;
-#pragma unroll
-            for (int rr = 0; rr < 4; ++rr) {
-                const int r = 4 * rg + rr;
-                const float4 g0 = *reinterpret_cast<const float4 *>(gs + r * D + 8 * cj);
-                const float4 g1 = *reinterpret_cast<const float4 *>(gs + r * D + 8 * cj + 4);
-                bsum[0] += g0.x; bsum[1] += g0.y; bsum[2] += g0.z; bsum[3] += g0.w;
-                bsum[4] += g1.x; bsum[5] += g1.y; bsum[6] += g1.z; bsum[7] += g1.w;
-                const float gq = gq_s[r], gk = gk_s[r];
-                const uint32_t off = half * HALF_BF16 + swz(r, chunk);
-                uint4 *qp = reinterpret_cast<uint4 *>(sm + OFF_Q + off);
-                uint4 *kp = reinterpret_cast<uint4 *>(sm + OFF_K + off);
-                uint4 qv = *qp, kv = *kp, ev;
-                uint32_t *qw = reinterpret_cast<uint32_t *>(&qv), *kw = reinterpret_cast<uint32_t *>(&kv);
-                uint32_t *ew = reinterpret_cast<uint32_t *>(&ev);
+            for (int c = 0; c < 4; ++c) {
+                const uint4 w = *reinterpret_cast<const uint4 *>(sm + OFF_S + wh * STATE_HALF + swz(row, 4 * part + c));
+                const uint32_t *ww = reinterpret_cast<const uint32_t *>(&w);
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                    const float e0 = __expf(bsum[2 * e]), e1 = __expf(bsum[2 * e + 1]);
-                    const float i0 = __expf(-bsum[2 * e]), i1 = __expf(-bsum[2 * e + 1]);
-                    float2 qf = unpack_bf16(qw[e]), kf = unpack_bf16(kw[e]);
-                    qw[e] = pack_bf16(qf.x * gq * e0, qf.y * gq * e1);
-                    kw[e] = pack_bf16(kf.x * gk * i0, kf.y * gk * i1);
-                    ew[e] = pack_bf16(e0, e1);
+                    const float2 sf = unpack_bf16(ww[e]);
+                    acc = fmaf(v[8 * c + 2 * e], sf.x, acc);
+                    acc = fmaf(v[8 * c + 2 * e + 1], sf.y, acc);
                 }
-                *qp = qv;
-                *kp = kv;
-                *reinterpret_cast<uint4 *>(sm + OFF_E + off) = ev;
             }
-            if (rg == 15) {
-#pragma unroll
-                for (int e = 0; e < 8; ++e) eblast[8 * cj + e] = __expf(bsum[e]);
-            }
-        }
-        fence_proxy_async();
-        tc_fence_before();
-        __syncthreads();
-        SLA_TS(2);
+            return acc;
+        };
 
-        if (tid == 0) {
-            if (n > 0) issue_g(n - 1);       // the log-decay tile is consumed: fetch the next one early
-            if (!failed && !mbar_wait_bounded(bar_vdo, ph_vdo)) failed = true;
-            tc_fence_after();
-#pragma unroll
-            for (int kk = 0; kk < 8; ++kk)   // A = qh kh^T
-                tc_mma_bf16(tmem + COL_A, desc_kmajor(base + OFF_Q, kk, HALF_BF16), desc_kmajor(base + OFF_K, kk, HALF_BF16),
-                            ID_A, kk > 0);
-#pragma unroll
-            for (int kk = 0; kk < 8; ++kk)   // dA = dO V^T
-                tc_mma_bf16(tmem + COL_DA, desc_kmajor(base + OFF_DO, kk, HALF_BF16), desc_kmajor(base + OFF_V, kk, HALF_BF16),
-                            ID_A, kk > 0);
-            tc_commit(bar_a);
-        }
-        ph_vdo ^= 1;
-
-        {   // dZ = diag(e^{b_last}) dS_{n+1}: fp32 back into TMEM (dS_n accumulates on it), bf16 operand copy
-            const float e = eblast[row];
+        {   // dS_NT = dht (or zero) into TMEM; R_{NT-1} = rowsum(dht * S_NT)
+            float rpart = 0.f;
+            if (p.dht) wait(INIT_FULL, 0);
+            const float *src = p.dht ? p.dht + ((size_t)bh * D + row) * D + 64 * wh : nullptr;
 #pragma unroll
             for (int part = 0; part < 2; ++part) {
                 float v[32];
-                const uint32_t ta = tmem + lane_base + COL_DS + 64 * wh + 32 * part;
-                tmem_ld32(ta, v);
-                tmem_wait_ld();
 #pragma unroll
-                for (int j = 0; j < 32; ++j) v[j] *= e;
-                tmem_st32(ta, v);
-                store_state_part(sm + OFF_DZ, row, wh, part, v);
+                for (int j = 0; j < 32; ++j) v[j] = src ? src[32 * part + j] : 0.f;
+                tmem_st32(tmem + lane_base + COL_DS + 64 * wh + 32 * part, v);
+                if (p.dht) rpart += rowdot_part(v, part);
             }
             tmem_wait_st();
+            Rs[((NT - 1) & 1) * 2 * D + wh * D + row] = rpart;
+            if (p.dht) mbar_arrive(bar(INIT_DONE));     // S_NT is no longer needed
         }
-        SLA_TS(3);
 
-        // A, dA: TMEM -> causal mask -> bf16 -> shared memory (row i of an M=64 tile sits in lane 32*(i/16) + i%16)
-        if (!failed && !mbar_wait_bounded(bar_a, ph_a)) failed = true;
-        ph_a ^= 1;
-        tc_fence_after();
-        SLA_TS(4);
-        {
-            const int i = 16 * (warp & 3) + lane;
-            const uint32_t col = wh ? COL_DA : COL_A;
-            uint8_t *dst = sm + (wh ? OFF_DA : OFF_A);
+        for (int k = 0; k < NT; ++k) {
+            const int n = NT - 1 - k, t0 = n * C;
+            const uint32_t par = k & 1;
+            uint8_t *qk = sm + ((k & 1) ? OFF_Y : OFF_X);          // this chunk's q, k tiles
+            SLA_TS(0);
+            // ---- prologue: cumulative decay, qh, kh in place, the (gq 2^b, gk 2^-b) tile ----
+            wait(GREADY + (k & 3), (k >> 2) & 1);
+            wait(FULL_G, par);
+            wait(FULL_QK, par);
+            SLA_TS(1);
+            {
+                const float *g = gate_s + (k & 3) * 2 * C;
+                chunk_prologue<true, true>(qk, qk + TILE_BF16, reinterpret_cast<const float *>(sm + OFF_G), tot, g, g + C,
+                                           eblast, sm + OFF_E2, tid);
+            }
+            fence_proxy_async();
+            mbar_arrive(bar(OPR));
+            mbar_arrive(bar(GFREE + (k & 3)));
+            SLA_TS(2);
+
+            // ---- dZ = diag(2^{b_last}) dS_{n+1}: fp32 back into TMEM (dS_n accumulates on it), bf16 operand copy ----
+            named_bar_sync(1, NCOMPUTE);                // eblast of this chunk is complete
+            if (k > 0) wait(DGFREE, (k - 1) & 1);       // the staged tiles of the previous chunk have left dZ and A|dA
+            {
+                const float e = eblast[row];
+                float v0[32], v1[32];
+                const uint32_t ta = tmem + lane_base + COL_DS + 64 * wh;
+                tmem_ld32(ta, v0);
+                tmem_ld32(ta + 32, v1);
+                tmem_wait_ld();
 #pragma unroll
-            for (int part = 0; part < 2; ++part) {
-                float v[32];
-                tmem_ld32(tmem + lane_base + col + 32 * part, v);
+                for (int j = 0; j < 32; ++j) { v0[j] *= e; v1[j] *= e; }
+                tmem_st32(ta, v0);
+                tmem_st32(ta + 32, v1);
+                store_state_part(sm + OFF_DZ, row, wh, 0, v0);
+                store_state_part(sm + OFF_DZ, row, wh, 1, v1);
+                tmem_wait_st();
+            }
+            fence_proxy_async();
+            tc_fence_before();
+            mbar_arrive(bar(ZREADY));
+            SLA_TS(3);
+
+            // ---- A, dA: TMEM -> causal mask -> bf16 -> shared memory (row i of an M=64 tile sits in lane 32*(i/16) + i%16) ----
+            wait(BAR_A, par);
+            tc_fence_after();
+            SLA_TS(4);
+            {
+                const int i = 16 * (warp & 3) + lane;
+                const uint32_t col = wh ? COL_DA : COL_A;
+                uint8_t *dst = sm + (wh ? OFF_DA : OFF_A);
+                float v0[32], v1[32];
+                tmem_ld32(tmem + lane_base + col, v0);
+                tmem_ld32(tmem + lane_base + col + 32, v1);
                 tmem_wait_ld();
                 if (lane < 16) {
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
-                        const int j0 = 32 * part + 8 * c;
+                        const int j0 = 8 * c;
                         uint4 w;
-                        w.x = pack_bf16(j0 + 0 <= i ? v[8 * c + 0] : 0.f, j0 + 1 <= i ? v[8 * c + 1] : 0.f);
-                        w.y = pack_bf16(j0 + 2 <= i ? v[8 * c + 2] : 0.f, j0 + 3 <= i ? v[8 * c + 3] : 0.f);
-                        w.z = pack_bf16(j0 + 4 <= i ? v[8 * c + 4] : 0.f, j0 + 5 <= i ? v[8 * c + 5] : 0.f);
-                        w.w = pack_bf16(j0 + 6 <= i ? v[8 * c + 6] : 0.f, j0 + 7 <= i ? v[8 * c + 7] : 0.f);
-                        *reinterpret_cast<uint4 *>(dst + swz(i, 4 * part + c)) = w;
+                        w.x = pack_bf16(j0 + 0 <= i ? v0[8 * c + 0] : 0.f, j0 + 1 <= i ? v0[8 * c + 1] : 0.f);
+                        w.y = pack_bf16(j0 + 2 <= i ? v0[8 * c + 2] : 0.f, j0 + 3 <= i ? v0[8 * c + 3] : 0.f);
+                        w.z = pack_bf16(j0 + 4 <= i ? v0[8 * c + 4] : 0.f, j0 + 5 <= i ? v0[8 * c + 5] : 0.f);
+                        w.w = pack_bf16(j0 + 6 <= i ? v0[8 * c + 6] : 0.f, j0 + 7 <= i ? v0[8 * c + 7] : 0.f);
+                        *reinterpret_cast<uint4 *>(dst + swz(i, c)) = w;
+                        const int j1 = 32 + 8 * c;
+                        w.x = pack_bf16(j1 + 0 <= i ? v1[8 * c + 0] : 0.f, j1 + 1 <= i ? v1[8 * c + 1] : 0.f);
+                        w.y = pack_bf16(j1 + 2 <= i ? v1[8 * c + 2] : 0.f, j1 + 3 <= i ? v1[8 * c + 3] : 0.f);
+                        w.z = pack_bf16(j1 + 4 <= i ? v1[8 * c + 4] : 0.f, j1 + 5 <= i ? v1[8 * c + 5] : 0.f);
+                        w.w = pack_bf16(j1 + 6 <= i ? v1[8 * c + 6] : 0.f, j1 + 7 <= i ? v1[8 * c + 7] : 0.f);
+                        *reinterpret_cast<uint4 *>(dst + swz(i, 4 + c)) = w;
                     }
                 }
             }
-        }
-        fence_proxy_async();
-        tc_fence_before();
-        __syncthreads();
-        SLA_TS(5);
+            fence_proxy_async();
+            tc_fence_before();
+            mbar_arrive(bar(AREADY));
+            SLA_TS(5);
 
-        if (tid == 0) {
-            if (!failed && !mbar_wait_bounded(bar_s, ph_s)) failed = true;
+            // ---- dqh^T, dkh^T: this thread owns key dimension `row` and tokens 32*wh .. 32*wh+31 ----
+            wait(BAR_M1, par);
             tc_fence_after();
-            const uint32_t sQ = base + OFF_Q, sK = base + OFF_K, sV = base + OFF_V, sDO = base + OFF_DO,
-                           sS = base + OFF_S, sDZ = base + OFF_DZ, sA = base + OFF_A, sDA = base + OFF_DA;
-            // dqh^T = kh^T dA^T + S_n dO^T
+            SLA_TS(6);
+            const float *Rcur = Rs + (n & 1) * 2 * D;
+            float sfx[32];
+            {
+                float dqh[32], dkh[32];
+                tmem_ld32(tmem + lane_base + COL_DQ + 32 * wh, dqh);
+                tmem_ld32(tmem + lane_base + COL_DK + 32 * wh, dkh);
+                tmem_wait_ld();
+                const uint32_t dhalf = (uint32_t)(row >> 6) * HALF_BF16, dchunk = (uint32_t)(row & 63) >> 3, dbyte = (row & 7) * 2;
+                float run = 0.f;
 #pragma unroll
-            for (int kk = 0; kk < 4; ++kk)
-                tc_mma_bf16(tmem + COL_DQ, desc_mnmajor(sK, kk, HALF_BF16), desc_kmajor(sDA, kk, 0),
-                            idesc_bf16(128, 64, 1, 0), kk > 0);
+                for (int ii = 31; ii >= 0; --ii) {
+                    const int i = 32 * wh + ii;
+                    const uint32_t off = dhalf + swz(i, dchunk) + dbyte;
+                    __nv_bfloat16 *qp = reinterpret_cast<__nv_bfloat16 *>(qk + off);
+                    __nv_bfloat16 *kp = reinterpret_cast<__nv_bfloat16 *>(qk + TILE_BF16 + off);
+                    const float2 ee = unpack_bf16(*reinterpret_cast<const uint32_t *>(sm + OFF_E2 + i * (D * 4) + row * 4));
+                    const float pq = __bfloat162float(*qp) * dqh[ii], pk = __bfloat162float(*kp) * dkh[ii];
+                    run += pq - pk;
+                    sfx[ii] = run;
+                    *qp = __float2bfloat16_rn(ee.x * dqh[ii]);       // dq = scale Gq 2^b dqh   (over qh, for the store)
+                    *kp = __float2bfloat16_rn(ee.y * dkh[ii]);       // dk = Gk 2^-b dkh
+                    dqh[ii] = pq;
+                    dkh[ii] = pk;
+                }
+                if (wh == 1) up[row] = run + Rcur[row] + Rcur[D + row];
+                const float sq = warp_transpose_sum(dqh, lane);
+                const float sk = warp_transpose_sum(dkh, lane);
+                red[warp * 32 + lane] = sq;
+                red[8 * 32 + warp * 32 + lane] = sk;
+            }
+            fence_proxy_async();
+            tc_fence_before();
+            mbar_arrive(bar(OUT1));
+            SLA_TS(7);
+
+            // ---- dV^T -> dv tile; R_{n-1} = rowsum(dS_n * S_n); dlog_decay tile; gate products ----
+            wait(BAR_M2, par);
+            tc_fence_after();
+            SLA_TS(8);
+            {
+                float dvt[32];
+                tmem_ld32(tmem + lane_base + COL_DV + 32 * wh, dvt);
+                tmem_wait_ld();
+                const uint32_t dhalf = (uint32_t)(row >> 6) * HALF_BF16, dchunk = (uint32_t)(row & 63) >> 3, dbyte = (row & 7) * 2;
 #pragma unroll
-            for (int kk = 0; kk < 8; ++kk)
-                tc_mma_bf16(tmem + COL_DQ, desc_kmajor(sS, kk, STATE_HALF), desc_kmajor(sDO, kk, HALF_BF16),
-                            idesc_bf16(128, 64, 0, 0), 1);
-            // dkh^T = qh^T dA + dZ V^T
+                for (int ii = 0; ii < 32; ++ii)
+                    *reinterpret_cast<__nv_bfloat16 *>(sm + OFF_A + dhalf + swz(32 * wh + ii, dchunk) + dbyte) =
+                        __float2bfloat16_rn(dvt[ii]);
+            }
+            {
+                float v0[32], v1[32];
+                tmem_ld32(tmem + lane_base + COL_DS + 64 * wh, v0);
+                tmem_ld32(tmem + lane_base + COL_DS + 64 * wh + 32, v1);
+                tmem_wait_ld();
+                Rs[((n & 1) ^ 1) * 2 * D + wh * D + row] = rowdot_part(v0, 0) + rowdot_part(v1, 1);
+            }
+            SLA_TS(9);
+            named_bar_sync(1, NCOMPUTE);                // up, red and the R partials are complete
+            {   // log-decay gradient: in-chunk suffix sum + what flows in from the right of the chunk
+                const float offs = wh == 1 ? Rcur[row] + Rcur[D + row] : up[row];
+                float *dgt = reinterpret_cast<float *>(sm + OFF_DZ);
 #pragma unroll
-            for (int kk = 0; kk < 4; ++kk)
-                tc_mma_bf16(tmem + COL_DK, desc_mnmajor(sQ, kk, HALF_BF16), desc_mnmajor(sDA, kk, HALF_BF16),
-                            idesc_bf16(128, 64, 1, 1), kk > 0);
+                for (int ii = 0; ii < 32; ++ii) dgt[(32 * wh + ii) * D + row] = sfx[ii] + offs;
+            }
+            if (tid < C) {   // Gq*dGq and Gk*dGk of token tid: sum over the four key-dimension quarters
+                const int cn = min(C, p.T - t0);
+                if (tid < cn) {
+                    const int w0 = 4 * (tid >> 5), l = tid & 31;
+                    float sq = 0.f, sk = 0.f;
 #pragma unroll
-            for (int kk = 0; kk < 8; ++kk)
-                tc_mma_bf16(tmem + COL_DK, desc_kmajor(sDZ, kk, STATE_HALF), desc_kmajor(sV, kk, HALF_BF16),
-                            idesc_bf16(128, 64, 0, 0), 1);
-            // dV^T = dO^T A + dZ^T kh^T
-#pragma unroll
-            for (int kk = 0; kk < 4; ++kk)
-                tc_mma_bf16(tmem + COL_DV, desc_mnmajor(sDO, kk, HALF_BF16), desc_mnmajor(sA, kk, HALF_BF16),
-                            idesc_bf16(128, 64, 1, 1), kk > 0);
-#pragma unroll
-            for (int kk = 0; kk < 8; ++kk)
-                tc_mma_bf16(tmem + COL_DV, desc_mnmajor(sDZ, kk, STATE_HALF), desc_kmajor(sK, kk, HALF_BF16),
-                            idesc_bf16(128, 64, 1, 0), 1);
-            // dS_n = dZ + qh^T dO
-#pragma unroll
-            for (int kk = 0; kk < 4; ++kk)
-                tc_mma_bf16(tmem + COL_DS, desc_mnmajor(sQ, kk, HALF_BF16), desc_mnmajor(sDO, kk, HALF_BF16),
-                            idesc_bf16(128, 128, 1, 1), 1);
-            tc_commit(bar_m);
+                    for (int w = 0; w < 4; ++w) {
+                        sq += red[(w0 + w) * 32 + l];
+                        sk += red[8 * 32 + (w0 + w) * 32 + l];
+                    }
+                    p.pq[(tokb + t0 + tid) * p.H + h] = sq;
+                    p.pk[(tokb + t0 + tid) * p.H + h] = sk;
+                }
+            }
+            fence_proxy_async();
+            tc_fence_before();
+            mbar_arrive(bar(OUT2));
+            SLA_TS(10);
         }
-        ph_s ^= 1;
 
-        if (!failed && !mbar_wait_bounded(bar_m, ph_m)) failed = true;
-        ph_m ^= 1;
-        tc_fence_after();
-        SLA_TS(6);
-
-        const float *Rcur = Rs + (n & 1) * 2 * D;
-        {   // R_{n-1} = rowsum(dS_n * S_n), this thread's 64 columns
-            float rpart = 0.f;
+        if (p.dh0) {   // dS_0, fp32 (the last chunk's MMAs were waited for above)
+            float *dst = p.dh0 + ((size_t)bh * D + row) * D + 64 * wh;
 #pragma unroll
             for (int part = 0; part < 2; ++part) {
                 float v[32];
                 tmem_ld32(tmem + lane_base + COL_DS + 64 * wh + 32 * part, v);
                 tmem_wait_ld();
-                rpart += rowdot_part(v, part);
+#pragma unroll
+                for (int j = 0; j < 32; j += 4)
+                    *reinterpret_cast<float4 *>(dst + 32 * part + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
             }
-            Rs[((n & 1) ^ 1) * 2 * D + wh * D + row] = rpart;
-        }
-
-        SLA_TS(7);
-        // gradient tiles: this thread owns key dimension `row` and tokens 32*wh .. 32*wh+31
-        const size_t tok0 = (size_t)b * p.T + t0;
-        float sfx[32];
-        {
-            float dqh[32], dkh[32];
-            tmem_ld32(tmem + lane_base + COL_DQ + 32 * wh, dqh);
-            tmem_ld32(tmem + lane_base + COL_DK + 32 * wh, dkh);
-            tmem_wait_ld();
-            const uint32_t dhalf = (uint32_t)(row >> 6) * HALF_BF16, dchunk = (uint32_t)(row & 63) >> 3, dbyte = (row & 7) * 2;
-            float run = 0.f;
-#pragma unroll
-            for (int ii = 31; ii >= 0; --ii) {
-                const int i = 32 * wh + ii;
-                const uint32_t off = dhalf + swz(i, dchunk) + dbyte;
-                const float qh = __bfloat162float(*reinterpret_cast<const __nv_bfloat16 *>(sm + OFF_Q + off));
-                const float kh = __bfloat162float(*reinterpret_cast<const __nv_bfloat16 *>(sm + OFF_K + off));
-                const float eb = __bfloat162float(*reinterpret_cast<const __nv_bfloat16 *>(sm + OFF_E + off));
-                const float pq = qh * dqh[ii], pk = kh * dkh[ii];
-                run += pq - pk;
-                sfx[ii] = run;
-                if (i < cn) {
-                    const size_t o = ((tok0 + i) * p.H + h) * D + row;
-                    p.dq[o] = __float2bfloat16_rn(gq_s[i] * eb * dqh[ii]);
-                    p.dk[o] = __float2bfloat16_rn(gk_s[i] * __fdividef(dkh[ii], eb));
-                }
-                dqh[ii] = pq;
-                dkh[ii] = pk;
-            }
-            if (wh == 1) up[row] = run + Rcur[row] + Rcur[D + row];
-            const float sq = warp_transpose_sum(dqh, lane);
-            const float sk = warp_transpose_sum(dkh, lane);
-            red[warp * 32 + lane] = sq;
-            red[8 * 32 + warp * 32 + lane] = sk;
-        }
-        SLA_TS(8);
-        {   // dV^T -> dv
-            float dvt[32];
-            tmem_ld32(tmem + lane_base + COL_DV + 32 * wh, dvt);
-            tmem_wait_ld();
-#pragma unroll
-            for (int ii = 0; ii < 32; ++ii) {
-                const int i = 32 * wh + ii;
-                if (i < cn) p.dv[((tok0 + i) * p.H + h) * D + row] = __float2bfloat16_rn(dvt[ii]);
-            }
-        }
-        SLA_TS(9);
-        fence_proxy_async();
-        tc_fence_before();
-        __syncthreads();
-        SLA_TS(10);
-        if (tid == 0 && n > 0) issue_rest(n - 1);      // every operand buffer is free again
-        tc_fence_after();
-        {   // log-decay gradient: in-chunk suffix sum + what flows in from the right of the chunk
-            const float offs = wh == 1 ? Rcur[row] + Rcur[D + row] : up[row];
-#pragma unroll
-            for (int ii = 0; ii < 32; ++ii) {
-                const int i = 32 * wh + ii;
-                if (i < cn) p.dg[((tok0 + i) * p.H + h) * D + row] = sfx[ii] + offs;
-            }
-        }
-        if (tid < C && tid < cn) {   // Gq*dGq and Gk*dGk of token tid: sum over the four key-dimension quarters
-            const int w0 = 4 * (tid >> 5), l = tid & 31;
-            float sq = 0.f, sk = 0.f;
-#pragma unroll
-            for (int w = 0; w < 4; ++w) {
-                sq += red[(w0 + w) * 32 + l];
-                sk += red[8 * 32 + (w0 + w) * 32 + l];
-            }
-            p.pq[(tok0 + tid) * p.H + h] = sq;
-            p.pk[(tok0 + tid) * p.H + h] = sk;
-        }
-        __syncthreads();     // red, up, Rs are rewritten by the next chunk
-        SLA_TS(11);
-    }
-
-    if (p.dh0) {   // dS_0, fp32
-        float *dst = p.dh0 + ((size_t)bh * D + row) * D + 64 * wh;
-#pragma unroll
-        for (int part = 0; part < 2; ++part) {
-            float v[32];
-            tmem_ld32(tmem + lane_base + COL_DS + 64 * wh + 32 * part, v);
-            tmem_wait_ld();
-#pragma unroll
-            for (int j = 0; j < 32; j += 4)
-                *reinterpret_cast<float4 *>(dst + 32 * part + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
         }
     }
     if (failed) atomicExch(p.status, 1);
@@ -745,10 +797,12 @@ int gla_tc_bwd_configure() {
 }
 
 int gla_tc_backward(const Dims &d, const BwdArgs &a, int *status, cudaStream_t st, Tracer &tr) {
-    CUtensorMap mq, mk, mv, mdo, mg;
-    if (!make_map(&mq, a.q, d.B, d.T, d.H, d.dk, false, 64) || !make_map(&mk, a.k, d.B, d.T, d.H, d.dk, false, 64) ||
-        !make_map(&mv, a.v, d.B, d.T, d.H, d.dv, false, 64) || !make_map(&mdo, a.dO, d.B, d.T, d.H, d.dv, false, 64) ||
-        !make_map(&mg, a.log_decay, d.B, d.T, d.H, d.dk, true, 128))
+    CUtensorMap mq, mk, mv, mdo, mg, mdq, mdk, mdv, mdg;
+    if (!make_tile_map(&mq, a.q, d.B, d.T, d.H) || !make_tile_map(&mk, a.k, d.B, d.T, d.H) ||
+        !make_tile_map(&mv, a.v, d.B, d.T, d.H) || !make_tile_map(&mdo, a.dO, d.B, d.T, d.H) ||
+        !make_map(&mg, a.log_decay, d.B, d.T, d.H, d.dk, true, 128) ||
+        !make_tile_map(&mdq, a.dq, d.B, d.T, d.H) || !make_tile_map(&mdk, a.dk, d.B, d.T, d.H) ||
+        !make_tile_map(&mdv, a.dv, d.B, d.T, d.H) || !make_map(&mdg, a.dlog_decay, d.B, d.T, d.H, d.dk, true, 128))
         return -1;
     // workspace: state images, then the two [B,T,H] gate products
     const size_t bth = (size_t)d.B * d.T * d.H;
@@ -758,11 +812,10 @@ int gla_tc_backward(const Dims &d, const BwdArgs &a, int *status, cudaStream_t s
     float *pk = pq + ((bth + 63) & ~(size_t)63);
 
     StatesParams sp{a.lq, a.lk, a.h0, simg, status, d.T, d.H, d.NT};
-    k_gla_states_tc<<<d.B * d.H, 256, st1::SMEM_BYTES, st>>>(mk, mv, mg, sp);
+    k_gla_states_tc<<<d.B * d.H, st1::NTHREADS, st1::SMEM_BYTES, st>>>(mk, mv, mg, sp);
     tr.mark("gla_states_tc");
-    BwdParams bp{a.lq, a.lk, a.dht, simg, (__nv_bfloat16 *)a.dq, (__nv_bfloat16 *)a.dk, (__nv_bfloat16 *)a.dv,
-                 a.dlog_decay, pq, pk, a.dh0, status, d.T, d.H, d.NT, d.scale, gla_tc_phase_ts()};
-    k_gla_bwd_tc<<<d.B * d.H, 256, st2::SMEM_BYTES, st>>>(mq, mk, mv, mdo, mg, bp);
+    BwdParams bp{a.lq, a.lk, a.dht, simg, pq, pk, a.dh0, status, d.T, d.H, d.NT, d.scale, gla_tc_phase_ts()};
+    k_gla_bwd_tc<<<d.B * d.H, st2::NTHREADS, st2::SMEM_BYTES, st>>>(mq, mk, mv, mdo, mg, mdq, mdk, mdv, mdg, bp);
     tr.mark("gla_bwd_tc");
     const long n_tok = (long)d.B * d.T;
     int hp = 1;
