@@ -47,12 +47,20 @@ def measured_peaks():
 
 
 def recorded_traffic(kernel: str):
-    """DRAM bytes per launch from the committed ncu summary, if one covers this kernel."""
+    """DRAM bytes per launch from the committed ncu summary, if one covers this kernel.  The record carries a hash
+    of the kernel sources it was taken on: once they have changed, the figure is stale and None is reported."""
+    import hashlib
     p = ROOT / "profiles" / "dram_traffic.json"
     if not p.exists():
         return None
     try:
-        e = json.loads(p.read_text()).get(kernel)
+        rec = json.loads(p.read_text())
+        h = hashlib.sha256()
+        for f in sorted((ROOT / "paper_2602_01744_b200" / "csrc").glob("*")):
+            h.update(f.read_bytes())
+        if rec.get("source_sha256") != h.hexdigest():
+            return None
+        e = rec.get(kernel)
         return None if e is None else e.get("bytes_per_launch_full_size")
     except Exception:
         return None
