@@ -576,28 +576,40 @@ k_grads_lin(Dims d, const TIO *__restrict__ q, const TIO *__restrict__ k, const 
 }
 
 // ------------------------------------------------------------------------------------------
-// a7: one recurrent step per (sequence, head); the fp32 state is read once and written once.
-// 256 threads: tx = lane owns columns tx+32c of the state, ty = warp owns rows ty, ty+8, ...
+// a7: one recurrent step per (sequence, head); the fp32 state is read once and written once (HBM-bound).
+// 256 threads: warp w owns state rows w, w+8, ...; lane l owns the four columns 4l..4l+3 (one 16-byte access per
+// row, a warp moves one 512-byte row per instruction).  The state loads are issued before anything else so that
+// the gate softmax and the operand set-up run under their latency.
 template <typename TIO>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 2)
 k_decode(Dims d, int Bdec, const TIO *__restrict__ q, const TIO *__restrict__ k,
          const TIO *__restrict__ v, const float *__restrict__ log_decay,
          const float *__restrict__ beta, const float *__restrict__ lq, const float *__restrict__ lk,
          float *__restrict__ state, TIO *__restrict__ o) {
-    __shared__ float qs[128], ks[128], as[128], red[8][128], us[128];
+    __shared__ float qs[128], ks[128], as[128], us[128];
+    __shared__ float4 red[8][32];
     __shared__ float gate[2];
-    int bh = blockIdx.x, b = bh / d.H, h = bh % d.H;
+    const int bh = blockIdx.x, b = bh / d.H, h = bh % d.H;
     const int ty = threadIdx.x >> 5, tx = threadIdx.x & 31;
-    if (threadIdx.x < 64) {       // two warps: gates of this head from the H logits of the token
+    const bool col_ok = 4 * tx < d.dv;
+    float4 *S4 = reinterpret_cast<float4 *>(state + (size_t)bh * d.dk * d.dv);
+    const int ld4 = d.dv >> 2;
+    float4 s[16];
+#pragma unroll
+    for (int r = 0; r < 16; ++r) {
+        const int row = ty + 8 * r;
+        s[r] = (row < d.dk && col_ok) ? S4[(size_t)row * ld4 + tx] : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    if (threadIdx.x < 64) {       // two warps: gates of this head from the H logits of the token (Eq. 4)
         const float *l = (ty == 0 ? lq : lk) + (size_t)b * d.H;
         float x = tx < d.H ? l[tx] : -INFINITY;
         float m = x;
 #pragma unroll
         for (int o2 = 16; o2 > 0; o2 >>= 1) m = fmaxf(m, __shfl_xor_sync(FULL, m, o2));
-        float e = tx < d.H ? expf(x - m) : 0.f, s = e;
+        float e = tx < d.H ? expf(x - m) : 0.f, sum = e;
 #pragma unroll
-        for (int o2 = 16; o2 > 0; o2 >>= 1) s += __shfl_xor_sync(FULL, s, o2);
-        if (tx == h) gate[ty] = e / s;
+        for (int o2 = 16; o2 > 0; o2 >>= 1) sum += __shfl_xor_sync(FULL, sum, o2);
+        if (tx == h) gate[ty] = e / sum;
     }
     __syncthreads();
     const float Gq = gate[0], Gk = gate[1];
@@ -612,58 +624,55 @@ k_decode(Dims d, int Bdec, const TIO *__restrict__ q, const TIO *__restrict__ k,
     for (int j = threadIdx.x; j < d.dv; j += blockDim.x)
         us[j] = (gdn ? Gk : 1.f) * ldf(v, (size_t)bh * d.dv + j);
     __syncthreads();
-    float *S = state + (size_t)bh * d.dk * d.dv;
-    float s[16][4];               // rows ty+8r, columns tx+32c
-    float part[4];
 #pragma unroll
-    for (int c = 0; c < 4; ++c) part[c] = 0.f;
-#pragma unroll
-    for (int r = 0; r < 16; ++r) {
-        int row = ty + 8 * r;
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            int col = tx + 32 * c;
-            float val = 0.f;
-            if (row < d.dk && col < d.dv) val = as[row] * S[(size_t)row * d.dv + col];
-            s[r][c] = val;
-            if (gdn && row < d.dk) part[c] = fmaf(ks[row], val, part[c]);
-        }
+    for (int r = 0; r < 16; ++r) {        // decay: Sbar = diag(a) S
+        const int row = ty + 8 * r;
+        const float a = row < d.dk ? as[row] : 0.f;
+        s[r].x *= a; s[r].y *= a; s[r].z *= a; s[r].w *= a;
     }
     if (gdn) {                    // u = beta (Gk v - k Sbar)
+        float4 part = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-        for (int c = 0; c < 4; ++c) red[ty][tx + 32 * c] = part[c];
+        for (int r = 0; r < 16; ++r) {
+            const int row = ty + 8 * r;
+            const float kr = row < d.dk ? ks[row] : 0.f;
+            part.x = fmaf(kr, s[r].x, part.x); part.y = fmaf(kr, s[r].y, part.y);
+            part.z = fmaf(kr, s[r].z, part.z); part.w = fmaf(kr, s[r].w, part.w);
+        }
+        red[ty][tx] = part;
         __syncthreads();
-        for (int j = threadIdx.x; j < d.dv; j += blockDim.x) {
+        if (threadIdx.x < d.dv) {
+            const int j = threadIdx.x;
             float acc = 0.f;
 #pragma unroll
-            for (int w = 0; w < 8; ++w) acc += red[w][j];
+            for (int w = 0; w < 8; ++w) acc += reinterpret_cast<const float *>(&red[w][j >> 2])[j & 3];
             us[j] = beta[bh] * (us[j] - acc);
         }
         __syncthreads();
     }
+    const float4 u4 = col_ok ? *reinterpret_cast<const float4 *>(&us[4 * tx]) : make_float4(0.f, 0.f, 0.f, 0.f);
+    float4 part = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-    for (int c = 0; c < 4; ++c) part[c] = 0.f;
-#pragma unroll
-    for (int r = 0; r < 16; ++r) {
-        int row = ty + 8 * r;
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            int col = tx + 32 * c;
-            if (row < d.dk && col < d.dv) {
-                float val = fmaf(ks[row], us[col], s[r][c]);
-                S[(size_t)row * d.dv + col] = val;
-                part[c] = fmaf(qs[row], val, part[c]);
-            }
+    for (int r = 0; r < 16; ++r) {        // write: S = Sbar + k^T u ; read: o = q S
+        const int row = ty + 8 * r;
+        if (row < d.dk && col_ok) {
+            const float kr = ks[row], qr = qs[row];
+            float4 val;
+            val.x = fmaf(kr, u4.x, s[r].x); val.y = fmaf(kr, u4.y, s[r].y);
+            val.z = fmaf(kr, u4.z, s[r].z); val.w = fmaf(kr, u4.w, s[r].w);
+            S4[(size_t)row * ld4 + tx] = val;
+            part.x = fmaf(qr, val.x, part.x); part.y = fmaf(qr, val.y, part.y);
+            part.z = fmaf(qr, val.z, part.z); part.w = fmaf(qr, val.w, part.w);
         }
     }
     __syncthreads();
-#pragma unroll
-    for (int c = 0; c < 4; ++c) red[ty][tx + 32 * c] = part[c];
+    red[ty][tx] = part;
     __syncthreads();
-    for (int j = threadIdx.x; j < d.dv; j += blockDim.x) {
+    if (threadIdx.x < d.dv) {
+        const int j = threadIdx.x;
         float acc = 0.f;
 #pragma unroll
-        for (int w = 0; w < 8; ++w) acc += red[w][j];
+        for (int w = 0; w < 8; ++w) acc += reinterpret_cast<const float *>(&red[w][j >> 2])[j & 3];
         stf(o, (size_t)bh * d.dv + j, acc);
     }
 }
