@@ -71,7 +71,8 @@ typedef struct {
 sla_status sla_plan_create(sla_plan **out, const sla_desc *desc);
 sla_status sla_plan_destroy(sla_plan *plan);
 
-/* Bytes of caller-provided scratch that sla_forward / sla_backward need for this plan. */
+/* Bytes of caller-provided scratch that sla_forward / sla_backward need for this plan (it depends on the kernels the
+ * plan selects; 0 means none is needed and the workspace pointer may then be NULL). */
 sla_status sla_plan_workspace_bytes(const sla_plan *plan, size_t *forward_bytes, size_t *backward_bytes);
 
 /* Synchronises with nothing; copies the plan's device status word back (on the legacy default
@@ -164,7 +165,8 @@ sla_status sla_decode_step(sla_plan *plan, int32_t Bdec,
  * routine.  Inputs and outputs are still the caller's, with the meanings, layouts and rules of
  * sla_forward.
  *
- *  - Size limit: if the plan's forward workspace (sla_plan_workspace_bytes) exceeds
+ *  - Size limit: if the forward workspace of the fp32 CUDA-core kernels for this shape (what
+ *    sla_plan_workspace_bytes reports for a plan created with SLA_FLAG_FORCE_GENERIC) exceeds
  *    SLA_NOALLOC_SCRATCH_BYTES the call does nothing and returns SLA_ERR_WORKSPACE.
  *  - First call on a device: looks up the device address of the array (one runtime query, made
  *    with that device current; result cached per device).  Where the CUDA runtime loads modules

@@ -97,6 +97,12 @@ sla_status sla_plan_create(sla_plan **out, const sla_desc *desc) {
     d.scale = desc->scale;
     p->ws = sla::plan_workspace(d);
     p->flags = desc->flags;
+    p->fwd_bytes = p->ws.fwd_floats * sizeof(float);
+    p->bwd_bytes = p->ws.bwd_floats * sizeof(float);
+    if (sla::gla_tc_supported(d) && !(desc->flags & SLA_FLAG_FORCE_GENERIC)) {
+        p->fwd_bytes = sla::gla_tc_forward_workspace_bytes(d);
+        p->bwd_bytes = sla::gla_tc_backward_workspace_bytes(d);
+    }
     p->device = dev;
     p->last_launches = 0;
     p->d_status = nullptr;
@@ -120,8 +126,8 @@ sla_status sla_plan_destroy(sla_plan *plan) {
 
 sla_status sla_plan_workspace_bytes(const sla_plan *plan, size_t *fwd, size_t *bwd) {
     if (!plan) return SLA_ERR_INVALID_ARG;
-    if (fwd) *fwd = plan->ws.fwd_floats * sizeof(float);
-    if (bwd) *bwd = plan->ws.bwd_floats * sizeof(float);
+    if (fwd) *fwd = plan->fwd_bytes;
+    if (bwd) *bwd = plan->bwd_bytes;
     return SLA_OK;
 }
 
@@ -185,7 +191,7 @@ sla_status sla_forward(sla_plan *plan, const void *q, const void *k, const void 
     const void *ptrs[] = {q, k, v, log_decay, beta, gq_logits, gk_logits, h0, o, ht, workspace};
     for (const void *p : ptrs)
         if (!aligned16(p)) return SLA_ERR_INVALID_ARG;
-    if (!workspace || workspace_bytes < plan->ws.fwd_floats * sizeof(float)) return SLA_ERR_WORKSPACE;
+    if (plan->fwd_bytes > 0 && (!workspace || workspace_bytes < plan->fwd_bytes)) return SLA_ERR_WORKSPACE;
     sla::FwdArgs a{q, k, v, log_decay, beta, gq_logits, gk_logits, h0, o, ht, (float *)workspace};
     plan->tracer.start((cudaStream_t)cuda_stream);
     const bool tc = sla::gla_tc_supported(d) && !(plan->flags & SLA_FLAG_FORCE_GENERIC);
@@ -217,7 +223,7 @@ sla_status sla_backward(sla_plan *plan, const void *q, const void *k, const void
                           dlog_decay, dbeta, dgq_logits, dgk_logits, dh0, workspace};
     for (const void *p : ptrs)
         if (!aligned16(p)) return SLA_ERR_INVALID_ARG;
-    if (!workspace || workspace_bytes < plan->ws.bwd_floats * sizeof(float)) return SLA_ERR_WORKSPACE;
+    if (plan->bwd_bytes > 0 && (!workspace || workspace_bytes < plan->bwd_bytes)) return SLA_ERR_WORKSPACE;
     sla::BwdArgs a{q, k, v, log_decay, beta, gq_logits, gk_logits, h0, dO, dht, dq, dk, dv,
                    dlog_decay, dbeta, dgq_logits, dgk_logits, dh0, (float *)workspace};
     plan->tracer.start((cudaStream_t)cuda_stream);

@@ -50,6 +50,7 @@ struct FwdParams {
     float *ht;
     int *status;
     int T, H, NT;
+    int P, L;                       // segments per sequence and chunks per segment (P = 1: L = NT)
     float scale;
     unsigned long long *phase_ts;   // optional: block 0 / thread 0 writes a timestamp at each phase of chunk 8
 };
@@ -71,7 +72,9 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t *sm = smem_raw + (base - raw);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int bh = blockIdx.x, b = bh / p.H, h = bh % p.H;
+    // a sequence may be cut into p.P segments of p.L chunks, one CTA each, every segment starting from its own state
+    const int bh = blockIdx.x / p.P, seg = blockIdx.x % p.P, b = bh / p.H, h = bh % p.H;
+    const int n0 = seg * p.L, NT = min(p.L, p.NT - n0);     // this CTA's chunks: n0 .. n0+NT-1
     auto bar = [&](int i) { return base + OFF_BAR + 8u * i; };
     float *tot = reinterpret_cast<float *>(sm + OFF_TOT);
     float *eblast = reinterpret_cast<float *>(sm + OFF_EB);
@@ -113,7 +116,7 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             constexpr uint32_t ID_A = idesc_bf16(64, 64, 0, 0);      // qh (K-major) x kh (K-major)
             constexpr uint32_t ID_O = idesc_bf16(64, 128, 0, 1);     // qh x S, A x V (B operand MN-major)
             constexpr uint32_t ID_Z = idesc_bf16(128, 128, 1, 1);    // kh^T (MN-major) x V (MN-major)
-            for (int n = 0; n < p.NT; ++n) {
+            for (int n = 0; n < NT; ++n) {
                 const uint32_t par = n & 1;
                 const uint32_t sQ = base + OFF_QK + (n % 3) * QK_BYTES, sK = sQ + TILE_BF16;
                 const uint32_t sV = base + OFF_V + (n & 1) * TILE_BF16;
@@ -153,51 +156,51 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
         if (lane == 0) {
             auto load_g = [&](int n) {
                 mbar_expect_tx(bar(FULL_G), TILE_G);
-                tma_load_4d(base + OFF_G, &tm_g, 0, h, n * C, b, bar(FULL_G));
+                tma_load_4d(base + OFF_G, &tm_g, 0, h, (n0 + n) * C, b, bar(FULL_G));
             };
             auto load_qk = [&](int n) {
                 const uint32_t bf = bar(FULL_QK + n % 3), dst = base + OFF_QK + (n % 3) * QK_BYTES;
                 mbar_expect_tx(bf, QK_BYTES);
-                tma_load_5d(dst, &tm_q, 0, n * C, 0, h, b, bf);
-                tma_load_5d(dst + TILE_BF16, &tm_k, 0, n * C, 0, h, b, bf);
+                tma_load_5d(dst, &tm_q, 0, (n0 + n) * C, 0, h, b, bf);
+                tma_load_5d(dst + TILE_BF16, &tm_k, 0, (n0 + n) * C, 0, h, b, bf);
             };
             auto load_v = [&](int n) {
                 const uint32_t bf = bar(FULL_V + (n & 1)), dst = base + OFF_V + (n & 1) * TILE_BF16;
                 mbar_expect_tx(bf, TILE_BF16);
-                tma_load_5d(dst, &tm_v, 0, n * C, 0, h, b, bf);
+                tma_load_5d(dst, &tm_v, 0, (n0 + n) * C, 0, h, b, bf);
             };
             auto store_o = [&](int m) {                // staged by the compute warps; rows past T are clipped
                 wait_relaxed(OSTAGED, m & 1);
                 if (failed) return;
-                tma_store_5d(&tm_o, base + OFF_OST, 0, m * C, 0, h, b);
+                tma_store_5d(&tm_o, base + OFF_OST, 0, (n0 + m) * C, 0, h, b);
                 bulk_commit();
                 bulk_wait_read0();
                 mbar_arrive(bar(OSFREE));
             };
             load_g(0);
-            for (int n = 0; n < 3 && n < p.NT; ++n) load_qk(n);
-            for (int n = 0; n < 2 && n < p.NT; ++n) load_v(n);
+            for (int n = 0; n < 3 && n < NT; ++n) load_qk(n);
+            for (int n = 0; n < 2 && n < NT; ++n) load_v(n);
             wait(OPR + 0, 0);                          // prologue of chunk 0 done: the log-decay buffer is free
-            if (p.NT > 1 && !failed) load_g(1);
-            for (int n = 0; n < p.NT && !failed; ++n) {
-                if (n + 3 < p.NT) {                    // q/k buffer: free once A, qh S and kh^T V have read it
+            if (NT > 1 && !failed) load_g(1);
+            for (int n = 0; n < NT && !failed; ++n) {
+                if (n + 3 < NT) {                    // q/k buffer: free once A, qh S and kh^T V have read it
                     wait(QKFREE + n % 3, (n / 3) & 1);
                     if (failed) break;
                     load_qk(n + 3);
                 }
-                if (n + 2 < p.NT) {                    // log-decay buffer: free once the prologue of chunk n+1 is done
+                if (n + 2 < NT) {                    // log-decay buffer: free once the prologue of chunk n+1 is done
                     wait(OPR + (n + 1) % 3, ((n + 1) / 3) & 1);
                     if (failed) break;
                     load_g(n + 2);
                 }
-                if (n + 2 < p.NT) {                    // v buffer: free once A V has read it
+                if (n + 2 < NT) {                    // v buffer: free once A V has read it
                     wait(BAR_O + (n & 1), (n >> 1) & 1);
                     if (failed) break;
                     load_v(n + 2);
                 }
                 if (n > 0) store_o(n - 1);
             }
-            if (!failed) store_o(p.NT - 1);
+            if (!failed) store_o(NT - 1);
             bulk_wait0();
             if (failed) {   // give loads that are still in flight time to land before shared memory goes away
                 const uint64_t t0 = globaltimer_ns();
@@ -209,11 +212,11 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
         const int g = tid - (NCOMPUTE + 32), t = g & (C - 1);
         const float *l = g < C ? p.lq : p.lk;
         const float mult = g < C ? p.scale : 1.f;
-        for (int n = 0; n < p.NT; ++n) {
+        for (int n = 0; n < NT; ++n) {
             if (n >= 4) wait_relaxed(GFREE + (n & 3), ((n >> 2) - 1) & 1);
             if (failed) break;
-            const int cn = min(C, p.T - n * C);
-            gate_s[(n & 3) * 2 * C + g] = t < cn ? mult * token_gate_any(l + (tokb + (size_t)n * C + t) * p.H, p.H, h) : 0.f;
+            const int cn = min(C, p.T - (n0 + n) * C);
+            gate_s[(n & 3) * 2 * C + g] = t < cn ? mult * token_gate_any(l + (tokb + (size_t)(n0 + n) * C + t) * p.H, p.H, h) : 0.f;
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(GREADY + (n & 3)));
         }
@@ -224,7 +227,7 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
         const int row = 32 * (warp & 3) + lane;
 
         {   // initial state: fp32 into TMEM, bf16 copy into shared memory (row = key dimension)
-            const float *src = p.h0 ? p.h0 + ((size_t)bh * D + row) * D + 64 * colhalf : nullptr;
+            const float *src = p.h0 ? p.h0 + ((size_t)blockIdx.x * D + row) * D + 64 * colhalf : nullptr;   // one state per CTA
 #pragma unroll
             for (int part = 0; part < 2; ++part) {
                 float v[32];
@@ -297,10 +300,10 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
         };
         prologue(0);
 
-        for (int n = 0; n < p.NT; ++n) {
+        for (int n = 0; n < NT; ++n) {
             const uint32_t par = n & 1;
             SLA_TS(0);
-            if (n + 1 < p.NT) prologue(n + 1);         // overlaps the MMAs of chunk n
+            if (n + 1 < NT) prologue(n + 1);         // overlaps the MMAs of chunk n
             SLA_TS(1);
 
             // A: TMEM -> causal mask -> bf16 -> shared memory (row i of the M=64 tile sits in lane 32*(i/16) + i%16)
@@ -365,9 +368,9 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             if (n > 0) stage_o(n - 1);                 // chunk n-1's output: its MMAs finished long ago
             SLA_TS(6);
         }
-        stage_o(p.NT - 1);
+        stage_o(NT - 1);
 
-        if (p.ht) {   // final state, fp32 (each thread reads back what it wrote in the last rescale)
+        if (p.ht && seg == p.P - 1) {   // final state, fp32 (each thread reads back what it wrote in the last rescale)
             float *dst = p.ht + ((size_t)bh * D + row) * D + 64 * colhalf;
 #pragma unroll
             for (int part = 0; part < 2; ++part) {
@@ -386,8 +389,47 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
     if (warp == 0) tmem_dealloc(tmem, TMEM_COLS);
 }
 
+// Segmented forward, second pass: S_start[p+1] = diag(gam_p) S_start[p] + fin_p along the segments of a sequence
+// (elementwise; thread = four consecutive state entries).  grid (B*H, 16), 256 threads.
+__global__ void k_segment_scan(const float *__restrict__ h0, const float *__restrict__ fin, const float *__restrict__ gam,
+                               float *__restrict__ start, int P) {
+    const int bh = blockIdx.x, e = (blockIdx.y * 256 + threadIdx.x) * 4, row = e / D;
+    float4 S = h0 ? *reinterpret_cast<const float4 *>(h0 + (size_t)bh * D * D + e) : make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int p = 0; p < P; ++p) {
+        const size_t c = (size_t)bh * P + p;
+        *reinterpret_cast<float4 *>(start + c * D * D + e) = S;
+        const float g = gam[c * D + row];
+        const float4 f = *reinterpret_cast<const float4 *>(fin + c * D * D + e);
+        S = make_float4(fmaf(g, S.x, f.x), fmaf(g, S.y, f.y), fmaf(g, S.z, f.z), fmaf(g, S.w, f.w));
+    }
+}
+
 // ---- host side ----
 unsigned long long *g_phase_ts = nullptr;   // set by sla_debug_set_phase_timestamps (profiling aid)
+
+int sm_count() {
+    static int n = 0;
+    if (!n) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+            n = 148;
+    }
+    return n;
+}
+// One CTA per sequence leaves most SMs idle when there are few sequences: then every sequence is cut into P segments
+// of L chunks (at least 8), so that B*H*P comes close to the SM count.
+void choose_segments(const Dims &d, int &P, int &L) {
+    const int BH = d.B * d.H, sms = sm_count();
+    P = 1;
+    L = d.NT;
+    if (BH > 0 && 2 * BH <= sms && d.NT >= 16) {
+        const int want = sms / BH;
+        L = (d.NT + want - 1) / want;
+        if (L < 8) L = 8;
+        P = (d.NT + L - 1) / L;
+    }
+}
 }  // namespace
 
 void gla_tc_set_phase_ts(unsigned long long *p) { g_phase_ts = p; }
@@ -403,16 +445,35 @@ int gla_tc_configure() {
                    cudaSuccess ? 0 : -1;
 }
 
+size_t gla_tc_forward_workspace_bytes(const Dims &d) {
+    int P, L;
+    choose_segments(d, P, L);
+    if (P == 1) return 0;
+    return (size_t)d.B * d.H * P * (2 * D * D + D) * sizeof(float);
+}
+
 int gla_tc_forward(const Dims &d, const FwdArgs &a, int *status, cudaStream_t st, Tracer &tr) {
     CUtensorMap mq, mk, mv, mg, mo;
     if (!make_tile_map(&mq, a.q, d.B, d.T, d.H) || !make_tile_map(&mk, a.k, d.B, d.T, d.H) ||
         !make_tile_map(&mv, a.v, d.B, d.T, d.H) || !make_map(&mg, a.log_decay, d.B, d.T, d.H, d.dk, true, 128) ||
         !make_tile_map(&mo, a.o, d.B, d.T, d.H))
         return -1;
-    FwdParams p{a.lq, a.lk, a.h0, (__nv_bfloat16 *)a.o, a.ht, status, d.T, d.H, d.NT, d.scale, g_phase_ts};
-    k_gla_fwd_tc<<<d.B * d.H, NTHREADS, SMEM_BYTES, st>>>(mq, mk, mv, mg, mo, p);
+    int P, L, launches = 1;
+    choose_segments(d, P, L);
+    const float *h0 = a.h0;
+    if (P > 1) {   // segment summaries from a zero state, scan over the segments, then the segments in parallel
+        const size_t nseg = (size_t)d.B * d.H * P;
+        float *fin = a.ws, *start = fin + nseg * D * D, *gam = start + nseg * D * D;
+        if (gla_tc_segment_summaries(d, a, P, L, fin, gam, status, st, tr) < 0) return -1;
+        k_segment_scan<<<dim3(d.B * d.H, 16), 256, 0, st>>>(a.h0, fin, gam, start, P);
+        tr.mark("segment_scan");
+        h0 = start;
+        launches = 3;
+    }
+    FwdParams p{a.lq, a.lk, h0, (__nv_bfloat16 *)a.o, a.ht, status, d.T, d.H, d.NT, P, L, d.scale, g_phase_ts};
+    k_gla_fwd_tc<<<d.B * d.H * P, NTHREADS, SMEM_BYTES, st>>>(mq, mk, mv, mg, mo, p);
     tr.mark("gla_fwd_tc");
-    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+    return cudaGetLastError() == cudaSuccess ? launches : -1;
 }
 
 }  // namespace sla

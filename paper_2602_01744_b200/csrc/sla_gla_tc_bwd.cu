@@ -51,9 +51,11 @@ static_assert(NBAR <= 32, "barrier slots");
 
 struct StatesParams {
     const float *lq, *lk, *h0;
-    uint8_t *simg;          // [B*H][NT+1][32 KiB] bf16 state images
+    uint8_t *simg;          // [B*H][NT+1][32 KiB] bf16 state images (image mode)
+    float *fin, *gam;       // summary mode: per CTA the state reached from a zero start [128][128] and the total decay [128]
     int *status;
     int T, H, NT;
+    int P, L;               // segments per sequence and chunks per segment (image mode: P = 1, L = NT)
 };
 
 // thread (row, colhalf) holds 32 consecutive state values of its row: bf16 them into the operand image
@@ -70,7 +72,10 @@ __device__ __forceinline__ void store_state_part(uint8_t *img, int row, int colh
 }
 
 // Per chunk: prologue of chunk n+1 (kh only) while the tensor core adds kh^T V of chunk n to S; then S is rescaled in
-// TMEM and its bf16 image goes to global memory through a staged bulk store.
+// TMEM and its bf16 image goes to global memory through a staged bulk store (image mode, for the backward pass).
+// Summary mode (simg == nullptr) serves the segmented forward of long sequences: every CTA runs one segment of a
+// sequence from a zero state and leaves only where it ended and the segment's total decay; a scan over the segments
+// then gives every segment its true starting state.
 __global__ void __launch_bounds__(st1::NTHREADS, 1)
 k_gla_states_tc(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                 const __grid_constant__ CUtensorMap tm_g, StatesParams p) {
@@ -80,7 +85,9 @@ k_gla_states_tc(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t *sm = smem_raw + (base - raw);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int bh = blockIdx.x, b = bh / p.H, h = bh % p.H;
+    const int bh = blockIdx.x / p.P, seg = blockIdx.x % p.P, b = bh / p.H, h = bh % p.H;
+    const int n0 = seg * p.L, NT = min(p.L, p.NT - n0);     // this CTA's chunks: n0 .. n0+NT-1
+    const bool images = p.simg != nullptr;
     auto bar = [&](int i) { return base + OFF_BAR + 8u * i; };
     float *tot = reinterpret_cast<float *>(sm + OFF_TOT);
     float *eblast = reinterpret_cast<float *>(sm + OFF_EB);
@@ -111,13 +118,13 @@ k_gla_states_tc(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
     tc_fence_after();
     const uint32_t tmem = *reinterpret_cast<volatile uint32_t *>(sm + OFF_TMEM);
     const size_t tokb = (size_t)b * p.T;
-    uint8_t *img0 = p.simg + (size_t)bh * (p.NT + 1) * STATE_BF16;
+    uint8_t *img0 = p.simg + (size_t)bh * (NT + 1) * STATE_BF16;      // (image mode: one segment, NT = p.NT)
 
     if (warp == 8) {
         // ---------------- MMA issue (one lane) ----------------
         if (lane == 0) {
             constexpr uint32_t ID_Z = idesc_bf16(128, 128, 1, 1);    // kh^T (MN-major) x V (MN-major)
-            for (int n = 0; n < p.NT; ++n) {
+            for (int n = 0; n < NT; ++n) {
                 const uint32_t sK = base + OFF_K + (n % 3) * TILE_BF16, sV = base + OFF_V + (n & 1) * TILE_BF16;
                 wait(OPR + n % 3, (n / 3) & 1);        // kh of chunk n is in place
                 wait(SREADY, n & 1);                   // S_n is in TMEM
@@ -140,37 +147,38 @@ k_gla_states_tc(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
         if (lane == 0) {
             auto load_g = [&](int n) {
                 mbar_expect_tx(bar(FULL_G + (n & 1)), TILE_G);
-                tma_load_4d(base + OFF_G + (n & 1) * TILE_G, &tm_g, 0, h, n * C, b, bar(FULL_G + (n & 1)));
+                tma_load_4d(base + OFF_G + (n & 1) * TILE_G, &tm_g, 0, h, (n0 + n) * C, b, bar(FULL_G + (n & 1)));
             };
             auto load_k = [&](int n) {
                 const uint32_t bf = bar(FULL_K + n % 3);
                 mbar_expect_tx(bf, TILE_BF16);
-                tma_load_5d(base + OFF_K + (n % 3) * TILE_BF16, &tm_k, 0, n * C, 0, h, b, bf);
+                tma_load_5d(base + OFF_K + (n % 3) * TILE_BF16, &tm_k, 0, (n0 + n) * C, 0, h, b, bf);
             };
             auto load_v = [&](int n) {
                 const uint32_t bf = bar(FULL_V + (n & 1));
                 mbar_expect_tx(bf, TILE_BF16);
-                tma_load_5d(base + OFF_V + (n & 1) * TILE_BF16, &tm_v, 0, n * C, 0, h, b, bf);
+                tma_load_5d(base + OFF_V + (n & 1) * TILE_BF16, &tm_v, 0, (n0 + n) * C, 0, h, b, bf);
             };
-            for (int n = 0; n < 2 && n < p.NT; ++n) load_g(n);
-            for (int n = 0; n < 3 && n < p.NT; ++n) load_k(n);
-            for (int n = 0; n < 2 && n < p.NT; ++n) load_v(n);
-            for (int n = 0; n < p.NT && !failed; ++n) {
-                if (n + 2 < p.NT) {                    // log-decay buffer: free once the prologue of chunk n is done
+            for (int n = 0; n < 2 && n < NT; ++n) load_g(n);
+            for (int n = 0; n < 3 && n < NT; ++n) load_k(n);
+            for (int n = 0; n < 2 && n < NT; ++n) load_v(n);
+            for (int n = 0; n < NT && !failed; ++n) {
+                if (n + 2 < NT) {                    // log-decay buffer: free once the prologue of chunk n is done
                     wait(OPR + n % 3, (n / 3) & 1);
                     if (failed) break;
                     load_g(n + 2);
                 }
-                if (n + 3 < p.NT) {
+                if (n + 3 < NT) {
                     wait(KFREE + n % 3, (n / 3) & 1);
                     if (failed) break;
                     load_k(n + 3);
                 }
-                if (n + 2 < p.NT) {
+                if (n + 2 < NT) {
                     wait(VFREE + (n & 1), (n >> 1) & 1);
                     if (failed) break;
                     load_v(n + 2);
                 }
+                if (!images) continue;
                 wait_relaxed(STAGED, n & 1);           // image of S_{n+1} is staged
                 if (failed) break;
                 asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
@@ -188,11 +196,11 @@ k_gla_states_tc(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
     } else if (warp >= 9) {
         // ---------------- gates (Gk only), up to four chunks ahead ----------------
         const int t = tid - (NCOMPUTE + 32);
-        for (int n = 0; n < p.NT; ++n) {
+        for (int n = 0; n < NT; ++n) {
             if (n >= 4) wait_relaxed(GFREE + (n & 3), ((n >> 2) - 1) & 1);
             if (failed) break;
-            const int cn = min(C, p.T - n * C);
-            gate_s[(n & 3) * C + t] = t < cn ? token_gate_any(p.lk + (tokb + (size_t)n * C + t) * p.H, p.H, h) : 0.f;
+            const int cn = min(C, p.T - (n0 + n) * C);
+            gate_s[(n & 3) * C + t] = t < cn ? token_gate_any(p.lk + (tokb + (size_t)(n0 + n) * C + t) * p.H, p.H, h) : 0.f;
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(GREADY + (n & 3)));
         }
@@ -202,14 +210,14 @@ k_gla_states_tc(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
         const int colhalf = warp >> 2;
         const int row = 32 * (warp & 3) + lane;
         {   // S_0: fp32 into TMEM, bf16 image into slot 0
-            const float *src = p.h0 ? p.h0 + ((size_t)bh * D + row) * D + 64 * colhalf : nullptr;
+            const float *src = (p.h0 && images) ? p.h0 + ((size_t)bh * D + row) * D + 64 * colhalf : nullptr;
 #pragma unroll
             for (int part = 0; part < 2; ++part) {
                 float v[32];
 #pragma unroll
                 for (int j = 0; j < 32; ++j) v[j] = src ? src[32 * part + j] : 0.f;
                 tmem_st32(tmem + lane_base + 64 * colhalf + 32 * part, v);
-                store_state_part(img0, row, colhalf, part, v);
+                if (images) store_state_part(img0, row, colhalf, part, v);
             }
             tmem_wait_st();
         }
@@ -228,12 +236,14 @@ k_gla_states_tc(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
             mbar_arrive(bar(GFREE + (n & 3)));
         };
         prologue(0);
-        for (int n = 0; n < p.NT; ++n) {
-            if (n + 1 < p.NT) prologue(n + 1);         // overlaps the MMA of chunk n
+        float gam = 1.f;                               // product of the chunks' 2^{b_last} for key dimension `row`
+        for (int n = 0; n < NT; ++n) {
+            if (n + 1 < NT) prologue(n + 1);         // overlaps the MMA of chunk n
             wait(BAR_Z, n & 1);
             tc_fence_after();
             {   // S_{n+1} = diag(2^{b_last}) (S_n + kh^T V): fp32 back into TMEM, bf16 image staged for slot n+1
                 const float e = eblast[(n & 1) * D + row];
+                gam *= e;
                 float v0[32], v1[32];
                 const uint32_t ta = tmem + lane_base + 64 * colhalf;
                 tmem_ld32(ta, v0);
@@ -243,9 +253,19 @@ k_gla_states_tc(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
                 for (int j = 0; j < 32; ++j) { v0[j] *= e; v1[j] *= e; }
                 tmem_st32(ta, v0);
                 tmem_st32(ta + 32, v1);
-                if (n > 0) wait(STFREE, (n - 1) & 1);  // the previous image has left the staging buffer
-                store_state_part(sm + OFF_IMG, row, colhalf, 0, v0);
-                store_state_part(sm + OFF_IMG, row, colhalf, 1, v1);
+                if (images) {
+                    if (n > 0) wait(STFREE, (n - 1) & 1);  // the previous image has left the staging buffer
+                    store_state_part(sm + OFF_IMG, row, colhalf, 0, v0);
+                    store_state_part(sm + OFF_IMG, row, colhalf, 1, v1);
+                } else if (n == NT - 1) {              // summary mode: where the segment ended, fp32
+                    float *dst = p.fin + ((size_t)blockIdx.x * D + row) * D + 64 * colhalf;
+#pragma unroll
+                    for (int j = 0; j < 32; j += 4) {
+                        *reinterpret_cast<float4 *>(dst + j) = make_float4(v0[j], v0[j + 1], v0[j + 2], v0[j + 3]);
+                        *reinterpret_cast<float4 *>(dst + 32 + j) = make_float4(v1[j], v1[j + 1], v1[j + 2], v1[j + 3]);
+                    }
+                    if (colhalf == 0) p.gam[(size_t)blockIdx.x * D + row] = gam;
+                }
                 tmem_wait_st();
             }
             fence_proxy_async();
@@ -796,6 +816,23 @@ int gla_tc_bwd_configure() {
     return 0;
 }
 
+size_t gla_tc_backward_workspace_bytes(const Dims &d) {
+    const size_t bth = (size_t)d.B * d.T * d.H;
+    return (size_t)d.B * d.H * (d.NT + 1) * STATE_BF16 + 2 * ((bth + 63) & ~(size_t)63) * sizeof(float);
+}
+
+int gla_tc_segment_summaries(const Dims &d, const FwdArgs &a, int P, int L, float *fin, float *gam, int *status,
+                             cudaStream_t st, Tracer &tr) {
+    CUtensorMap mk, mv, mg;
+    if (!make_tile_map(&mk, a.k, d.B, d.T, d.H) || !make_tile_map(&mv, a.v, d.B, d.T, d.H) ||
+        !make_map(&mg, a.log_decay, d.B, d.T, d.H, d.dk, true, 128))
+        return -1;
+    StatesParams sp{a.lq, a.lk, nullptr, nullptr, fin, gam, status, d.T, d.H, d.NT, P, L};
+    k_gla_states_tc<<<d.B * d.H * P, st1::NTHREADS, st1::SMEM_BYTES, st>>>(mk, mv, mg, sp);
+    tr.mark("gla_segment_states_tc");
+    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+}
+
 int gla_tc_backward(const Dims &d, const BwdArgs &a, int *status, cudaStream_t st, Tracer &tr) {
     CUtensorMap mq, mk, mv, mdo, mg, mdq, mdk, mdv, mdg;
     if (!make_tile_map(&mq, a.q, d.B, d.T, d.H) || !make_tile_map(&mk, a.k, d.B, d.T, d.H) ||
@@ -811,7 +848,7 @@ int gla_tc_backward(const Dims &d, const BwdArgs &a, int *status, cudaStream_t s
     float *pq = a.ws + img_floats;
     float *pk = pq + ((bth + 63) & ~(size_t)63);
 
-    StatesParams sp{a.lq, a.lk, a.h0, simg, status, d.T, d.H, d.NT};
+    StatesParams sp{a.lq, a.lk, a.h0, simg, nullptr, nullptr, status, d.T, d.H, d.NT, 1, d.NT};
     k_gla_states_tc<<<d.B * d.H, st1::NTHREADS, st1::SMEM_BYTES, st>>>(mk, mv, mg, sp);
     tr.mark("gla_states_tc");
     BwdParams bp{a.lq, a.lk, a.dht, simg, pq, pk, a.dh0, status, d.T, d.H, d.NT, d.scale, gla_tc_phase_ts()};

@@ -101,6 +101,13 @@ int gla_tc_forward(const Dims &d, const FwdArgs &a, int *status, cudaStream_t st
 // Backward: chunk-state sweep, gradient sweep, gate softmax backward.  Needs the first
 // B*H*(NT+1)*32 KiB + 2*B*T*H*4 bytes (rounded up) of the workspace, less than the generic path.
 int gla_tc_bwd_configure();
+// Segmented forward of long sequences, first pass: every (sequence, segment of L chunks) from a zero state; leaves
+// the state it reaches (fin [B*H*P][128][128]) and the segment's total decay (gam [B*H*P][128]).
+int gla_tc_segment_summaries(const Dims &d, const FwdArgs &a, int P, int L, float *fin, float *gam, int *status,
+                             cudaStream_t st, Tracer &tr);
+// Bytes of workspace the tensor-core forward / backward need (the generic kernels need more).
+size_t gla_tc_forward_workspace_bytes(const Dims &d);
+size_t gla_tc_backward_workspace_bytes(const Dims &d);
 int gla_tc_backward(const Dims &d, const BwdArgs &a, int *status, cudaStream_t st, Tracer &tr);
 
 // GDN per-tile gradient kernels (after the recompute pass and the state-gradient scan).
@@ -111,7 +118,8 @@ int gdn_backward_tiles(const Dims &d, const Workspace &w, const BwdArgs &a, cuda
 // The opaque plan of the C ABI.
 struct sla_plan {
     sla::Dims dims;
-    sla::Workspace ws;
+    sla::Workspace ws;          // carve-up for the generic kernels
+    size_t fwd_bytes, bwd_bytes; // what the kernels this plan selects need (tensor-core plans need less than ws says)
     uint32_t flags;
     int device;
     int *d_status;          // device status word (bounded waits report here)

@@ -10,7 +10,8 @@ from tests import gpu_util as gu
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("B,T,H,with_h0", [(1, 64, 1, False), (2, 200, 3, True), (1, 1000, 16, True), (3, 65, 4, False)])
+@pytest.mark.parametrize("B,T,H,with_h0", [(1, 64, 1, False), (2, 200, 3, True), (1, 1000, 16, True), (3, 65, 4, False),
+                                           (1, 1297, 2, True), (2, 2048, 4, False)])    # the last two run segmented
 def test_gla_forward_tc(B, T, H, with_h0):
     cfg = small(CONFIGS["C1"], B=B, T=T, H=H, seed=300 + T)
     errs = gu.check_forward(cfg, with_h0=with_h0)
@@ -21,7 +22,7 @@ def test_gla_forward_tc_is_the_path_taken_and_agrees_with_generic():
     cfg = small(CONFIGS["C1"], B=2, T=300, H=4, seed=310, scale=0.5)
     x = gu.to_dev(make_inputs(cfg, with_h0=True))
     o1, ht1, plan = gu.gpu_forward(cfg, x, h0=x["h0"])
-    assert plan.last_launch_count == 1                 # the fused kernel, not the multi-kernel generic path
+    assert plan.last_launch_count == 1                 # the fused kernel (a short batch: one CTA per sequence)
     o2, ht2, plan2 = gu.gpu_forward(cfg, x, h0=x["h0"], flags=api.SLA_FLAG_FORCE_GENERIC)
     assert plan2.last_launch_count > 1
     assert gu.rel_l2(o1, o2.double().cpu().numpy()) <= 1e-2

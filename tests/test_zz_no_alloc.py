@@ -46,7 +46,8 @@ def test_noalloc_forward_matches_workspace_forward_twice_in_a_row(variant, dtype
 
 def test_noalloc_forward_refuses_problems_beyond_its_scratch():
     cfg = small(CONFIGS["C1"], B=4, T=2048, H=8)        # forward workspace far above 32 MiB
-    plan = api.sla_plan_create(cfg.variant, cfg.dtype, cfg.B, cfg.T, cfg.H, cfg.d_k, cfg.d_v, cfg.chunk)
+    plan = api.sla_plan_create(cfg.variant, cfg.dtype, cfg.B, cfg.T, cfg.H, cfg.d_k, cfg.d_v, cfg.chunk,
+                               flags=api.SLA_FLAG_FORCE_GENERIC)   # (the entry point always runs these kernels)
     assert plan.forward_workspace_bytes > api.SLA_NOALLOC_SCRATCH_BYTES
     z = torch.zeros(16, device="cuda")
     with pytest.raises(api.SLAError) as e:
