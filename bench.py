@@ -80,7 +80,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=self.tmp, stderr=subprocess.DEVNULL)
+                 "-lms", "20"], stdout=self.tmp, stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
@@ -150,7 +150,7 @@ def run_reference(args, cfg, rank):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -272,6 +272,40 @@ def main():
         ms_e2e = float(t.item())
     e2e_value = world * tokens_step * e2e_steps / (ms_e2e * 1e-3)
 
+    # ---- the decode step of the long-context configuration (C3): batch 64, fp32 state of 64 MiB, updated in place ----
+    decode = None
+    if rank == 0 and args.batch <= 0:
+        from paper_2602_01744_b200.inputs import C3_DECODE_BATCH, make_decode_inputs
+        c3 = CONFIGS["C3"]
+        dplan = api.sla_plan_create(c3.variant, c3.dtype, 1, 64, c3.H, c3.d_k, c3.d_v, c3.chunk)
+        dec = {n: (None if t is None else t.cuda()) for n, t in make_decode_inputs(c3, C3_DECODE_BATCH, 8, seed=5).items()}
+        state = torch.zeros((C3_DECODE_BATCH, c3.H, c3.d_k, c3.d_v), dtype=torch.float32, device="cuda")
+        o_t = torch.empty((C3_DECODE_BATCH, c3.H, c3.d_v), dtype=torch.bfloat16, device="cuda")
+        dsteps = 64
+
+        def dstep(i):
+            j = i % 8
+            api.sla_decode_step(dplan, dec["q"][j], dec["k"][j], dec["v"][j], dec["log_decay"][j], dec["gq_logits"][j],
+                                dec["gk_logits"][j], state, o_t=o_t)
+
+        for i in range(8):
+            dstep(i)
+        torch.cuda.synchronize()
+        e0.record()
+        for i in range(dsteps):
+            dstep(i)
+        e1.record()
+        torch.cuda.synchronize()
+        us = 1e3 * e0.elapsed_time(e1) / dsteps
+        dbytes = 2 * state.numel() * 4 + sum(dec[n][0].numel() * dec[n][0].element_size() for n in
+                                             ("q", "k", "v", "log_decay", "gq_logits", "gk_logits")) + o_t.numel() * 2
+        dpeak, _ = measured_peaks()
+        decode = {"workload": f"C3 decode: batch {C3_DECODE_BATCH}, H={c3.H}, d={c3.d_k}, fp32 state updated in place",
+                  "us_per_step": us, "tokens_per_s": C3_DECODE_BATCH / (us * 1e-6), "bound": "hbm",
+                  "algorithmic_bytes_per_step": dbytes, "achieved": dbytes / (us * 1e-6) / 1e9, "peak": dpeak,
+                  "unit": "GB/s", "frac": dbytes / (us * 1e-6) / 1e9 / dpeak,
+                  "note": "the 64 MiB state fits the 126 MB L2, so part of the traffic may be served there"}
+
     # ---- roofline of the dominant kernel, from the per-kernel CUDA events of the timed region ----
     peak, peak_kind = measured_peaks()
     roof = None
@@ -319,6 +353,7 @@ def main():
             "gpu_launches": n_launch,
             "roofline": roof,
             "step_hbm": {"algorithmic_bytes_per_step": step_bytes, "achieved_gbs": step_gbs, "frac": step_gbs / peak},
+            "decode_step": decode,
             "cpu_baseline": cpu,
         }
         print(json.dumps(line), flush=True)
