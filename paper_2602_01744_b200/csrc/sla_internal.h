@@ -110,6 +110,11 @@ size_t gla_tc_forward_workspace_bytes(const Dims &d);
 size_t gla_tc_backward_workspace_bytes(const Dims &d);
 int gla_tc_backward(const Dims &d, const BwdArgs &a, int *status, cudaStream_t st, Tracer &tr);
 
+// ---- tensor-core Softmax-GatedDeltaNet forward (WY form): sla_gdn_tc.cu.  Needs no workspace. ----
+bool gdn_tc_supported(const Dims &d);
+int gdn_tc_configure();
+int gdn_tc_forward(const Dims &d, const FwdArgs &a, int *status, cudaStream_t st, Tracer &tr);
+
 // GDN per-tile gradient kernels (after the recompute pass and the state-gradient scan).
 int gdn_backward_tiles(const Dims &d, const Workspace &w, const BwdArgs &a, cudaStream_t st, Tracer &tr);
 

@@ -1,4 +1,4 @@
-"""GPU parity of the tcgen05/TMEM/TMA Softmax-GLA kernels (bf16, d_k = d_v = 128, chunk 64) against
+"""GPU parity of the tcgen05/TMEM/TMA Softmax-GLA and Softmax-GatedDeltaNet kernels (bf16, d_k = d_v = 128, chunk 64) against
 the fp64 oracle, through the C ABI with default kernel selection."""
 import pytest
 import torch
@@ -46,3 +46,21 @@ def test_gla_backward_tc_is_the_path_taken_and_agrees_with_generic():
     assert plan2.last_launch_count > 3
     for name in ("dq", "dk", "dv", "dlog_decay", "dgq_logits", "dgk_logits", "dh0"):
         assert gu.rel_l2(g1[name], g2[name].double().cpu().numpy()) <= 1e-2, name
+
+
+@pytest.mark.parametrize("B,T,H,with_h0", [(1, 64, 1, False), (2, 200, 3, True), (1, 1000, 16, True), (3, 65, 4, True)])
+def test_gdn_forward_tc(B, T, H, with_h0):
+    cfg = small(CONFIGS["C4"], B=B, T=T, H=H, seed=500 + T, backward=False)
+    errs = gu.check_forward(cfg, with_h0=with_h0)
+    assert max(errs.values()) <= 1e-2
+
+
+def test_gdn_forward_tc_is_the_path_taken_and_agrees_with_generic():
+    cfg = small(CONFIGS["C4"], B=2, T=300, H=4, seed=510, scale=0.5, backward=False)
+    x = gu.to_dev(make_inputs(cfg, with_h0=True))
+    o1, ht1, plan = gu.gpu_forward(cfg, x, h0=x["h0"])
+    assert plan.last_launch_count == 1 and plan.forward_workspace_bytes == 0
+    o2, ht2, plan2 = gu.gpu_forward(cfg, x, h0=x["h0"], flags=api.SLA_FLAG_FORCE_GENERIC)
+    assert plan2.last_launch_count > 1
+    assert gu.rel_l2(o1, o2.double().cpu().numpy()) <= 1e-2
+    assert gu.rel_l2(ht1, ht2.double().cpu().numpy()) <= 1e-2
