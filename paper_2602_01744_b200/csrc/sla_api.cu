@@ -83,7 +83,8 @@ sla_status sla_plan_create(sla_plan **out, const sla_desc *desc) {
     if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return SLA_ERR_CUDA;
     if (prop.major != 10) return SLA_ERR_ARCH;
     if (sla::generic_configure() != 0 || sla::gdn_configure() != 0 || sla::gla_tc_configure() != 0 ||
-        sla::gla_tc_bwd_configure() != 0 || sla::gdn_tc_configure() != 0)
+        sla::gla_tc_bwd_configure() != 0 || sla::gdn_tc_configure() != 0 ||
+        sla::gdn_tc_bwd_configure() != 0)
         return SLA_ERR_CUDA;
 
     sla_plan *p = new (std::nothrow) sla_plan();
@@ -103,7 +104,10 @@ sla_status sla_plan_create(sla_plan **out, const sla_desc *desc) {
         p->fwd_bytes = sla::gla_tc_forward_workspace_bytes(d);
         p->bwd_bytes = sla::gla_tc_backward_workspace_bytes(d);
     }
-    if (sla::gdn_tc_supported(d) && !(desc->flags & SLA_FLAG_FORCE_GENERIC)) p->fwd_bytes = 0;
+    if (sla::gdn_tc_supported(d) && !(desc->flags & SLA_FLAG_FORCE_GENERIC)) {
+        p->fwd_bytes = 0;
+        p->bwd_bytes = sla::gdn_tc_backward_workspace_bytes(d);
+    }
     p->device = dev;
     p->last_launches = 0;
     p->d_status = nullptr;
@@ -231,9 +235,12 @@ sla_status sla_backward(sla_plan *plan, const void *q, const void *k, const void
     sla::BwdArgs a{q, k, v, log_decay, beta, gq_logits, gk_logits, h0, dO, dht, dq, dk, dv,
                    dlog_decay, dbeta, dgq_logits, dgk_logits, dh0, (float *)workspace};
     plan->tracer.start((cudaStream_t)cuda_stream);
-    const bool tc = sla::gla_tc_supported(d) && !(plan->flags & SLA_FLAG_FORCE_GENERIC);
-    int n = tc ? sla::gla_tc_backward(d, a, plan->d_status, (cudaStream_t)cuda_stream, plan->tracer)
-               : sla::generic_backward(d, plan->ws, a, (cudaStream_t)cuda_stream, plan->tracer);
+    const bool generic = plan->flags & SLA_FLAG_FORCE_GENERIC;
+    int n = (!generic && sla::gla_tc_supported(d))
+                ? sla::gla_tc_backward(d, a, plan->d_status, (cudaStream_t)cuda_stream, plan->tracer)
+            : (!generic && sla::gdn_tc_supported(d))
+                ? sla::gdn_tc_backward(d, a, plan->d_status, (cudaStream_t)cuda_stream, plan->tracer)
+                : sla::generic_backward(d, plan->ws, a, (cudaStream_t)cuda_stream, plan->tracer);
     if (n == -2) return SLA_ERR_UNSUPPORTED;
     if (n < 0) return SLA_ERR_CUDA;
     plan->last_launches = n;

@@ -46,9 +46,15 @@ static_assert(NBAR <= 32, "barrier slots");
 enum Sc { SC_B = 0, SC_GAM, SC_IGAM, SC_FQ, SC_FKB, SC_FVB, SC_BETA, SC_MISC };
 }  // namespace gd
 
+// Per-chunk record the forward leaves for the gradient sweep (save mode): bf16 S_n image, bf16 U tile, bf16 T tile,
+// each in MMA-operand layout.  Record n of sequence bh sits at save + (bh * (NT + 1) + n) * GDN_REC_BYTES; record NT
+// holds only S_NT.
+constexpr uint32_t REC_S = 0, REC_U = STATE_BF16, REC_T = STATE_BF16 + TILE_BF16, REC_BYTES = STATE_BF16 + TILE_BF16 + HALF_BF16;
+
 struct GdnParams {
     const float *lq, *lk, *g, *beta, *h0;
     float *ht;
+    uint8_t *save;          // nullptr: plain forward (o is stored); else: records are written and o is not stored
     int *status;
     int T, H, NT;
     float scale;
@@ -174,8 +180,10 @@ k_gdn_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             for (int n = 0; n < NT && !failed; ++n) {
                 wait_relaxed(OSTAGED + (n & 1), (n >> 1) & 1);   // O staged in the v buffer; every MMA of the chunk is done
                 if (failed) break;
-                tma_store_5d(&tm_o, base + (n & 1) * STAGE + OFF_V, 0, n * C, 0, h, b);
-                bulk_commit();
+                if (!p.save) {
+                    tma_store_5d(&tm_o, base + (n & 1) * STAGE + OFF_V, 0, n * C, 0, h, b);
+                    bulk_commit();
+                }
                 if (n + 2 < NT) {
                     bulk_wait_read0();
                     load(n + 2);
@@ -213,6 +221,7 @@ k_gdn_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
         const int row = 32 * (warp & 3) + lane;                          // state row (M = 128 tiles)
         const int ti = 16 * (warp & 3) + lane;                           // token row (M = 64 tiles, lanes 0..15)
 
+        uint8_t *rec0 = p.save ? p.save + (size_t)bh * (NT + 1) * REC_BYTES : nullptr;   // this sequence's records
         {   // initial state: fp32 into TMEM, bf16 copy into shared memory (row = key dimension)
             const float *src = p.h0 ? p.h0 + ((size_t)bh * D + row) * D + 64 * colhalf : nullptr;
 #pragma unroll
@@ -229,6 +238,7 @@ k_gdn_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
                     w.z = pack_bf16(v[8 * c + 4], v[8 * c + 5]);
                     w.w = pack_bf16(v[8 * c + 6], v[8 * c + 7]);
                     *reinterpret_cast<uint4 *>(sm + OFF_S + colhalf * STATE_HALF + swz(row, 4 * part + c)) = w;
+                    if (rec0) *reinterpret_cast<uint4 *>(rec0 + REC_S + colhalf * STATE_HALF + swz(row, 4 * part + c)) = w;
                 }
             }
             tmem_wait_st();
@@ -238,7 +248,7 @@ k_gdn_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
         mbar_arrive(bar(SREADY));
 
         // a 64x128 accumulator tile (M = 64: row i in lane 32*(i/16) + i%16) -> sign * bf16 -> swizzled tile at dst
-        auto tile_to_bf16 = [&](uint32_t col, uint8_t *dst, float sign) {
+        auto tile_to_bf16 = [&](uint32_t col, uint8_t *dst, float sign, uint8_t *gdst) {
             float v0[32], v1[32];
             tmem_ld32(tmem + lane_base + col + 64 * colhalf, v0);
             tmem_ld32(tmem + lane_base + col + 64 * colhalf + 32, v1);
@@ -252,11 +262,13 @@ k_gdn_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
                     w.z = pack_bf16(sign * v0[8 * c + 4], sign * v0[8 * c + 5]);
                     w.w = pack_bf16(sign * v0[8 * c + 6], sign * v0[8 * c + 7]);
                     *reinterpret_cast<uint4 *>(dst + colhalf * HALF_BF16 + swz(ti, c)) = w;
+                    if (gdst) *reinterpret_cast<uint4 *>(gdst + colhalf * HALF_BF16 + swz(ti, c)) = w;
                     w.x = pack_bf16(sign * v1[8 * c + 0], sign * v1[8 * c + 1]);
                     w.y = pack_bf16(sign * v1[8 * c + 2], sign * v1[8 * c + 3]);
                     w.z = pack_bf16(sign * v1[8 * c + 4], sign * v1[8 * c + 5]);
                     w.w = pack_bf16(sign * v1[8 * c + 6], sign * v1[8 * c + 7]);
                     *reinterpret_cast<uint4 *>(dst + colhalf * HALF_BF16 + swz(ti, 4 + c)) = w;
+                    if (gdst) *reinterpret_cast<uint4 *>(gdst + colhalf * HALF_BF16 + swz(ti, 4 + c)) = w;
                 }
             }
         };
@@ -423,6 +435,7 @@ k_gdn_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
                         ww[e] = pack_bf16(t0, t1);
                     }
                     *reinterpret_cast<uint4 *>(sm + OFF_T + swz(i, 2 * jq + hh)) = w;
+                    if (rec0) *reinterpret_cast<uint4 *>(rec0 + (size_t)n * REC_BYTES + REC_T + swz(i, 2 * jq + hh)) = w;
                 }
             }
             fence_proxy_async();
@@ -432,7 +445,7 @@ k_gdn_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             // ---- C: -W as bf16 over the q tile ----
             wait(BAR_2, par);
             tc_fence_after();
-            tile_to_bf16(COL_W, st + OFF_Q, -1.f);
+            tile_to_bf16(COL_W, st + OFF_Q, -1.f, nullptr);
             fence_proxy_async();
             tc_fence_before();
             mbar_arrive(bar(WREADY));
@@ -440,7 +453,7 @@ k_gdn_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             // ---- D: U as bf16 over the k tile ----
             wait(BAR_3, par);
             tc_fence_after();
-            tile_to_bf16(COL_U, st + OFF_K, 1.f);
+            tile_to_bf16(COL_U, st + OFF_K, 1.f, rec0 ? rec0 + (size_t)n * REC_BYTES + REC_U : nullptr);
             fence_proxy_async();
             tc_fence_before();
             mbar_arrive(bar(UREADY));
@@ -467,18 +480,20 @@ k_gdn_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
                     w.z = pack_bf16(v0[8 * c + 4], v0[8 * c + 5]);
                     w.w = pack_bf16(v0[8 * c + 6], v0[8 * c + 7]);
                     *reinterpret_cast<uint4 *>(sm + OFF_S + colhalf * STATE_HALF + swz(row, c)) = w;
+                    if (rec0) *reinterpret_cast<uint4 *>(rec0 + (size_t)(n + 1) * REC_BYTES + REC_S + colhalf * STATE_HALF + swz(row, c)) = w;
                     w.x = pack_bf16(v1[8 * c + 0], v1[8 * c + 1]);
                     w.y = pack_bf16(v1[8 * c + 2], v1[8 * c + 3]);
                     w.z = pack_bf16(v1[8 * c + 4], v1[8 * c + 5]);
                     w.w = pack_bf16(v1[8 * c + 6], v1[8 * c + 7]);
                     *reinterpret_cast<uint4 *>(sm + OFF_S + colhalf * STATE_HALF + swz(row, 4 + c)) = w;
+                    if (rec0) *reinterpret_cast<uint4 *>(rec0 + (size_t)(n + 1) * REC_BYTES + REC_S + colhalf * STATE_HALF + swz(row, 4 + c)) = w;
                 }
                 tmem_wait_st();
             }
             fence_proxy_async();
             tc_fence_before();
             mbar_arrive(bar(SREADY));
-            tile_to_bf16(COL_O, st + OFF_V, 1.f);
+            tile_to_bf16(COL_O, st + OFF_V, 1.f, nullptr);
             fence_proxy_async();
             tc_fence_before();
             mbar_arrive(bar(OSTAGED + (n & 1)));
@@ -515,12 +530,24 @@ int gdn_tc_configure() {
                    cudaSuccess ? 0 : -1;
 }
 
+// Forward sweep in save mode, for the gradient sweep: writes the per-chunk records (S_n, U, T), stores no output.
+int gdn_tc_forward_save(const Dims &d, const FwdArgs &a, uint8_t *save, int *status, cudaStream_t st, Tracer &tr) {
+    CUtensorMap mq, mk, mv;
+    if (!make_tile_map(&mq, a.q, d.B, d.T, d.H) || !make_tile_map(&mk, a.k, d.B, d.T, d.H) ||
+        !make_tile_map(&mv, a.v, d.B, d.T, d.H))
+        return -1;
+    GdnParams p{a.lq, a.lk, a.log_decay, a.beta, a.h0, nullptr, save, status, d.T, d.H, d.NT, d.scale};
+    k_gdn_fwd_tc<<<d.B * d.H, gd::NTHREADS, gd::SMEM_BYTES, st>>>(mq, mk, mv, mq /* unused: nothing is stored */, p);
+    tr.mark("gdn_states_tc");
+    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+}
+
 int gdn_tc_forward(const Dims &d, const FwdArgs &a, int *status, cudaStream_t st, Tracer &tr) {
     CUtensorMap mq, mk, mv, mo;
     if (!make_tile_map(&mq, a.q, d.B, d.T, d.H) || !make_tile_map(&mk, a.k, d.B, d.T, d.H) ||
         !make_tile_map(&mv, a.v, d.B, d.T, d.H) || !make_tile_map(&mo, a.o, d.B, d.T, d.H))
         return -1;
-    GdnParams p{a.lq, a.lk, a.log_decay, a.beta, a.h0, a.ht, status, d.T, d.H, d.NT, d.scale};
+    GdnParams p{a.lq, a.lk, a.log_decay, a.beta, a.h0, a.ht, nullptr, status, d.T, d.H, d.NT, d.scale};
     k_gdn_fwd_tc<<<d.B * d.H, gd::NTHREADS, gd::SMEM_BYTES, st>>>(mq, mk, mv, mo, p);
     tr.mark("gdn_fwd_tc");
     return cudaGetLastError() == cudaSuccess ? 1 : -1;

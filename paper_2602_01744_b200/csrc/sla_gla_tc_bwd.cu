@@ -816,6 +816,22 @@ int gla_tc_bwd_configure() {
     return 0;
 }
 
+// Softmax backward over the heads from the gate products P = G dG (shared by the GLA and GDN tensor-core paths).
+int gate_bwd_prod(const float *lq, const float *lk, const float *pq, const float *pk, float *dlq, float *dlk, long n_tok,
+                  int H, cudaStream_t st) {
+    int hp = 1;
+    while (hp < H) hp <<= 1;
+    switch (hp) {
+        case 1: launch_gate_bwd_prod<1>(lq, lk, pq, pk, dlq, dlk, n_tok, H, st); break;
+        case 2: launch_gate_bwd_prod<2>(lq, lk, pq, pk, dlq, dlk, n_tok, H, st); break;
+        case 4: launch_gate_bwd_prod<4>(lq, lk, pq, pk, dlq, dlk, n_tok, H, st); break;
+        case 8: launch_gate_bwd_prod<8>(lq, lk, pq, pk, dlq, dlk, n_tok, H, st); break;
+        case 16: launch_gate_bwd_prod<16>(lq, lk, pq, pk, dlq, dlk, n_tok, H, st); break;
+        default: launch_gate_bwd_prod<32>(lq, lk, pq, pk, dlq, dlk, n_tok, H, st); break;
+    }
+    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+}
+
 size_t gla_tc_backward_workspace_bytes(const Dims &d) {
     const size_t bth = (size_t)d.B * d.T * d.H;
     return (size_t)d.B * d.H * (d.NT + 1) * STATE_BF16 + 2 * ((bth + 63) & ~(size_t)63) * sizeof(float);
@@ -854,17 +870,7 @@ int gla_tc_backward(const Dims &d, const BwdArgs &a, int *status, cudaStream_t s
     BwdParams bp{a.lq, a.lk, a.dht, simg, pq, pk, a.dh0, status, d.T, d.H, d.NT, d.scale, gla_tc_phase_ts()};
     k_gla_bwd_tc<<<d.B * d.H, st2::NTHREADS, st2::SMEM_BYTES, st>>>(mq, mk, mv, mdo, mg, mdq, mdk, mdv, mdg, bp);
     tr.mark("gla_bwd_tc");
-    const long n_tok = (long)d.B * d.T;
-    int hp = 1;
-    while (hp < d.H) hp <<= 1;
-    switch (hp) {
-        case 1: launch_gate_bwd_prod<1>(a.lq, a.lk, pq, pk, a.dlq, a.dlk, n_tok, d.H, st); break;
-        case 2: launch_gate_bwd_prod<2>(a.lq, a.lk, pq, pk, a.dlq, a.dlk, n_tok, d.H, st); break;
-        case 4: launch_gate_bwd_prod<4>(a.lq, a.lk, pq, pk, a.dlq, a.dlk, n_tok, d.H, st); break;
-        case 8: launch_gate_bwd_prod<8>(a.lq, a.lk, pq, pk, a.dlq, a.dlk, n_tok, d.H, st); break;
-        case 16: launch_gate_bwd_prod<16>(a.lq, a.lk, pq, pk, a.dlq, a.dlk, n_tok, d.H, st); break;
-        default: launch_gate_bwd_prod<32>(a.lq, a.lk, pq, pk, a.dlq, a.dlk, n_tok, d.H, st); break;
-    }
+    if (gate_bwd_prod(a.lq, a.lk, pq, pk, a.dlq, a.dlk, (long)d.B * d.T, d.H, st) < 0) return -1;
     tr.mark("gate_bwd");
     return cudaGetLastError() == cudaSuccess ? 3 : -1;
 }

@@ -114,6 +114,13 @@ int gla_tc_backward(const Dims &d, const BwdArgs &a, int *status, cudaStream_t s
 bool gdn_tc_supported(const Dims &d);
 int gdn_tc_configure();
 int gdn_tc_forward(const Dims &d, const FwdArgs &a, int *status, cudaStream_t st, Tracer &tr);
+int gdn_tc_forward_save(const Dims &d, const FwdArgs &a, uint8_t *save, int *status, cudaStream_t st, Tracer &tr);
+// backward: forward sweep in save mode (per-chunk S_n, U, T records), reverse gradient sweep, gate softmax backward
+int gdn_tc_bwd_configure();
+size_t gdn_tc_backward_workspace_bytes(const Dims &d);
+int gdn_tc_backward(const Dims &d, const BwdArgs &a, int *status, cudaStream_t st, Tracer &tr);
+int gate_bwd_prod(const float *lq, const float *lk, const float *pq, const float *pk, float *dlq, float *dlk, long n_tok,
+                  int H, cudaStream_t st);
 
 // GDN per-tile gradient kernels (after the recompute pass and the state-gradient scan).
 int gdn_backward_tiles(const Dims &d, const Workspace &w, const BwdArgs &a, cudaStream_t st, Tracer &tr);

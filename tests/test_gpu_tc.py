@@ -64,3 +64,22 @@ def test_gdn_forward_tc_is_the_path_taken_and_agrees_with_generic():
     assert plan2.last_launch_count > 1
     assert gu.rel_l2(o1, o2.double().cpu().numpy()) <= 1e-2
     assert gu.rel_l2(ht1, ht2.double().cpu().numpy()) <= 1e-2
+
+
+@pytest.mark.parametrize("B,T,H,with_h0", [(1, 64, 1, False), (1, 128, 2, False), (2, 200, 3, True), (1, 1000, 16, True),
+                                           (3, 65, 4, True)])
+def test_gdn_backward_tc(B, T, H, with_h0):
+    cfg = small(CONFIGS["C4"], B=B, T=T, H=H, seed=600 + T)
+    errs = gu.check_backward(cfg, with_h0=with_h0)
+    assert max(errs.values()) <= 1e-2
+
+
+def test_gdn_backward_tc_is_the_path_taken_and_agrees_with_generic():
+    cfg = small(CONFIGS["C4"], B=2, T=300, H=4, seed=610, scale=0.5)
+    x = gu.to_dev(make_inputs(cfg, with_dO=True, with_h0=True))
+    g1, plan = gu.gpu_backward(cfg, x, h0=x["h0"], dht=x["dht"], want_dh0=True)
+    assert plan.last_launch_count == 3                 # forward sweep in save mode, gradient sweep, gate softmax backward
+    g2, plan2 = gu.gpu_backward(cfg, x, h0=x["h0"], dht=x["dht"], want_dh0=True, flags=api.SLA_FLAG_FORCE_GENERIC)
+    assert plan2.last_launch_count > 3
+    for name in ("dq", "dk", "dv", "dlog_decay", "dbeta", "dgq_logits", "dgk_logits", "dh0"):
+        assert gu.rel_l2(g1[name], g2[name].double().cpu().numpy()) <= 1e-2, name
