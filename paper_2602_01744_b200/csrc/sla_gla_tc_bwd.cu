@@ -418,11 +418,10 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
                 if (failed) break;
                 tc_fence_after();
 #pragma unroll
-                for (int kk = 0; kk < 8; ++kk)         // A = qh kh^T
+                for (int kk = 0; kk < 8; ++kk) {       // A = qh kh^T and dA = dO V^T, the two accumulation chains interleaved
                     tc_mma_bf16(tmem + COL_A, kQ + kstep_kmajor(kk, HALF_BF16), kK + kstep_kmajor(kk, HALF_BF16), ID_A, kk > 0);
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk)         // dA = dO V^T
                     tc_mma_bf16(tmem + COL_DA, kDO + kstep_kmajor(kk, HALF_BF16), kV + kstep_kmajor(kk, HALF_BF16), ID_A, kk > 0);
+                }
                 tc_commit(bar(BAR_A));
                 if (k > 0) wait(OUT1, (k - 1) & 1);    // dqh^T, dkh^T of the previous chunk have been read out
                 wait(FULL_S, par);
@@ -436,23 +435,19 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
                 if (failed) break;
                 tc_fence_after();
 #pragma unroll
-                for (int kk = 0; kk < 8; ++kk)         // dkh^T = dZ V^T ...
-                    tc_mma_bf16(tmem + COL_DK, kDZ + kstep_kmajor(kk, STATE_HALF), kV + kstep_kmajor(kk, HALF_BF16), ID_KK, kk > 0);
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk)         // dV^T = dZ^T kh^T ...
-                    tc_mma_bf16(tmem + COL_DV, mDZ + kstep_mnmajor(kk), kK + kstep_kmajor(kk, HALF_BF16), ID_MK, kk > 0);
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk)         // dS_n = dZ + qh^T dO
-                    tc_mma_bf16(tmem + COL_DS, mQ + kstep_mnmajor(kk), mDO + kstep_mnmajor(kk), ID_S, 1);
+                for (int kk = 0; kk < 8; ++kk) {       // three independent accumulation chains, interleaved
+                    tc_mma_bf16(tmem + COL_DK, kDZ + kstep_kmajor(kk, STATE_HALF), kV + kstep_kmajor(kk, HALF_BF16), ID_KK, kk > 0);   // dkh^T = dZ V^T ...
+                    tc_mma_bf16(tmem + COL_DV, mDZ + kstep_mnmajor(kk), kK + kstep_kmajor(kk, HALF_BF16), ID_MK, kk > 0);            // dV^T = dZ^T kh^T ...
+                    if (kk < 4) tc_mma_bf16(tmem + COL_DS, mQ + kstep_mnmajor(kk), mDO + kstep_mnmajor(kk), ID_S, 1);                // dS_n = dZ + qh^T dO
+                }
                 wait(AREADY, par);                     // masked A, dA in shared memory
                 if (failed) break;
                 tc_fence_after();
 #pragma unroll
-                for (int kk = 0; kk < 4; ++kk)         // ... + kh^T dA^T
+                for (int kk = 0; kk < 4; ++kk) {       // ... + kh^T dA^T  and  ... + qh^T dA, interleaved
                     tc_mma_bf16(tmem + COL_DQ, mK + kstep_mnmajor(kk), kDA + kstep_kmajor(kk, 0), ID_MK, 1);
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk)         // ... + qh^T dA
                     tc_mma_bf16(tmem + COL_DK, mQ + kstep_mnmajor(kk), mDA + kstep_mnmajor(kk), ID_MM, 1);
+                }
                 tc_commit(bar(BAR_M1));
 #pragma unroll
                 for (int kk = 0; kk < 4; ++kk)         // ... + dO^T A
@@ -606,10 +601,12 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             SLA_TS(2);
 
             // ---- dZ = diag(2^{b_last}) dS_{n+1}: fp32 back into TMEM (dS_n accumulates on it), bf16 operand copy ----
-            named_bar_sync(1, NCOMPUTE);                // eblast of this chunk is complete
             if (k > 0) wait(DGFREE, (k - 1) & 1);       // the staged tiles of the previous chunk have left dZ and A|dA
             {
-                const float e = eblast[row];
+                float bl = 0.f;                         // b_last of key dimension `row` from the prologue's 8-row sums
+#pragma unroll
+                for (int g8 = 0; g8 < 8; ++g8) bl += tot[g8 * D + row];
+                const float e = ex2f(bl * LOG2E);
                 float v0[32], v1[32];
                 const uint32_t ta = tmem + lane_base + COL_DS + 64 * wh;
                 tmem_ld32(ta, v0);
@@ -633,7 +630,8 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             tc_fence_after();
             SLA_TS(4);
             {
-                const int i = 16 * (warp & 3) + lane;
+                // rows 16q..16q+15 of this warp: a block of 8 columns c is empty for c >= 2q+2, full for c < 2q
+                const int q4 = warp & 3, i = 16 * q4 + lane;
                 const uint32_t col = wh ? COL_DA : COL_A;
                 uint8_t *dst = sm + (wh ? OFF_DA : OFF_A);
                 float v0[32], v1[32];
@@ -641,22 +639,24 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
                 tmem_ld32(tmem + lane_base + col + 32, v1);
                 tmem_wait_ld();
                 if (lane < 16) {
+#define SLA_MASK_BLOCK(V, CL, CB)                                                                                          \
+    {                                                                                                                      \
+        uint4 w = make_uint4(0u, 0u, 0u, 0u);                                                                              \
+        if ((CB) < 2 * q4 + 2) {                                                                                           \
+            const int j0 = 8 * (CB);                                                                                       \
+            const bool full = (CB) < 2 * q4;                                                                               \
+            w.x = pack_bf16(full || j0 + 0 <= i ? V[8 * (CL) + 0] : 0.f, full || j0 + 1 <= i ? V[8 * (CL) + 1] : 0.f);     \
+            w.y = pack_bf16(full || j0 + 2 <= i ? V[8 * (CL) + 2] : 0.f, full || j0 + 3 <= i ? V[8 * (CL) + 3] : 0.f);     \
+            w.z = pack_bf16(full || j0 + 4 <= i ? V[8 * (CL) + 4] : 0.f, full || j0 + 5 <= i ? V[8 * (CL) + 5] : 0.f);     \
+            w.w = pack_bf16(full || j0 + 6 <= i ? V[8 * (CL) + 6] : 0.f, full || j0 + 7 <= i ? V[8 * (CL) + 7] : 0.f);     \
+        }                                                                                                                  \
+        *reinterpret_cast<uint4 *>(dst + swz(i, (CB))) = w;                                                                \
+    }
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        const int j0 = 8 * c;
-                        uint4 w;
-                        w.x = pack_bf16(j0 + 0 <= i ? v0[8 * c + 0] : 0.f, j0 + 1 <= i ? v0[8 * c + 1] : 0.f);
-                        w.y = pack_bf16(j0 + 2 <= i ? v0[8 * c + 2] : 0.f, j0 + 3 <= i ? v0[8 * c + 3] : 0.f);
-                        w.z = pack_bf16(j0 + 4 <= i ? v0[8 * c + 4] : 0.f, j0 + 5 <= i ? v0[8 * c + 5] : 0.f);
-                        w.w = pack_bf16(j0 + 6 <= i ? v0[8 * c + 6] : 0.f, j0 + 7 <= i ? v0[8 * c + 7] : 0.f);
-                        *reinterpret_cast<uint4 *>(dst + swz(i, c)) = w;
-                        const int j1 = 32 + 8 * c;
-                        w.x = pack_bf16(j1 + 0 <= i ? v1[8 * c + 0] : 0.f, j1 + 1 <= i ? v1[8 * c + 1] : 0.f);
-                        w.y = pack_bf16(j1 + 2 <= i ? v1[8 * c + 2] : 0.f, j1 + 3 <= i ? v1[8 * c + 3] : 0.f);
-                        w.z = pack_bf16(j1 + 4 <= i ? v1[8 * c + 4] : 0.f, j1 + 5 <= i ? v1[8 * c + 5] : 0.f);
-                        w.w = pack_bf16(j1 + 6 <= i ? v1[8 * c + 6] : 0.f, j1 + 7 <= i ? v1[8 * c + 7] : 0.f);
-                        *reinterpret_cast<uint4 *>(dst + swz(i, 4 + c)) = w;
-                    }
+                    for (int c = 0; c < 4; ++c) SLA_MASK_BLOCK(v0, c, c)
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) SLA_MASK_BLOCK(v1, c, 4 + c)
+#undef SLA_MASK_BLOCK
                 }
             }
             fence_proxy_async();
