@@ -29,9 +29,13 @@ CPU_ROWS = 2          # batch rows of the workload the CPU oracle is timed on (a
 # (+ its gradient), fp32 gate logits (+ their gradients).
 FWD_BYTES_PER_TOKEN_HEAD = 4 * 256 + 512 + 8            # 1544
 BWD_BYTES_PER_TOKEN_HEAD = 4 * 256 + 512 + 3 * 256 + 512 + 16   # 2832
+# The gated delta rule has a scalar decay and beta per (token, head): 4 B each instead of 512 B.
+GDN_FWD_BYTES_PER_TOKEN_HEAD = 4 * 256 + 8 + 8          # 1040
+GDN_BWD_BYTES_PER_TOKEN_HEAD = 4 * 256 + 3 * 256 + 8 + 8 + 16   # 1824
 KERNEL_BYTES = {  # which share of the compulsory traffic each kernel is accountable for
     "output": FWD_BYTES_PER_TOKEN_HEAD, "grads_lin": BWD_BYTES_PER_TOKEN_HEAD,
     "gla_fwd_tc": FWD_BYTES_PER_TOKEN_HEAD, "gla_bwd_tc": BWD_BYTES_PER_TOKEN_HEAD,
+    "gdn_fwd_tc": GDN_FWD_BYTES_PER_TOKEN_HEAD, "gdn_bwd_tc": GDN_BWD_BYTES_PER_TOKEN_HEAD,
 }
 
 
@@ -106,22 +110,25 @@ class ClockSampler:
 
 
 def cpu_oracle_sample(cfg, x, steps=1, warmup=0):
-    """fp64 oracle, forward + backward, on the first CPU_ROWS batch rows of the workload (all T tokens, all heads)."""
+    """fp64 oracle, forward (+ backward where the workload has one), on the first CPU_ROWS batch rows of the workload
+    (all T tokens, all heads)."""
     from oracle import sla_oracle as orc
     s = lambda t: t[0:CPU_ROWS]
     args = (s(x["q"]), s(x["k"]), s(x["v"]), s(x["log_decay"]), s(x["gq_logits"]), s(x["gk_logits"]))
     # widen once outside the timed region, as the GPU arm holds its inputs resident
     args = tuple(a.double().numpy() for a in args)
-    dO = s(x["dO"]).double().numpy()
+    beta = None if x.get("beta") is None else s(x["beta"]).double().numpy()
+    dO = s(x["dO"]).double().numpy() if cfg.backward else None
     times = []
     for i in range(warmup + steps):
         t0 = time.perf_counter()
-        orc.forward(cfg.variant, *args, scale=cfg.scale)
-        orc.backward(cfg.variant, *args, dO, scale=cfg.scale)
+        orc.forward(cfg.variant, *args, beta=beta, scale=cfg.scale)
+        if cfg.backward:
+            orc.backward(cfg.variant, *args, dO, beta=beta, scale=cfg.scale)
         dt = time.perf_counter() - t0
         if i >= warmup:
             times.append(dt)
-    tokens = cfg.T * CPU_ROWS
+    tokens = cfg.T * min(CPU_ROWS, cfg.B)
     return tokens, times, orc.num_threads()
 
 
@@ -129,16 +136,17 @@ def run_reference(args, cfg, rank):
     if rank != 0:
         return
     from paper_2602_01744_b200.inputs import make_inputs, small
-    x = make_inputs(small(cfg, B=CPU_ROWS))
+    x = make_inputs(small(cfg, B=min(CPU_ROWS, cfg.B)))
     tokens, times, cores = cpu_oracle_sample(cfg, x, steps=args.steps, warmup=min(args.warmup, 1))
     total = sum(times)
     value = tokens * len(times) / total
-    sample = f"first {CPU_ROWS} batch rows of {WORKLOAD}: T={cfg.T}, H={cfg.H}, d={cfg.d_k}, forward+backward, fp64 recurrent oracle"
+    sample = (f"first {min(CPU_ROWS, cfg.B)} batch rows of {WORKLOAD}: T={cfg.T}, H={cfg.H}, d={cfg.d_k}, "
+              f"{'forward+backward' if cfg.backward else 'forward'}, fp64 recurrent oracle")
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / len(times),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "variant": cfg.variant, "B": CPU_ROWS, "T": cfg.T, "H": cfg.H,
+        "config": {"workload": WORKLOAD, "variant": cfg.variant, "B": min(CPU_ROWS, cfg.B), "T": cfg.T, "H": cfg.H,
                    "d_k": cfg.d_k, "d_v": cfg.d_v, "sample": sample},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -155,6 +163,9 @@ def main():
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--generic", action="store_true", help="force the fp32 CUDA-core kernels")
+    ap.add_argument("--workload", default="C2", choices=["C1", "C2", "C3", "C4"],
+                    help="C2 is the benchmark; the other configurations (C1, C3: forward only; C4: gated delta rule, "
+                         "forward + backward) are timed the same way for the per-configuration figures and profiles")
     ap.add_argument("--batch", type=int, default=0,
                     help="profiling aid: shrink the batch of the workload (0 = the full configuration; "
                          "a reduced batch is not the benchmark and is labelled in config)")
@@ -162,7 +173,12 @@ def main():
     args.warmup = max(args.warmup, 3) if args.impl == "b200" else args.warmup
 
     from paper_2602_01744_b200.inputs import CONFIGS, make_inputs
+    global WORKLOAD, METRIC
+    WORKLOAD = args.workload
     cfg = CONFIGS[WORKLOAD]
+    passes = "forward+backward" if cfg.backward else "forward"
+    if WORKLOAD != "C2":
+        METRIC = f"SLA-{cfg.variant.upper()} {passes} tokens/s ({WORKLOAD}: B={cfg.B},T={cfg.T},H={cfg.H},d={cfg.d_k},{cfg.dtype})"
     if args.batch > 0:
         from paper_2602_01744_b200.inputs import small
         cfg = small(cfg, B=args.batch)
@@ -191,27 +207,33 @@ def main():
         torch.cuda.synchronize()
 
     x = make_inputs(cfg)                        # every replica draws the same seeded batch
-    names = ["q", "k", "v", "log_decay", "gq_logits", "gk_logits", "dO"]
+    names = ["q", "k", "v", "log_decay", "gq_logits", "gk_logits"] + (["beta"] if x.get("beta") is not None else []) + \
+            (["dO"] if cfg.backward else [])
     host = {n: x[n].pin_memory() for n in names}
     dev = {n: host[n].cuda() for n in names}
+    dev.setdefault("beta", None)
     flags = api.SLA_FLAG_FORCE_GENERIC if args.generic else 0
     plan = api.sla_plan_create(cfg.variant, cfg.dtype, cfg.B, cfg.T, cfg.H, cfg.d_k, cfg.d_v, cfg.chunk,
                                cfg.scale, flags)
-    ws = plan.workspace(backward=True)
+    ws = plan.workspace(backward=cfg.backward)
     o = torch.empty_like(dev["v"])
-    grads = dict(dq=torch.empty_like(dev["q"]), dk=torch.empty_like(dev["k"]), dv=torch.empty_like(dev["v"]),
-                 dlog_decay=torch.empty_like(dev["log_decay"]), dbeta=None,
-                 dgq_logits=torch.empty_like(dev["gq_logits"]), dgk_logits=torch.empty_like(dev["gk_logits"]),
-                 dh0=None)
+    grads = None
+    if cfg.backward:
+        grads = dict(dq=torch.empty_like(dev["q"]), dk=torch.empty_like(dev["k"]), dv=torch.empty_like(dev["v"]),
+                     dlog_decay=torch.empty_like(dev["log_decay"]),
+                     dbeta=None if dev["beta"] is None else torch.empty_like(dev["beta"]),
+                     dgq_logits=torch.empty_like(dev["gq_logits"]), dgk_logits=torch.empty_like(dev["gk_logits"]),
+                     dh0=None)
     launches = [0]
 
     def step(d):
-        api.sla_forward(plan, d["q"], d["k"], d["v"], d["log_decay"], d["gq_logits"], d["gk_logits"], o=o,
-                        workspace=ws)
+        api.sla_forward(plan, d["q"], d["k"], d["v"], d["log_decay"], d["gq_logits"], d["gk_logits"], beta=d.get("beta"),
+                        o=o, workspace=ws)
         launches[0] += plan.last_launch_count
-        api.sla_backward(plan, d["q"], d["k"], d["v"], d["log_decay"], d["gq_logits"], d["gk_logits"], d["dO"],
-                         workspace=ws, out=grads)
-        launches[0] += plan.last_launch_count
+        if cfg.backward:
+            api.sla_backward(plan, d["q"], d["k"], d["v"], d["log_decay"], d["gq_logits"], d["gk_logits"], d["dO"],
+                             beta=d.get("beta"), workspace=ws, out=grads)
+            launches[0] += plan.last_launch_count
 
     for _ in range(args.warmup):
         step(dev)
@@ -244,7 +266,8 @@ def main():
     value = world * tokens_step * args.steps / (ms * 1e-3)
 
     # ---- end to end: pinned host inputs -> device, run, results -> pinned host, every step ----
-    outs = [o, grads["dq"], grads["dk"], grads["dv"], grads["dlog_decay"], grads["dgq_logits"], grads["dgk_logits"]]
+    outs = [o] + ([t for t in (grads["dq"], grads["dk"], grads["dv"], grads["dlog_decay"], grads["dbeta"],
+                               grads["dgq_logits"], grads["dgk_logits"]) if t is not None] if cfg.backward else [])
     host_out = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in outs]
     stage = {n: torch.empty_like(dev[n]) for n in names}
     h2d = sum(host[n].numel() * host[n].element_size() for n in names)
@@ -274,7 +297,7 @@ def main():
 
     # ---- the decode step of the long-context configuration (C3): batch 64, fp32 state of 64 MiB, updated in place ----
     decode = None
-    if rank == 0 and args.batch <= 0:
+    if rank == 0 and args.batch <= 0 and WORKLOAD == "C2":
         from paper_2602_01744_b200.inputs import C3_DECODE_BATCH, make_decode_inputs
         c3 = CONFIGS["C3"]
         dplan = api.sla_plan_create(c3.variant, c3.dtype, 1, 64, c3.H, c3.d_k, c3.d_v, c3.chunk)
@@ -326,7 +349,9 @@ def main():
                     "peak_kind": f"of {peak_kind}", "traffic": None, "avg_launch_ms": avg_ms,
                     "kernel_time_share": share}
     # whole-step figure against the same peak: all compulsory bytes of forward + backward / step time
-    step_bytes = (FWD_BYTES_PER_TOKEN_HEAD + BWD_BYTES_PER_TOKEN_HEAD) * cfg.B * cfg.T * cfg.H
+    gdn = cfg.variant == "gdn"
+    step_bytes = ((GDN_FWD_BYTES_PER_TOKEN_HEAD if gdn else FWD_BYTES_PER_TOKEN_HEAD) +
+                  ((GDN_BWD_BYTES_PER_TOKEN_HEAD if gdn else BWD_BYTES_PER_TOKEN_HEAD) if cfg.backward else 0)) * cfg.B * cfg.T * cfg.H
     step_gbs = step_bytes / (ms / args.steps * 1e-3) / 1e9
 
     if rank == 0:
@@ -334,7 +359,7 @@ def main():
         if world == 1 and not args.no_cpu_baseline:
             tokens, times, cores = cpu_oracle_sample(cfg, x, steps=1)
             cpu = {"value": tokens / times[0], "unit": UNIT, "cores": cores, "kind": "oracle",
-                   "sample": f"first {CPU_ROWS} batch rows of {WORKLOAD} (T={cfg.T}, H={cfg.H}), forward+backward, "
+                   "sample": f"first {min(CPU_ROWS, cfg.B)} batch rows of {WORKLOAD} (T={cfg.T}, H={cfg.H}), {passes}, "
                              f"{times[0]:.1f} s of fp64 recurrent oracle"}
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -342,9 +367,9 @@ def main():
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": WORKLOAD if args.batch <= 0 else f"{WORKLOAD} reduced to batch {cfg.B} (profiling only)",
                        "variant": cfg.variant, "B": cfg.B, "T": cfg.T, "H": cfg.H,
-                       "d_k": cfg.d_k, "d_v": cfg.d_v, "chunk": cfg.chunk, "pass": "forward+backward",
+                       "d_k": cfg.d_k, "d_v": cfg.d_v, "chunk": cfg.chunk, "pass": passes,
                        "io": "bf16 q,k,v,o and gradients; fp32 decay, logits, state; fp32 accumulation",
-                       "l2": "inputs (0.77 GB per step) exceed the 126 MB L2; no flush needed",
+                       "l2": f"inputs ({h2d / 1e9:.2f} GB per step) exceed the 126 MB L2; no flush needed",
                        "parallelism": "replicas only" if world > 1 else "single GPU",
                        "kernels": "generic fp32 CUDA-core" if args.generic else "default"},
             "clocks": clocks,

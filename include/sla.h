@@ -80,6 +80,12 @@ sla_status sla_plan_workspace_bytes(const sla_plan *plan, size_t *forward_bytes,
  * kernel gave up a bounded wait since the last poll, SLA_OK otherwise. */
 sla_status sla_plan_poll(sla_plan *plan);
 
+/* Diagnostic of the failure path (the paper has no counterpart): enqueues a one-warp kernel whose bounded wait can
+ * never be satisfied (limit 2 ms).  It gives up, raises the plan's status word like a tensor-core kernel whose wait
+ * expired, and returns normally: after synchronising the stream, sla_plan_poll reports SLA_ERR_TIMEOUT once and the
+ * context stays usable. */
+sla_status sla_plan_selftest_timeout(sla_plan *plan, void *cuda_stream);
+
 /* Number of kernel launches the last sla_forward / sla_backward / sla_decode_step on this plan
  * enqueued (for launch accounting in benchmarks). */
 int32_t sla_plan_last_launch_count(const sla_plan *plan);

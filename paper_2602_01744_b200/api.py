@@ -23,7 +23,7 @@ EXPORTS = (
     "sla_plan_create", "sla_plan_destroy", "sla_plan_workspace_bytes", "sla_plan_poll",
     "sla_plan_last_launch_count", "sla_plan_set_kernel_timing", "sla_plan_kernel_timing_collect",
     "sla_plan_kernel_timing_get", "sla_status_string", "sla_forward", "sla_backward", "sla_decode_step",
-    "sla_forward_noalloc",
+    "sla_forward_noalloc", "sla_plan_selftest_timeout",
 )
 SLA_NOALLOC_SCRATCH_BYTES = 32 << 20
 
@@ -59,6 +59,8 @@ def lib():
         L.sla_plan_destroy.argtypes = [vp]
         L.sla_plan_workspace_bytes.argtypes = [vp, ctypes.POINTER(sz), ctypes.POINTER(sz)]
         L.sla_plan_poll.argtypes = [vp]
+        L.sla_plan_selftest_timeout.argtypes = [vp, vp]
+        L.sla_plan_selftest_timeout.restype = ctypes.c_int
         L.sla_plan_last_launch_count.argtypes = [vp]
         L.sla_plan_last_launch_count.restype = i32
         L.sla_plan_set_kernel_timing.argtypes = [vp, i32]
@@ -123,6 +125,10 @@ class Plan:
 
     def poll(self):
         _check("sla_plan_poll", lib().sla_plan_poll(self.handle))
+
+    def selftest_timeout(self):
+        """Enqueue the bounded-wait self test (see sla_plan_selftest_timeout); poll() raises afterwards."""
+        _check("sla_plan_selftest_timeout", lib().sla_plan_selftest_timeout(self.handle, _stream()))
 
     @property
     def last_launch_count(self) -> int:

@@ -1,5 +1,6 @@
 // Host side of the C ABI: plan validation, workspace carve-up, launch order.
 #include "sla_internal.h"
+#include "sla_ptx.cuh"
 
 #include <new>
 #include <string.h>
@@ -41,6 +42,19 @@ Workspace plan_workspace(const Dims &d) {
 }  // namespace sla
 
 static bool aligned16(const void *p) { return ((uintptr_t)p & 15u) == 0; }
+
+// One warp waits on an mbarrier that nobody ever arrives at, with the same bounded wait the tensor-core kernels use
+// but a limit of `limit_ns`; when the wait gives up it raises the plan's status word, exactly as those kernels do.
+__global__ void k_selftest_bounded_wait(int *status, unsigned long long limit_ns) {
+    __shared__ __align__(8) unsigned long long mbar;
+    const uint32_t bar = sla::ptx::smem_u32(&mbar);
+    if (threadIdx.x == 0) {
+        sla::ptx::mbar_init(bar, 1);
+        sla::ptx::fence_mbar_init();
+    }
+    __syncthreads();
+    if (!sla::ptx::mbar_wait_bounded(bar, 0, nullptr, limit_ns) && threadIdx.x == 0) atomicExch(status, 1);
+}
 
 extern "C" {
 
@@ -148,6 +162,12 @@ sla_status sla_plan_poll(sla_plan *plan) {
 }
 
 int32_t sla_plan_last_launch_count(const sla_plan *plan) { return plan ? plan->last_launches : 0; }
+
+sla_status sla_plan_selftest_timeout(sla_plan *plan, void *cuda_stream) {
+    if (!plan) return SLA_ERR_INVALID_ARG;
+    k_selftest_bounded_wait<<<1, 32, 0, (cudaStream_t)cuda_stream>>>(plan->d_status, 2000000ull);   // 2 ms
+    return cudaGetLastError() == cudaSuccess ? SLA_OK : SLA_ERR_CUDA;
+}
 
 sla_status sla_plan_set_kernel_timing(sla_plan *plan, int32_t enable) {
     if (!plan) return SLA_ERR_INVALID_ARG;

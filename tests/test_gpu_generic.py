@@ -111,3 +111,18 @@ def test_rejections():
     z = torch.empty(0, device="cuda")
     api.sla_forward(p0, z, z, z, z, z, z, o=z)
     assert p0.last_launch_count == 0
+
+
+def test_bounded_wait_expiry_is_reported_and_the_context_survives():
+    plan = api.sla_plan_create("gla", "bf16", 1, 64, 2, 128, 128)
+    plan.selftest_timeout()                     # a wait nobody satisfies: gives up after 2 ms
+    torch.cuda.synchronize()
+    with pytest.raises(api.SLAError) as e:
+        plan.poll()
+    assert e.value.status == 6                  # SLA_ERR_TIMEOUT
+    plan.poll()                                 # reported once, then clear again
+    x = gu.to_dev(make_inputs(small(CONFIGS["C1"], B=1, T=64, H=2)))
+    o, _ = api.sla_forward(plan, x["q"], x["k"], x["v"], x["log_decay"], x["gq_logits"], x["gk_logits"])
+    torch.cuda.synchronize()
+    plan.poll()
+    assert torch.isfinite(o.float()).all()
