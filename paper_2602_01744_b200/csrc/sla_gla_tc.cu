@@ -251,14 +251,9 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
         mbar_arrive(bar(SREADY));
 
         auto prologue = [&](int n) {
-#define SLA_TSP(k) do { if (p.phase_ts && bh == 0 && tid == 0 && n == 9) p.phase_ts[k] = globaltimer_ns(); } while (0)
-            SLA_TSP(16);
             wait(GREADY + (n & 3), (n >> 2) & 1);
-            SLA_TSP(17);
             wait(FULL_G, n & 1);
-            SLA_TSP(18);
             wait(FULL_QK + n % 3, (n / 3) & 1);
-            SLA_TSP(19);
             uint8_t *qk = sm + OFF_QK + (n % 3) * QK_BYTES;
             const float *g = gate_s + (n & 3) * 2 * C;
             chunk_prologue<true, false>(qk, qk + TILE_BF16, reinterpret_cast<const float *>(sm + OFF_G), tot, g, g + C,
