@@ -258,12 +258,9 @@ def main():
     plan.set_kernel_timing(False)
     plan.poll()
     n_launch = launches[0]
-    if dist is not None:
-        t = torch.tensor([ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    from paper_2602_01744_b200.replicas import whole_job_throughput
     tokens_step = cfg.B * cfg.T
-    value = world * tokens_step * args.steps / (ms * 1e-3)
+    value, ms = whole_job_throughput(tokens_step, args.steps, ms, dist, "cuda")
 
     # ---- end to end: pinned host inputs -> device, run, results -> pinned host, every step ----
     outs = [o] + ([t for t in (grads["dq"], grads["dk"], grads["dv"], grads["dlog_decay"], grads["dbeta"],
@@ -288,12 +285,7 @@ def main():
         e2e_step()
     e1.record()
     barrier()
-    ms_e2e = e0.elapsed_time(e1)
-    if dist is not None:
-        t = torch.tensor([ms_e2e], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_e2e = float(t.item())
-    e2e_value = world * tokens_step * e2e_steps / (ms_e2e * 1e-3)
+    e2e_value, ms_e2e = whole_job_throughput(tokens_step, e2e_steps, e0.elapsed_time(e1), dist, "cuda")
 
     # ---- the decode step of the long-context configuration (C3): batch 64, fp32 state of 64 MiB, updated in place ----
     decode = None
