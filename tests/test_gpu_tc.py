@@ -83,3 +83,18 @@ def test_gdn_backward_tc_is_the_path_taken_and_agrees_with_generic():
     assert plan2.last_launch_count > 3
     for name in ("dq", "dk", "dv", "dlog_decay", "dbeta", "dgq_logits", "dgk_logits", "dh0"):
         assert gu.rel_l2(g1[name], g2[name].double().cpu().numpy()) <= 1e-2, name
+
+
+@pytest.mark.parametrize("base", ["C2", "C4"])
+@pytest.mark.parametrize("T", [1, 5, 193])
+def test_tc_paths_on_very_short_and_ragged_sequences(base, T):
+    cfg = small(CONFIGS[base], B=2, T=T, H=2, seed=700 + T)
+    assert max(gu.check_forward(small(cfg, backward=False), with_h0=True).values()) <= 1e-2
+    assert max(gu.check_backward(cfg, with_h0=True).values()) <= 1e-2
+
+
+def test_tc_paths_with_thirty_two_heads():
+    for base in ("C2", "C4"):
+        cfg = small(CONFIGS[base], B=1, T=130, H=32, seed=720)
+        assert max(gu.check_forward(small(cfg, backward=False)).values()) <= 1e-2
+        assert max(gu.check_backward(cfg).values()) <= 1e-2
