@@ -226,13 +226,13 @@ def main():
                      dh0=None)
     launches = [0]
 
-    def step(d):
+    def step(d, o_=None, grads_=None):
         api.sla_forward(plan, d["q"], d["k"], d["v"], d["log_decay"], d["gq_logits"], d["gk_logits"], beta=d.get("beta"),
-                        o=o, workspace=ws)
+                        o=o if o_ is None else o_, workspace=ws)
         launches[0] += plan.last_launch_count
         if cfg.backward:
             api.sla_backward(plan, d["q"], d["k"], d["v"], d["log_decay"], d["gq_logits"], d["gk_logits"], d["dO"],
-                             beta=d.get("beta"), workspace=ws, out=grads)
+                             beta=d.get("beta"), workspace=ws, out=grads if grads_ is None else grads_)
             launches[0] += plan.last_launch_count
 
     for _ in range(args.warmup):
@@ -263,26 +263,57 @@ def main():
     value, ms = whole_job_throughput(tokens_step, args.steps, ms, dist, "cuda")
 
     # ---- end to end: pinned host inputs -> device, run, results -> pinned host, every step ----
-    outs = [o] + ([t for t in (grads["dq"], grads["dk"], grads["dv"], grads["dlog_decay"], grads["dbeta"],
-                               grads["dgq_logits"], grads["dgk_logits"]) if t is not None] if cfg.backward else [])
-    host_out = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in outs]
-    stage = {n: torch.empty_like(dev[n]) for n in names}
+    # Every step copies all of its inputs in and all of its results out.  The three legs run on three streams with
+    # double-buffered device staging, so that the copy-in of step i+1 and the copy-out of step i-1 overlap the compute
+    # of step i (PCIe is full duplex); the kernels themselves still run one step after the other.
+    def out_list(o_, g_):
+        return [o_] + ([t for t in (g_["dq"], g_["dk"], g_["dv"], g_["dlog_decay"], g_["dbeta"], g_["dgq_logits"],
+                                    g_["dgk_logits"]) if t is not None] if cfg.backward else [])
+
+    o2 = [o, torch.empty_like(o)]
+    g2 = [grads, None if grads is None else {n: (None if t is None else torch.empty_like(t)) for n, t in grads.items()}]
+    outs2 = [out_list(o2[j], g2[j]) for j in range(2)]
+    host_out = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in outs2[0]]
+    stage2 = [{n: torch.empty_like(dev[n]) for n in names} for _ in range(2)]
+    for st_ in stage2:
+        st_.setdefault("beta", None)
     h2d = sum(host[n].numel() * host[n].element_size() for n in names)
-    d2h = sum(t.numel() * t.element_size() for t in outs)
+    d2h = sum(t.numel() * t.element_size() for t in outs2[0])
     e2e_steps = max(3, min(args.steps, 10))
+    s_in, s_out, s_c = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.current_stream()
 
-    def e2e_step():
-        for n in names:
-            stage[n].copy_(host[n], non_blocking=True)
-        step(stage)
-        for src, dst in zip(outs, host_out):
-            dst.copy_(src, non_blocking=True)
+    def e2e_run(nsteps):
+        in_ready, done, copied = [], [], []
+        for i in range(nsteps):
+            j = i % 2
+            with torch.cuda.stream(s_in):
+                if i >= 2:
+                    s_in.wait_event(done[i - 2])            # the staging buffer's previous step has been computed
+                for n in names:
+                    stage2[j][n].copy_(host[n], non_blocking=True)
+                ev = torch.cuda.Event()
+                ev.record(s_in)
+                in_ready.append(ev)
+            s_c.wait_event(in_ready[i])
+            if i >= 2:
+                s_c.wait_event(copied[i - 2])               # the output buffers' previous results are on the host
+            step(stage2[j], o2[j], g2[j])
+            ev = torch.cuda.Event()
+            ev.record(s_c)
+            done.append(ev)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(done[i])
+                for src, dst in zip(outs2[j], host_out):
+                    dst.copy_(src, non_blocking=True)
+                ev = torch.cuda.Event()
+                ev.record(s_out)
+                copied.append(ev)
+        s_c.wait_event(copied[-1])
 
-    e2e_step()
+    e2e_run(2)
     barrier()
     e0.record()
-    for _ in range(e2e_steps):
-        e2e_step()
+    e2e_run(e2e_steps)
     e1.record()
     barrier()
     e2e_value, ms_e2e = whole_job_throughput(tokens_step, e2e_steps, e0.elapsed_time(e1), dist, "cuda")

@@ -50,6 +50,14 @@ def lib():
     """Load libsla.so (built in-tree by paper_2602_01744_b200.build); raises if it is absent."""
     global _lib
     if _lib is None:
+        try:                                    # (re)build in-tree when the sources are newer than the library
+            from . import build as _build
+            _build.build()
+        except Exception as e:                  # no nvcc here: an existing, current library is still fine
+            if not _SO.exists():
+                raise FileNotFoundError(
+                    f"{_SO} is missing and could not be built ({e}): run `python -m paper_2602_01744_b200.build` "
+                    "(there is no fallback path)") from e
         if not _SO.exists():
             raise FileNotFoundError(
                 f"{_SO} is missing: run `python -m paper_2602_01744_b200.build` (there is no fallback path)")
