@@ -304,7 +304,7 @@ constexpr uint32_t SMEM_BYTES = OFF_TMEM + 16 + 1024;
 constexpr uint32_t COL_DS = 0, COL_A = 128, COL_DA = 192, COL_DQ = 256, COL_DK = 320, COL_DV = 384, TMEM_COLS = 512;
 constexpr int NTHREADS = NCOMPUTE + 32 + NGATE + 32;    // warps 0..7 compute, 8 MMA issue, 9..12 gates, 13 TMA
 enum Bar { FULL_G = 0, FULL_QK, FULL_V, FULL_DO, FULL_S, OPR, GREADY /*[4]*/, GFREE = GREADY + 4 /*[4]*/, ZREADY = GFREE + 4,
-           AREADY, OUT1, OUT2, INIT_DONE, DGFREE, BAR_A, BAR_M1, BAR_M2, DOFREE, INIT_FULL, DRAIN, NBAR };
+           AREADY, OUT1, OUT2, SNFREE, INIT_DONE, DGFREE, BAR_A, BAR_M1, BAR_M2, DOFREE, INIT_FULL, DRAIN, NBAR };
 static_assert(SMEM_BYTES <= 232448, "shared memory budget");
 static_assert(NBAR <= 32, "barrier slots");
 }  // namespace st2
@@ -412,24 +412,41 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
                 const uint64_t kQ = desc_kmajor(sQ), kK = desc_kmajor(sK), kV = desc_kmajor(sV), kDO = desc_kmajor(sDO),
                                mQ = desc_mnmajor(sQ, HALF_BF16), mK = desc_mnmajor(sK, HALF_BF16),
                                mDO = desc_mnmajor(sDO, HALF_BF16);
-                wait(OPR, par);                        // qh, kh in place
+                // dA = dO V^T and S_n dO^T need no prologue: they are issued while the compute warps still scale q and k
                 wait(FULL_V, par);
                 wait(FULL_DO, par);
                 if (failed) break;
                 tc_fence_after();
 #pragma unroll
-                for (int kk = 0; kk < 8; ++kk) {       // A = qh kh^T and dA = dO V^T, the two accumulation chains interleaved
-                    tc_mma_bf16(tmem + COL_A, kQ + kstep_kmajor(kk, HALF_BF16), kK + kstep_kmajor(kk, HALF_BF16), ID_A, kk > 0);
+                for (int kk = 0; kk < 8; ++kk)         // dA = dO V^T
                     tc_mma_bf16(tmem + COL_DA, kDO + kstep_kmajor(kk, HALF_BF16), kV + kstep_kmajor(kk, HALF_BF16), ID_A, kk > 0);
+                bool sdo_done = false;
+                auto issue_sdo = [&]() {               // dqh^T = S_n dO^T ...
+                    if (k > 0) wait(OUT1, (k - 1) & 1);    // dqh^T, dkh^T of the previous chunk have been read out (long ago)
+                    tc_fence_after();
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk)
+                        tc_mma_bf16(tmem + COL_DQ, kS + kstep_kmajor(kk, STATE_HALF), kDO + kstep_kmajor(kk, HALF_BF16), ID_KK, kk > 0);
+                    sdo_done = true;
+                };
+                {   // whichever comes first: S_n landed, or the prologue done
+                    const uint64_t t0 = globaltimer_ns();
+                    for (uint32_t it = 0; !failed && !mbar_test_wait(bar(OPR), par); ++it) {
+                        if (!sdo_done && mbar_test_wait(bar(FULL_S), par)) issue_sdo();
+                        if ((it & 63u) == 63u && (*abort_flag || globaltimer_ns() - t0 > 2000000000ull)) { failed = true; *abort_flag = 1; }
+                    }
                 }
-                tc_commit(bar(BAR_A));
-                if (k > 0) wait(OUT1, (k - 1) & 1);    // dqh^T, dkh^T of the previous chunk have been read out
-                wait(FULL_S, par);
                 if (failed) break;
                 tc_fence_after();
 #pragma unroll
-                for (int kk = 0; kk < 8; ++kk)         // dqh^T = S_n dO^T ...
-                    tc_mma_bf16(tmem + COL_DQ, kS + kstep_kmajor(kk, STATE_HALF), kDO + kstep_kmajor(kk, HALF_BF16), ID_KK, kk > 0);
+                for (int kk = 0; kk < 8; ++kk)         // A = qh kh^T
+                    tc_mma_bf16(tmem + COL_A, kQ + kstep_kmajor(kk, HALF_BF16), kK + kstep_kmajor(kk, HALF_BF16), ID_A, kk > 0);
+                tc_commit(bar(BAR_A));
+                if (!sdo_done) {
+                    wait(FULL_S, par);
+                    if (failed) break;
+                    issue_sdo();
+                }
                 if (k > 0) wait(OUT2, (k - 1) & 1);    // dV^T and dS of the previous chunk have been read out
                 wait(ZREADY, par);                     // dZ: fp32 in TMEM, bf16 in shared memory
                 if (failed) break;
@@ -511,12 +528,16 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
                 bulk_commit();
                 bulk_wait_read0();
                 if (n > 0) load_vdo(n - 1, k + 1);     // ... and this buffer takes the next v, dO
-                wait_relaxed(OUT2, par);               // dv, dlog_decay staged; S_n no longer needed
+                if (n > 0) {
+                    wait_relaxed(SNFREE, par);         // rowsum(dS_n * S_n) done: S_n no longer needed
+                    if (failed) break;
+                    load_s(n - 1);
+                }
+                wait_relaxed(OUT2, par);               // dv, dlog_decay staged
                 if (failed) break;
                 tma_store_5d(&tm_dv, base + OFF_A, 0, n * C, 0, h, b);
                 tma_store_4d(&tm_dg, base + OFF_DZ, 0, h, n * C, b);
                 bulk_commit();
-                if (n > 0) load_s(n - 1);
                 bulk_wait_read0();
                 mbar_arrive(bar(DGFREE));
             }
@@ -724,6 +745,7 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
                 tmem_wait_ld();
                 Rs[((n & 1) ^ 1) * 2 * D + wh * D + row] = rowdot_part(v0, 0) + rowdot_part(v1, 1);
             }
+            mbar_arrive(bar(SNFREE));
             SLA_TS(9);
             named_bar_sync(1, NCOMPUTE);                // up, red and the R partials are complete
             {   // log-decay gradient: in-chunk suffix sum + what flows in from the right of the chunk
