@@ -163,6 +163,9 @@ def main():
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--generic", action="store_true", help="force the fp32 CUDA-core kernels")
+    ap.add_argument("--recompute", action="store_true",
+                    help="plan without SLA_FLAG_SAVE_FOR_BACKWARD: the backward pass recomputes the chunk states "
+                         "instead of reading what the forward pass of the same step left in the workspace")
     ap.add_argument("--workload", default="C2", choices=["C1", "C2", "C3", "C4"],
                     help="C2 is the benchmark; the other configurations (C1, C3: forward only; C4: gated delta rule, "
                          "forward + backward) are timed the same way for the per-configuration figures and profiles")
@@ -213,6 +216,9 @@ def main():
     dev = {n: host[n].cuda() for n in names}
     dev.setdefault("beta", None)
     flags = api.SLA_FLAG_FORCE_GENERIC if args.generic else 0
+    saving = cfg.backward and not args.recompute and not args.generic
+    if saving:      # a training step: the forward leaves the chunk states for the backward of the same step
+        flags |= api.SLA_FLAG_SAVE_FOR_BACKWARD
     plan = api.sla_plan_create(cfg.variant, cfg.dtype, cfg.B, cfg.T, cfg.H, cfg.d_k, cfg.d_v, cfg.chunk,
                                cfg.scale, flags)
     ws = plan.workspace(backward=cfg.backward)
@@ -394,7 +400,10 @@ def main():
                        "io": "bf16 q,k,v,o and gradients; fp32 decay, logits, state; fp32 accumulation",
                        "l2": f"inputs ({h2d / 1e9:.2f} GB per step) exceed the 126 MB L2; no flush needed",
                        "parallelism": "replicas only" if world > 1 else "single GPU",
-                       "kernels": "generic fp32 CUDA-core" if args.generic else "default"},
+                       "kernels": "generic fp32 CUDA-core" if args.generic else "default",
+                       "chunk_states": ("written by the forward pass of each step into the workspace, read by the backward "
+                                        "pass of the same step" if saving else
+                                        "recomputed by the backward pass" if cfg.backward else "not kept")},
             "clocks": clocks,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": e2e_steps, "ms_per_step": ms_e2e / e2e_steps},

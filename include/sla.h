@@ -54,6 +54,17 @@ typedef enum { SLA_FP32 = 0, SLA_BF16 = 1 } sla_dtype;
 /* flags */
 #define SLA_FLAG_FORCE_GENERIC 1u  /* use the fp32 CUDA-core chunk kernels even where a tensor-core
                                       kernel exists for the shape (same function, other rounding) */
+#define SLA_FLAG_SAVE_FOR_BACKWARD 2u
+/* Training plans: sla_forward also leaves in its workspace what the chunkwise backward pass would
+ * otherwise recompute first (Softmax-GLA: the state before every chunk; Softmax-GDN: per chunk the
+ * state, the corrected values U and the inverse T of the WY form).  sla_plan_workspace_bytes then
+ * reports the backward size for the forward too.  A following sla_backward on the same plan that is
+ * given the same workspace, the same q, k, v, log_decay, beta, logits and h0 pointers and the same
+ * stream as that sla_forward uses what was left and skips its recomputation; any other call
+ * recomputes, so results never depend on the flag.  Contract: between the two calls the caller
+ * changes neither the workspace nor the contents of those inputs.  Ignored (nothing is left, the
+ * backward recomputes) by the fp32 CUDA-core kernels and where the forward cuts long sequences
+ * into segments. */
 
 typedef struct {
     uint32_t struct_size;      /* sizeof(sla_desc) */

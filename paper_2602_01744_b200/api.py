@@ -17,6 +17,7 @@ _SO = _PKG / "libsla.so"
 SLA_RETNET, SLA_GLA, SLA_GDN = 0, 1, 2
 SLA_FP32, SLA_BF16 = 0, 1
 SLA_FLAG_FORCE_GENERIC = 1
+SLA_FLAG_SAVE_FOR_BACKWARD = 2
 VARIANTS = {"retnet": SLA_RETNET, "gla": SLA_GLA, "gdn": SLA_GDN}
 DTYPES = {"fp32": SLA_FP32, "bf16": SLA_BF16, torch.float32: SLA_FP32, torch.bfloat16: SLA_BF16}
 EXPORTS = (

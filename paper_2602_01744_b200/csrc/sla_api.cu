@@ -56,6 +56,14 @@ __global__ void k_selftest_bounded_wait(int *status, unsigned long long limit_ns
     if (!sla::ptx::mbar_wait_bounded(bar, 0, nullptr, limit_ns) && threadIdx.x == 0) atomicExch(status, 1);
 }
 
+// Can sla_forward of this plan leave what sla_backward needs (SLA_FLAG_SAVE_FOR_BACKWARD)?  Only the tensor-core
+// paths do, and Softmax-GLA only where the forward runs each sequence in one piece.
+static bool forward_can_save(const sla_plan &p) {
+    if (p.flags & SLA_FLAG_FORCE_GENERIC) return false;
+    if (sla::gla_tc_supported(p.dims)) return sla::gla_tc_forward_can_save(p.dims);
+    return sla::gdn_tc_supported(p.dims);
+}
+
 extern "C" {
 
 // Profiling aid (not declared in sla.h): device buffer of >= 16 uint64 that block 0 of the tensor-core
@@ -122,6 +130,8 @@ sla_status sla_plan_create(sla_plan **out, const sla_desc *desc) {
         p->fwd_bytes = 0;
         p->bwd_bytes = sla::gdn_tc_backward_workspace_bytes(d);
     }
+    if ((desc->flags & SLA_FLAG_SAVE_FOR_BACKWARD) && forward_can_save(*p) && p->bwd_bytes > p->fwd_bytes)
+        p->fwd_bytes = p->bwd_bytes;     // the forward writes into the backward pass's workspace layout
     p->device = dev;
     p->last_launches = 0;
     p->d_status = nullptr;
@@ -220,13 +230,23 @@ sla_status sla_forward(sla_plan *plan, const void *q, const void *k, const void 
     sla::FwdArgs a{q, k, v, log_decay, beta, gq_logits, gk_logits, h0, o, ht, (float *)workspace};
     plan->tracer.start((cudaStream_t)cuda_stream);
     const bool generic = plan->flags & SLA_FLAG_FORCE_GENERIC;
+    const bool save = (plan->flags & SLA_FLAG_SAVE_FOR_BACKWARD) && forward_can_save(*plan);
+    plan->saved.valid = false;
     int n = (!generic && sla::gla_tc_supported(d))
-                ? sla::gla_tc_forward(d, a, plan->d_status, (cudaStream_t)cuda_stream, plan->tracer)
+                ? sla::gla_tc_forward(d, a, save ? sla::gla_tc_state_images(a.ws) : nullptr, plan->d_status,
+                                      (cudaStream_t)cuda_stream, plan->tracer)
             : (!generic && sla::gdn_tc_supported(d))
-                ? sla::gdn_tc_forward(d, a, plan->d_status, (cudaStream_t)cuda_stream, plan->tracer)
+                ? sla::gdn_tc_forward(d, a, save ? sla::gdn_tc_records(a.ws) : nullptr, plan->d_status,
+                                      (cudaStream_t)cuda_stream, plan->tracer)
                 : sla::generic_forward(d, plan->ws, a, true, (cudaStream_t)cuda_stream, plan->tracer);
     if (n < 0) return SLA_ERR_CUDA;
     plan->last_launches = n;
+    if (save) {
+        sla_plan::Saved &sv = plan->saved;
+        sv.valid = true;
+        sv.ws = workspace; sv.q = q; sv.k = k; sv.v = v; sv.log_decay = log_decay; sv.beta = beta;
+        sv.lq = gq_logits; sv.lk = gk_logits; sv.h0 = h0; sv.stream = cuda_stream;
+    }
     return SLA_OK;
 }
 
@@ -256,10 +276,15 @@ sla_status sla_backward(sla_plan *plan, const void *q, const void *k, const void
                    dlog_decay, dbeta, dgq_logits, dgk_logits, dh0, (float *)workspace};
     plan->tracer.start((cudaStream_t)cuda_stream);
     const bool generic = plan->flags & SLA_FLAG_FORCE_GENERIC;
+    // the states (GLA) or per-chunk records (GDN) are taken from the workspace only if the last sla_forward of this plan
+    // left them there for exactly these inputs, on this stream; anything else recomputes them
+    const sla_plan::Saved &sv = plan->saved;
+    const bool have = sv.valid && sv.ws == workspace && sv.q == q && sv.k == k && sv.v == v && sv.log_decay == log_decay &&
+                      sv.beta == beta && sv.lq == gq_logits && sv.lk == gk_logits && sv.h0 == h0 && sv.stream == cuda_stream;
     int n = (!generic && sla::gla_tc_supported(d))
-                ? sla::gla_tc_backward(d, a, plan->d_status, (cudaStream_t)cuda_stream, plan->tracer)
+                ? sla::gla_tc_backward(d, a, have, plan->d_status, (cudaStream_t)cuda_stream, plan->tracer)
             : (!generic && sla::gdn_tc_supported(d))
-                ? sla::gdn_tc_backward(d, a, plan->d_status, (cudaStream_t)cuda_stream, plan->tracer)
+                ? sla::gdn_tc_backward(d, a, have, plan->d_status, (cudaStream_t)cuda_stream, plan->tracer)
                 : sla::generic_backward(d, plan->ws, a, (cudaStream_t)cuda_stream, plan->tracer);
     if (n == -2) return SLA_ERR_UNSUPPORTED;
     if (n < 0) return SLA_ERR_CUDA;

@@ -54,7 +54,8 @@ constexpr uint32_t REC_S = 0, REC_U = STATE_BF16, REC_T = STATE_BF16 + TILE_BF16
 struct GdnParams {
     const float *lq, *lk, *g, *beta, *h0;
     float *ht;
-    uint8_t *save;          // nullptr: plain forward (o is stored); else: records are written and o is not stored
+    uint8_t *save;          // not nullptr: the per-chunk records are written
+    int write_o;            // 0: o is not stored (the gradient sweep's own recomputation)
     int *status;
     int T, H, NT;
     float scale;
@@ -180,7 +181,7 @@ k_gdn_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             for (int n = 0; n < NT && !failed; ++n) {
                 wait_relaxed(OSTAGED + (n & 1), (n >> 1) & 1);   // O staged in the v buffer; every MMA of the chunk is done
                 if (failed) break;
-                if (!p.save) {
+                if (p.write_o) {
                     tma_store_5d(&tm_o, base + (n & 1) * STAGE + OFF_V, 0, n * C, 0, h, b);
                     bulk_commit();
                 }
@@ -536,18 +537,19 @@ int gdn_tc_forward_save(const Dims &d, const FwdArgs &a, uint8_t *save, int *sta
     if (!make_tile_map(&mq, a.q, d.B, d.T, d.H) || !make_tile_map(&mk, a.k, d.B, d.T, d.H) ||
         !make_tile_map(&mv, a.v, d.B, d.T, d.H))
         return -1;
-    GdnParams p{a.lq, a.lk, a.log_decay, a.beta, a.h0, nullptr, save, status, d.T, d.H, d.NT, d.scale};
+    GdnParams p{a.lq, a.lk, a.log_decay, a.beta, a.h0, nullptr, save, 0, status, d.T, d.H, d.NT, d.scale};
     k_gdn_fwd_tc<<<d.B * d.H, gd::NTHREADS, gd::SMEM_BYTES, st>>>(mq, mk, mv, mq /* unused: nothing is stored */, p);
     tr.mark("gdn_states_tc");
     return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 
-int gdn_tc_forward(const Dims &d, const FwdArgs &a, int *status, cudaStream_t st, Tracer &tr) {
+// Forward; with `save` not null it also leaves the per-chunk records for a later gradient sweep over the same inputs.
+int gdn_tc_forward(const Dims &d, const FwdArgs &a, uint8_t *save, int *status, cudaStream_t st, Tracer &tr) {
     CUtensorMap mq, mk, mv, mo;
     if (!make_tile_map(&mq, a.q, d.B, d.T, d.H) || !make_tile_map(&mk, a.k, d.B, d.T, d.H) ||
         !make_tile_map(&mv, a.v, d.B, d.T, d.H) || !make_tile_map(&mo, a.o, d.B, d.T, d.H))
         return -1;
-    GdnParams p{a.lq, a.lk, a.log_decay, a.beta, a.h0, a.ht, nullptr, status, d.T, d.H, d.NT, d.scale};
+    GdnParams p{a.lq, a.lk, a.log_decay, a.beta, a.h0, a.ht, save, 1, status, d.T, d.H, d.NT, d.scale};
     k_gdn_fwd_tc<<<d.B * d.H, gd::NTHREADS, gd::SMEM_BYTES, st>>>(mq, mk, mv, mo, p);
     tr.mark("gdn_fwd_tc");
     return cudaGetLastError() == cudaSuccess ? 1 : -1;

@@ -748,7 +748,9 @@ size_t gdn_tc_backward_workspace_bytes(const Dims &d) {
     return (size_t)d.B * d.H * (d.NT + 1) * REC_BYTES + 2 * ((bth + 63) & ~(size_t)63) * sizeof(float);
 }
 
-int gdn_tc_backward(const Dims &d, const BwdArgs &a, int *status, cudaStream_t st, Tracer &tr) {
+uint8_t *gdn_tc_records(float *ws) { return reinterpret_cast<uint8_t *>(ws); }
+
+int gdn_tc_backward(const Dims &d, const BwdArgs &a, bool have_records, int *status, cudaStream_t st, Tracer &tr) {
     CUtensorMap mq, mk, mv, mdo, mdq, mdk, mdv;
     if (!make_tile_map(&mq, a.q, d.B, d.T, d.H) || !make_tile_map(&mk, a.k, d.B, d.T, d.H) ||
         !make_tile_map(&mv, a.v, d.B, d.T, d.H) || !make_tile_map(&mdo, a.dO, d.B, d.T, d.H) ||
@@ -760,14 +762,15 @@ int gdn_tc_backward(const Dims &d, const BwdArgs &a, int *status, cudaStream_t s
     float *pq = reinterpret_cast<float *>(save + (size_t)d.B * d.H * (d.NT + 1) * REC_BYTES);
     float *pk = pq + ((bth + 63) & ~(size_t)63);
     FwdArgs f{a.q, a.k, a.v, a.log_decay, a.beta, a.lq, a.lk, a.h0, nullptr, nullptr, a.ws};
-    if (gdn_tc_forward_save(d, f, save, status, st, tr) < 0) return -1;
+    // (with have_records the forward pass of the same inputs has left the records in this workspace)
+    if (!have_records && gdn_tc_forward_save(d, f, save, status, st, tr) < 0) return -1;
     GdnBwdParams bp{a.lq, a.lk, a.log_decay, a.beta, a.dht, save, a.dlog_decay, a.dbeta, pq, pk, a.dh0, status,
                     d.T, d.H, d.NT, d.scale};
     k_gdn_bwd_tc<<<d.B * d.H, gb::NTHREADS, gb::SMEM_BYTES, st>>>(mq, mk, mv, mdo, mdq, mdk, mdv, bp);
     tr.mark("gdn_bwd_tc");
     if (gate_bwd_prod(a.lq, a.lk, pq, pk, a.dlq, a.dlk, (long)d.B * d.T, d.H, st) < 0) return -1;
     tr.mark("gate_bwd");
-    return cudaGetLastError() == cudaSuccess ? 3 : -1;
+    return cudaGetLastError() == cudaSuccess ? (have_records ? 2 : 3) : -1;
 }
 
 }  // namespace sla

@@ -42,12 +42,14 @@ constexpr int NTHREADS = NCOMPUTE + 32 + NGATE + 32;   // warps 0..7 compute, 8 
 
 // mbarrier slots (8 bytes each)
 enum Bar { FULL_G = 0, FULL_QK = 1, FULL_V = 4, OPR = 6, GREADY = 9, GFREE = 13, SREADY = 17, OFREE, AREADY, BAR_A, BAR_Z,
-           BAR_O /* [2], one per O accumulator */, OSTAGED = BAR_O + 2, OSFREE, DRAIN, QKFREE /* [3] */, NBAR = QKFREE + 3 };
+           BAR_O /* [2], one per O accumulator */, OSTAGED = BAR_O + 2, OSFREE, DRAIN, QKFREE /* [3] */, SSAVED = QKFREE + 3, NBAR };
+static_assert(NBAR <= 32, "barrier slots");
 
 struct FwdParams {
     const float *lq, *lk, *h0;
     __nv_bfloat16 *o;
     float *ht;
+    uint8_t *simg;                  // optional: [B*H][NT+1][32 KiB] bf16 images of the state before every chunk (P = 1 only)
     int *status;
     int T, H, NT;
     int P, L;                       // segments per sequence and chunks per segment (P = 1: L = NT)
@@ -169,12 +171,26 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
                 mbar_expect_tx(bf, TILE_BF16);
                 tma_load_5d(dst, &tm_v, 0, (n0 + n) * C, 0, h, b, bf);
             };
+            // save mode: S_m (the bf16 operand copy, as it stands in shared memory) -> image slot m, for the backward pass
+            uint8_t *img0 = p.simg ? p.simg + (size_t)bh * (p.NT + 1) * STATE_BF16 : nullptr;
+            bool save_pending = false;
+            auto save_s = [&](int m) {
+                wait_relaxed(SREADY, m & 1);
+                if (failed) return;
+                bulk_store(img0 + (size_t)m * STATE_BF16, base + OFF_S, STATE_BF16);
+                bulk_commit();
+                save_pending = true;
+            };
+            auto reads_done = [&]() {                  // every store issued so far has read its shared-memory source
+                bulk_wait_read0();
+                if (save_pending) { mbar_arrive(bar(SSAVED)); save_pending = false; }
+            };
             auto store_o = [&](int m) {                // staged by the compute warps; rows past T are clipped
                 wait_relaxed(OSTAGED, m & 1);
                 if (failed) return;
                 tma_store_5d(&tm_o, base + OFF_OST, 0, (n0 + m) * C, 0, h, b);
                 bulk_commit();
-                bulk_wait_read0();
+                reads_done();
                 mbar_arrive(bar(OSFREE));
             };
             load_g(0);
@@ -182,6 +198,7 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             for (int n = 0; n < 2 && n < NT; ++n) load_v(n);
             wait(OPR + 0, 0);                          // prologue of chunk 0 done: the log-decay buffer is free
             if (NT > 1 && !failed) load_g(1);
+            if (img0 && !failed) { save_s(0); reads_done(); }
             for (int n = 0; n < NT && !failed; ++n) {
                 if (n + 3 < NT) {                    // q/k buffer: free once A, qh S and kh^T V have read it
                     wait(QKFREE + n % 3, (n / 3) & 1);
@@ -198,7 +215,10 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
                     if (failed) break;
                     load_v(n + 2);
                 }
+                if (img0) save_s(n + 1);               // (the rescale of chunk n has just produced S_{n+1})
+                if (failed) break;
                 if (n > 0) store_o(n - 1);
+                else if (img0) reads_done();
             }
             if (!failed) store_o(NT - 1);
             bulk_wait0();
@@ -332,6 +352,7 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             wait(BAR_Z, par);
             tc_fence_after();
             SLA_TS(4);
+            if (p.simg) wait(SSAVED, par);             // the image store of S_n has read the operand copy
             {
                 const float e = eblast[(n & 1) * D + row];
 #pragma unroll
@@ -447,7 +468,13 @@ size_t gla_tc_forward_workspace_bytes(const Dims &d) {
     return (size_t)d.B * d.H * P * (2 * D * D + D) * sizeof(float);
 }
 
-int gla_tc_forward(const Dims &d, const FwdArgs &a, int *status, cudaStream_t st, Tracer &tr) {
+bool gla_tc_forward_can_save(const Dims &d) {
+    int P, L;
+    choose_segments(d, P, L);
+    return P == 1;
+}
+
+int gla_tc_forward(const Dims &d, const FwdArgs &a, uint8_t *simg, int *status, cudaStream_t st, Tracer &tr) {
     CUtensorMap mq, mk, mv, mg, mo;
     if (!make_tile_map(&mq, a.q, d.B, d.T, d.H) || !make_tile_map(&mk, a.k, d.B, d.T, d.H) ||
         !make_tile_map(&mv, a.v, d.B, d.T, d.H) || !make_map(&mg, a.log_decay, d.B, d.T, d.H, d.dk, true, 128) ||
@@ -465,7 +492,8 @@ int gla_tc_forward(const Dims &d, const FwdArgs &a, int *status, cudaStream_t st
         h0 = start;
         launches = 3;
     }
-    FwdParams p{a.lq, a.lk, h0, (__nv_bfloat16 *)a.o, a.ht, status, d.T, d.H, d.NT, P, L, d.scale, g_phase_ts};
+    if (P > 1) simg = nullptr;
+    FwdParams p{a.lq, a.lk, h0, (__nv_bfloat16 *)a.o, a.ht, simg, status, d.T, d.H, d.NT, P, L, d.scale, g_phase_ts};
     k_gla_fwd_tc<<<d.B * d.H * P, NTHREADS, SMEM_BYTES, st>>>(mq, mk, mv, mg, mo, p);
     tr.mark("gla_fwd_tc");
     return cudaGetLastError() == cudaSuccess ? launches : -1;

@@ -181,8 +181,7 @@ k_gla_states_tc(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
                 if (!images) continue;
                 wait_relaxed(STAGED, n & 1);           // image of S_{n+1} is staged
                 if (failed) break;
-                asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
-                             ::"l"((uint64_t)(img0 + (size_t)(n + 1) * STATE_BF16)), "r"(base + OFF_IMG), "r"(STATE_BF16) : "memory");
+                bulk_store(img0 + (size_t)(n + 1) * STATE_BF16, base + OFF_IMG, STATE_BF16);
                 bulk_commit();
                 bulk_wait_read0();
                 mbar_arrive(bar(STFREE));
@@ -871,7 +870,9 @@ int gla_tc_segment_summaries(const Dims &d, const FwdArgs &a, int P, int L, floa
     return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 
-int gla_tc_backward(const Dims &d, const BwdArgs &a, int *status, cudaStream_t st, Tracer &tr) {
+uint8_t *gla_tc_state_images(float *ws) { return reinterpret_cast<uint8_t *>(ws); }
+
+int gla_tc_backward(const Dims &d, const BwdArgs &a, bool have_states, int *status, cudaStream_t st, Tracer &tr) {
     CUtensorMap mq, mk, mv, mdo, mg, mdq, mdk, mdv, mdg;
     if (!make_tile_map(&mq, a.q, d.B, d.T, d.H) || !make_tile_map(&mk, a.k, d.B, d.T, d.H) ||
         !make_tile_map(&mv, a.v, d.B, d.T, d.H) || !make_tile_map(&mdo, a.dO, d.B, d.T, d.H) ||
@@ -886,15 +887,17 @@ int gla_tc_backward(const Dims &d, const BwdArgs &a, int *status, cudaStream_t s
     float *pq = a.ws + img_floats;
     float *pk = pq + ((bth + 63) & ~(size_t)63);
 
-    StatesParams sp{a.lq, a.lk, a.h0, simg, nullptr, nullptr, status, d.T, d.H, d.NT, 1, d.NT};
-    k_gla_states_tc<<<d.B * d.H, st1::NTHREADS, st1::SMEM_BYTES, st>>>(mk, mv, mg, sp);
-    tr.mark("gla_states_tc");
+    if (!have_states) {   // (otherwise the forward pass of the same inputs has left the images in this workspace)
+        StatesParams sp{a.lq, a.lk, a.h0, simg, nullptr, nullptr, status, d.T, d.H, d.NT, 1, d.NT};
+        k_gla_states_tc<<<d.B * d.H, st1::NTHREADS, st1::SMEM_BYTES, st>>>(mk, mv, mg, sp);
+        tr.mark("gla_states_tc");
+    }
     BwdParams bp{a.lq, a.lk, a.dht, simg, pq, pk, a.dh0, status, d.T, d.H, d.NT, d.scale, gla_tc_phase_ts()};
     k_gla_bwd_tc<<<d.B * d.H, st2::NTHREADS, st2::SMEM_BYTES, st>>>(mq, mk, mv, mdo, mg, mdq, mdk, mdv, mdg, bp);
     tr.mark("gla_bwd_tc");
     if (gate_bwd_prod(a.lq, a.lk, pq, pk, a.dlq, a.dlk, (long)d.B * d.T, d.H, st) < 0) return -1;
     tr.mark("gate_bwd");
-    return cudaGetLastError() == cudaSuccess ? 3 : -1;
+    return cudaGetLastError() == cudaSuccess ? (have_states ? 2 : 3) : -1;
 }
 
 }  // namespace sla

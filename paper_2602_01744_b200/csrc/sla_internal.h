@@ -97,7 +97,11 @@ bool gla_tc_supported(const Dims &d);
 int gla_tc_configure();
 void gla_tc_set_phase_ts(unsigned long long *device_buffer);
 unsigned long long *gla_tc_phase_ts();
-int gla_tc_forward(const Dims &d, const FwdArgs &a, int *status, cudaStream_t st, Tracer &tr);
+// With `simg` not null (and gla_tc_forward_can_save) the forward also leaves the bf16 image of the state before every
+// chunk there, in the layout the gradient sweep reads: the backward pass of the same inputs then needs no state sweep.
+bool gla_tc_forward_can_save(const Dims &d);
+uint8_t *gla_tc_state_images(float *ws);   // where in the backward workspace the images sit
+int gla_tc_forward(const Dims &d, const FwdArgs &a, uint8_t *simg, int *status, cudaStream_t st, Tracer &tr);
 // Backward: chunk-state sweep, gradient sweep, gate softmax backward.  Needs the first
 // B*H*(NT+1)*32 KiB + 2*B*T*H*4 bytes (rounded up) of the workspace, less than the generic path.
 int gla_tc_bwd_configure();
@@ -108,17 +112,18 @@ int gla_tc_segment_summaries(const Dims &d, const FwdArgs &a, int P, int L, floa
 // Bytes of workspace the tensor-core forward / backward need (the generic kernels need more).
 size_t gla_tc_forward_workspace_bytes(const Dims &d);
 size_t gla_tc_backward_workspace_bytes(const Dims &d);
-int gla_tc_backward(const Dims &d, const BwdArgs &a, int *status, cudaStream_t st, Tracer &tr);
+int gla_tc_backward(const Dims &d, const BwdArgs &a, bool have_states, int *status, cudaStream_t st, Tracer &tr);
 
 // ---- tensor-core Softmax-GatedDeltaNet forward (WY form): sla_gdn_tc.cu.  Needs no workspace. ----
 bool gdn_tc_supported(const Dims &d);
 int gdn_tc_configure();
-int gdn_tc_forward(const Dims &d, const FwdArgs &a, int *status, cudaStream_t st, Tracer &tr);
+int gdn_tc_forward(const Dims &d, const FwdArgs &a, uint8_t *save, int *status, cudaStream_t st, Tracer &tr);
+uint8_t *gdn_tc_records(float *ws);        // where in the backward workspace the per-chunk records sit
 int gdn_tc_forward_save(const Dims &d, const FwdArgs &a, uint8_t *save, int *status, cudaStream_t st, Tracer &tr);
 // backward: forward sweep in save mode (per-chunk S_n, U, T records), reverse gradient sweep, gate softmax backward
 int gdn_tc_bwd_configure();
 size_t gdn_tc_backward_workspace_bytes(const Dims &d);
-int gdn_tc_backward(const Dims &d, const BwdArgs &a, int *status, cudaStream_t st, Tracer &tr);
+int gdn_tc_backward(const Dims &d, const BwdArgs &a, bool have_records, int *status, cudaStream_t st, Tracer &tr);
 int gate_bwd_prod(const float *lq, const float *lk, const float *pq, const float *pk, float *dlq, float *dlk, long n_tok,
                   int H, cudaStream_t st);
 
@@ -136,6 +141,13 @@ struct sla_plan {
     int device;
     int *d_status;          // device status word (bounded waits report here)
     int last_launches;
+    // SLA_FLAG_SAVE_FOR_BACKWARD: what the last sla_forward left in its workspace, and for which inputs
+    struct Saved {
+        bool valid = false;
+        const void *ws = nullptr, *q = nullptr, *k = nullptr, *v = nullptr, *log_decay = nullptr, *beta = nullptr, *lq = nullptr,
+                   *lk = nullptr, *h0 = nullptr;
+        void *stream = nullptr;
+    } saved;
     sla::Tracer tracer;
     std::vector<std::pair<const char *, std::pair<int, float>>> agg;   // name -> (launches, total ms)
 };

@@ -88,3 +88,37 @@ def check_backward(cfg, with_h0=False, flags=0, bsel=None):
         errs[gname] = rel_l2(g[gname][sel] if g[gname].dim() > 1 else g[gname], ref[rname])
     assert all(np.isfinite(e) and e <= tol for e in errs.values()), (cfg, errs)
     return errs
+
+
+def gpu_training_step(cfg, x, h0=None, dht=None, want_dh0=False):
+    """Forward then backward on one SLA_FLAG_SAVE_FOR_BACKWARD plan and one workspace, as a training step runs them.
+    Returns (o, ht, gradients, plan, launches of the forward, launches of the backward)."""
+    plan = api.sla_plan_create(cfg.variant, cfg.dtype, cfg.B, cfg.T, cfg.H, cfg.d_k, cfg.d_v, cfg.chunk, cfg.scale,
+                               api.SLA_FLAG_SAVE_FOR_BACKWARD)
+    ws = plan.workspace(backward=True)
+    ht = torch.empty((cfg.B, cfg.H, cfg.d_k, cfg.d_v), dtype=torch.float32, device="cuda")
+    o, ht = api.sla_forward(plan, x["q"], x["k"], x["v"], x["log_decay"], x["gq_logits"], x["gk_logits"],
+                            beta=x["beta"], h0=h0, ht=ht, workspace=ws)
+    lf = plan.last_launch_count
+    g = api.sla_backward(plan, x["q"], x["k"], x["v"], x["log_decay"], x["gq_logits"], x["gk_logits"], x["dO"],
+                         beta=x["beta"], h0=h0, dht=dht, want_dh0=want_dh0, workspace=ws)
+    lb = plan.last_launch_count
+    torch.cuda.synchronize()
+    plan.poll()
+    return o, ht, g, plan, ws, lf, lb
+
+
+def check_training_step(cfg, with_h0=False):
+    """Parity of o, ht and every gradient when the backward reads what the forward left in the workspace."""
+    x = make_inputs(cfg, with_dO=True, with_h0=with_h0)
+    xd = to_dev(x)
+    o, ht, g, plan, ws, lf, lb = gpu_training_step(cfg, xd, h0=xd.get("h0"), dht=xd.get("dht"), want_dh0=with_h0)
+    oref, htref = oracle_forward(cfg, x, h0=x.get("h0"))
+    ref = oracle_backward(cfg, x, h0=x.get("h0"), dht=x.get("dht"))
+    errs = {"o": rel_l2(o, oref), "ht": rel_l2(ht, htref)}
+    for gname, rname in GRAD_NAMES.items():
+        if g.get(gname) is not None:
+            errs[gname] = rel_l2(g[gname], ref[rname])
+    tol = TOL[cfg.dtype]
+    assert all(np.isfinite(e) and e <= tol for e in errs.values()), (cfg, errs)
+    return errs, lf, lb

@@ -98,3 +98,45 @@ def test_tc_paths_with_thirty_two_heads():
         cfg = small(CONFIGS[base], B=1, T=130, H=32, seed=720)
         assert max(gu.check_forward(small(cfg, backward=False)).values()) <= 1e-2
         assert max(gu.check_backward(cfg).values()) <= 1e-2
+
+
+@pytest.mark.parametrize("base", ["C2", "C4"])
+@pytest.mark.parametrize("B,T,H,with_h0", [(1, 64, 1, False), (2, 200, 3, True), (1, 960, 8, True), (3, 65, 4, True), (1, 5, 2, False)])
+def test_training_step_backward_reads_what_the_forward_left(base, B, T, H, with_h0):
+    cfg = small(CONFIGS[base], B=B, T=T, H=H, seed=900 + T)
+    errs, lf, lb = gu.check_training_step(cfg, with_h0=with_h0)
+    assert (lf, lb) == (1, 2)                          # no state sweep (GLA) / no forward recomputation (GDN) in the backward
+    assert max(errs.values()) <= 1e-2
+
+
+@pytest.mark.parametrize("base", ["C2", "C4"])
+def test_saved_states_are_used_only_for_the_same_inputs_and_never_change_the_result(base):
+    cfg = small(CONFIGS[base], B=2, T=300, H=4, seed=910)
+    x = gu.to_dev(make_inputs(cfg, with_dO=True))
+    o, ht, g, plan, ws, lf, lb = gu.gpu_training_step(cfg, x)
+    args = (x["q"], x["k"], x["v"], x["log_decay"], x["gq_logits"], x["gk_logits"], x["dO"])
+    # another workspace: nothing was left there, so the backward recomputes (3 launches) and gives the same bits
+    g2 = api.sla_backward(plan, *args, beta=x["beta"])
+    assert plan.last_launch_count == 3
+    # other inputs (a copy of k at another address) with the forward's workspace: recomputed as well
+    k2 = x["k"].clone()
+    g3 = api.sla_backward(plan, x["q"], k2, *args[2:], beta=x["beta"], workspace=ws)
+    assert plan.last_launch_count == 3
+    # a plan without the flag leaves nothing and asks for no forward workspace beyond its own
+    plain = api.sla_plan_create(cfg.variant, cfg.dtype, cfg.B, cfg.T, cfg.H, cfg.d_k, cfg.d_v, cfg.chunk, cfg.scale)
+    assert plain.forward_workspace_bytes == 0 and plan.forward_workspace_bytes == plan.backward_workspace_bytes
+    api.sla_forward(plain, *args[:6], beta=x["beta"], workspace=ws)
+    g4 = api.sla_backward(plain, *args, beta=x["beta"], workspace=ws)
+    assert plain.last_launch_count == 3
+    torch.cuda.synchronize()
+    for other in (g2, g3, g4):
+        for n, t in g.items():
+            if t is not None:
+                assert torch.equal(t, other[n]), n
+
+
+def test_segmented_forward_leaves_nothing_and_the_backward_recomputes():
+    cfg = small(CONFIGS["C2"], B=1, T=2048, H=4, seed=920)     # few long sequences: the forward runs in segments
+    errs, lf, lb = gu.check_training_step(cfg)
+    assert lf == 3 and lb == 3
+    assert max(errs.values()) <= 1e-2
