@@ -298,10 +298,10 @@ k_gdn_bwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             const size_t tok = tokb + (size_t)n * C + t;
             float *dst = gate_s + (k & 3) * 4 * C;
             if (g < C) {
-                dst[t] = t < cn ? p.scale * token_gate_any(p.lq + tok * p.H, p.H, h) : 0.f;
+                chunk_gate(p.lq + (tok - t) * p.H, p.H, cn, h, p.scale, dst, t);
                 dst[2 * C + t] = t < cn ? p.g[tok * p.H + h] : 0.f;
             } else {
-                dst[C + t] = t < cn ? token_gate_any(p.lk + tok * p.H, p.H, h) : 0.f;
+                chunk_gate(p.lk + (tok - t) * p.H, p.H, cn, h, 1.f, dst + C, t);
                 dst[3 * C + t] = t < cn ? p.beta[tok * p.H + h] : 0.f;
             }
             __syncwarp();

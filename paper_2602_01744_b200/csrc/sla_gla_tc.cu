@@ -30,19 +30,20 @@ constexpr uint32_t OFF_S = OFF_V + 2 * TILE_BF16;               // bf16 state op
 constexpr uint32_t OFF_A = OFF_S + STATE_BF16;                  // masked A, [64 rows][128 B]
 constexpr uint32_t OFF_OST = OFF_A + HALF_BF16;                 // bf16 output tile staged for the TMA store
 constexpr uint32_t OFF_TOT = OFF_OST + TILE_BF16;               // prologue scratch
-constexpr uint32_t OFF_EB = OFF_TOT + TOT_BYTES;                // [2][128] 2^{b_last}
-constexpr uint32_t OFF_GATE = OFF_EB + 2 * D * 4;               // [4][2][64]: scale*Gq, Gk of four chunks
+constexpr uint32_t OFF_EB = OFF_TOT + TOT_BYTES;                // [4][128] 2^{b_last} of four chunks
+constexpr uint32_t OFF_GATE = OFF_EB + 4 * D * 4;               // [4][2][64]: scale*Gq, Gk of four chunks
 constexpr uint32_t OFF_BAR = OFF_GATE + 4 * 2 * C * 4;          // mbarriers, see Bar
 constexpr uint32_t OFF_TMEM = OFF_BAR + 32 * 8;                 // TMEM base address, then the abort flag
 constexpr uint32_t SMEM_BYTES = OFF_TMEM + 16 + 1024;           // + slack to align the base to 1024 B
 static_assert(SMEM_BYTES <= 232448, "shared memory budget");
 
 constexpr uint32_t COL_A = 0, COL_O = 64, COL_S = 320, TMEM_COLS = 512;   // O: two buffers of 128 columns
-constexpr int NTHREADS = NCOMPUTE + 32 + NGATE + 32;   // warps 0..7 compute, 8 MMA issue, 9..12 gates, 13 TMA
+constexpr int W_PRO = 8, W_MMA = 16, W_GATE = 17, W_TMA = 21;      // first warp of each role
+constexpr int NTHREADS = 2 * NCOMPUTE + 32 + NGATE + 32;
 
 // mbarrier slots (8 bytes each)
 enum Bar { FULL_G = 0, FULL_QK = 1, FULL_V = 4, OPR = 6, GREADY = 9, GFREE = 13, SREADY = 17, OFREE, AREADY, BAR_A, BAR_Z,
-           BAR_O /* [2], one per O accumulator */, OSTAGED = BAR_O + 2, OSFREE, DRAIN, QKFREE /* [3] */, SSAVED = QKFREE + 3, NBAR };
+           BAR_O /* [2], one per O accumulator */, OSTAGED = BAR_O + 2, OSFREE, DRAIN, QKFREE /* [3] */, SSAVED = QKFREE + 3, GTFREE, NBAR };
 static_assert(NBAR <= 32, "barrier slots");
 
 struct FwdParams {
@@ -58,13 +59,14 @@ struct FwdParams {
 };
 #define SLA_TS(k) do { if (p.phase_ts && bh == 0 && tid == 0 && n == 8) p.phase_ts[k] = globaltimer_ns(); } while (0)
 
-// One CTA per (batch, head) sequence, four roles:
-//   warp 8 (one lane)  every tcgen05.mma
-//   warp 13 (one lane) TMA: loads (log-decay one chunk ahead, q/k three, v two) and the output store
-//   warps 9..12        head-softmax gates (Eq. 4) up to four chunks ahead, one thread per (token, gate)
-//   warps 0..7         prologue (cumulative decay, qh, kh), causal mask of A, state rescale, output staging
-// While the tensor core works on chunk n the compute warps already run the prologue of chunk n+1, so per chunk
-// the critical path is prologue -> mask -> rescale -> store.
+// One CTA per (batch, head) sequence, five roles that only meet on mbarriers:
+//   warps 8..15        prologue: cumulative decay, qh, kh of the chunks ahead (as far as the three q/k buffers allow)
+//   warps 0..7         causal mask of A, state rescale, output staging (TMEM lane quarter = warp % 4)
+//   warp 16 (one lane) every tcgen05.mma
+//   warp 21 (one lane) TMA: loads (log-decay one chunk ahead, q/k three, v two) and the output store
+//   warps 17..20       head-softmax gates (Eq. 4) up to four chunks ahead, one thread per (token, gate)
+// The prologue of chunk n+1.. runs beside the mask / rescale / store work of chunk n, so the shared-memory,
+// special-function and FMA phases of the two groups overlap instead of following one another.
 __global__ void __launch_bounds__(NTHREADS, 1)
 k_gla_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
              const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_g,
@@ -95,7 +97,7 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
     if (tid == 0) {
         *abort_flag = 0;
         for (int i = 0; i < NBAR; ++i) {
-            const bool all = (i >= OPR && i < GREADY) || (i >= GFREE && i <= AREADY) || i == OSTAGED;
+            const bool all = (i >= OPR && i < GREADY) || (i >= GFREE && i <= AREADY) || i == OSTAGED || i == GTFREE;   // 256 arrivals
             mbar_init(bar(i), all ? NCOMPUTE : (i >= GREADY && i < GFREE) ? NGATE / 32 : 1);
         }
         fence_mbar_init();
@@ -112,7 +114,7 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
     const uint32_t tmem = *reinterpret_cast<volatile uint32_t *>(sm + OFF_TMEM);
     const size_t tokb = (size_t)b * p.T;
 
-    if (warp == 8) {
+    if (warp == W_MMA) {
         // ---------------- MMA issue (one lane) ----------------
         if (lane == 0) {
             constexpr uint32_t ID_A = idesc_bf16(64, 64, 0, 0);      // qh (K-major) x kh (K-major)
@@ -153,7 +155,7 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             tc_commit(bar(DRAIN));
             mbar_wait_bounded(bar(DRAIN), 0, nullptr, 20000000ull);
         }
-    } else if (warp == 13) {
+    } else if (warp == W_TMA) {
         // ---------------- TMA (one lane): loads ahead of the compute warps, output stores behind them ----------------
         if (lane == 0) {
             auto load_g = [&](int n) {
@@ -173,75 +175,89 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             };
             // save mode: S_m (the bf16 operand copy, as it stands in shared memory) -> image slot m, for the backward pass
             uint8_t *img0 = p.simg ? p.simg + (size_t)bh * (p.NT + 1) * STATE_BF16 : nullptr;
-            bool save_pending = false;
-            auto save_s = [&](int m) {
-                wait_relaxed(SREADY, m & 1);
-                if (failed) return;
-                bulk_store(img0 + (size_t)m * STATE_BF16, base + OFF_S, STATE_BF16);
-                bulk_commit();
-                save_pending = true;
-            };
-            auto reads_done = [&]() {                  // every store issued so far has read its shared-memory source
-                bulk_wait_read0();
-                if (save_pending) { mbar_arrive(bar(SSAVED)); save_pending = false; }
-            };
-            auto store_o = [&](int m) {                // staged by the compute warps; rows past T are clipped
-                wait_relaxed(OSTAGED, m & 1);
-                if (failed) return;
-                tma_store_5d(&tm_o, base + OFF_OST, 0, (n0 + m) * C, 0, h, b);
-                bulk_commit();
-                reads_done();
-                mbar_arrive(bar(OSFREE));
-            };
             load_g(0);
             for (int n = 0; n < 3 && n < NT; ++n) load_qk(n);
             for (int n = 0; n < 2 && n < NT; ++n) load_v(n);
-            wait(OPR + 0, 0);                          // prologue of chunk 0 done: the log-decay buffer is free
-            if (NT > 1 && !failed) load_g(1);
-            if (img0 && !failed) { save_s(0); reads_done(); }
-            for (int n = 0; n < NT && !failed; ++n) {
-                if (n + 3 < NT) {                    // q/k buffer: free once A, qh S and kh^T V have read it
-                    wait(QKFREE + n % 3, (n / 3) & 1);
-                    if (failed) break;
-                    load_qk(n + 3);
+            // From here on the lane serves whichever buffer falls free or fills first (no fixed order: the prologue warps
+            // run ahead of the tensor core by a varying distance).  Next chunk to load / store per stream:
+            int ng = 1, nqk = 3, nv = 2, nst = 0, nsv = img0 ? 0 : NT + 1;
+            auto ready = [&](int i, uint32_t parity) { return mbar_test_wait(bar(i), parity) != 0; };
+            uint64_t t_idle = globaltimer_ns();
+            for (uint32_t it = 0; !failed && (nst < NT || nsv <= NT); ++it) {
+                bool progress = false;
+                if (ng < NT && ready(GTFREE, (ng - 1) & 1)) {                   // the prologue of chunk ng-1 has read the tile
+                    load_g(ng++);
+                    progress = true;
                 }
-                if (n + 2 < NT) {                    // log-decay buffer: free once the prologue of chunk n+1 is done
-                    wait(OPR + (n + 1) % 3, ((n + 1) / 3) & 1);
-                    if (failed) break;
-                    load_g(n + 2);
+                if (nqk < NT && ready(QKFREE + nqk % 3, ((nqk - 3) / 3) & 1)) { // A, qh S and kh^T V of chunk nqk-3 have read it
+                    load_qk(nqk++);
+                    progress = true;
                 }
-                if (n + 2 < NT) {                    // v buffer: free once A V has read it
-                    wait(BAR_O + (n & 1), (n >> 1) & 1);
-                    if (failed) break;
-                    load_v(n + 2);
+                if (nv < NT && ready(BAR_O + (nv & 1), ((nv - 2) >> 1) & 1)) {  // A V of chunk nv-2 has read it
+                    load_v(nv++);
+                    progress = true;
                 }
-                if (img0) save_s(n + 1);               // (the rescale of chunk n has just produced S_{n+1})
-                if (failed) break;
-                if (n > 0) store_o(n - 1);
-                else if (img0) reads_done();
+                if (nsv <= NT && ready(SREADY, nsv & 1)) {                       // S_nsv stands in shared memory
+                    bulk_store(img0 + (size_t)nsv * STATE_BF16, base + OFF_S, STATE_BF16);
+                    bulk_commit();
+                    bulk_wait_read0();
+                    mbar_arrive(bar(SSAVED));
+                    ++nsv;
+                    progress = true;
+                }
+                if (nst < NT && ready(OSTAGED, nst & 1)) {                       // O of chunk nst is staged; rows past T are clipped
+                    tma_store_5d(&tm_o, base + OFF_OST, 0, (n0 + nst) * C, 0, h, b);
+                    bulk_commit();
+                    bulk_wait_read0();
+                    mbar_arrive(bar(OSFREE));
+                    ++nst;
+                    progress = true;
+                }
+                if (progress) {
+                    t_idle = globaltimer_ns();
+                } else if ((it & 31u) == 31u) {
+                    if (*abort_flag || globaltimer_ns() - t_idle > 2000000000ull) { failed = true; *abort_flag = 1; }
+                    __nanosleep(64);
+                }
             }
-            if (!failed) store_o(NT - 1);
             bulk_wait0();
             if (failed) {   // give loads that are still in flight time to land before shared memory goes away
                 const uint64_t t0 = globaltimer_ns();
                 while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
             }
         }
-    } else if (warp >= 9) {
+    } else if (warp >= W_GATE) {
         // ---------------- gates: softmax over the heads, up to four chunks ahead ----------------
-        const int g = tid - (NCOMPUTE + 32), t = g & (C - 1);
+        const int g = tid - 32 * W_GATE, t = g & (C - 1);
         const float *l = g < C ? p.lq : p.lk;
         const float mult = g < C ? p.scale : 1.f;
         for (int n = 0; n < NT; ++n) {
             if (n >= 4) wait_relaxed(GFREE + (n & 3), ((n >> 2) - 1) & 1);
             if (failed) break;
             const int cn = min(C, p.T - (n0 + n) * C);
-            gate_s[(n & 3) * 2 * C + g] = t < cn ? mult * token_gate_any(l + (tokb + (size_t)(n0 + n) * C + t) * p.H, p.H, h) : 0.f;
+            chunk_gate(l + (tokb + (size_t)(n0 + n) * C) * p.H, p.H, cn, h, mult, gate_s + (n & 3) * 2 * C + (g < C ? 0 : C), t);
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(GREADY + (n & 3)));
         }
+    } else if (warp >= W_PRO) {
+        // ---------------- prologue warps: qh, kh of every chunk, ahead of the tensor core ----------------
+        const int ptid = tid - 32 * W_PRO;
+        for (int n = 0; n < NT; ++n) {
+            wait(GREADY + (n & 3), (n >> 2) & 1);
+            wait(FULL_G, n & 1);
+            wait(FULL_QK + n % 3, (n / 3) & 1);
+            if (failed) break;
+            uint8_t *qk = sm + OFF_QK + (n % 3) * QK_BYTES;
+            const float *g = gate_s + (n & 3) * 2 * C;
+            // eblast has four slots: these warps are never more than three chunks ahead of the rescale that reads one
+            chunk_prologue<true, false>(qk, qk + TILE_BF16, reinterpret_cast<const float *>(sm + OFF_G), tot, g, g + C,
+                                        eblast + (n & 3) * D, nullptr, ptid, 2, bar(GTFREE));
+            fence_proxy_async();
+            mbar_arrive(bar(OPR + n % 3));
+            mbar_arrive(bar(GFREE + (n & 3)));
+        }
     } else {
-        // ---------------- compute warps ----------------
+        // ---------------- mask / rescale / store warps ----------------
         const uint32_t lane_base = (uint32_t)(32 * (warp & 3)) << 16;   // this warp's TMEM lane quarter
         const int colhalf = warp >> 2;                                   // which 64 state / output columns
         const int row = 32 * (warp & 3) + lane;
@@ -270,18 +286,6 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
         tc_fence_before();
         mbar_arrive(bar(SREADY));
 
-        auto prologue = [&](int n) {
-            wait(GREADY + (n & 3), (n >> 2) & 1);
-            wait(FULL_G, n & 1);
-            wait(FULL_QK + n % 3, (n / 3) & 1);
-            uint8_t *qk = sm + OFF_QK + (n % 3) * QK_BYTES;
-            const float *g = gate_s + (n & 3) * 2 * C;
-            chunk_prologue<true, false>(qk, qk + TILE_BF16, reinterpret_cast<const float *>(sm + OFF_G), tot, g, g + C,
-                                        eblast + (n & 1) * D, nullptr, tid);
-            fence_proxy_async();
-            mbar_arrive(bar(OPR + n % 3));
-            mbar_arrive(bar(GFREE + (n & 3)));
-        };
         // O of chunk m: TMEM -> bf16 -> staging tile (the TMA warp stores it)
         auto stage_o = [&](int m) {
             wait(BAR_O + (m & 1), (m >> 1) & 1);
@@ -313,12 +317,9 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             fence_proxy_async();
             mbar_arrive(bar(OSTAGED));
         };
-        prologue(0);
-
         for (int n = 0; n < NT; ++n) {
             const uint32_t par = n & 1;
             SLA_TS(0);
-            if (n + 1 < NT) prologue(n + 1);         // overlaps the MMAs of chunk n
             SLA_TS(1);
 
             // A: TMEM -> causal mask -> bf16 -> shared memory (row i of the M=64 tile sits in lane 32*(i/16) + i%16)
@@ -354,7 +355,7 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             SLA_TS(4);
             if (p.simg) wait(SSAVED, par);             // the image store of S_n has read the operand copy
             {
-                const float e = eblast[(n & 1) * D + row];
+                const float e = eblast[(n & 3) * D + row];
 #pragma unroll
                 for (int part = 0; part < 2; ++part) {
                     float v[32];

@@ -102,7 +102,7 @@ __device__ __forceinline__ float ex2f(float x) {
 constexpr uint32_t NCOMPUTE = 256;      // compute threads (warps 0..7); they meet on named barrier 1
 constexpr float LOG2E = 1.4426950408889634f;
 
-// Chunk prologue, run by the 256 compute threads on one landed stage (Eq. 12's decay made chunk-local):
+// Chunk prologue, run by 256 threads (tid 0..255, meeting on named barrier bar_id) on one landed stage (Eq. 12's decay made chunk-local):
 //   b_i = inclusive cumulative log-decay (kept in log2 units), two-level: per-8-row sums, then a running sum
 //   qh_i = gq_i * q_i * 2^{b_i}   (gq_i = scale*Gq_i)      kh_i = gk_i * k_i * 2^{-b_i}
 // written over q and k in place (the swizzled tiles are the MMA operands); eblast[d] = 2^{b_last,d}.
@@ -114,19 +114,21 @@ constexpr uint32_t TOT_BYTES = 8 * D * 4;
 template <bool WITH_Q, bool WITH_E>
 __device__ __forceinline__ void chunk_prologue(uint8_t *q_tile, uint8_t *k_tile, const float *gs, float *tot,
                                                const float *gq_s, const float *gk_s, float *eblast,
-                                               uint8_t *e2_tile, int tid) {
+                                               uint8_t *e2_tile, int tid, int bar_id = 1, uint32_t g_free_bar = 0) {
     using namespace ptx;
     const int rg = tid >> 5, cj = tid & 31;
+    float4 gl[8];                               // this thread's log-decay rows: read once, kept for the second pass
     {
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
         for (int rr = 0; rr < 8; ++rr) {
-            const float4 g = *reinterpret_cast<const float4 *>(gs + (8 * rg + rr) * D + 4 * cj);
-            acc.x += g.x; acc.y += g.y; acc.z += g.z; acc.w += g.w;
+            gl[rr] = *reinterpret_cast<const float4 *>(gs + (8 * rg + rr) * D + 4 * cj);
+            acc.x += gl[rr].x; acc.y += gl[rr].y; acc.z += gl[rr].z; acc.w += gl[rr].w;
         }
         *reinterpret_cast<float4 *>(tot + rg * D + 4 * cj) = acc;
     }
-    named_bar_sync(1, NCOMPUTE);
+    if (g_free_bar) mbar_arrive(g_free_bar);    // the log-decay tile may be overwritten once every thread has said so
+    named_bar_sync(bar_id, NCOMPUTE);
     float bsum[4] = {0.f, 0.f, 0.f, 0.f};
     for (int g = 0; g < rg; ++g) {
         const float4 a = *reinterpret_cast<const float4 *>(tot + g * D + 4 * cj);
@@ -139,7 +141,7 @@ __device__ __forceinline__ void chunk_prologue(uint8_t *q_tile, uint8_t *k_tile,
 #pragma unroll
     for (int rr = 0; rr < 8; ++rr) {
         const int r = 8 * rg + rr;
-        const float4 g = *reinterpret_cast<const float4 *>(gs + r * D + 4 * cj);
+        const float4 g = gl[rr];
         bsum[0] = fmaf(g.x, LOG2E, bsum[0]); bsum[1] = fmaf(g.y, LOG2E, bsum[1]);
         bsum[2] = fmaf(g.z, LOG2E, bsum[2]); bsum[3] = fmaf(g.w, LOG2E, bsum[3]);
         const float gq = WITH_Q ? gq_s[r] : 0.f, gk = gk_s[r];
@@ -198,6 +200,43 @@ __device__ __forceinline__ float token_gate_any(const float *row, int H, int h) 
     if (H <= 8) return token_gate<8>(row, H, h);
     if (H <= 16) return token_gate<16>(row, H, h);
     return token_gate<32>(row, H, h);
+}
+// Gates of one chunk for head h, by the 64 threads (t = 0..63, two whole warps) that serve one of the two gates:
+// dst[i] = mult * softmax(L[i*H .. i*H+H))[h] for token i < cn, 0 for cn <= i < 64.  L points at the chunk's first
+// logit; consecutive tokens are consecutive rows of H floats, so for H = 4, 8, 16, 32 the block is read as whole
+// float4s, fully coalesced, H/4 lanes per token, and max / sum travel over shuffles (one exponential per logit).
+// Other H: one thread per token reads its own row.
+template <int LPT>
+__device__ __forceinline__ void chunk_gate_vec(const float *__restrict__ L, int cn, int h, float mult, float *dst, int t) {
+    float4 x[LPT];
+#pragma unroll
+    for (int i = 0; i < LPT; ++i) {
+        const int f = i * 64 + t;                      // float4 index inside the chunk's block; token f / LPT
+        x[i] = f / LPT < cn ? __ldg(reinterpret_cast<const float4 *>(L) + f) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+#pragma unroll
+    for (int i = 0; i < LPT; ++i) {
+        const int token = (i * 64 + t) / LPT;
+        float m = fmaxf(fmaxf(x[i].x, x[i].y), fmaxf(x[i].z, x[i].w));
+#pragma unroll
+        for (int o = 1; o < LPT; o <<= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+        const float e0 = __expf(x[i].x - m), e1 = __expf(x[i].y - m), e2 = __expf(x[i].z - m), e3 = __expf(x[i].w - m);
+        float sum = (e0 + e1) + (e2 + e3);
+#pragma unroll
+        for (int o = 1; o < LPT; o <<= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+        if ((t % LPT) == (h >> 2)) {
+            const int j = h & 3;
+            const float eh = j == 0 ? e0 : j == 1 ? e1 : j == 2 ? e2 : e3;
+            dst[token] = token < cn ? mult * eh / sum : 0.f;
+        }
+    }
+}
+__device__ __forceinline__ void chunk_gate(const float *L, int H, int cn, int h, float mult, float *dst, int t) {
+    if (H == 16) chunk_gate_vec<4>(L, cn, h, mult, dst, t);
+    else if (H == 8) chunk_gate_vec<2>(L, cn, h, mult, dst, t);
+    else if (H == 4) chunk_gate_vec<1>(L, cn, h, mult, dst, t);
+    else if (H == 32) chunk_gate_vec<8>(L, cn, h, mult, dst, t);
+    else dst[t] = t < cn ? mult * token_gate_any(L + (size_t)t * H, H, h) : 0.f;
 }
 constexpr int NGATE = 128;   // gate threads: g < 64 -> scale*Gq of token g, g >= 64 -> Gk of token g-64
 

@@ -199,7 +199,7 @@ k_gla_states_tc(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
             if (n >= 4) wait_relaxed(GFREE + (n & 3), ((n >> 2) - 1) & 1);
             if (failed) break;
             const int cn = min(C, p.T - (n0 + n) * C);
-            gate_s[(n & 3) * C + t] = t < cn ? token_gate_any(p.lk + (tokb + (size_t)(n0 + n) * C + t) * p.H, p.H, h) : 0.f;
+            chunk_gate(p.lk + (tokb + (size_t)(n0 + n) * C) * p.H, p.H, cn, h, 1.f, gate_s + (n & 3) * C, t);
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(GREADY + (n & 3)));
         }
@@ -556,7 +556,7 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             if (k >= 4) wait_relaxed(GFREE + (k & 3), ((k >> 2) - 1) & 1);
             if (failed) break;
             const int cn = min(C, p.T - n * C);
-            gate_s[(k & 3) * 2 * C + g] = t < cn ? mult * token_gate_any(l + (tokb + (size_t)n * C + t) * p.H, p.H, h) : 0.f;
+            chunk_gate(l + (tokb + (size_t)n * C) * p.H, p.H, cn, h, mult, gate_s + (k & 3) * 2 * C + (g < C ? 0 : C), t);
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(GREADY + (k & 3)));
         }
