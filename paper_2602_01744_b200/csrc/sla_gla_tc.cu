@@ -33,7 +33,7 @@ constexpr uint32_t OFF_TOT = OFF_OST + TILE_BF16;               // prologue scra
 constexpr uint32_t OFF_EB = OFF_TOT + TOT_BYTES;                // [4][128] 2^{b_last} of four chunks
 constexpr uint32_t OFF_GATE = OFF_EB + 4 * D * 4;               // [4][2][64]: scale*Gq, Gk of four chunks
 constexpr uint32_t OFF_BAR = OFF_GATE + 4 * 2 * C * 4;          // mbarriers, see Bar
-constexpr uint32_t OFF_TMEM = OFF_BAR + 32 * 8;                 // TMEM base address, then the abort flag
+constexpr uint32_t OFF_TMEM = OFF_BAR + 40 * 8;                 // TMEM base address, then the abort flag
 constexpr uint32_t SMEM_BYTES = OFF_TMEM + 16 + 1024;           // + slack to align the base to 1024 B
 static_assert(SMEM_BYTES <= 232448, "shared memory budget");
 
@@ -43,8 +43,9 @@ constexpr int NTHREADS = 2 * NCOMPUTE + 32 + NGATE + 32;
 
 // mbarrier slots (8 bytes each)
 enum Bar { FULL_G = 0, FULL_QK = 1, FULL_V = 4, OPR = 6, GREADY = 9, GFREE = 13, SREADY = 17, OFREE, AREADY, BAR_A, BAR_Z,
-           BAR_O /* [2], one per O accumulator */, OSTAGED = BAR_O + 2, OSFREE, DRAIN, QKFREE /* [3] */, SSAVED = QKFREE + 3, GTFREE, NBAR };
-static_assert(NBAR <= 32, "barrier slots");
+           BAR_O /* [2], one per O accumulator */, OSTAGED = BAR_O + 2, OSFREE, DRAIN, QKFREE /* [3] */, SSAVED = QKFREE + 3, ATAKEN,
+           OFREE2 /* OFREE, OFREE2: one per O accumulator (the output warps may be a chunk ahead of the waiter) */, NBAR };
+static_assert(NBAR <= 40, "barrier slots");
 
 struct FwdParams {
     const float *lq, *lk, *h0;
@@ -97,7 +98,7 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
     if (tid == 0) {
         *abort_flag = 0;
         for (int i = 0; i < NBAR; ++i) {
-            const bool all = (i >= OPR && i < GREADY) || (i >= GFREE && i <= AREADY) || i == OSTAGED || i == GTFREE;   // 256 arrivals
+            const bool all = (i >= OPR && i < GREADY) || (i >= GFREE && i <= AREADY) || i == OSTAGED || i == ATAKEN || i == OFREE2;   // 256 arrivals
             mbar_init(bar(i), all ? NCOMPUTE : (i >= GREADY && i < GFREE) ? NGATE / 32 : 1);
         }
         fence_mbar_init();
@@ -120,30 +121,40 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             constexpr uint32_t ID_A = idesc_bf16(64, 64, 0, 0);      // qh (K-major) x kh (K-major)
             constexpr uint32_t ID_O = idesc_bf16(64, 128, 0, 1);     // qh x S, A x V (B operand MN-major)
             constexpr uint32_t ID_Z = idesc_bf16(128, 128, 1, 1);    // kh^T (MN-major) x V (MN-major)
-            for (int n = 0; n < NT; ++n) {
+            auto issue_a = [&](int n) {                              // A_n = qh kh^T, one chunk ahead of the recurrence
+                const uint32_t sQ = base + OFF_QK + (n % 3) * QK_BYTES, sK = sQ + TILE_BF16;
+                wait(OPR + n % 3, (n / 3) & 1);                      // qh, kh of chunk n are in place
+                if (n > 0) wait(ATAKEN, (n - 1) & 1);                // A_{n-1} has been read out of tensor memory
+                if (failed) return;
+                tc_fence_after();
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk)
+                    tc_mma_bf16(tmem + COL_A, (desc_kmajor(sQ) + kstep_kmajor(kk, HALF_BF16)), (desc_kmajor(sK) + kstep_kmajor(kk, HALF_BF16)), ID_A, kk > 0);
+                tc_commit(bar(BAR_A));
+            };
+            issue_a(0);
+            for (int n = 0; n < NT && !failed; ++n) {
                 const uint32_t par = n & 1;
                 const uint32_t sQ = base + OFF_QK + (n % 3) * QK_BYTES, sK = sQ + TILE_BF16;
                 const uint32_t sV = base + OFF_V + (n & 1) * TILE_BF16;
                 const uint32_t tO = tmem + COL_O + (n & 1) * D;
-                wait(OPR + n % 3, (n / 3) & 1);        // qh, kh of chunk n are in place
                 wait(SREADY, par);                     // S_n: fp32 in TMEM, bf16 in shared memory
-                if (n > 1) wait(OFREE, n & 1);         // O of chunk n-2 (same TMEM buffer) has been read out
+                if (n > 1) wait((n & 1) ? OFREE2 : OFREE, ((n - 2) >> 1) & 1);   // O of chunk n-2 (same TMEM buffer) has been read out
                 wait(FULL_V + (n & 1), (n >> 1) & 1);
                 if (failed) break;
                 tc_fence_after();
+                // the recurrence: S += kh^T V and O = qh S_n; their commit releases the rescale
 #pragma unroll
-                for (int kk = 0; kk < 8; ++kk)         // A = qh kh^T
-                    tc_mma_bf16(tmem + COL_A, (desc_kmajor(sQ) + kstep_kmajor(kk, HALF_BF16)), (desc_kmajor(sK) + kstep_kmajor(kk, HALF_BF16)), ID_A, kk > 0);
-                tc_commit(bar(BAR_A));
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk)         // O = qh S_n
-                    tc_mma_bf16(tO, (desc_kmajor(sQ) + kstep_kmajor(kk, HALF_BF16)), (desc_mnmajor(base + OFF_S, STATE_HALF) + kstep_mnmajor(kk)), ID_O, kk > 0);
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk)         // S += kh^T V
+                for (int kk = 0; kk < 4; ++kk)
                     tc_mma_bf16(tmem + COL_S, (desc_mnmajor(sK, HALF_BF16) + kstep_mnmajor(kk)), (desc_mnmajor(sV, HALF_BF16) + kstep_mnmajor(kk)), ID_Z, 1);
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk)
+                    tc_mma_bf16(tO, (desc_kmajor(sQ) + kstep_kmajor(kk, HALF_BF16)), (desc_mnmajor(base + OFF_S, STATE_HALF) + kstep_mnmajor(kk)), ID_O, kk > 0);
                 tc_commit(bar(BAR_Z));
                 tc_commit(bar(QKFREE + n % 3));        // (same event, own barrier: the TMA lane may look at it much later)
-                wait(AREADY, par);                     // masked A is in shared memory
+                // beside the rescale: A of the next chunk, then A V of this one
+                if (n + 1 < NT) issue_a(n + 1);
+                wait(AREADY, par);                     // masked A_n is in shared memory
                 if (failed) break;
                 tc_fence_after();
 #pragma unroll
@@ -158,10 +169,6 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
     } else if (warp == W_TMA) {
         // ---------------- TMA (one lane): loads ahead of the compute warps, output stores behind them ----------------
         if (lane == 0) {
-            auto load_g = [&](int n) {
-                mbar_expect_tx(bar(FULL_G), TILE_G);
-                tma_load_4d(base + OFF_G, &tm_g, 0, h, (n0 + n) * C, b, bar(FULL_G));
-            };
             auto load_qk = [&](int n) {
                 const uint32_t bf = bar(FULL_QK + n % 3), dst = base + OFF_QK + (n % 3) * QK_BYTES;
                 mbar_expect_tx(bf, QK_BYTES);
@@ -175,20 +182,15 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             };
             // save mode: S_m (the bf16 operand copy, as it stands in shared memory) -> image slot m, for the backward pass
             uint8_t *img0 = p.simg ? p.simg + (size_t)bh * (p.NT + 1) * STATE_BF16 : nullptr;
-            load_g(0);
             for (int n = 0; n < 3 && n < NT; ++n) load_qk(n);
             for (int n = 0; n < 2 && n < NT; ++n) load_v(n);
             // From here on the lane serves whichever buffer falls free or fills first (no fixed order: the prologue warps
             // run ahead of the tensor core by a varying distance).  Next chunk to load / store per stream:
-            int ng = 1, nqk = 3, nv = 2, nst = 0, nsv = img0 ? 0 : NT + 1;
+            int nqk = 3, nv = 2, nst = 0, nsv = img0 ? 0 : NT + 1;
             auto ready = [&](int i, uint32_t parity) { return mbar_test_wait(bar(i), parity) != 0; };
             uint64_t t_idle = globaltimer_ns();
             for (uint32_t it = 0; !failed && (nst < NT || nsv <= NT); ++it) {
                 bool progress = false;
-                if (ng < NT && ready(GTFREE, (ng - 1) & 1)) {                   // the prologue of chunk ng-1 has read the tile
-                    load_g(ng++);
-                    progress = true;
-                }
                 if (nqk < NT && ready(QKFREE + nqk % 3, ((nqk - 3) / 3) & 1)) { // A, qh S and kh^T V of chunk nqk-3 have read it
                     load_qk(nqk++);
                     progress = true;
@@ -242,6 +244,11 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
     } else if (warp >= W_PRO) {
         // ---------------- prologue warps: qh, kh of every chunk, ahead of the tensor core ----------------
         const int ptid = tid - 32 * W_PRO;
+        auto load_g = [&](int n) {                     // (one thread) log-decay tile of chunk n
+            mbar_expect_tx(bar(FULL_G), TILE_G);
+            tma_load_4d(base + OFF_G, &tm_g, 0, h, (n0 + n) * C, b, bar(FULL_G));
+        };
+        if (ptid == 0) load_g(0);
         for (int n = 0; n < NT; ++n) {
             wait(GREADY + (n & 3), (n >> 2) & 1);
             wait(FULL_G, n & 1);
@@ -251,7 +258,8 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             const float *g = gate_s + (n & 3) * 2 * C;
             // eblast has four slots: these warps are never more than three chunks ahead of the rescale that reads one
             chunk_prologue<true, false>(qk, qk + TILE_BF16, reinterpret_cast<const float *>(sm + OFF_G), tot, g, g + C,
-                                        eblast + (n & 3) * D, nullptr, ptid, 2, bar(GTFREE));
+                                        eblast + (n & 3) * D, nullptr, ptid, 2,
+                                        [&]() { if (ptid == 0 && n + 1 < NT) load_g(n + 1); });
             fence_proxy_async();
             mbar_arrive(bar(OPR + n % 3));
             mbar_arrive(bar(GFREE + (n & 3)));
@@ -296,7 +304,7 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             tmem_ld32(tmem + lane_base + COL_O + (m & 1) * D + 64 * colhalf + 32, v1);
             tmem_wait_ld();
             tc_fence_before();
-            mbar_arrive(bar(OFREE));
+            mbar_arrive(bar((m & 1) ? OFREE2 : OFREE));
             if (m > 0) wait(OSFREE, (m - 1) & 1);      // the previous store has left the staging tile
             if (lane < 16) {
 #pragma unroll
@@ -317,42 +325,46 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             fence_proxy_async();
             mbar_arrive(bar(OSTAGED));
         };
-        for (int n = 0; n < NT; ++n) {
-            const uint32_t par = n & 1;
-            SLA_TS(0);
-            SLA_TS(1);
-
-            // A: TMEM -> causal mask -> bf16 -> shared memory (row i of the M=64 tile sits in lane 32*(i/16) + i%16)
-            wait(BAR_A, par);
+        // A_m: TMEM -> registers as soon as it is there (the tensor core may then start on A_{m+1}) -> causal mask -> bf16 ->
+        // shared memory once A_{m-1} V has read the tile (row i of the M=64 tile sits in lane 32*(i/16) + i%16)
+        auto mask_a = [&](int m) {
+            wait(BAR_A, m & 1);
             tc_fence_after();
-            SLA_TS(2);
-            {
-                const int i = 16 * (warp & 3) + lane, part = colhalf;
-                float v[32];
-                tmem_ld32(tmem + lane_base + COL_A + 32 * part, v);
-                tmem_wait_ld();
-                if (lane < 16) {
+            const int i = 16 * (warp & 3) + lane, part = colhalf;
+            float v[32];
+            tmem_ld32(tmem + lane_base + COL_A + 32 * part, v);
+            tmem_wait_ld();
+            tc_fence_before();
+            mbar_arrive(bar(ATAKEN));
+            if (m > 0) {
+                wait(BAR_O + ((m - 1) & 1), ((m - 1) >> 1) & 1);
+                tc_fence_after();
+            }
+            if (lane < 16) {
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        const int j0 = 32 * part + 8 * c;
-                        uint4 w;
-                        w.x = pack_bf16(j0 + 0 <= i ? v[8 * c + 0] : 0.f, j0 + 1 <= i ? v[8 * c + 1] : 0.f);
-                        w.y = pack_bf16(j0 + 2 <= i ? v[8 * c + 2] : 0.f, j0 + 3 <= i ? v[8 * c + 3] : 0.f);
-                        w.z = pack_bf16(j0 + 4 <= i ? v[8 * c + 4] : 0.f, j0 + 5 <= i ? v[8 * c + 5] : 0.f);
-                        w.w = pack_bf16(j0 + 6 <= i ? v[8 * c + 6] : 0.f, j0 + 7 <= i ? v[8 * c + 7] : 0.f);
-                        *reinterpret_cast<uint4 *>(sm + OFF_A + swz(i, 4 * part + c)) = w;
-                    }
+                for (int c = 0; c < 4; ++c) {
+                    const int j0 = 32 * part + 8 * c;
+                    uint4 w;
+                    w.x = pack_bf16(j0 + 0 <= i ? v[8 * c + 0] : 0.f, j0 + 1 <= i ? v[8 * c + 1] : 0.f);
+                    w.y = pack_bf16(j0 + 2 <= i ? v[8 * c + 2] : 0.f, j0 + 3 <= i ? v[8 * c + 3] : 0.f);
+                    w.z = pack_bf16(j0 + 4 <= i ? v[8 * c + 4] : 0.f, j0 + 5 <= i ? v[8 * c + 5] : 0.f);
+                    w.w = pack_bf16(j0 + 6 <= i ? v[8 * c + 6] : 0.f, j0 + 7 <= i ? v[8 * c + 7] : 0.f);
+                    *reinterpret_cast<uint4 *>(sm + OFF_A + swz(i, 4 * part + c)) = w;
                 }
             }
             fence_proxy_async();
             tc_fence_before();
             mbar_arrive(bar(AREADY));
-            SLA_TS(3);
-
-            // S_{n+1} = diag(2^{b_last}) (S_n + kh^T V): fp32 back into TMEM, bf16 copy for the next chunk's qh S
+        };
+        mask_a(0);
+        for (int n = 0; n < NT; ++n) {
+            const uint32_t par = n & 1;
+            SLA_TS(0);
+            // the recurrence first: S_{n+1} = diag(2^{b_last}) (S_n + kh^T V), fp32 back into TMEM, bf16 copy for the next
+            // chunk's qh S; the tensor core goes on with chunk n+1 the moment this is done
             wait(BAR_Z, par);
             tc_fence_after();
-            SLA_TS(4);
+            SLA_TS(1);
             if (p.simg) wait(SSAVED, par);             // the image store of S_n has read the operand copy
             {
                 const float e = eblast[(n & 3) * D + row];
@@ -380,12 +392,12 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             fence_proxy_async();
             tc_fence_before();
             mbar_arrive(bar(SREADY));
-            SLA_TS(5);
-
-            if (n > 0) stage_o(n - 1);                 // chunk n-1's output: its MMAs finished long ago
-            SLA_TS(6);
+            SLA_TS(2);
+            if (n + 1 < NT) mask_a(n + 1);             // beside the MMAs of chunk n+1: its A tile ...
+            SLA_TS(3);
+            stage_o(n);                                // ... and this chunk's output
+            SLA_TS(4);
         }
-        stage_o(NT - 1);
 
         if (p.ht && seg == p.P - 1) {   // final state, fp32 (each thread reads back what it wrote in the last rescale)
             float *dst = p.ht + ((size_t)bh * D + row) * D + 64 * colhalf;

@@ -2,6 +2,7 @@
 // bf16 I/O, d_k = d_v = 128, 64-token chunks.  Shared-memory tiles are rows of 128 bytes (64 bf16) in the
 // 128-byte swizzle; a 128-wide tile is two such halves side by side.
 #pragma once
+#include <type_traits>
 #include "sla_internal.h"
 #include "sla_ptx.cuh"
 
@@ -111,10 +112,11 @@ constexpr float LOG2E = 1.4426950408889634f;
 // columns 4cj..4cj+3.
 // tot: [8][128] floats of scratch.
 constexpr uint32_t TOT_BYTES = 8 * D * 4;
-template <bool WITH_Q, bool WITH_E>
+struct NoHook { __device__ __forceinline__ void operator()() const {} };
+template <bool WITH_Q, bool WITH_E, class Hook = NoHook>
 __device__ __forceinline__ void chunk_prologue(uint8_t *q_tile, uint8_t *k_tile, const float *gs, float *tot,
                                                const float *gq_s, const float *gk_s, float *eblast,
-                                               uint8_t *e2_tile, int tid, int bar_id = 1, uint32_t g_free_bar = 0) {
+                                               uint8_t *e2_tile, int tid, int bar_id = 1, Hook tile_read = Hook()) {
     using namespace ptx;
     const int rg = tid >> 5, cj = tid & 31;
     float4 gl[8];                               // this thread's log-decay rows: read once, kept for the second pass
@@ -127,8 +129,8 @@ __device__ __forceinline__ void chunk_prologue(uint8_t *q_tile, uint8_t *k_tile,
         }
         *reinterpret_cast<float4 *>(tot + rg * D + 4 * cj) = acc;
     }
-    if (g_free_bar) mbar_arrive(g_free_bar);    // the log-decay tile may be overwritten once every thread has said so
     named_bar_sync(bar_id, NCOMPUTE);
+    tile_read();                                // every thread has read its rows: the log-decay tile may be overwritten
     float bsum[4] = {0.f, 0.f, 0.f, 0.f};
     for (int g = 0; g < rg; ++g) {
         const float4 a = *reinterpret_cast<const float4 *>(tot + g * D + 4 * cj);
@@ -201,42 +203,70 @@ __device__ __forceinline__ float token_gate_any(const float *row, int H, int h) 
     if (H <= 16) return token_gate<16>(row, H, h);
     return token_gate<32>(row, H, h);
 }
-// Gates of one chunk for head h, by the 64 threads (t = 0..63, two whole warps) that serve one of the two gates:
+// Gates of one chunk for head h, by the NTH threads (whole warps) that serve one of the two gates:
 // dst[i] = mult * softmax(L[i*H .. i*H+H))[h] for token i < cn, 0 for cn <= i < 64.  L points at the chunk's first
 // logit; consecutive tokens are consecutive rows of H floats, so for H = 4, 8, 16, 32 the block is read as whole
 // float4s, fully coalesced, H/4 lanes per token, and max / sum travel over shuffles (one exponential per logit).
 // Other H: one thread per token reads its own row.
-template <int LPT>
-__device__ __forceinline__ void chunk_gate_vec(const float *__restrict__ L, int cn, int h, float mult, float *dst, int t) {
-    float4 x[LPT];
+// fetch: this thread's float4s of the chunk's logit block (LPT = H/4 lanes per token, NTH threads per gate)
+template <int LPT, int NTH>
+__device__ __forceinline__ void gate_fetch(const float *__restrict__ L, int cn, int t, float4 (&x)[LPT * 64 / NTH]) {
 #pragma unroll
-    for (int i = 0; i < LPT; ++i) {
-        const int f = i * 64 + t;                      // float4 index inside the chunk's block; token f / LPT
+    for (int i = 0; i < LPT * 64 / NTH; ++i) {
+        const int f = i * NTH + t;                     // float4 index inside the chunk's block; token f / LPT
         x[i] = f / LPT < cn ? __ldg(reinterpret_cast<const float4 *>(L) + f) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
+}
+// finish: softmax over the H/4 lanes of every token, dst[token] = mult * G[token][h].  Stage by stage over all of the
+// thread's float4s, so that the shuffles and exponentials of different tokens overlap.
+template <int LPT, int NTH>
+__device__ __forceinline__ void gate_finish(float4 (&x)[LPT * 64 / NTH], int cn, int h, float mult, float *dst, int t) {
+    constexpr int NF = LPT * 64 / NTH;
+    float m[NF], sum[NF];
 #pragma unroll
-    for (int i = 0; i < LPT; ++i) {
-        const int token = (i * 64 + t) / LPT;
-        float m = fmaxf(fmaxf(x[i].x, x[i].y), fmaxf(x[i].z, x[i].w));
+    for (int i = 0; i < NF; ++i) m[i] = fmaxf(fmaxf(x[i].x, x[i].y), fmaxf(x[i].z, x[i].w));
 #pragma unroll
-        for (int o = 1; o < LPT; o <<= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-        const float e0 = __expf(x[i].x - m), e1 = __expf(x[i].y - m), e2 = __expf(x[i].z - m), e3 = __expf(x[i].w - m);
-        float sum = (e0 + e1) + (e2 + e3);
+    for (int o = 1; o < LPT; o <<= 1) {
 #pragma unroll
-        for (int o = 1; o < LPT; o <<= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-        if ((t % LPT) == (h >> 2)) {
-            const int j = h & 3;
-            const float eh = j == 0 ? e0 : j == 1 ? e1 : j == 2 ? e2 : e3;
-            dst[token] = token < cn ? mult * eh / sum : 0.f;
+        for (int i = 0; i < NF; ++i) m[i] = fmaxf(m[i], __shfl_xor_sync(0xffffffffu, m[i], o));
+    }
+#pragma unroll
+    for (int i = 0; i < NF; ++i) {
+        x[i].x = __expf(x[i].x - m[i]); x[i].y = __expf(x[i].y - m[i]);
+        x[i].z = __expf(x[i].z - m[i]); x[i].w = __expf(x[i].w - m[i]);
+        sum[i] = (x[i].x + x[i].y) + (x[i].z + x[i].w);
+    }
+#pragma unroll
+    for (int o = 1; o < LPT; o <<= 1) {
+#pragma unroll
+        for (int i = 0; i < NF; ++i) sum[i] += __shfl_xor_sync(0xffffffffu, sum[i], o);
+    }
+    if ((t % LPT) == (h >> 2)) {
+        const int j = h & 3;
+#pragma unroll
+        for (int i = 0; i < NF; ++i) {
+            const int token = (i * NTH + t) / LPT;
+            const float eh = j == 0 ? x[i].x : j == 1 ? x[i].y : j == 2 ? x[i].z : x[i].w;
+            dst[token] = token < cn ? mult * __fdividef(eh, sum[i]) : 0.f;
         }
     }
 }
+template <int LPT, int NTH>
+__device__ __forceinline__ void chunk_gate_vec(const float *__restrict__ L, int cn, int h, float mult, float *dst, int t) {
+    float4 x[LPT * 64 / NTH];
+    gate_fetch<LPT, NTH>(L, cn, t, x);
+    gate_finish<LPT, NTH>(x, cn, h, mult, dst, t);
+}
+// NTH = 64 (threads t = 0..63, two whole warps) or 32 (one warp) serve one gate of one chunk.
+template <int NTH = 64>
 __device__ __forceinline__ void chunk_gate(const float *L, int H, int cn, int h, float mult, float *dst, int t) {
-    if (H == 16) chunk_gate_vec<4>(L, cn, h, mult, dst, t);
-    else if (H == 8) chunk_gate_vec<2>(L, cn, h, mult, dst, t);
-    else if (H == 4) chunk_gate_vec<1>(L, cn, h, mult, dst, t);
-    else if (H == 32) chunk_gate_vec<8>(L, cn, h, mult, dst, t);
-    else dst[t] = t < cn ? mult * token_gate_any(L + (size_t)t * H, H, h) : 0.f;
+    if (H == 16) chunk_gate_vec<4, NTH>(L, cn, h, mult, dst, t);
+    else if (H == 8) chunk_gate_vec<2, NTH>(L, cn, h, mult, dst, t);
+    else if (H == 4) chunk_gate_vec<1, NTH>(L, cn, h, mult, dst, t);
+    else if (H == 32) chunk_gate_vec<8, NTH>(L, cn, h, mult, dst, t);
+    else {
+        for (int i = t; i < C; i += NTH) dst[i] = i < cn ? mult * token_gate_any(L + (size_t)i * H, H, h) : 0.f;
+    }
 }
 constexpr int NGATE = 128;   // gate threads: g < 64 -> scale*Gq of token g, g >= 64 -> Gk of token g-64
 
