@@ -50,8 +50,9 @@ def measured_peaks():
     return 6650.0, "fallback"
 
 
-def recorded_traffic(kernel: str):
-    """DRAM bytes per launch from the committed ncu summary, if one covers this kernel.  The record carries a hash
+def recorded_traffic(workload: str, kernel: str):
+    """DRAM bytes per launch from the committed ncu summary, if one covers this kernel on this workload (full size,
+    plan flags as in the default run).  The record carries a hash
     of the kernel sources it was taken on: once they have changed, the figure is stale and None is reported."""
     import hashlib
     p = ROOT / "profiles" / "dram_traffic.json"
@@ -64,7 +65,7 @@ def recorded_traffic(kernel: str):
             h.update(f.read_bytes())
         if rec.get("source_sha256") != h.hexdigest():
             return None
-        e = rec.get(kernel)
+        e = rec.get(workload, {}).get(kernel)
         return None if e is None else e.get("bytes_per_launch_full_size")
     except Exception:
         return None
@@ -371,7 +372,7 @@ def main():
             alg = per_unit * cfg.B * cfg.T * cfg.H
             achieved = alg / (avg_ms * 1e-3) / 1e9
             roof = {"bound": "hbm", "kernel": top, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                    "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": recorded_traffic(top),
+                    "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": recorded_traffic(WORKLOAD, top) if (args.batch <= 0 and saving) else None,
                     "algorithmic_bytes_per_launch": alg, "avg_launch_ms": avg_ms, "kernel_time_share": share}
         else:
             roof = {"bound": "hbm", "kernel": top, "achieved": None, "peak": peak, "unit": "GB/s", "frac": None,
