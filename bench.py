@@ -358,6 +358,37 @@ def main():
                   "algorithmic_bytes_per_step": dbytes, "achieved": dbytes / (us * 1e-6) / 1e9, "peak": dpeak,
                   "unit": "GB/s", "frac": dbytes / (us * 1e-6) / 1e9 / dpeak,
                   "note": "the 64 MiB state fits the 126 MB L2, so part of the traffic may be served there"}
+        # a single sequence (1 MiB of state): launch bound, so the serving loop replays its steps as one CUDA graph
+        s1 = torch.zeros((1, c3.H, c3.d_k, c3.d_v), dtype=torch.float32, device="cuda")
+        o1 = torch.empty((1, c3.H, c3.d_v), dtype=torch.bfloat16, device="cuda")
+        d1 = {n: (None if t is None else t[:, :1].contiguous()) for n, t in dec.items()}
+
+        def steps1():
+            for j in range(8):
+                api.sla_decode_step(dplan, d1["q"][j], d1["k"][j], d1["v"][j], d1["log_decay"][j], d1["gq_logits"][j],
+                                    d1["gk_logits"][j], s1, o_t=o1)
+
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            steps1()
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            steps1()
+        timings = {}
+        for name, fn in (("launched", steps1), ("graph", graph.replay)):
+            fn()
+            torch.cuda.synchronize()
+            e0.record()
+            for _ in range(16):
+                fn()
+            e1.record()
+            torch.cuda.synchronize()
+            timings[name] = 1e3 * e0.elapsed_time(e1) / (16 * 8)
+        decode["batch_1"] = {"us_per_step_launched_one_by_one": timings["launched"],
+                             "us_per_step_as_one_cuda_graph_of_8_steps": timings["graph"]}
 
     # ---- roofline of the dominant kernel, from the per-kernel CUDA events of the timed region ----
     peak, peak_kind = measured_peaks()
