@@ -30,7 +30,7 @@ constexpr uint32_t OFF_PQ = OFF_T + HALF_BF16;          // bf16 Pq
 constexpr int LDL = 68;                                 // row stride (floats) of the fp32 64x64 work arrays
 constexpr uint32_t OFF_LS = OFF_PQ + HALF_BF16;         // fp32 L
 constexpr uint32_t OFF_TS = OFF_LS + 64 * LDL * 4;      // fp32 T
-constexpr uint32_t OFF_XS = OFF_TS + 64 * LDL * 4;      // fp32 [3][16][17] block products
+constexpr uint32_t OFF_XS = OFF_TS + 64 * LDL * 4;      // fp32 block-product scratch, [6 warps][16][8] (816 floats reserved)
 constexpr uint32_t OFF_SC = OFF_XS + 3 * 16 * 17 * 4;   // per-token scalars of the chunk: 8 arrays of 64 floats
 constexpr uint32_t OFF_GATE = OFF_SC + 8 * C * 4;       // [4 chunks][4][64]: scale*Gq, Gk, log-decay, beta
 constexpr uint32_t OFF_BAR = OFF_GATE + 4 * 4 * C * 4;
@@ -399,30 +399,52 @@ k_gdn_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
                 for (int i = 0; i < 16; ++i) Ts[(16 * bb + i) * LDL + 16 * bb + c] = x[i];
             }
             named_bar_sync(1, NCOMPUTE);
-            for (int dlev = 1; dlev < 4; ++dlev) {     // block T_ba (b = a + dlev) = -T_bb sum_{a <= c < b} L_bc T_ca
-                const int nel = (4 - dlev) * 256;
-                for (int e = tid; e < nel; e += NCOMPUTE) {
-                    const int a = e >> 8, r = (e >> 4) & 15, c = e & 15, bI = a + dlev;
-                    float acc = 0.f;
+            // Off-diagonal blocks, top down within a block column a:  T_ba = -T_bb sum_{a <= c < b} L_bc T_ca,  b = a+1 .. 3.
+            // A column of T depends on no other column, so two warps share a block column, eight columns each, and no
+            // barrier is needed inside.  16x16x16 products on the warp-level tf32 MMA (T is rounded to bf16 afterwards, so
+            // tf32 operands cost nothing).
+            if (warp < 6) {
+                const int a = warp >> 1, nh = warp & 1, g = lane >> 2, t = lane & 3;
+                float *Xw = Xs + warp * 16 * 8;          // this warp's 16x8 scratch
+                auto frag_a = [&](const float *M, uint32_t (&fa)[4]) {       // 16x8 slice at M (row stride LDL)
+                    fa[0] = to_tf32(M[g * LDL + t]);
+                    fa[1] = to_tf32(M[(g + 8) * LDL + t]);
+                    fa[2] = to_tf32(M[g * LDL + t + 4]);
+                    fa[3] = to_tf32(M[(g + 8) * LDL + t + 4]);
+                };
+                const int col0 = 16 * a + 8 * nh;        // this warp's columns of T
+                for (int bI = a + 1; bI < 4; ++bI) {
+                    float x[4] = {0.f, 0.f, 0.f, 0.f};
                     for (int cc = a; cc < bI; ++cc) {
-                        const float *Lr = Ls + (16 * bI + r) * LDL + 16 * cc;
-                        const float *Tc = Ts + (16 * cc) * LDL + 16 * a + c;
 #pragma unroll
-                        for (int m = 0; m < 16; ++m) acc = fmaf(Lr[m], Tc[m * LDL], acc);
+                        for (int ks = 0; ks < 2; ++ks) {
+                            uint32_t fa[4], fb[2];
+                            frag_a(Ls + (16 * bI) * LDL + 16 * cc + 8 * ks, fa);
+                            const float *Tb = Ts + (16 * cc + 8 * ks) * LDL + col0;
+                            fb[0] = to_tf32(Tb[t * LDL + g]);
+                            fb[1] = to_tf32(Tb[(t + 4) * LDL + g]);
+                            mma_tf32_16x8x8(x, fa, fb);
+                        }
                     }
-                    Xs[(a * 16 + r) * 17 + c] = acc;
-                }
-                named_bar_sync(1, NCOMPUTE);
-                for (int e = tid; e < nel; e += NCOMPUTE) {
-                    const int a = e >> 8, r = (e >> 4) & 15, c = e & 15, bI = a + dlev;
-                    const float *Tb = Ts + (16 * bI + r) * LDL + 16 * bI;
-                    float acc = 0.f;
+                    Xw[g * 8 + 2 * t] = x[0];       Xw[g * 8 + 2 * t + 1] = x[1];
+                    Xw[(g + 8) * 8 + 2 * t] = x[2]; Xw[(g + 8) * 8 + 2 * t + 1] = x[3];
+                    __syncwarp();
+                    float y[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                    for (int m = 0; m < 16; ++m) acc = fmaf(Tb[m], Xs[(a * 16 + m) * 17 + c], acc);
-                    Ts[(16 * bI + r) * LDL + 16 * a + c] = -acc;
+                    for (int ks = 0; ks < 2; ++ks) {
+                        uint32_t fa[4], fb[2];
+                        frag_a(Ts + (16 * bI) * LDL + 16 * bI + 8 * ks, fa);
+                        fb[0] = to_tf32(Xw[(8 * ks + t) * 8 + g]);
+                        fb[1] = to_tf32(Xw[(8 * ks + t + 4) * 8 + g]);
+                        mma_tf32_16x8x8(y, fa, fb);
+                    }
+                    float *To = Ts + (16 * bI) * LDL + col0;
+                    To[g * LDL + 2 * t] = -y[0];       To[g * LDL + 2 * t + 1] = -y[1];
+                    To[(g + 8) * LDL + 2 * t] = -y[2]; To[(g + 8) * LDL + 2 * t + 1] = -y[3];
+                    __syncwarp();
                 }
-                named_bar_sync(1, NCOMPUTE);
             }
+            named_bar_sync(1, NCOMPUTE);
             {   // bf16 T (A operand, K-major): thread = (row i, 16 columns)
                 const int i = tid >> 2, jq = tid & 3;
 #pragma unroll
