@@ -40,7 +40,7 @@ static_assert(SMEM_BYTES <= 232448, "shared memory budget");
 constexpr uint32_t COL_KK = 0, COL_QK = 64, COL_W = 0, COL_U = 128, COL_O = 256, COL_S = 384, TMEM_COLS = 512;
 constexpr int NTHREADS = NCOMPUTE + 32 + NGATE + 32;    // warps 0..7 compute, 8 MMA issue, 9..12 gates, 13 TMA
 enum Bar { FULL = 0 /*[2]*/, GREADY = 2 /*[4]*/, GFREE = 6 /*[4]*/, OPR = 10, TREADY, WREADY, UREADY, SREADY, OSTAGED /*[2]*/,
-           BAR_1 = OSTAGED + 2, BAR_2, BAR_3, BAR_4, DRAIN, NBAR };
+           BAR_1 = OSTAGED + 2, BAR_2, BAR_3, BAR_4, DRAIN, SAVED, NBAR };
 static_assert(NBAR <= 32, "barrier slots");
 // scalar arrays in OFF_SC
 enum Sc { SC_B = 0, SC_GAM, SC_IGAM, SC_FQ, SC_FKB, SC_FVB, SC_BETA, SC_MISC };
@@ -185,10 +185,16 @@ k_gdn_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
                     tma_store_5d(&tm_o, base + (n & 1) * STAGE + OFF_V, 0, n * C, 0, h, b);
                     bulk_commit();
                 }
-                if (n + 2 < NT) {
-                    bulk_wait_read0();
-                    load(n + 2);
+                if (p.save) {   // the chunk's record: T, U and S_{n+1} stand in shared memory in exactly the record's layout
+                    uint8_t *rec = p.save + ((size_t)bh * (NT + 1) + n) * REC_BYTES;
+                    bulk_store(rec + REC_T, base + OFF_T, HALF_BF16);
+                    bulk_store(rec + REC_U, base + (n & 1) * STAGE + OFF_K, TILE_BF16);
+                    bulk_store(rec + REC_BYTES + REC_S, base + OFF_S, STATE_BF16);
+                    bulk_commit();
                 }
+                if (n + 2 < NT || p.save) bulk_wait_read0();
+                if (p.save) mbar_arrive(bar(SAVED));   // T and the S copy may be overwritten
+                if (n + 2 < NT) load(n + 2);
             }
             bulk_wait0();
             if (failed) {
@@ -249,7 +255,7 @@ k_gdn_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
         mbar_arrive(bar(SREADY));
 
         // a 64x128 accumulator tile (M = 64: row i in lane 32*(i/16) + i%16) -> sign * bf16 -> swizzled tile at dst
-        auto tile_to_bf16 = [&](uint32_t col, uint8_t *dst, float sign, uint8_t *gdst) {
+        auto tile_to_bf16 = [&](uint32_t col, uint8_t *dst, float sign) {
             float v0[32], v1[32];
             tmem_ld32(tmem + lane_base + col + 64 * colhalf, v0);
             tmem_ld32(tmem + lane_base + col + 64 * colhalf + 32, v1);
@@ -263,13 +269,11 @@ k_gdn_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
                     w.z = pack_bf16(sign * v0[8 * c + 4], sign * v0[8 * c + 5]);
                     w.w = pack_bf16(sign * v0[8 * c + 6], sign * v0[8 * c + 7]);
                     *reinterpret_cast<uint4 *>(dst + colhalf * HALF_BF16 + swz(ti, c)) = w;
-                    if (gdst) *reinterpret_cast<uint4 *>(gdst + colhalf * HALF_BF16 + swz(ti, c)) = w;
                     w.x = pack_bf16(sign * v1[8 * c + 0], sign * v1[8 * c + 1]);
                     w.y = pack_bf16(sign * v1[8 * c + 2], sign * v1[8 * c + 3]);
                     w.z = pack_bf16(sign * v1[8 * c + 4], sign * v1[8 * c + 5]);
                     w.w = pack_bf16(sign * v1[8 * c + 6], sign * v1[8 * c + 7]);
                     *reinterpret_cast<uint4 *>(dst + colhalf * HALF_BF16 + swz(ti, 4 + c)) = w;
-                    if (gdst) *reinterpret_cast<uint4 *>(gdst + colhalf * HALF_BF16 + swz(ti, 4 + c)) = w;
                 }
             }
         };
@@ -445,6 +449,7 @@ k_gdn_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
                 }
             }
             named_bar_sync(1, NCOMPUTE);
+            if (p.save && n > 0) wait(SAVED, (n - 1) & 1);   // the previous chunk's record has left T and the S copy
             {   // bf16 T (A operand, K-major): thread = (row i, 16 columns)
                 const int i = tid >> 2, jq = tid & 3;
 #pragma unroll
@@ -458,7 +463,6 @@ k_gdn_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
                         ww[e] = pack_bf16(t0, t1);
                     }
                     *reinterpret_cast<uint4 *>(sm + OFF_T + swz(i, 2 * jq + hh)) = w;
-                    if (rec0) *reinterpret_cast<uint4 *>(rec0 + (size_t)n * REC_BYTES + REC_T + swz(i, 2 * jq + hh)) = w;
                 }
             }
             fence_proxy_async();
@@ -468,7 +472,7 @@ k_gdn_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             // ---- C: -W as bf16 over the q tile ----
             wait(BAR_2, par);
             tc_fence_after();
-            tile_to_bf16(COL_W, st + OFF_Q, -1.f, nullptr);
+            tile_to_bf16(COL_W, st + OFF_Q, -1.f);
             fence_proxy_async();
             tc_fence_before();
             mbar_arrive(bar(WREADY));
@@ -476,7 +480,7 @@ k_gdn_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             // ---- D: U as bf16 over the k tile ----
             wait(BAR_3, par);
             tc_fence_after();
-            tile_to_bf16(COL_U, st + OFF_K, 1.f, rec0 ? rec0 + (size_t)n * REC_BYTES + REC_U : nullptr);
+            tile_to_bf16(COL_U, st + OFF_K, 1.f);
             fence_proxy_async();
             tc_fence_before();
             mbar_arrive(bar(UREADY));
@@ -503,20 +507,18 @@ k_gdn_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
                     w.z = pack_bf16(v0[8 * c + 4], v0[8 * c + 5]);
                     w.w = pack_bf16(v0[8 * c + 6], v0[8 * c + 7]);
                     *reinterpret_cast<uint4 *>(sm + OFF_S + colhalf * STATE_HALF + swz(row, c)) = w;
-                    if (rec0) *reinterpret_cast<uint4 *>(rec0 + (size_t)(n + 1) * REC_BYTES + REC_S + colhalf * STATE_HALF + swz(row, c)) = w;
                     w.x = pack_bf16(v1[8 * c + 0], v1[8 * c + 1]);
                     w.y = pack_bf16(v1[8 * c + 2], v1[8 * c + 3]);
                     w.z = pack_bf16(v1[8 * c + 4], v1[8 * c + 5]);
                     w.w = pack_bf16(v1[8 * c + 6], v1[8 * c + 7]);
                     *reinterpret_cast<uint4 *>(sm + OFF_S + colhalf * STATE_HALF + swz(row, 4 + c)) = w;
-                    if (rec0) *reinterpret_cast<uint4 *>(rec0 + (size_t)(n + 1) * REC_BYTES + REC_S + colhalf * STATE_HALF + swz(row, 4 + c)) = w;
                 }
                 tmem_wait_st();
             }
             fence_proxy_async();
             tc_fence_before();
             mbar_arrive(bar(SREADY));
-            tile_to_bf16(COL_O, st + OFF_V, 1.f, nullptr);
+            tile_to_bf16(COL_O, st + OFF_V, 1.f);
             fence_proxy_async();
             tc_fence_before();
             mbar_arrive(bar(OSTAGED + (n & 1)));
