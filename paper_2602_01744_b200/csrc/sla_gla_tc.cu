@@ -49,6 +49,7 @@ static_assert(NBAR <= 40, "barrier slots");
 
 struct FwdParams {
     const float *lq, *lk, *h0;
+    const float *fin, *gam;         // segmented run (P > 1): per (sequence, segment) the state reached from zero and the total decay
     __nv_bfloat16 *o;
     float *ht;
     uint8_t *simg;                  // optional: [B*H][NT+1][32 KiB] bf16 images of the state before every chunk (P = 1 only)
@@ -270,13 +271,26 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
         const int colhalf = warp >> 2;                                   // which 64 state / output columns
         const int row = 32 * (warp & 3) + lane;
 
-        {   // initial state: fp32 into TMEM, bf16 copy into shared memory (row = key dimension)
-            const float *src = p.h0 ? p.h0 + ((size_t)blockIdx.x * D + row) * D + 64 * colhalf : nullptr;   // one state per CTA
+        {   // initial state: fp32 into TMEM, bf16 copy into shared memory (row = key dimension).  A segment that is not the
+            // first starts from S <- diag(gam_s) S + fin_s taken over the segments s before it (a short scan over their
+            // summaries, elementwise, done here rather than in a launch of its own).
+            const float *src = p.h0 ? p.h0 + ((size_t)bh * D + row) * D + 64 * colhalf : nullptr;
 #pragma unroll
             for (int part = 0; part < 2; ++part) {
                 float v[32];
 #pragma unroll
                 for (int j = 0; j < 32; ++j) v[j] = src ? src[32 * part + j] : 0.f;
+                for (int sgm = 0; sgm < seg; ++sgm) {
+                    const size_t c = (size_t)bh * p.P + sgm;
+                    const float gmm = p.gam[c * D + row];
+                    const float4 *f = reinterpret_cast<const float4 *>(p.fin + (c * D + row) * D + 64 * colhalf + 32 * part);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const float4 x = f[j];
+                        v[4 * j] = fmaf(gmm, v[4 * j], x.x);         v[4 * j + 1] = fmaf(gmm, v[4 * j + 1], x.y);
+                        v[4 * j + 2] = fmaf(gmm, v[4 * j + 2], x.z); v[4 * j + 3] = fmaf(gmm, v[4 * j + 3], x.w);
+                    }
+                }
                 tmem_st32(tmem + lane_base + COL_S + 64 * colhalf + 32 * part, v);
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
@@ -418,21 +432,6 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
     if (warp == 0) tmem_dealloc(tmem, TMEM_COLS);
 }
 
-// Segmented forward, second pass: S_start[p+1] = diag(gam_p) S_start[p] + fin_p along the segments of a sequence
-// (elementwise; thread = four consecutive state entries).  grid (B*H, 16), 256 threads.
-__global__ void k_segment_scan(const float *__restrict__ h0, const float *__restrict__ fin, const float *__restrict__ gam,
-                               float *__restrict__ start, int P) {
-    const int bh = blockIdx.x, e = (blockIdx.y * 256 + threadIdx.x) * 4, row = e / D;
-    float4 S = h0 ? *reinterpret_cast<const float4 *>(h0 + (size_t)bh * D * D + e) : make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int p = 0; p < P; ++p) {
-        const size_t c = (size_t)bh * P + p;
-        *reinterpret_cast<float4 *>(start + c * D * D + e) = S;
-        const float g = gam[c * D + row];
-        const float4 f = *reinterpret_cast<const float4 *>(fin + c * D * D + e);
-        S = make_float4(fmaf(g, S.x, f.x), fmaf(g, S.y, f.y), fmaf(g, S.z, f.z), fmaf(g, S.w, f.w));
-    }
-}
-
 // ---- host side ----
 unsigned long long *g_phase_ts = nullptr;   // set by sla_debug_set_phase_timestamps (profiling aid)
 
@@ -478,7 +477,7 @@ size_t gla_tc_forward_workspace_bytes(const Dims &d) {
     int P, L;
     choose_segments(d, P, L);
     if (P == 1) return 0;
-    return (size_t)d.B * d.H * P * (2 * D * D + D) * sizeof(float);
+    return (size_t)d.B * d.H * P * (D * D + D) * sizeof(float);
 }
 
 bool gla_tc_forward_can_save(const Dims &d) {
@@ -495,18 +494,16 @@ int gla_tc_forward(const Dims &d, const FwdArgs &a, uint8_t *simg, int *status, 
         return -1;
     int P, L, launches = 1;
     choose_segments(d, P, L);
-    const float *h0 = a.h0;
-    if (P > 1) {   // segment summaries from a zero state, scan over the segments, then the segments in parallel
+    float *fin = nullptr, *gam = nullptr;
+    if (P > 1) {   // segment summaries from a zero state, then the segments in parallel (each scans the summaries before it)
         const size_t nseg = (size_t)d.B * d.H * P;
-        float *fin = a.ws, *start = fin + nseg * D * D, *gam = start + nseg * D * D;
+        fin = a.ws;
+        gam = fin + nseg * D * D;
         if (gla_tc_segment_summaries(d, a, P, L, fin, gam, status, st, tr) < 0) return -1;
-        k_segment_scan<<<dim3(d.B * d.H, 16), 256, 0, st>>>(a.h0, fin, gam, start, P);
-        tr.mark("segment_scan");
-        h0 = start;
-        launches = 3;
+        launches = 2;
+        simg = nullptr;
     }
-    if (P > 1) simg = nullptr;
-    FwdParams p{a.lq, a.lk, h0, (__nv_bfloat16 *)a.o, a.ht, simg, status, d.T, d.H, d.NT, P, L, d.scale, g_phase_ts};
+    FwdParams p{a.lq, a.lk, a.h0, fin, gam, (__nv_bfloat16 *)a.o, a.ht, simg, status, d.T, d.H, d.NT, P, L, d.scale, g_phase_ts};
     k_gla_fwd_tc<<<d.B * d.H * P, NTHREADS, SMEM_BYTES, st>>>(mq, mk, mv, mg, mo, p);
     tr.mark("gla_fwd_tc");
     return cudaGetLastError() == cudaSuccess ? launches : -1;
