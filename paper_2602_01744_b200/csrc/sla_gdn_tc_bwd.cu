@@ -251,6 +251,11 @@ k_gdn_bwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             for (int k = 0; k < NT && !failed; ++k) {
                 const int n = NT - 1 - k;
                 const uint32_t par = k & 1;
+                if (n > 0) {   // the next chunk's q, k and record can only be loaded late in this chunk: have them in L2 by then
+                    tma_prefetch_l2_5d(&tm_q, 0, (n - 1) * C, 0, h, b);
+                    tma_prefetch_l2_5d(&tm_k, 0, (n - 1) * C, 0, h, b);
+                    bulk_prefetch_l2(rec0 + (size_t)(n - 1) * REC_BYTES, REC_BYTES);                        // S, U, T
+                }
                 wait_relaxed(S3R, par);                // dq staged over dO
                 if (failed) break;
                 tma_store_5d(&tm_dq, base + B_DO, 0, n * C, 0, h, b);

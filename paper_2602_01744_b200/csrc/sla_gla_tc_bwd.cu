@@ -513,6 +513,12 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
                 const uint32_t par = k & 1;
                 const uint32_t sQK = base + ((k & 1) ? OFF_Y : OFF_X);
                 if (n > 0) {
+                    // the next chunk's tiles can only be loaded as this chunk's buffers fall free: have them in L2 by then
+                    tma_prefetch_l2_5d(&tm_q, 0, (n - 1) * C, 0, h, b);
+                    tma_prefetch_l2_5d(&tm_k, 0, (n - 1) * C, 0, h, b);
+                    tma_prefetch_l2_5d(&tm_v, 0, (n - 1) * C, 0, h, b);
+                    tma_prefetch_l2_5d(&tm_do, 0, (n - 1) * C, 0, h, b);
+                    bulk_prefetch_l2(img0 + (size_t)(n - 1) * STATE_BF16, STATE_BF16);
                     wait(OPR, par);                    // prologue done: the log-decay buffer is free
                     if (failed) break;
                     load_g(n - 1);
