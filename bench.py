@@ -32,6 +32,11 @@ BWD_BYTES_PER_TOKEN_HEAD = 4 * 256 + 512 + 3 * 256 + 512 + 16   # 2832
 # The gated delta rule has a scalar decay and beta per (token, head): 4 B each instead of 512 B.
 GDN_FWD_BYTES_PER_TOKEN_HEAD = 4 * 256 + 8 + 8          # 1040
 GDN_BWD_BYTES_PER_TOKEN_HEAD = 4 * 256 + 3 * 256 + 8 + 8 + 16   # 1824
+# Tensor-core work per (token, head) at chunk 64, d_k = d_v = 128 (2 FLOP per multiply-add).  "algorithmic" counts the
+# causal half of the 64x64 products only; "executed" is what the MMAs issue (full 64x64 tiles; the chunk-state
+# recomputation of the backward is counted only when the plan recomputes).
+GLA_FLOP = {"fwd_algorithmic": 82176, "bwd_algorithmic": 205440, "fwd_executed": 98304, "bwd_executed": 212992,
+            "state_recompute_executed": 32768}
 KERNEL_BYTES = {  # which share of the compulsory traffic each kernel is accountable for
     "output": FWD_BYTES_PER_TOKEN_HEAD, "grads_lin": BWD_BYTES_PER_TOKEN_HEAD,
     "gla_fwd_tc": FWD_BYTES_PER_TOKEN_HEAD, "gla_bwd_tc": BWD_BYTES_PER_TOKEN_HEAD,
@@ -50,10 +55,22 @@ def measured_peaks():
     return 6650.0, "fallback"
 
 
-def recorded_traffic(workload: str, kernel: str):
-    """DRAM bytes per launch from the committed ncu summary, if one covers this kernel on this workload (full size,
-    plan flags as in the default run).  The record carries a hash
-    of the kernel sources it was taken on: once they have changed, the figure is stale and None is reported."""
+def measured_tensor_peaks():
+    """(burst, sustained) dense bf16 TFLOP/s and where they come from."""
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        try:
+            d = json.loads(p.read_text())
+            return float(d["bf16_tflops"]), float(d["bf16_tflops_sustained"]), "measured"
+        except Exception:
+            pass
+    return 1590.0, 1400.0, "fallback"
+
+
+def recorded_counters(workload: str, kernel: str, key: str = "bytes_per_launch_full_size"):
+    """A figure from the committed ncu summary (DRAM bytes per launch, tensor-pipe activity), if one covers this kernel
+    on this workload (full size, plan flags as in the default run).  The record carries a hash of the kernel sources
+    it was taken on: once they have changed, the figure is stale and None is reported."""
     import hashlib
     p = ROOT / "profiles" / "dram_traffic.json"
     if not p.exists():
@@ -66,9 +83,13 @@ def recorded_traffic(workload: str, kernel: str):
         if rec.get("source_sha256") != h.hexdigest():
             return None
         e = rec.get(workload, {}).get(kernel)
-        return None if e is None else e.get("bytes_per_launch_full_size")
+        return None if e is None else e.get(key)
     except Exception:
         return None
+
+
+def recorded_traffic(workload: str, kernel: str):
+    return recorded_counters(workload, kernel)
 
 
 class ClockSampler:
@@ -249,7 +270,6 @@ def main():
 
     # ---- device-resident timing (inputs in HBM; 0.77 GB of inputs per step, far beyond the 126 MB L2) ----
     launches[0] = 0
-    plan.set_kernel_timing(True)
     sampler = ClockSampler(local)
     sampler.start()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -261,10 +281,22 @@ def main():
     barrier()
     ms = e0.elapsed_time(e1)
     clocks = sampler.stop()
+    plan.poll()
+    n_launch = launches[0]
+    # second pass of the same steps with one CUDA event after every kernel (on the launch stream, inside the library):
+    # per-kernel durations and shares.  Kept out of the pass above so that `value` carries no measurement overhead.
+    plan.set_kernel_timing(True)
+    barrier()
+    e0.record()
+    for _ in range(args.steps):
+        step(dev)
+    e1.record()
+    barrier()
+    ms_traced = e0.elapsed_time(e1)
     ktimes = plan.kernel_times()
     plan.set_kernel_timing(False)
     plan.poll()
-    n_launch = launches[0]
+    launches[0] = n_launch
     from paper_2602_01744_b200.replicas import whole_job_throughput
     tokens_step = cfg.B * cfg.T
     value, ms = whole_job_throughput(tokens_step, args.steps, ms, dist, "cuda")
@@ -332,14 +364,19 @@ def main():
         c3 = CONFIGS["C3"]
         dplan = api.sla_plan_create(c3.variant, c3.dtype, 1, 64, c3.H, c3.d_k, c3.d_v, c3.chunk)
         dec = {n: (None if t is None else t.cuda()) for n, t in make_decode_inputs(c3, C3_DECODE_BATCH, 8, seed=5).items()}
-        state = torch.zeros((C3_DECODE_BATCH, c3.H, c3.d_k, c3.d_v), dtype=torch.float32, device="cuda")
+        # four independent 64 MiB states taken in turn: between two visits of one state 192 MiB of other states pass
+        # through the 126 MB L2, so every step reads its state from HBM and its writes are evicted to HBM
+        NSTATE = 4
+        states = [torch.zeros((C3_DECODE_BATCH, c3.H, c3.d_k, c3.d_v), dtype=torch.float32, device="cuda")
+                  for _ in range(NSTATE)]
+        state = states[0]
         o_t = torch.empty((C3_DECODE_BATCH, c3.H, c3.d_v), dtype=torch.bfloat16, device="cuda")
         dsteps = 64
 
         def dstep(i):
             j = i % 8
             api.sla_decode_step(dplan, dec["q"][j], dec["k"][j], dec["v"][j], dec["log_decay"][j], dec["gq_logits"][j],
-                                dec["gk_logits"][j], state, o_t=o_t)
+                                dec["gk_logits"][j], states[i % NSTATE], o_t=o_t)
 
         for i in range(8):
             dstep(i)
@@ -357,7 +394,9 @@ def main():
                   "us_per_step": us, "tokens_per_s": C3_DECODE_BATCH / (us * 1e-6), "bound": "hbm",
                   "algorithmic_bytes_per_step": dbytes, "achieved": dbytes / (us * 1e-6) / 1e9, "peak": dpeak,
                   "unit": "GB/s", "frac": dbytes / (us * 1e-6) / 1e9 / dpeak,
-                  "note": "the 64 MiB state fits the 126 MB L2, so part of the traffic may be served there"}
+                  "l2": f"{NSTATE} independent 64 MiB states visited in turn ({NSTATE * 64} MiB > 126 MB L2): no step "
+                        "finds its state in L2",
+                  "traffic": recorded_counters("C3_decode", "decode")}
         # a single sequence (1 MiB of state): launch bound, so the serving loop replays its steps as one CUDA graph
         s1 = torch.zeros((1, c3.H, c3.d_k, c3.d_v), dtype=torch.float32, device="cuda")
         o1 = torch.empty((1, c3.H, c3.d_v), dtype=torch.bfloat16, device="cuda")
@@ -415,6 +454,28 @@ def main():
                   ((GDN_BWD_BYTES_PER_TOKEN_HEAD if gdn else BWD_BYTES_PER_TOKEN_HEAD) if cfg.backward else 0)) * cfg.B * cfg.T * cfg.H
     step_gbs = step_bytes / (ms / args.steps * 1e-3) / 1e9
 
+    # the tensor-core side of the metric: algorithmic MMA FLOP of a step / step time against the dense bf16 peaks.
+    # The step is HBM-bound (66 FLOP/B against a ridge near 256), so the fraction it could reach at the HBM roofline
+    # is stated beside it.
+    tensor = None
+    if cfg.variant == "gla" and cfg.d_k == 128 and cfg.d_v == 128 and not args.generic:
+        pairs = cfg.B * cfg.T * cfg.H
+        alg = GLA_FLOP["fwd_algorithmic"] + (GLA_FLOP["bwd_algorithmic"] if cfg.backward else 0)
+        exe = GLA_FLOP["fwd_executed"] + ((GLA_FLOP["bwd_executed"] + (0 if saving else GLA_FLOP["state_recompute_executed"]))
+                                          if cfg.backward else 0)
+        burst, sustained, tkind = measured_tensor_peaks()
+        sec = ms / args.steps * 1e-3
+        tf_alg, tf_exe = alg * pairs / sec / 1e12, exe * pairs / sec / 1e12
+        ceiling_s = step_bytes / (peak * 1e9)
+        tensor = {"algorithmic_flop_per_step": alg * pairs, "executed_mma_flop_per_step": exe * pairs,
+                  "achieved_tflops": tf_alg, "achieved_tflops_executed": tf_exe,
+                  "peak_burst_tflops": burst, "peak_sustained_tflops": sustained, "peak_kind": f"of {tkind}",
+                  "frac_of_burst": tf_alg / burst, "frac_of_sustained": tf_alg / sustained,
+                  "frac_of_burst_executed": tf_exe / burst,
+                  "hbm_bound_ceiling_frac_of_burst": alg * pairs / ceiling_s / 1e12 / burst,
+                  "ncu_tensor_pipe_pct_of_elapsed": {k: recorded_counters(WORKLOAD, k, "tensor_pipe_pct_of_elapsed")
+                                                     for k in ("gla_fwd_tc", "gla_bwd_tc")} if args.batch <= 0 else None}
+
     if rank == 0:
         cpu = None
         if world == 1 and not args.no_cpu_baseline:
@@ -441,6 +502,8 @@ def main():
                     "steps": e2e_steps, "ms_per_step": ms_e2e / e2e_steps},
             "gpu_launches": n_launch,
             "roofline": roof,
+            "tensor": tensor,
+            "ms_per_step_with_kernel_events": ms_traced / args.steps,
             "step_hbm": {"algorithmic_bytes_per_step": step_bytes, "achieved_gbs": step_gbs, "frac": step_gbs / peak},
             "decode_step": decode,
             "cpu_baseline": cpu,

@@ -25,9 +25,19 @@
  *          log_decay  RETNET [H] (log gamma_h) | GLA [B,T,H,d_k] | GDN [B,T,H]   (all <= 0)
  *          beta       GDN [B,T,H] in (0,1), else NULL
  *          h0, ht, dht, dh0 [B,H,d_k,d_v]  (row = key dimension)
+ *
+ * Decay range.  The recurrences of Eq. 10-16 are defined for every log_decay <= 0, but the chunkwise kernels
+ * split the decay between two tokens of a chunk as e^{b_i} * e^{-b_j} (b = cumulative log-decay inside the chunk)
+ * and keep both factors in fp32 / bf16.  They are exact re-associations as long as the cumulative log-decay over
+ * one chunk stays above -SLA_MAX_CHUNK_DECAY (about -1.2 per token at the largest chunk of 64, -4.7 per token at
+ * chunk 16).  Every chunk is checked on the device: a chunk beyond the limit raises the plan's status word, the
+ * call still completes (its results for that sequence are then not meaningful and may hold inf or NaN), and the next
+ * sla_plan_poll returns SLA_ERR_RANGE.  A smaller chunk widens the range; decode steps have no limit.
  */
 #ifndef SLA_H
 #define SLA_H
+
+#define SLA_MAX_CHUNK_DECAY 76.0f    /* see "Decay range" above */
 
 #include <stddef.h>
 #include <stdint.h>
@@ -45,7 +55,9 @@ typedef enum {
     SLA_ERR_WORKSPACE = 3,     /* workspace NULL or smaller than sla_plan_workspace_bytes      */
     SLA_ERR_ARCH = 4,          /* current device is not compute capability 10.x                */
     SLA_ERR_CUDA = 5,          /* a CUDA runtime call failed (launch, attribute, allocation)   */
-    SLA_ERR_TIMEOUT = 6        /* a bounded device-side wait expired (reported by sla_plan_poll) */
+    SLA_ERR_TIMEOUT = 6,       /* a bounded device-side wait expired (reported by sla_plan_poll) */
+    SLA_ERR_RANGE = 7          /* a chunk's cumulative log-decay left the range the chunkwise kernels can
+                                  represent (reported by sla_plan_poll; see "Decay range" below)       */
 } sla_status;
 
 typedef enum { SLA_RETNET = 0, SLA_GLA = 1, SLA_GDN = 2 } sla_variant;
@@ -87,8 +99,9 @@ sla_status sla_plan_destroy(sla_plan *plan);
 sla_status sla_plan_workspace_bytes(const sla_plan *plan, size_t *forward_bytes, size_t *backward_bytes);
 
 /* Synchronises with nothing; copies the plan's device status word back (on the legacy default
- * stream, so call it after synchronising the stream that ran the work).  SLA_ERR_TIMEOUT if a
- * kernel gave up a bounded wait since the last poll, SLA_OK otherwise. */
+ * stream, so call it after synchronising the stream that ran the work) and clears it.  SLA_ERR_TIMEOUT if a
+ * kernel gave up a bounded wait since the last poll; else SLA_ERR_RANGE if a chunk's cumulative log-decay
+ * was beyond SLA_MAX_CHUNK_DECAY; SLA_OK otherwise. */
 sla_status sla_plan_poll(sla_plan *plan);
 
 /* Diagnostic of the failure path (the paper has no counterpart): enqueues a one-warp kernel whose bounded wait can
@@ -125,6 +138,7 @@ const char *sla_status_string(sla_status s);
  *   o_t     = (scale Gq q_t) S_t, heads concatenated along the last axes      (Eq. 6-7, 11, 13, 16)
  * h0 may be NULL (zero state); ht may be NULL (final state not wanted).
  * gq_logits and gk_logits may alias.  Outputs must not alias inputs.
+ * With T == 0 (and B > 0) there is nothing to read: o is not touched and ht, if given, receives h0 (or zeros).
  */
 sla_status sla_forward(sla_plan *plan,
                        const void *q, const void *k, const void *v,

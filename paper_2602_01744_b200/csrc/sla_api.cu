@@ -53,7 +53,7 @@ __global__ void k_selftest_bounded_wait(int *status, unsigned long long limit_ns
         sla::ptx::fence_mbar_init();
     }
     __syncthreads();
-    if (!sla::ptx::mbar_wait_bounded(bar, 0, nullptr, limit_ns) && threadIdx.x == 0) atomicExch(status, 1);
+    if (!sla::ptx::mbar_wait_bounded(bar, 0, nullptr, limit_ns) && threadIdx.x == 0) atomicOr(status, sla::STATUS_TIMEOUT);
 }
 
 // Can sla_forward of this plan leave what sla_backward needs (SLA_FLAG_SAVE_FOR_BACKWARD)?  Only the tensor-core
@@ -66,12 +66,6 @@ static bool forward_can_save(const sla_plan &p) {
 
 extern "C" {
 
-// Profiling aid (not declared in sla.h): device buffer of >= 16 uint64 that block 0 of the tensor-core
-// kernels fills with %globaltimer stamps at the phase boundaries of one chunk; NULL switches it off.
-void sla_debug_set_phase_timestamps(void *device_buffer) {
-    sla::gla_tc_set_phase_ts((unsigned long long *)device_buffer);
-}
-
 const char *sla_status_string(sla_status s) {
     switch (s) {
         case SLA_OK: return "ok";
@@ -81,6 +75,7 @@ const char *sla_status_string(sla_status s) {
         case SLA_ERR_ARCH: return "device is not sm_100";
         case SLA_ERR_CUDA: return "CUDA runtime error";
         case SLA_ERR_TIMEOUT: return "device-side wait timed out";
+        case SLA_ERR_RANGE: return "cumulative log-decay of a chunk beyond the representable range";
     }
     return "unknown status";
 }
@@ -166,7 +161,7 @@ sla_status sla_plan_poll(sla_plan *plan) {
     if (cudaMemcpy(&v, plan->d_status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return SLA_ERR_CUDA;
     if (v != 0) {
         cudaMemset(plan->d_status, 0, sizeof(int));
-        return SLA_ERR_TIMEOUT;
+        return (v & sla::STATUS_TIMEOUT) ? SLA_ERR_TIMEOUT : SLA_ERR_RANGE;
     }
     return SLA_OK;
 }
@@ -220,14 +215,22 @@ sla_status sla_forward(sla_plan *plan, const void *q, const void *k, const void 
     if (!plan) return SLA_ERR_INVALID_ARG;
     const sla::Dims &d = plan->dims;
     plan->last_launches = 0;
-    if (d.B == 0 || d.T == 0) return SLA_OK;
+    if (d.B == 0) return SLA_OK;
+    if (d.T == 0) {     // nothing to read: the final state is the initial one
+        if (!ht) return SLA_OK;
+        if (!aligned16(ht) || !aligned16(h0)) return SLA_ERR_INVALID_ARG;
+        const size_t bytes = (size_t)d.B * d.H * d.dk * d.dv * sizeof(float);
+        cudaError_t e = h0 ? cudaMemcpyAsync(ht, h0, bytes, cudaMemcpyDeviceToDevice, (cudaStream_t)cuda_stream)
+                           : cudaMemsetAsync(ht, 0, bytes, (cudaStream_t)cuda_stream);
+        return e == cudaSuccess ? SLA_OK : SLA_ERR_CUDA;
+    }
     if (!q || !k || !v || !log_decay || !gq_logits || !gk_logits || !o) return SLA_ERR_INVALID_ARG;
     if (d.variant == SLA_GDN && !beta) return SLA_ERR_INVALID_ARG;
     const void *ptrs[] = {q, k, v, log_decay, beta, gq_logits, gk_logits, h0, o, ht, workspace};
     for (const void *p : ptrs)
         if (!aligned16(p)) return SLA_ERR_INVALID_ARG;
     if (plan->fwd_bytes > 0 && (!workspace || workspace_bytes < plan->fwd_bytes)) return SLA_ERR_WORKSPACE;
-    sla::FwdArgs a{q, k, v, log_decay, beta, gq_logits, gk_logits, h0, o, ht, (float *)workspace};
+    sla::FwdArgs a{q, k, v, log_decay, beta, gq_logits, gk_logits, h0, o, ht, (float *)workspace, plan->d_status};
     plan->tracer.start((cudaStream_t)cuda_stream);
     const bool generic = plan->flags & SLA_FLAG_FORCE_GENERIC;
     const bool save = (plan->flags & SLA_FLAG_SAVE_FOR_BACKWARD) && forward_can_save(*plan);
@@ -259,7 +262,15 @@ sla_status sla_backward(sla_plan *plan, const void *q, const void *k, const void
     if (!plan) return SLA_ERR_INVALID_ARG;
     const sla::Dims &d = plan->dims;
     plan->last_launches = 0;
-    if (d.B == 0 || d.T == 0) return SLA_OK;
+    if (d.B == 0) return SLA_OK;
+    if (d.T == 0) {     // no tokens: the gradient of the initial state is the gradient of the final one
+        if (!dh0) return SLA_OK;
+        if (!aligned16(dh0) || !aligned16(dht)) return SLA_ERR_INVALID_ARG;
+        const size_t bytes = (size_t)d.B * d.H * d.dk * d.dv * sizeof(float);
+        cudaError_t e = dht ? cudaMemcpyAsync(dh0, dht, bytes, cudaMemcpyDeviceToDevice, (cudaStream_t)cuda_stream)
+                            : cudaMemsetAsync(dh0, 0, bytes, (cudaStream_t)cuda_stream);
+        return e == cudaSuccess ? SLA_OK : SLA_ERR_CUDA;
+    }
     if (!q || !k || !v || !log_decay || !gq_logits || !gk_logits || !dO || !dq || !dk || !dv ||
         !dgq_logits || !dgk_logits)
         return SLA_ERR_INVALID_ARG;
@@ -273,14 +284,17 @@ sla_status sla_backward(sla_plan *plan, const void *q, const void *k, const void
         if (!aligned16(p)) return SLA_ERR_INVALID_ARG;
     if (plan->bwd_bytes > 0 && (!workspace || workspace_bytes < plan->bwd_bytes)) return SLA_ERR_WORKSPACE;
     sla::BwdArgs a{q, k, v, log_decay, beta, gq_logits, gk_logits, h0, dO, dht, dq, dk, dv,
-                   dlog_decay, dbeta, dgq_logits, dgk_logits, dh0, (float *)workspace};
+                   dlog_decay, dbeta, dgq_logits, dgk_logits, dh0, (float *)workspace, plan->d_status};
     plan->tracer.start((cudaStream_t)cuda_stream);
     const bool generic = plan->flags & SLA_FLAG_FORCE_GENERIC;
     // the states (GLA) or per-chunk records (GDN) are taken from the workspace only if the last sla_forward of this plan
     // left them there for exactly these inputs, on this stream; anything else recomputes them
-    const sla_plan::Saved &sv = plan->saved;
+    sla_plan::Saved &sv = plan->saved;
     const bool have = sv.valid && sv.ws == workspace && sv.q == q && sv.k == k && sv.v == v && sv.log_decay == log_decay &&
                       sv.beta == beta && sv.lq == gq_logits && sv.lk == gk_logits && sv.h0 == h0 && sv.stream == cuda_stream;
+    // a backward pass that recomputes writes its own states into `workspace`: whatever an earlier forward left there
+    // (for other inputs) is gone, and must not be taken for valid by a later call
+    if (!have && sv.ws == workspace) sv.valid = false;
     int n = (!generic && sla::gla_tc_supported(d))
                 ? sla::gla_tc_backward(d, a, have, plan->d_status, (cudaStream_t)cuda_stream, plan->tracer)
             : (!generic && sla::gdn_tc_supported(d))

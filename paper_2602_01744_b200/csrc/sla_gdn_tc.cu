@@ -305,7 +305,10 @@ k_gdn_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
                 sc[SC_FKB * C + tid] = beta * gam;
                 sc[SC_FVB * C + tid] = beta * gt[C + tid];         // beta Gk
                 sc[SC_BETA * C + tid] = beta;
-                if (tid == C - 1) sc[SC_MISC * C] = gam;           // e^{b_last}
+                if (tid == C - 1) {
+                    sc[SC_MISC * C] = gam;                          // e^{b_last}
+                    if (bi < -SLA_MAX_CHUNK_DECAY) atomicOr(p.status, STATUS_RANGE);
+                }
             }
             named_bar_sync(1, NCOMPUTE);
             mbar_arrive(bar(GFREE + (n & 3)));
@@ -537,7 +540,7 @@ k_gdn_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             }
         }
     }
-    if (failed) atomicExch(p.status, 1);
+    if (failed) atomicOr(p.status, STATUS_TIMEOUT);
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, TMEM_COLS);

@@ -437,7 +437,10 @@ k_gdn_bwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
                 sc[SC_BETA * C + tid] = beta;
                 sc[SC_FVB * C + tid] = beta * gk;
                 sc[SC_GK * C + tid] = gk;
-                if (tid == C - 1) red[20] = gam;                   // e^{b_last}
+                if (tid == C - 1) {
+                    red[20] = gam;                                  // e^{b_last}
+                    if (bi < -SLA_MAX_CHUNK_DECAY) atomicOr(p.status, STATUS_RANGE);
+                }
             }
             named_bar_sync(1, NCOMPUTE);
             mbar_arrive(bar(GFREE + (k & 3)));
@@ -735,7 +738,7 @@ k_gdn_bwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             }
         }
     }
-    if (failed) atomicExch(p.status, 1);
+    if (failed) atomicOr(p.status, STATUS_TIMEOUT);
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, TMEM_COLS);
@@ -766,7 +769,7 @@ int gdn_tc_backward(const Dims &d, const BwdArgs &a, bool have_records, int *sta
     uint8_t *save = reinterpret_cast<uint8_t *>(a.ws);
     float *pq = reinterpret_cast<float *>(save + (size_t)d.B * d.H * (d.NT + 1) * REC_BYTES);
     float *pk = pq + ((bth + 63) & ~(size_t)63);
-    FwdArgs f{a.q, a.k, a.v, a.log_decay, a.beta, a.lq, a.lk, a.h0, nullptr, nullptr, a.ws};
+    FwdArgs f{a.q, a.k, a.v, a.log_decay, a.beta, a.lq, a.lk, a.h0, nullptr, nullptr, a.ws, a.status};
     // (with have_records the forward pass of the same inputs has left the records in this workspace)
     if (!have_records && gdn_tc_forward_save(d, f, save, status, st, tr) < 0) return -1;
     GdnBwdParams bp{a.lq, a.lk, a.log_decay, a.beta, a.dht, save, a.dlog_decay, a.dbeta, pq, pk, a.dh0, status,

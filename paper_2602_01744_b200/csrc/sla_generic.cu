@@ -60,7 +60,8 @@ __global__ void k_gate_bwd(const float *__restrict__ Gq, const float *__restrict
 
 // ------------------------------------------------------------------------------------------
 // a2: chunk-local inclusive cumulative log-decay.  grid (NT, B*H).
-__global__ void k_cumdecay(Dims d, const float *__restrict__ log_decay, float *__restrict__ bcum) {
+// A chunk whose cumulative log-decay is beyond the range of the e^{b}, e^{-b} factors raises STATUS_RANGE.
+__global__ void k_cumdecay(Dims d, const float *__restrict__ log_decay, float *__restrict__ bcum, int *status) {
     int n = blockIdx.x, bh = blockIdx.y, b = bh / d.H, h = bh % d.H;
     int t0 = n * d.C, cn = min(d.C, d.T - t0);
     if (d.variant == SLA_GLA) {
@@ -71,6 +72,7 @@ __global__ void k_cumdecay(Dims d, const float *__restrict__ log_decay, float *_
                 acc += log_decay[idx];
                 bcum[idx] = acc;
             }
+            if (acc < -SLA_MAX_CHUNK_DECAY) atomicOr(status, STATUS_RANGE);
         }
     } else if (threadIdx.x == 0) {
         float acc = 0.f;
@@ -79,6 +81,7 @@ __global__ void k_cumdecay(Dims d, const float *__restrict__ log_decay, float *_
             acc += (d.variant == SLA_RETNET) ? log_decay[h] : log_decay[row];
             bcum[row] = acc;
         }
+        if (acc < -SLA_MAX_CHUNK_DECAY) atomicOr(status, STATUS_RANGE);
     }
 }
 
@@ -731,7 +734,7 @@ int forward_t(const Dims &d, const Workspace &w, const FwdArgs &a, bool write_o,
     tr.mark("gate_fwd");
     ++launches;
     dim3 tiles(d.NT, d.B * d.H);
-    k_cumdecay<<<tiles, d.variant == SLA_GLA ? 128 : 32, 0, st>>>(d, a.log_decay, bcum);
+    k_cumdecay<<<tiles, d.variant == SLA_GLA ? 128 : 32, 0, st>>>(d, a.log_decay, bcum, a.status);
     tr.mark("cumdecay");
     ++launches;
     const TIO *q = (const TIO *)a.q, *k = (const TIO *)a.k, *v = (const TIO *)a.v;
@@ -797,7 +800,7 @@ int generic_forward(const Dims &d, const Workspace &w, const FwdArgs &a, bool wr
 
 int generic_backward(const Dims &d, const Workspace &w, const BwdArgs &a, cudaStream_t st, Tracer &tr) {
     // recompute gates, cumulative decays and the per-chunk states (no output store)
-    FwdArgs f{a.q, a.k, a.v, a.log_decay, a.beta, a.lq, a.lk, a.h0, nullptr, nullptr, a.ws};
+    FwdArgs f{a.q, a.k, a.v, a.log_decay, a.beta, a.lq, a.lk, a.h0, nullptr, nullptr, a.ws, a.status};
     int n1 = generic_forward(d, w, f, false, st, tr);
     if (n1 < 0) return -1;
     int n2;

@@ -57,9 +57,7 @@ struct FwdParams {
     int T, H, NT;
     int P, L;                       // segments per sequence and chunks per segment (P = 1: L = NT)
     float scale;
-    unsigned long long *phase_ts;   // optional: block 0 / thread 0 writes a timestamp at each phase of chunk 8
 };
-#define SLA_TS(k) do { if (p.phase_ts && bh == 0 && tid == 0 && n == 8) p.phase_ts[k] = globaltimer_ns(); } while (0)
 
 // One CTA per (batch, head) sequence, five roles that only meet on mbarriers:
 //   warps 8..15        prologue: cumulative decay, qh, kh of the chunks ahead (as far as the three q/k buffers allow)
@@ -259,7 +257,7 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             const float *g = gate_s + (n & 3) * 2 * C;
             // eblast has four slots: these warps are never more than three chunks ahead of the rescale that reads one
             chunk_prologue<true, false>(qk, qk + TILE_BF16, reinterpret_cast<const float *>(sm + OFF_G), tot, g, g + C,
-                                        eblast + (n & 3) * D, nullptr, ptid, 2,
+                                        eblast + (n & 3) * D, nullptr, p.status, ptid, 2,
                                         [&]() { if (ptid == 0 && n + 1 < NT) load_g(n + 1); });
             fence_proxy_async();
             mbar_arrive(bar(OPR + n % 3));
@@ -373,12 +371,10 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
         mask_a(0);
         for (int n = 0; n < NT; ++n) {
             const uint32_t par = n & 1;
-            SLA_TS(0);
             // the recurrence first: S_{n+1} = diag(2^{b_last}) (S_n + kh^T V), fp32 back into TMEM, bf16 copy for the next
             // chunk's qh S; the tensor core goes on with chunk n+1 the moment this is done
             wait(BAR_Z, par);
             tc_fence_after();
-            SLA_TS(1);
             if (p.simg) wait(SSAVED, par);             // the image store of S_n has read the operand copy
             {
                 const float e = eblast[(n & 3) * D + row];
@@ -406,11 +402,8 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             fence_proxy_async();
             tc_fence_before();
             mbar_arrive(bar(SREADY));
-            SLA_TS(2);
             if (n + 1 < NT) mask_a(n + 1);             // beside the MMAs of chunk n+1: its A tile ...
-            SLA_TS(3);
             stage_o(n);                                // ... and this chunk's output
-            SLA_TS(4);
         }
 
         if (p.ht && seg == p.P - 1) {   // final state, fp32 (each thread reads back what it wrote in the last rescale)
@@ -426,15 +419,13 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             }
         }
     }
-    if (failed) atomicExch(p.status, 1);
+    if (failed) atomicOr(p.status, STATUS_TIMEOUT);
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, TMEM_COLS);
 }
 
 // ---- host side ----
-unsigned long long *g_phase_ts = nullptr;   // set by sla_debug_set_phase_timestamps (profiling aid)
-
 int sm_count() {
     static int n = 0;
     if (!n) {
@@ -459,9 +450,6 @@ void choose_segments(const Dims &d, int &P, int &L) {
     }
 }
 }  // namespace
-
-void gla_tc_set_phase_ts(unsigned long long *p) { g_phase_ts = p; }
-unsigned long long *gla_tc_phase_ts() { return g_phase_ts; }
 
 bool gla_tc_supported(const Dims &d) {
     return d.variant == SLA_GLA && d.io_bf16 && d.dk == 128 && d.dv == 128 && d.C == 64;
@@ -503,7 +491,7 @@ int gla_tc_forward(const Dims &d, const FwdArgs &a, uint8_t *simg, int *status, 
         launches = 2;
         simg = nullptr;
     }
-    FwdParams p{a.lq, a.lk, a.h0, fin, gam, (__nv_bfloat16 *)a.o, a.ht, simg, status, d.T, d.H, d.NT, P, L, d.scale, g_phase_ts};
+    FwdParams p{a.lq, a.lk, a.h0, fin, gam, (__nv_bfloat16 *)a.o, a.ht, simg, status, d.T, d.H, d.NT, P, L, d.scale};
     k_gla_fwd_tc<<<d.B * d.H * P, NTHREADS, SMEM_BYTES, st>>>(mq, mk, mv, mg, mo, p);
     tr.mark("gla_fwd_tc");
     return cudaGetLastError() == cudaSuccess ? launches : -1;

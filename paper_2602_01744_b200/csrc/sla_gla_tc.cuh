@@ -110,13 +110,15 @@ constexpr float LOG2E = 1.4426950408889634f;
 // With WITH_E also leaves the tile e2[i][d] = (bf16 gq_i 2^{b_i}, bf16 gk_i 2^{-b_i}), 4 bytes per element, rows of 512 B,
 // unswizzled: the factors that turn dqh, dkh into dq, dk.  Thread (rg = warp, cj = lane) owns rows 8rg..8rg+7,
 // columns 4cj..4cj+3.
-// tot: [8][128] floats of scratch.
+// tot: [8][128] floats of scratch.  status: the plan's device status word (a chunk whose cumulative log-decay is
+// beyond the representable range raises STATUS_RANGE there).
 constexpr uint32_t TOT_BYTES = 8 * D * 4;
 struct NoHook { __device__ __forceinline__ void operator()() const {} };
 template <bool WITH_Q, bool WITH_E, class Hook = NoHook>
 __device__ __forceinline__ void chunk_prologue(uint8_t *q_tile, uint8_t *k_tile, const float *gs, float *tot,
                                                const float *gq_s, const float *gk_s, float *eblast,
-                                               uint8_t *e2_tile, int tid, int bar_id = 1, Hook tile_read = Hook()) {
+                                               uint8_t *e2_tile, int *status, int tid, int bar_id = 1,
+                                               Hook tile_read = Hook()) {
     using namespace ptx;
     const int rg = tid >> 5, cj = tid & 31;
     float4 gl[8];                               // this thread's log-decay rows: read once, kept for the second pass
@@ -175,6 +177,8 @@ __device__ __forceinline__ void chunk_prologue(uint8_t *q_tile, uint8_t *k_tile,
     if (rg == 7) {
 #pragma unroll
         for (int e = 0; e < 4; ++e) eblast[4 * cj + e] = ex2f(bsum[e]);
+        // beyond this the factors 2^{b}, 2^{-b} leave the exponent range of their fp32 / bf16 carriers
+        if (fminf(fminf(bsum[0], bsum[1]), fminf(bsum[2], bsum[3])) < -SLA_MAX_CHUNK_DECAY * LOG2E) atomicOr(status, STATUS_RANGE);
     }
 }
 

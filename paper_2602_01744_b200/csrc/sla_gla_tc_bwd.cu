@@ -229,7 +229,7 @@ k_gla_states_tc(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
             wait(FULL_K + n % 3, (n / 3) & 1);
             chunk_prologue<false, false>(nullptr, sm + OFF_K + (n % 3) * TILE_BF16,
                                          reinterpret_cast<const float *>(sm + OFF_G + (n & 1) * TILE_G), tot, nullptr,
-                                         gate_s + (n & 3) * C, eblast + (n & 1) * D, nullptr, tid);
+                                         gate_s + (n & 3) * C, eblast + (n & 1) * D, nullptr, p.status, tid);
             fence_proxy_async();
             mbar_arrive(bar(OPR + n % 3));
             mbar_arrive(bar(GFREE + (n & 3)));
@@ -273,7 +273,7 @@ k_gla_states_tc(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
             mbar_arrive(bar(STAGED));
         }
     }
-    if (failed) atomicExch(p.status, 1);
+    if (failed) atomicOr(p.status, STATUS_TIMEOUT);
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, TMEM_COLS);
@@ -315,9 +315,7 @@ struct BwdParams {
     int *status;
     int T, H, NT;
     float scale;
-    unsigned long long *phase_ts;   // optional: block 0 / thread 0 stamps the phases of one chunk
 };
-#define SLA_TS(k) do { if (p.phase_ts && bh == 0 && tid == 0 && n == 8) p.phase_ts[k] = globaltimer_ns(); } while (0)
 
 // Sum v[j] over the 32 lanes for every j: afterwards lane l holds the total of v[l] in v[0].
 __device__ __forceinline__ float warp_transpose_sum(float (&v)[32], int lane) {
@@ -610,21 +608,18 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             const int n = NT - 1 - k, t0 = n * C;
             const uint32_t par = k & 1;
             uint8_t *qk = sm + ((k & 1) ? OFF_Y : OFF_X);          // this chunk's q, k tiles
-            SLA_TS(0);
             // ---- prologue: cumulative decay, qh, kh in place, the (gq 2^b, gk 2^-b) tile ----
             wait(GREADY + (k & 3), (k >> 2) & 1);
             wait(FULL_G, par);
             wait(FULL_QK, par);
-            SLA_TS(1);
             {
                 const float *g = gate_s + (k & 3) * 2 * C;
                 chunk_prologue<true, true>(qk, qk + TILE_BF16, reinterpret_cast<const float *>(sm + OFF_G), tot, g, g + C,
-                                           eblast, sm + OFF_E2, tid);
+                                           eblast, sm + OFF_E2, p.status, tid);
             }
             fence_proxy_async();
             mbar_arrive(bar(OPR));
             mbar_arrive(bar(GFREE + (k & 3)));
-            SLA_TS(2);
 
             // ---- dZ = diag(2^{b_last}) dS_{n+1}: fp32 back into TMEM (dS_n accumulates on it), bf16 operand copy ----
             if (k > 0) wait(DGFREE, (k - 1) & 1);       // the staged tiles of the previous chunk have left dZ and A|dA
@@ -649,12 +644,10 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             fence_proxy_async();
             tc_fence_before();
             mbar_arrive(bar(ZREADY));
-            SLA_TS(3);
 
             // ---- A, dA: TMEM -> causal mask -> bf16 -> shared memory (row i of an M=64 tile sits in lane 32*(i/16) + i%16) ----
             wait(BAR_A, par);
             tc_fence_after();
-            SLA_TS(4);
             {
                 // rows 16q..16q+15 of this warp: a block of 8 columns c is empty for c >= 2q+2, full for c < 2q
                 const int q4 = warp & 3, i = 16 * q4 + lane;
@@ -688,12 +681,10 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             fence_proxy_async();
             tc_fence_before();
             mbar_arrive(bar(AREADY));
-            SLA_TS(5);
 
             // ---- dqh^T, dkh^T: this thread owns key dimension `row` and tokens 32*wh .. 32*wh+31 ----
             wait(BAR_M1, par);
             tc_fence_after();
-            SLA_TS(6);
             const float *Rcur = Rs + (n & 1) * 2 * D;
             float sfx[32];
             {
@@ -727,12 +718,10 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             fence_proxy_async();
             tc_fence_before();
             mbar_arrive(bar(OUT1));
-            SLA_TS(7);
 
             // ---- dV^T -> dv tile; R_{n-1} = rowsum(dS_n * S_n); dlog_decay tile; gate products ----
             wait(BAR_M2, par);
             tc_fence_after();
-            SLA_TS(8);
             {
                 float dvt[32];
                 tmem_ld32(tmem + lane_base + COL_DV + 32 * wh, dvt);
@@ -751,7 +740,6 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
                 Rs[((n & 1) ^ 1) * 2 * D + wh * D + row] = rowdot_part(v0, 0) + rowdot_part(v1, 1);
             }
             mbar_arrive(bar(SNFREE));
-            SLA_TS(9);
             named_bar_sync(1, NCOMPUTE);                // up, red and the R partials are complete
             {   // log-decay gradient: in-chunk suffix sum + what flows in from the right of the chunk
                 const float offs = wh == 1 ? Rcur[row] + Rcur[D + row] : up[row];
@@ -776,7 +764,6 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             fence_proxy_async();
             tc_fence_before();
             mbar_arrive(bar(OUT2));
-            SLA_TS(10);
         }
 
         if (p.dh0) {   // dS_0, fp32 (the last chunk's MMAs were waited for above)
@@ -792,7 +779,7 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             }
         }
     }
-    if (failed) atomicExch(p.status, 1);
+    if (failed) atomicOr(p.status, STATUS_TIMEOUT);
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, TMEM_COLS);
@@ -898,7 +885,7 @@ int gla_tc_backward(const Dims &d, const BwdArgs &a, bool have_states, int *stat
         k_gla_states_tc<<<d.B * d.H, st1::NTHREADS, st1::SMEM_BYTES, st>>>(mk, mv, mg, sp);
         tr.mark("gla_states_tc");
     }
-    BwdParams bp{a.lq, a.lk, a.dht, simg, pq, pk, a.dh0, status, d.T, d.H, d.NT, d.scale, gla_tc_phase_ts()};
+    BwdParams bp{a.lq, a.lk, a.dht, simg, pq, pk, a.dh0, status, d.T, d.H, d.NT, d.scale};
     k_gla_bwd_tc<<<d.B * d.H, st2::NTHREADS, st2::SMEM_BYTES, st>>>(mq, mk, mv, mdo, mg, mdq, mdk, mdv, mdg, bp);
     tr.mark("gla_bwd_tc");
     if (gate_bwd_prod(a.lq, a.lk, pq, pk, a.dlq, a.dlk, (long)d.B * d.T, d.H, st) < 0) return -1;

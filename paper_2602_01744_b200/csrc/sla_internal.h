@@ -11,6 +11,10 @@
 
 namespace sla {
 
+// bits of a plan's device status word
+constexpr int STATUS_TIMEOUT = 1;    // a bounded wait expired
+constexpr int STATUS_RANGE = 2;      // a chunk's cumulative log-decay went below -SLA_MAX_CHUNK_DECAY
+
 struct Dims {
     int variant;      // sla_variant
     int io_bf16;      // 1: q,k,v,o are bf16, 0: fp32
@@ -41,6 +45,7 @@ struct FwdArgs {
     void *o;
     float *ht;
     float *ws;
+    int *status;            // the plan's device status word
 };
 struct BwdArgs {
     const void *q, *k, *v;
@@ -50,6 +55,7 @@ struct BwdArgs {
     void *dq, *dk, *dv;
     float *dlog_decay, *dbeta, *dlq, *dlk, *dh0;
     float *ws;
+    int *status;
 };
 struct DecArgs {
     const void *q, *k, *v;
@@ -95,8 +101,6 @@ int gdn_configure();
 // ---- tensor-core (tcgen05 / TMEM / TMA) Softmax-GLA kernels: sla_gla_tc.cu ----
 bool gla_tc_supported(const Dims &d);
 int gla_tc_configure();
-void gla_tc_set_phase_ts(unsigned long long *device_buffer);
-unsigned long long *gla_tc_phase_ts();
 // With `simg` not null (and gla_tc_forward_can_save) the forward also leaves the bf16 image of the state before every
 // chunk there, in the layout the gradient sweep reads: the backward pass of the same inputs then needs no state sweep.
 bool gla_tc_forward_can_save(const Dims &d);

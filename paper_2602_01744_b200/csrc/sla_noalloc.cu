@@ -56,7 +56,7 @@ extern "C" sla_status sla_forward_noalloc(sla_plan *plan, const void *q, const v
     if (s != SLA_OK) return s;
     // Every region of the scratch the kernels read (gates, cumulative decays, chunk states, WY factors)
     // is written earlier in the same call, so nothing has to be cleared between calls.
-    sla::FwdArgs a{q, k, v, log_decay, beta, gq_logits, gk_logits, h0, o, ht, (float *)scratch};
+    sla::FwdArgs a{q, k, v, log_decay, beta, gq_logits, gk_logits, h0, o, ht, (float *)scratch, plan->d_status};
     plan->tracer.start((cudaStream_t)cuda_stream);
     int n = sla::generic_forward(d, plan->ws, a, true, (cudaStream_t)cuda_stream, plan->tracer);
     if (n < 0) return SLA_ERR_CUDA;

@@ -1,5 +1,7 @@
 """Helpers for the GPU parity tests: run the CUDA path through the C-ABI binding and the oracle on
-the same seeded tensors, and compare per tensor by relative L2 error."""
+the same seeded tensors, and compare per tensor by relative L2 error - once over the whole tensor (the stated
+tolerance) and once row by row (so that a fault confined to one chunk, tail row or segment boundary cannot hide
+in the global figure)."""
 import numpy as np
 import torch
 
@@ -15,6 +17,38 @@ def rel_l2(x, ref):
     ref = np.asarray(ref, dtype=np.float64)
     den = np.linalg.norm(ref)
     return float(np.linalg.norm(x - ref) / den) if den > 0 else float(np.abs(x).max())
+
+
+# Per-row bound.  A row is a vector along the last axis (the d_k / d_v features of one (b, t, h), the H logits of one
+# token, one state row); its error is measured against the RMS row norm of the reference tensor, so the RMS over rows
+# of this figure IS the global relative L2 error.  Rounding noise is not uniform over rows: a row's error scales with
+# its own operands (rows two to three times the RMS norm are common among 10^5..10^6 rows), and the log-decay
+# gradient is a suffix sum whose rounding error grows like a random walk towards the start of a sequence.  Four times
+# the global tolerance covers that spread with margin (measured maxima are noted in the tests); a chunk, tail row or
+# segment boundary that is wrong by more than a few per cent of a typical row fails it.
+ROW_TOL = {"bf16": 4e-2, "fp32": 4e-4}
+
+
+def row_err(x, ref):
+    """max over rows of ||x_row - ref_row|| / rms_rows(||ref_row||); rows run along the last axis."""
+    x = x.detach().double().cpu().numpy() if hasattr(x, "detach") else np.asarray(x, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    if ref.size == 0:
+        return 0.0
+    x = x.reshape(-1, ref.shape[-1])
+    r = ref.reshape(-1, ref.shape[-1])
+    if not np.isfinite(x).all():
+        return float("inf")
+    rms = np.sqrt(np.mean(np.sum(r * r, axis=1)))
+    err = np.sqrt(np.sum((x - r) ** 2, axis=1))
+    return float(err.max() / rms) if rms > 0 else float(err.max())
+
+
+def assert_close(errs_global, errs_row, dtype, what=""):
+    tol, rtol = TOL[dtype], ROW_TOL[dtype]
+    bad = {n: e for n, e in errs_global.items() if not (np.isfinite(e) and e <= tol)}
+    bad_rows = {n: e for n, e in errs_row.items() if not (np.isfinite(e) and e <= rtol)}
+    assert not bad and not bad_rows, (what, "global", bad, "worst row", bad_rows)
 
 
 def to_dev(x):
@@ -68,9 +102,9 @@ def check_forward(cfg, with_h0=False, flags=0, bsel=None):
     o, ht, _ = gpu_forward(cfg, xd, h0=xd.get("h0"), flags=flags)
     oref, htref = oracle_forward(cfg, x, h0=x.get("h0"), bsel=bsel)
     sel = slice(None) if bsel is None else bsel
-    tol = TOL[cfg.dtype]
     errs = {"o": rel_l2(o[sel], oref), "ht": rel_l2(ht[sel], htref)}
-    assert all(np.isfinite(e) and e <= tol for e in errs.values()), (cfg, errs)
+    rows = {"o": row_err(o[sel], oref), "ht": row_err(ht[sel], htref)}
+    assert_close(errs, rows, cfg.dtype, cfg)
     return errs
 
 
@@ -80,13 +114,14 @@ def check_backward(cfg, with_h0=False, flags=0, bsel=None):
     g, _ = gpu_backward(cfg, xd, h0=xd.get("h0"), dht=xd.get("dht"), want_dh0=with_h0, flags=flags)
     ref = oracle_backward(cfg, x, h0=x.get("h0"), dht=x.get("dht"), bsel=bsel)
     sel = slice(None) if bsel is None else bsel
-    tol = TOL[cfg.dtype]
-    errs = {}
+    errs, rows = {}, {}
     for gname, rname in GRAD_NAMES.items():
         if g.get(gname) is None:
             continue
-        errs[gname] = rel_l2(g[gname][sel] if g[gname].dim() > 1 else g[gname], ref[rname])
-    assert all(np.isfinite(e) and e <= tol for e in errs.values()), (cfg, errs)
+        t = g[gname][sel] if g[gname].dim() > 1 else g[gname]
+        errs[gname] = rel_l2(t, ref[rname])
+        rows[gname] = row_err(t, ref[rname])
+    assert_close(errs, rows, cfg.dtype, cfg)
     return errs
 
 
@@ -116,9 +151,50 @@ def check_training_step(cfg, with_h0=False):
     oref, htref = oracle_forward(cfg, x, h0=x.get("h0"))
     ref = oracle_backward(cfg, x, h0=x.get("h0"), dht=x.get("dht"))
     errs = {"o": rel_l2(o, oref), "ht": rel_l2(ht, htref)}
+    rows = {"o": row_err(o, oref), "ht": row_err(ht, htref)}
     for gname, rname in GRAD_NAMES.items():
         if g.get(gname) is not None:
             errs[gname] = rel_l2(g[gname], ref[rname])
-    tol = TOL[cfg.dtype]
-    assert all(np.isfinite(e) and e <= tol for e in errs.values()), (cfg, errs)
+            rows[gname] = row_err(g[gname], ref[rname])
+    assert_close(errs, rows, cfg.dtype, cfg)
     return errs, lf, lb
+
+
+class Guarded:
+    """Device buffers carved out of one pattern-filled arena with guard bands on both sides of each, standing in
+    for a memory checker: after the calls, `check()` asserts that not one guard byte changed."""
+    GUARD = 1 << 16
+    PATTERN = 0xA5
+
+    def __init__(self, total_bytes):
+        self.arena = torch.full((total_bytes,), self.PATTERN, dtype=torch.uint8, device="cuda")
+        self.off = 0
+        self.spans = []
+
+    @classmethod
+    def for_sizes(cls, sizes):
+        return cls(sum(((n + 255) & ~255) + 2 * cls.GUARD for n in sizes) + 512)
+
+    def take(self, nbytes, dtype=torch.uint8, shape=None, fill=None):
+        base = self.arena.data_ptr()
+        start = self.off + self.GUARD
+        start += (-(base + start)) % 256                   # 256-byte aligned, as torch allocations are
+        end = start + nbytes
+        assert end + self.GUARD <= self.arena.numel()
+        self.spans.append((start, end))
+        self.off = end
+        t = self.arena[start:end].view(dtype)
+        if shape is not None:
+            t = t.view(shape)
+        if fill is not None:
+            t.fill_(fill)
+        return t
+
+    def check(self):
+        keep = torch.ones(self.arena.numel(), dtype=torch.bool, device="cuda")
+        for a, b in self.spans:
+            keep[a:b] = False
+        touched = (self.arena != self.PATTERN) & keep
+        n = int(touched.sum())
+        where = int(torch.nonzero(touched)[0]) if n else -1
+        assert n == 0, f"{n} bytes outside the buffers handed to the library were written (first at arena offset {where}; spans {self.spans})"

@@ -1,6 +1,7 @@
 """The five benchmark configurations at full size, in the launch configuration bench.py times
-(default kernel selection), against the oracle on whole batch rows (sequences are independent, so
-a batch row is a set of outputs the oracle can compute on its own)."""
+(default kernel selection, and for the training configurations the plan flags of the benchmark), against the
+oracle on EVERY batch row (the oracle runs a few rows at a time to bound host memory: sequences are independent),
+per tensor and per row."""
 import numpy as np
 import pytest
 import torch
@@ -19,20 +20,47 @@ def test_c0_retnet_fp32():
     assert max(errs.values()) <= 1e-4
 
 
-def test_c1_gla_forward_full_size():
-    gu.check_forward(CONFIGS["C1"], bsel=slice(0, 1))
+def _all_rows(cfg, rows_per_pass):
+    """One GPU pass over the whole configuration (a training step where it has a backward, as bench.py runs it), then
+    the oracle over all batch rows, `rows_per_pass` at a time."""
+    x = make_inputs(cfg)
+    xd = gu.to_dev(x)
+    if cfg.backward:
+        o, ht, g, plan, ws, lf, lb = gu.gpu_training_step(cfg, xd)
+        assert (lf, lb) == (1, 2)
+    else:
+        o, ht, plan = gu.gpu_forward(cfg, xd)
+        g = {}
+    worst, worst_row = {}, {}
+    for b0 in range(0, cfg.B, rows_per_pass):
+        sel = slice(b0, min(cfg.B, b0 + rows_per_pass))
+        oref, htref = gu.oracle_forward(cfg, x, bsel=sel)
+        pairs = {"o": (o[sel], oref), "ht": (ht[sel], htref)}
+        if cfg.backward:
+            ref = gu.oracle_backward(cfg, x, bsel=sel)
+            for gname, rname in gu.GRAD_NAMES.items():
+                if g.get(gname) is not None:
+                    pairs[gname] = (g[gname][sel], ref[rname])
+        errs = {n: gu.rel_l2(a, r) for n, (a, r) in pairs.items()}
+        rows = {n: gu.row_err(a, r) for n, (a, r) in pairs.items()}
+        gu.assert_close(errs, rows, cfg.dtype, (cfg.name, "batch rows", sel))
+        for n in errs:
+            worst[n] = max(worst.get(n, 0.0), errs[n])
+            worst_row[n] = max(worst_row.get(n, 0.0), rows[n])
+    print(cfg.name, "worst relative L2 per tensor:", {n: f"{e:.2e}" for n, e in worst.items()})
+    print(cfg.name, "worst row:", {n: f"{e:.2e}" for n, e in worst_row.items()})
 
 
-def test_c2_gla_forward_backward_full_size():
-    cfg = CONFIGS["C2"]
-    gu.check_forward(cfg, bsel=slice(3, 4))
-    gu.check_backward(cfg, bsel=slice(5, 6))
+def test_c1_gla_forward_full_size_every_row():
+    _all_rows(CONFIGS["C1"], 4)
 
 
-def test_c4_gdn_forward_backward_full_size():
-    cfg = CONFIGS["C4"]
-    gu.check_forward(cfg, bsel=slice(1, 2))
-    gu.check_backward(cfg, bsel=slice(2, 3))
+def test_c2_gla_forward_backward_full_size_every_row():
+    _all_rows(CONFIGS["C2"], 2)
+
+
+def test_c4_gdn_forward_backward_full_size_every_row():
+    _all_rows(CONFIGS["C4"], 2)
 
 
 def test_c3_long_context_prefill_then_decode():
@@ -44,6 +72,9 @@ def test_c3_long_context_prefill_then_decode():
     oref, htref = gu.oracle_forward(cfg, x)
     assert gu.rel_l2(o, oref) <= tol
     assert gu.rel_l2(ht, htref) <= tol
+    # row by row: covers the tokens on both sides of every segment boundary of the segmented forward
+    assert gu.row_err(o, oref) <= gu.ROW_TOL[cfg.dtype]
+    assert gu.row_err(ht, htref) <= gu.ROW_TOL[cfg.dtype]
     # split-sequence property at full size: forward(T1) -> ht -> forward(T2, h0 = ht)
     T1 = 40000 - 40000 % cfg.chunk + 17                 # an uneven cut: ragged chunk on both sides
     parts = []
@@ -54,6 +85,7 @@ def test_c3_long_context_prefill_then_decode():
         o_p, state, _ = gu.gpu_forward(c, sub, h0=state)
         parts.append(o_p)
     assert gu.rel_l2(torch.cat(parts, 1), oref) <= tol
+    assert gu.row_err(torch.cat(parts, 1), oref) <= gu.ROW_TOL[cfg.dtype]
     assert gu.rel_l2(state, htref) <= tol
 
     # decode: the final state replicated into 64 slots, each continuing with its own tokens
@@ -71,6 +103,7 @@ def test_c3_long_context_prefill_then_decode():
                                   dec["gq_logits"][t], dec["gk_logits"][t], ref_state)
     torch.cuda.synchronize()
     assert gu.rel_l2(outs, refs) <= tol
+    assert gu.row_err(outs, refs) <= gu.ROW_TOL[cfg.dtype]
     assert gu.rel_l2(state, ref_state) <= tol
     # the same continuation through the chunkwise kernels with h0 = replicated prefill state
     tr = lambda t: t.transpose(0, 1).contiguous()

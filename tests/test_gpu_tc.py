@@ -135,6 +135,99 @@ def test_saved_states_are_used_only_for_the_same_inputs_and_never_change_the_res
                 assert torch.equal(t, other[n]), n
 
 
+@pytest.mark.parametrize("base", ["C2", "C4"])
+def test_saved_states_are_not_reused_once_another_backward_has_overwritten_them(base):
+    """forward(A) leaves A's chunk states in the workspace; a backward for OTHER contents through the same workspace
+    recomputes and overwrites them; a backward for A's pointers afterwards must recompute too (not read B's states)."""
+    cfg_a = small(CONFIGS[base], B=2, T=300, H=4, seed=911)
+    cfg_b = small(cfg_a, seed=912)
+    xa_host, xb_host = make_inputs(cfg_a, with_dO=True), make_inputs(cfg_b, with_dO=True)
+    xa, xb = gu.to_dev(xa_host), gu.to_dev(xb_host)
+    plan = api.sla_plan_create(cfg_a.variant, cfg_a.dtype, cfg_a.B, cfg_a.T, cfg_a.H, cfg_a.d_k, cfg_a.d_v, cfg_a.chunk,
+                               cfg_a.scale, api.SLA_FLAG_SAVE_FOR_BACKWARD)
+    ws = plan.workspace(backward=True)
+    args = lambda x: (x["q"], x["k"], x["v"], x["log_decay"], x["gq_logits"], x["gk_logits"])
+    api.sla_forward(plan, *args(xa), beta=xa["beta"], workspace=ws)
+    g_a1 = api.sla_backward(plan, *args(xa), xa["dO"], beta=xa["beta"], workspace=ws)
+    assert plan.last_launch_count == 2                 # read what the forward left
+    api.sla_forward(plan, *args(xa), beta=xa["beta"], workspace=ws)
+    g_b = api.sla_backward(plan, *args(xb), xb["dO"], beta=xb["beta"], workspace=ws)
+    assert plan.last_launch_count == 3                 # other inputs: recomputed, into the same workspace
+    g_a2 = api.sla_backward(plan, *args(xa), xa["dO"], beta=xa["beta"], workspace=ws)
+    assert plan.last_launch_count == 3                 # A's states are gone from the workspace: recomputed again
+    g_b2 = api.sla_backward(plan, *args(xb), xb["dO"], beta=xb["beta"], workspace=ws)
+    assert plan.last_launch_count == 3
+    torch.cuda.synchronize()
+    plan.poll()
+    for cfg, xh, grads in ((cfg_a, xa_host, (g_a1, g_a2)), (cfg_b, xb_host, (g_b, g_b2))):
+        ref = gu.oracle_backward(cfg, xh)
+        for g in grads:
+            errs = {n: gu.rel_l2(g[n], ref[r]) for n, r in gu.GRAD_NAMES.items() if g.get(n) is not None}
+            rows = {n: gu.row_err(g[n], ref[r]) for n, r in gu.GRAD_NAMES.items() if g.get(n) is not None}
+            gu.assert_close(errs, rows, cfg.dtype, cfg)
+    for n, t in g_a1.items():
+        if t is not None:
+            assert torch.equal(t, g_a2[n]) and torch.equal(g_b[n], g_b2[n]), n
+
+
+@pytest.mark.parametrize("base,T", [("C2", 200), ("C2", 64), ("C4", 200), ("C4", 65)])
+def test_nothing_is_written_outside_the_buffers_handed_in(base, T):
+    """In place of a memory checker: outputs and workspace are carved out of one pattern-filled arena with guard bands
+    around each; after a training step and a recomputing backward no guard byte may differ, every output element must
+    have been written (they start as NaN) and the results must still match the oracle."""
+    cfg = small(CONFIGS[base], B=2, T=T, H=3, seed=940 + T)
+    xh = make_inputs(cfg, with_dO=True, with_h0=True)
+    x = gu.to_dev(xh)
+    plan = api.sla_plan_create(cfg.variant, cfg.dtype, cfg.B, cfg.T, cfg.H, cfg.d_k, cfg.d_v, cfg.chunk, cfg.scale,
+                               api.SLA_FLAG_SAVE_FOR_BACKWARD)
+    nio = cfg.B * cfg.T * cfg.H * cfg.d_k * 2
+    nst = cfg.B * cfg.H * cfg.d_k * cfg.d_v * 4
+    nl = cfg.B * cfg.T * cfg.H * 4
+    ndec = x["log_decay"].numel() * 4
+    wsb = max(plan.backward_workspace_bytes, plan.forward_workspace_bytes, 16)
+    arena = gu.Guarded.for_sizes([wsb, nio, nst, nio, nio, nio, ndec, nl, nl, nl, nst])
+    nan = float("nan")
+    ws = arena.take(wsb)
+    shape_io = (cfg.B, cfg.T, cfg.H, cfg.d_k)
+    shape_st = (cfg.B, cfg.H, cfg.d_k, cfg.d_v)
+    o = arena.take(nio, torch.bfloat16, shape_io, nan)
+    ht = arena.take(nst, torch.float32, shape_st, nan)
+    out = dict(dq=arena.take(nio, torch.bfloat16, shape_io, nan), dk=arena.take(nio, torch.bfloat16, shape_io, nan),
+               dv=arena.take(nio, torch.bfloat16, shape_io, nan),
+               dlog_decay=arena.take(ndec, torch.float32, tuple(x["log_decay"].shape), nan),
+               dbeta=arena.take(nl, torch.float32, (cfg.B, cfg.T, cfg.H), nan) if cfg.variant == "gdn" else None,
+               dgq_logits=arena.take(nl, torch.float32, (cfg.B, cfg.T, cfg.H), nan),
+               dgk_logits=arena.take(nl, torch.float32, (cfg.B, cfg.T, cfg.H), nan),
+               dh0=arena.take(nst, torch.float32, shape_st, nan))
+    args = (x["q"], x["k"], x["v"], x["log_decay"], x["gq_logits"], x["gk_logits"])
+    api.sla_forward(plan, *args, beta=x["beta"], h0=x["h0"], o=o, ht=ht, workspace=ws)
+    api.sla_backward(plan, *args, x["dO"], beta=x["beta"], h0=x["h0"], dht=x["dht"], workspace=ws, out=out)
+    assert plan.last_launch_count == 2
+    torch.cuda.synchronize()
+    plan.poll()
+    arena.check()
+    oref, htref = gu.oracle_forward(cfg, xh, h0=xh["h0"])
+    ref = gu.oracle_backward(cfg, xh, h0=xh["h0"], dht=xh["dht"])
+    pairs = {"o": (o, oref), "ht": (ht, htref)}
+    pairs.update({n: (out[n], ref[r]) for n, r in gu.GRAD_NAMES.items() if out.get(n) is not None})
+    gu.assert_close({n: gu.rel_l2(a, r) for n, (a, r) in pairs.items()},
+                    {n: gu.row_err(a, r) for n, (a, r) in pairs.items()}, cfg.dtype, cfg)   # (a NaN left in place fails here)
+    # the recomputing backward (state sweep / record sweep into the same workspace) under the same watch
+    for t in out.values():
+        if t is not None:
+            t.fill_(nan)
+    plain = api.sla_plan_create(cfg.variant, cfg.dtype, cfg.B, cfg.T, cfg.H, cfg.d_k, cfg.d_v, cfg.chunk, cfg.scale)
+    assert plain.backward_workspace_bytes <= wsb
+    api.sla_backward(plain, *args, x["dO"], beta=x["beta"], h0=x["h0"], dht=x["dht"], workspace=ws, out=out)
+    assert plain.last_launch_count == 3
+    torch.cuda.synchronize()
+    plain.poll()
+    arena.check()
+    pairs = {n: (out[n], ref[r]) for n, r in gu.GRAD_NAMES.items() if out.get(n) is not None}
+    gu.assert_close({n: gu.rel_l2(a, r) for n, (a, r) in pairs.items()},
+                    {n: gu.row_err(a, r) for n, (a, r) in pairs.items()}, cfg.dtype, cfg)
+
+
 def test_segmented_forward_leaves_nothing_and_the_backward_recomputes():
     cfg = small(CONFIGS["C2"], B=1, T=2048, H=4, seed=920)     # few long sequences: the forward runs in segments
     errs, lf, lb = gu.check_training_step(cfg)

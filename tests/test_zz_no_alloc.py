@@ -18,7 +18,8 @@ def test_noalloc_forward_matches_workspace_forward_twice_in_a_row(variant, dtype
     plan = None
     for call, seed in enumerate((200, 201)):            # two calls in a row on the shared scratch
         cfg = small(base, B=2, T=200 - 36 * call, H=4, d_k=64, d_v=64, dtype=dtype, seed=seed)
-        x = gu.to_dev(make_inputs(cfg, with_h0=True))
+        xh = make_inputs(cfg, with_h0=True)
+        x = gu.to_dev(xh)
         plan = api.sla_plan_create(cfg.variant, cfg.dtype, cfg.B, cfg.T, cfg.H, cfg.d_k, cfg.d_v, cfg.chunk,
                                    cfg.scale, api.SLA_FLAG_FORCE_GENERIC)
         assert plan.forward_workspace_bytes <= api.SLA_NOALLOC_SCRATCH_BYTES
@@ -42,6 +43,12 @@ def test_noalloc_forward_matches_workspace_forward_twice_in_a_row(variant, dtype
             assert torch.cuda.mem_get_info()[0] >= free_before
         assert gu.rel_l2(o, o_ref.double().cpu().numpy()) <= tol
         assert gu.rel_l2(ht, ht_ref.double().cpu().numpy()) <= tol
+        # both calls run the same kernels on the same inputs, only the scratch differs: the bits must agree too
+        assert torch.equal(o, o_ref) and torch.equal(ht, ht_ref)
+        # and against the oracle directly
+        oref, htref = gu.oracle_forward(cfg, xh, h0=xh["h0"])
+        assert gu.rel_l2(o, oref) <= tol and gu.rel_l2(ht, htref) <= tol
+        assert gu.row_err(o, oref) <= gu.ROW_TOL[dtype]
 
 
 def test_noalloc_forward_refuses_problems_beyond_its_scratch():
