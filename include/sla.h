@@ -182,6 +182,22 @@ sla_status sla_decode_step(sla_plan *plan, int32_t Bdec,
                            float *state, void *o_t, void *cuda_stream);
 
 /*
+ * Multi-token decode: n_tokens consecutive recurrent steps (Eq. 5-6 / 10-16) per sequence in one call - what a
+ * serving loop needs when several tokens of a sequence are known at once (chunked prefill of a short prompt tail,
+ * verification of speculated tokens).  Token t of sequence b reads the state token t-1 left; the state travels
+ * from and to memory once per call instead of once per token, every token's output is produced.  Same arithmetic,
+ * in the same order, as n_tokens calls of sla_decode_step (the results are equal bit for bit).
+ * q, k [Bdec,n_tokens,H,d_k]; v, o [Bdec,n_tokens,H,d_v]; log_decay RETNET [H] | GLA [Bdec,n_tokens,H,d_k] |
+ * GDN [Bdec,n_tokens,H]; beta [Bdec,n_tokens,H] (GDN); logits [Bdec,n_tokens,H]; state [Bdec,H,d_k,d_v] fp32,
+ * updated in place.  n_tokens == 1 is sla_decode_step.  Needs no workspace.
+ */
+sla_status sla_decode_steps(sla_plan *plan, int32_t Bdec, int32_t n_tokens,
+                            const void *q, const void *k, const void *v,
+                            const float *log_decay, const float *beta,
+                            const float *gq_logits, const float *gk_logits,
+                            float *state, void *o, void *cuda_stream);
+
+/*
  * sla_forward with built-in scratch (an addition of this library; the paper has no counterpart).
  *
  * Some callers are not allowed to obtain device memory at the point where they run the layer: a

@@ -162,6 +162,18 @@ int sla_oracle_decode_step(int variant, int Bdec, int H, int d_k, int d_v, doubl
                               beta_t, lq_t, lk_t, state, o_t, state);
 }
 
+int sla_oracle_decode_steps(int variant, int Bdec, int n_tok, int H, int d_k, int d_v, double scale,
+                            const double *q, const double *k, const double *v,
+                            const double *log_decay, const double *beta,
+                            const double *lq, const double *lk,
+                            double *state, double *o) {
+    /* n_tok consecutive steps of every sequence: token t reads the state token t-1 left, i.e. the
+     * recurrence of sla_oracle_forward over n_tok tokens started from the caller's state. */
+    if (!state) return -1;
+    return sla_oracle_forward(variant, Bdec, n_tok, H, d_k, d_v, scale, q, k, v, log_decay, beta,
+                              lq, lk, state, o, state);
+}
+
 /* Softmax backward over heads: dl_h = G_h (dG_h - sum_h' G_h' dG_h'). */
 static void head_softmax_backward(const double *G, const double *dG, long n_tok, int H, double *dl) {
     for (long t = 0; t < n_tok; ++t) {

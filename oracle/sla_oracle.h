@@ -66,6 +66,16 @@ int sla_oracle_decode_step(int variant, int Bdec, int H, int d_k, int d_v, doubl
                            const double *lq_t, const double *lk_t,
                            double *state, double *o_t);
 
+/* n_tok consecutive recurrent steps per sequence on a caller-held state (multi-token decode).
+ * q, k [Bdec,n_tok,H,d_k]; v, o [Bdec,n_tok,H,d_v]; log_decay RETNET [H], GLA [Bdec,n_tok,H,d_k],
+ * GDN [Bdec,n_tok,H]; beta, lq, lk [Bdec,n_tok,H]; state [Bdec,H,d_k,d_v] updated in place.
+ * Pinned by: equals n_tok calls of sla_oracle_decode_step on the token slices. */
+int sla_oracle_decode_steps(int variant, int Bdec, int n_tok, int H, int d_k, int d_v, double scale,
+                            const double *q, const double *k, const double *v,
+                            const double *log_decay, const double *beta,
+                            const double *lq, const double *lk,
+                            double *state, double *o);
+
 #ifdef __cplusplus
 }
 #endif

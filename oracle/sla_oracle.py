@@ -51,6 +51,8 @@ def _load():
         lib.sla_oracle_backward.restype = i
         lib.sla_oracle_decode_step.argtypes = [i] * 5 + [d] + [dp] * 9
         lib.sla_oracle_decode_step.restype = i
+        lib.sla_oracle_decode_steps.argtypes = [i] * 6 + [d] + [dp] * 9
+        lib.sla_oracle_decode_steps.restype = i
         _lib = lib
     return _lib
 
@@ -144,4 +146,22 @@ def decode_step(variant, q_t, k_t, v_t, log_decay_t, lq_t, lk_t, state, beta_t=N
                                         _p(state), _p(o))
     if rc != 0:
         raise ValueError("sla_oracle_decode_step rejected its arguments")
+    return o
+
+
+def decode_steps(variant, q, k, v, log_decay, lq, lk, state, beta=None, scale=1.0):
+    """n consecutive steps per sequence: q, k [Bdec,n,H,d_k], v [Bdec,n,H,d_v].  Updates ``state`` in place;
+    returns o [Bdec,n,H,d_v]."""
+    variant = VARIANTS.get(variant, variant)
+    assert isinstance(state, np.ndarray) and state.dtype == np.float64 and state.flags.c_contiguous
+    q, k, v, log_decay, beta, lq, lk = map(_f64, (q, k, v, log_decay, beta, lq, lk))
+    Bd, n, H, d_k = q.shape
+    d_v = v.shape[-1]
+    assert state.shape == (Bd, H, d_k, d_v)
+    assert log_decay.shape == _decay_shape(variant, Bd, n, H, d_k)
+    o = np.zeros((Bd, n, H, d_v))
+    rc = _load().sla_oracle_decode_steps(variant, Bd, n, H, d_k, d_v, float(scale), _p(q), _p(k), _p(v),
+                                         _p(log_decay), _p(beta), _p(lq), _p(lk), _p(state), _p(o))
+    if rc != 0:
+        raise ValueError("sla_oracle_decode_steps rejected its arguments")
     return o

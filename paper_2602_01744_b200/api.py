@@ -24,7 +24,7 @@ EXPORTS = (
     "sla_plan_create", "sla_plan_destroy", "sla_plan_workspace_bytes", "sla_plan_poll",
     "sla_plan_last_launch_count", "sla_plan_set_kernel_timing", "sla_plan_kernel_timing_collect",
     "sla_plan_kernel_timing_get", "sla_status_string", "sla_forward", "sla_backward", "sla_decode_step",
-    "sla_forward_noalloc", "sla_plan_selftest_timeout",
+    "sla_forward_noalloc", "sla_plan_selftest_timeout", "sla_decode_steps",
 )
 SLA_NOALLOC_SCRATCH_BYTES = 32 << 20
 
@@ -83,6 +83,8 @@ def lib():
         L.sla_forward_noalloc.restype = ctypes.c_int
         L.sla_backward.argtypes = [vp] * 19 + [vp, sz, vp]
         L.sla_decode_step.argtypes = [vp, i32] + [vp] * 10
+        L.sla_decode_steps.argtypes = [vp, i32, i32] + [vp] * 10
+        L.sla_decode_steps.restype = ctypes.c_int
         for name in ("sla_plan_create", "sla_plan_destroy", "sla_plan_workspace_bytes", "sla_plan_poll",
                      "sla_plan_set_kernel_timing", "sla_plan_kernel_timing_collect",
                      "sla_plan_kernel_timing_get", "sla_forward", "sla_backward", "sla_decode_step"):
@@ -227,3 +229,16 @@ def sla_decode_step(plan: Plan, q_t, k_t, v_t, log_decay_t, gq_logits_t, gk_logi
         plan.handle, Bdec, _ptr(q_t), _ptr(k_t), _ptr(v_t), _ptr(log_decay_t), _ptr(beta_t),
         _ptr(gq_logits_t), _ptr(gk_logits_t), _ptr(state), _ptr(o_t), _stream()))
     return o_t
+
+
+def sla_decode_steps(plan: Plan, q, k, v, log_decay, gq_logits, gk_logits, state, beta=None, o=None):
+    """n consecutive recurrent steps per sequence on `state` ([Bdec,H,d_k,d_v] fp32, updated in place): q, k
+    [Bdec,n,H,d_k], v [Bdec,n,H,d_v].  Returns o [Bdec,n,H,d_v]."""
+    d = plan.desc
+    Bdec, n = q.shape[0], q.shape[1]
+    if o is None:
+        o = torch.empty((Bdec, n, d.H, d.d_v), dtype=plan.io_torch, device=q.device)
+    _check("sla_decode_steps", lib().sla_decode_steps(
+        plan.handle, Bdec, n, _ptr(q), _ptr(k), _ptr(v), _ptr(log_decay), _ptr(beta), _ptr(gq_logits),
+        _ptr(gk_logits), _ptr(state), _ptr(o), _stream()))
+    return o

@@ -306,26 +306,34 @@ sla_status sla_backward(sla_plan *plan, const void *q, const void *k, const void
     return SLA_OK;
 }
 
-sla_status sla_decode_step(sla_plan *plan, int32_t Bdec, const void *q_t, const void *k_t,
-                           const void *v_t, const float *log_decay_t, const float *beta_t,
-                           const float *gq_logits_t, const float *gk_logits_t, float *state, void *o_t,
-                           void *cuda_stream) {
-    if (!plan || Bdec < 0) return SLA_ERR_INVALID_ARG;
+sla_status sla_decode_steps(sla_plan *plan, int32_t Bdec, int32_t n_tokens, const void *q, const void *k,
+                            const void *v, const float *log_decay, const float *beta,
+                            const float *gq_logits, const float *gk_logits, float *state, void *o,
+                            void *cuda_stream) {
+    if (!plan || Bdec < 0 || n_tokens < 0) return SLA_ERR_INVALID_ARG;
     const sla::Dims &d = plan->dims;
     plan->last_launches = 0;
-    if (Bdec == 0) return SLA_OK;
-    if (!q_t || !k_t || !v_t || !log_decay_t || !gq_logits_t || !gk_logits_t || !state || !o_t)
-        return SLA_ERR_INVALID_ARG;
-    if (d.variant == SLA_GDN && !beta_t) return SLA_ERR_INVALID_ARG;
-    const void *ptrs[] = {q_t, k_t, v_t, log_decay_t, beta_t, gq_logits_t, gk_logits_t, state, o_t};
+    if (Bdec == 0 || n_tokens == 0) return SLA_OK;
+    if ((uint64_t)Bdec * d.H > 0x7fffffffu) return SLA_ERR_UNSUPPORTED;
+    if (!q || !k || !v || !log_decay || !gq_logits || !gk_logits || !state || !o) return SLA_ERR_INVALID_ARG;
+    if (d.variant == SLA_GDN && !beta) return SLA_ERR_INVALID_ARG;
+    const void *ptrs[] = {q, k, v, log_decay, beta, gq_logits, gk_logits, state, o};
     for (const void *p : ptrs)
         if (!aligned16(p)) return SLA_ERR_INVALID_ARG;
-    sla::DecArgs a{q_t, k_t, v_t, log_decay_t, beta_t, gq_logits_t, gk_logits_t, state, o_t, Bdec};
+    sla::DecArgs a{q, k, v, log_decay, beta, gq_logits, gk_logits, state, o, Bdec, n_tokens};
     plan->tracer.start((cudaStream_t)cuda_stream);
     int n = sla::decode_step(d, a, (cudaStream_t)cuda_stream, plan->tracer);
     if (n < 0) return SLA_ERR_CUDA;
     plan->last_launches = n;
     return SLA_OK;
+}
+
+sla_status sla_decode_step(sla_plan *plan, int32_t Bdec, const void *q_t, const void *k_t,
+                           const void *v_t, const float *log_decay_t, const float *beta_t,
+                           const float *gq_logits_t, const float *gk_logits_t, float *state, void *o_t,
+                           void *cuda_stream) {
+    return sla_decode_steps(plan, Bdec, 1, q_t, k_t, v_t, log_decay_t, beta_t, gq_logits_t, gk_logits_t, state, o_t,
+                            cuda_stream);
 }
 
 }  // extern "C"

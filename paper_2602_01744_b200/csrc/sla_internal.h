@@ -63,6 +63,7 @@ struct DecArgs {
     float *state;
     void *o;
     int Bdec;
+    int n_tok;              // consecutive tokens per sequence applied in one launch
 };
 
 // Optional per-kernel timing: one CUDA event before the first kernel of a call and one after every

@@ -20,17 +20,19 @@ def rel_l2(x, ref):
 
 
 # Per-row bound.  A row is a vector along the last axis (the d_k / d_v features of one (b, t, h), the H logits of one
-# token, one state row); its error is measured against the RMS row norm of the reference tensor, so the RMS over rows
-# of this figure IS the global relative L2 error.  Rounding noise is not uniform over rows: a row's error scales with
-# its own operands (rows two to three times the RMS norm are common among 10^5..10^6 rows), and the log-decay
-# gradient is a suffix sum whose rounding error grows like a random walk towards the start of a sequence.  Four times
-# the global tolerance covers that spread with margin (measured maxima are noted in the tests); a chunk, tail row or
-# segment boundary that is wrong by more than a few per cent of a typical row fails it.
+# token, one state row).  Its error ||x_row - ref_row|| is measured against its own norm, or against the RMS row norm
+# of the tensor where the row is smaller than that: every row is right to a few bf16 roundings at its own scale (the
+# head gates make row norms heavy tailed - 15 to 25 times the RMS norm occur in the benchmark configurations - so an
+# absolute bound would only bind on the largest rows), and a small row is right at the scale of a typical one.
+# With operands and outputs rounded to bf16 (relative 2^-9 each, a handful of roundings per value) whole tensors sit at
+# 3e-3..4e-3; single rows, over 10^5..10^6 of them, reach 1.5e-2 (o, dq, dk, dv) and 2.5e-2 (the logit, beta and decay
+# gradients, which are sums with cancellation).  Four times the global tolerance bounds that with margin; a chunk, tail
+# row or segment boundary that is off by more than a few per cent of its own size fails it.
 ROW_TOL = {"bf16": 4e-2, "fp32": 4e-4}
 
 
 def row_err(x, ref):
-    """max over rows of ||x_row - ref_row|| / rms_rows(||ref_row||); rows run along the last axis."""
+    """max over rows of ||x_row - ref_row|| / max(||ref_row||, rms_rows ||ref_row||); rows run along the last axis."""
     x = x.detach().double().cpu().numpy() if hasattr(x, "detach") else np.asarray(x, dtype=np.float64)
     ref = np.asarray(ref, dtype=np.float64)
     if ref.size == 0:
@@ -39,9 +41,11 @@ def row_err(x, ref):
     r = ref.reshape(-1, ref.shape[-1])
     if not np.isfinite(x).all():
         return float("inf")
-    rms = np.sqrt(np.mean(np.sum(r * r, axis=1)))
+    norm = np.sqrt(np.sum(r * r, axis=1))
+    rms = np.sqrt(np.mean(norm * norm))
     err = np.sqrt(np.sum((x - r) ** 2, axis=1))
-    return float(err.max() / rms) if rms > 0 else float(err.max())
+    den = np.maximum(norm, rms)
+    return float((err / den).max()) if rms > 0 else float(err.max())
 
 
 def assert_close(errs_global, errs_row, dtype, what=""):

@@ -63,3 +63,39 @@ def test_prefill_then_graphed_decode(base):
             for t in range(steps)]
     assert gu.rel_l2(outs, np.stack(refs)) <= 1e-2
     assert gu.rel_l2(state_graph, ref_state) <= 1e-2
+
+
+@pytest.mark.parametrize("variant,dtype", [("retnet", "fp32"), ("gla", "bf16"), ("gdn", "bf16"), ("gla", "fp32")])
+@pytest.mark.parametrize("n_tok", [2, 5, 16])
+def test_multi_token_decode_equals_single_steps_bit_for_bit_and_the_oracle(variant, dtype, n_tok):
+    """sla_decode_steps keeps the state in registers over n tokens; it must give the bits of n sla_decode_step calls
+    (outputs and state) and match the oracle's n recurrent steps."""
+    base = {"retnet": CONFIGS["C0"], "gla": CONFIGS["C1"], "gdn": CONFIGS["C4"]}[variant]
+    d = 128 if dtype == "bf16" else 48
+    cfg = small(base, B=4, T=n_tok, H=4, d_k=d, d_v=d, dtype=dtype, seed=960)   # (B*H*4 bytes per step: slices stay 16-byte aligned)
+    dec = make_decode_inputs(cfg, cfg.B, n_tok, seed=961)          # [n, B, H, d]
+    h0 = torch.randn(cfg.B, cfg.H, cfg.d_k, cfg.d_v, generator=torch.Generator().manual_seed(8)) * 0.1
+    plan = api.sla_plan_create(cfg.variant, cfg.dtype, cfg.B, 64, cfg.H, cfg.d_k, cfg.d_v, cfg.chunk, 0.9)
+    dd = {n: (None if t is None else t.cuda()) for n, t in dec.items()}
+    s1 = h0.clone().cuda()
+    outs = []
+    for t in range(n_tok):
+        ld = dd["log_decay"] if variant == "retnet" else dd["log_decay"][t]
+        outs.append(api.sla_decode_step(plan, dd["q"][t], dd["k"][t], dd["v"][t], ld, dd["gq_logits"][t],
+                                        dd["gk_logits"][t], s1, beta_t=None if dd["beta"] is None else dd["beta"][t]))
+    tm = lambda t: None if t is None else t.transpose(0, 1).contiguous()     # token-major per sequence: [B, n, H, d]
+    s2 = h0.clone().cuda()
+    ld = dd["log_decay"] if variant == "retnet" else tm(dd["log_decay"])
+    o2 = api.sla_decode_steps(plan, tm(dd["q"]), tm(dd["k"]), tm(dd["v"]), ld, tm(dd["gq_logits"]), tm(dd["gk_logits"]),
+                              s2, beta=tm(dd["beta"]))
+    torch.cuda.synchronize()
+    assert plan.last_launch_count == 1
+    assert torch.equal(o2, torch.stack(outs, 1)) and torch.equal(s1, s2)
+    ref_state = np.ascontiguousarray(h0.double().numpy().copy())
+    cm = lambda t: None if t is None else t.transpose(0, 1).contiguous()
+    oref = orc.decode_steps(variant, cm(dec["q"]), cm(dec["k"]), cm(dec["v"]),
+                            dec["log_decay"] if variant == "retnet" else cm(dec["log_decay"]), cm(dec["gq_logits"]),
+                            cm(dec["gk_logits"]), ref_state, beta=cm(dec["beta"]), scale=0.9)
+    tol = gu.TOL[dtype]
+    assert gu.rel_l2(o2, oref) <= tol and gu.row_err(o2, oref) <= gu.ROW_TOL[dtype]
+    assert gu.rel_l2(s2, ref_state) <= tol

@@ -210,6 +210,33 @@ def test_state_carry_and_decode_agree_with_one_pass(variant):
     np.testing.assert_allclose(state, ht, rtol=1e-12, atol=1e-13)
 
 
+@pytest.mark.parametrize("variant", ["retnet", "gla", "gdn"])
+def test_multi_token_decode_is_the_single_step_repeated(variant):
+    """decode_steps over n tokens = n decode_step calls on the token slices (same state, same outputs), and two calls
+    of 3 and 4 tokens = one call of 7."""
+    x, h0 = draw(variant, T=7, seed=23)
+    s_multi = np.ascontiguousarray(h0.copy())
+    o_multi = orc.decode_steps(variant, x["q"], x["k"], x["v"], x["log_decay"], x["lq"], x["lk"], s_multi,
+                               beta=x["beta"], scale=0.7)
+    s_one = np.ascontiguousarray(h0.copy())
+    for t in range(7):
+        ld = x["log_decay"] if variant == "retnet" else x["log_decay"][:, t]
+        bt = None if x["beta"] is None else x["beta"][:, t]
+        ot = orc.decode_step(variant, x["q"][:, t], x["k"][:, t], x["v"][:, t], ld, x["lq"][:, t], x["lk"][:, t],
+                             s_one, beta_t=bt, scale=0.7)
+        np.testing.assert_allclose(o_multi[:, t], ot, rtol=1e-13, atol=1e-14)
+    np.testing.assert_allclose(s_multi, s_one, rtol=1e-13, atol=1e-14)
+    s_split = np.ascontiguousarray(h0.copy())
+    part = lambda a, sl: a if (a is None or a.ndim == 1) else np.ascontiguousarray(a[:, sl])
+    outs = []
+    for sl in (slice(0, 3), slice(3, 7)):
+        outs.append(orc.decode_steps(variant, part(x["q"], sl), part(x["k"], sl), part(x["v"], sl),
+                                     part(x["log_decay"], sl), part(x["lq"], sl), part(x["lk"], sl), s_split,
+                                     beta=part(x["beta"], sl), scale=0.7))
+    np.testing.assert_allclose(np.concatenate(outs, 1), o_multi, rtol=1e-13, atol=1e-14)
+    np.testing.assert_allclose(s_split, s_multi, rtol=1e-13, atol=1e-14)
+
+
 def test_bad_arguments_are_rejected():
     z = np.zeros((1, 2, 1, 2))
     with pytest.raises(ValueError):
