@@ -428,6 +428,30 @@ def main():
             timings[name] = 1e3 * e0.elapsed_time(e1) / (16 * 8)
         decode["batch_1"] = {"us_per_step_launched_one_by_one": timings["launched"],
                              "us_per_step_as_one_cuda_graph_of_8_steps": timings["graph"]}
+        # multi-token decode (sla_decode_steps): n tokens per sequence per call, the state read and written once per call
+        multi = {}
+        for nt in (4, 16):
+            md = make_decode_inputs(c3, C3_DECODE_BATCH, nt, seed=6)
+            tm = lambda t: None if t is None else t.transpose(0, 1).contiguous().cuda()      # [batch, n, H, d]
+            mq, mk, mv, mg, mlq, mlk = (tm(md[n]) for n in ("q", "k", "v", "log_decay", "gq_logits", "gk_logits"))
+            mo = torch.empty((C3_DECODE_BATCH, nt, c3.H, c3.d_v), dtype=torch.bfloat16, device="cuda")
+            row = {}
+            for label, bsz in (("batch_64", C3_DECODE_BATCH), ("batch_1", 1)):
+                sts = states if bsz > 1 else [st_[:1] for st_ in states]
+                call = lambda i: api.sla_decode_steps(dplan, mq[:bsz], mk[:bsz], mv[:bsz], mg[:bsz], mlq[:bsz], mlk[:bsz],
+                                                      sts[i % NSTATE], o=mo[:bsz])
+                for i in range(4):
+                    call(i)
+                torch.cuda.synchronize()
+                e0.record()
+                for i in range(32):
+                    call(i)
+                e1.record()
+                torch.cuda.synchronize()
+                us_call = 1e3 * e0.elapsed_time(e1) / 32
+                row[label] = {"us_per_call": us_call, "us_per_token": us_call / nt}
+            multi[f"{nt}_tokens_per_call"] = row
+        decode["multi_token"] = multi
 
     # ---- roofline of the dominant kernel, from the per-kernel CUDA events of the timed region ----
     peak, peak_kind = measured_peaks()

@@ -101,7 +101,7 @@ sla_status sla_plan_create(sla_plan **out, const sla_desc *desc) {
     if (prop.major != 10) return SLA_ERR_ARCH;
     if (sla::generic_configure() != 0 || sla::gdn_configure() != 0 || sla::gla_tc_configure() != 0 ||
         sla::gla_tc_bwd_configure() != 0 || sla::gdn_tc_configure() != 0 ||
-        sla::gdn_tc_bwd_configure() != 0)
+        sla::gdn_tc_bwd_configure() != 0 || sla::decode_configure() != 0)
         return SLA_ERR_CUDA;
 
     sla_plan *p = new (std::nothrow) sla_plan();
@@ -314,7 +314,7 @@ sla_status sla_decode_steps(sla_plan *plan, int32_t Bdec, int32_t n_tokens, cons
     const sla::Dims &d = plan->dims;
     plan->last_launches = 0;
     if (Bdec == 0 || n_tokens == 0) return SLA_OK;
-    if ((uint64_t)Bdec * d.H > 0x7fffffffu) return SLA_ERR_UNSUPPORTED;
+    if ((uint64_t)Bdec * d.H * d.dk > 0x7fffffffu) return SLA_ERR_UNSUPPORTED;   // (row coordinate of the state's tensor map)
     if (!q || !k || !v || !log_decay || !gq_logits || !gk_logits || !state || !o) return SLA_ERR_INVALID_ARG;
     if (d.variant == SLA_GDN && !beta) return SLA_ERR_INVALID_ARG;
     const void *ptrs[] = {q, k, v, log_decay, beta, gq_logits, gk_logits, state, o};
@@ -322,7 +322,7 @@ sla_status sla_decode_steps(sla_plan *plan, int32_t Bdec, int32_t n_tokens, cons
         if (!aligned16(p)) return SLA_ERR_INVALID_ARG;
     sla::DecArgs a{q, k, v, log_decay, beta, gq_logits, gk_logits, state, o, Bdec, n_tokens};
     plan->tracer.start((cudaStream_t)cuda_stream);
-    int n = sla::decode_step(d, a, (cudaStream_t)cuda_stream, plan->tracer);
+    int n = sla::decode_step(d, a, plan->d_status, (cudaStream_t)cuda_stream, plan->tracer);
     if (n < 0) return SLA_ERR_CUDA;
     plan->last_launches = n;
     return SLA_OK;

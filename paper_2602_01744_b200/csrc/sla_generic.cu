@@ -579,113 +579,6 @@ k_grads_lin(Dims d, const TIO *__restrict__ q, const TIO *__restrict__ k, const 
 }
 
 // ------------------------------------------------------------------------------------------
-// a7: recurrent decode, one CTA per (sequence, head): n_tok consecutive tokens of the sequence are applied to the fp32
-// state, which is read from HBM once, kept in registers across the tokens and written back once (HBM-bound).
-// Inputs are token-major per sequence, [Bdec, n_tok, H, d]; n_tok = 1 is the single decode step.
-// 256 threads: warp w owns state rows w, w+8, ...; lane l owns the four columns 4l..4l+3 (one 16-byte access per
-// row, a warp moves one 512-byte row per instruction).  The state loads are issued before anything else so that
-// the gate softmax and the operand set-up of the first token run under their latency.
-template <typename TIO>
-__global__ void __launch_bounds__(256, 2)
-k_decode(Dims d, int Bdec, int n_tok, const TIO *__restrict__ q, const TIO *__restrict__ k,
-         const TIO *__restrict__ v, const float *__restrict__ log_decay,
-         const float *__restrict__ beta, const float *__restrict__ lq, const float *__restrict__ lk,
-         float *__restrict__ state, TIO *__restrict__ o) {
-    __shared__ float qs[128], ks[128], as[128], us[128];
-    __shared__ float4 red[8][32];
-    __shared__ float gate[2];
-    const int bh = blockIdx.x, b = bh / d.H, h = bh % d.H;
-    const int ty = threadIdx.x >> 5, tx = threadIdx.x & 31;
-    const bool col_ok = 4 * tx < d.dv;
-    float4 *S4 = reinterpret_cast<float4 *>(state + (size_t)bh * d.dk * d.dv);
-    const int ld4 = d.dv >> 2;
-    float4 s[16];
-#pragma unroll
-    for (int r = 0; r < 16; ++r) {
-        const int row = ty + 8 * r;
-        s[r] = (row < d.dk && col_ok) ? S4[(size_t)row * ld4 + tx] : make_float4(0.f, 0.f, 0.f, 0.f);
-    }
-    const bool gdn = d.variant == SLA_GDN;
-    for (int t = 0; t < n_tok; ++t) {
-        const size_t tok = (size_t)b * n_tok + t, th = tok * d.H + h;   // token row, (token, head) row
-        if (threadIdx.x < 64) {       // two warps: gates of this head from the H logits of the token (Eq. 4)
-            const float *l = (ty == 0 ? lq : lk) + tok * d.H;
-            float x = tx < d.H ? l[tx] : -INFINITY;
-            float m = x;
-#pragma unroll
-            for (int o2 = 16; o2 > 0; o2 >>= 1) m = fmaxf(m, __shfl_xor_sync(FULL, m, o2));
-            float e = tx < d.H ? expf(x - m) : 0.f, sum = e;
-#pragma unroll
-            for (int o2 = 16; o2 > 0; o2 >>= 1) sum += __shfl_xor_sync(FULL, sum, o2);
-            if (tx == h) gate[ty] = e / sum;
-        }
-        __syncthreads();
-        const float Gq = gate[0], Gk = gate[1];
-        for (int c = threadIdx.x; c < d.dk; c += blockDim.x) {
-            size_t idx = th * d.dk + c;
-            qs[c] = d.scale * Gq * ldf(q, idx);
-            ks[c] = (gdn ? 1.f : Gk) * ldf(k, idx);
-            float g = d.variant == SLA_RETNET ? log_decay[h] : (d.variant == SLA_GLA ? log_decay[idx] : log_decay[th]);
-            as[c] = expf(g);
-        }
-        for (int j = threadIdx.x; j < d.dv; j += blockDim.x)
-            us[j] = (gdn ? Gk : 1.f) * ldf(v, th * d.dv + j);
-        __syncthreads();
-#pragma unroll
-        for (int r = 0; r < 16; ++r) {        // decay: Sbar = diag(a) S
-            const int row = ty + 8 * r;
-            const float a = row < d.dk ? as[row] : 0.f;
-            s[r].x *= a; s[r].y *= a; s[r].z *= a; s[r].w *= a;
-        }
-        if (gdn) {                    // u = beta (Gk v - k Sbar)
-            float4 part = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-            for (int r = 0; r < 16; ++r) {
-                const int row = ty + 8 * r;
-                const float kr = row < d.dk ? ks[row] : 0.f;
-                part.x = fmaf(kr, s[r].x, part.x); part.y = fmaf(kr, s[r].y, part.y);
-                part.z = fmaf(kr, s[r].z, part.z); part.w = fmaf(kr, s[r].w, part.w);
-            }
-            red[ty][tx] = part;
-            __syncthreads();
-            if (threadIdx.x < d.dv) {
-                const int j = threadIdx.x;
-                float acc = 0.f;
-#pragma unroll
-                for (int w = 0; w < 8; ++w) acc += reinterpret_cast<const float *>(&red[w][j >> 2])[j & 3];
-                us[j] = beta[th] * (us[j] - acc);
-            }
-            __syncthreads();
-        }
-        const float4 u4 = col_ok ? *reinterpret_cast<const float4 *>(&us[4 * tx]) : make_float4(0.f, 0.f, 0.f, 0.f);
-        float4 part = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-        for (int r = 0; r < 16; ++r) {        // write: S = Sbar + k^T u ; read: o = q S
-            const int row = ty + 8 * r;
-            if (row < d.dk && col_ok) {
-                const float kr = ks[row], qr = qs[row];
-                s[r].x = fmaf(kr, u4.x, s[r].x); s[r].y = fmaf(kr, u4.y, s[r].y);
-                s[r].z = fmaf(kr, u4.z, s[r].z); s[r].w = fmaf(kr, u4.w, s[r].w);
-                if (t == n_tok - 1) S4[(size_t)row * ld4 + tx] = s[r];      // the state goes back once, after the last token
-                part.x = fmaf(qr, s[r].x, part.x); part.y = fmaf(qr, s[r].y, part.y);
-                part.z = fmaf(qr, s[r].z, part.z); part.w = fmaf(qr, s[r].w, part.w);
-            }
-        }
-        __syncthreads();
-        red[ty][tx] = part;
-        __syncthreads();
-        if (threadIdx.x < d.dv) {
-            const int j = threadIdx.x;
-            float acc = 0.f;
-#pragma unroll
-            for (int w = 0; w < 8; ++w) acc += reinterpret_cast<const float *>(&red[w][j >> 2])[j & 3];
-            stf(o, th * d.dv + j, acc);
-        }
-        __syncthreads();              // red, us and the operand arrays are rewritten for the next token
-    }
-}
-
-// ------------------------------------------------------------------------------------------
 // host side
 size_t smem_prepare(const Dims &d) {
     return sizeof(float) * (CMAX * (d.dk + 1) + CMAX * (CMAX + 1) + CMAX * (d.dk + d.dv) + 2 * CMAX);
@@ -844,21 +737,6 @@ int generic_backward(const Dims &d, const Workspace &w, const BwdArgs &a, cudaSt
     tr.mark("gate_bwd");
     if (cudaGetLastError() != cudaSuccess) return -1;
     return n1 + n2 + 1;
-}
-
-int decode_step(const Dims &d, const DecArgs &a, cudaStream_t st, Tracer &tr) {
-    dim3 grid(a.Bdec * d.H);
-    if (d.io_bf16)
-        k_decode<__nv_bfloat16><<<grid, 256, 0, st>>>(d, a.Bdec, a.n_tok, (const __nv_bfloat16 *)a.q,
-                                                      (const __nv_bfloat16 *)a.k, (const __nv_bfloat16 *)a.v,
-                                                      a.log_decay, a.beta, a.lq, a.lk, a.state,
-                                                      (__nv_bfloat16 *)a.o);
-    else
-        k_decode<float><<<grid, 256, 0, st>>>(d, a.Bdec, a.n_tok, (const float *)a.q, (const float *)a.k,
-                                              (const float *)a.v, a.log_decay, a.beta, a.lq, a.lk, a.state,
-                                              (float *)a.o);
-    tr.mark("decode");
-    return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 
 }  // namespace sla

@@ -94,7 +94,9 @@ struct Tracer {
 // Each returns the number of kernels launched (>0) or -1 after a CUDA launch error.
 int generic_forward(const Dims &d, const Workspace &w, const FwdArgs &a, bool write_o, cudaStream_t st, Tracer &tr);
 int generic_backward(const Dims &d, const Workspace &w, const BwdArgs &a, cudaStream_t st, Tracer &tr);
-int decode_step(const Dims &d, const DecArgs &a, cudaStream_t st, Tracer &tr);
+// recurrent decode (sla_decode.cu): streaming kernel over 32-column slices of the state
+int decode_step(const Dims &d, const DecArgs &a, int *status, cudaStream_t st, Tracer &tr);
+int decode_configure();
 // Opt the kernels into the shared memory they need (once per device).
 int generic_configure();
 int gdn_configure();
