@@ -37,11 +37,22 @@ GDN_BWD_BYTES_PER_TOKEN_HEAD = 4 * 256 + 3 * 256 + 8 + 8 + 16   # 1824
 # recomputation of the backward is counted only when the plan recomputes).
 GLA_FLOP = {"fwd_algorithmic": 82176, "bwd_algorithmic": 205440, "fwd_executed": 98304, "bwd_executed": 212992,
             "state_recompute_executed": 32768}
+# Softmax-RetNet: the decay is a constant per head, so no decay tensor is read and no decay gradient written.
+RETNET_FWD_BYTES_PER_TOKEN_HEAD = 4 * 256 + 8           # 1032
+RETNET_BWD_BYTES_PER_TOKEN_HEAD = 4 * 256 + 3 * 256 + 16   # 1808
 KERNEL_BYTES = {  # which share of the compulsory traffic each kernel is accountable for
     "output": FWD_BYTES_PER_TOKEN_HEAD, "grads_lin": BWD_BYTES_PER_TOKEN_HEAD,
     "gla_fwd_tc": FWD_BYTES_PER_TOKEN_HEAD, "gla_bwd_tc": BWD_BYTES_PER_TOKEN_HEAD,
     "gdn_fwd_tc": GDN_FWD_BYTES_PER_TOKEN_HEAD, "gdn_bwd_tc": GDN_BWD_BYTES_PER_TOKEN_HEAD,
 }
+KERNEL_BYTES_RETNET = {"gla_fwd_tc": RETNET_FWD_BYTES_PER_TOKEN_HEAD, "gla_bwd_tc": RETNET_BWD_BYTES_PER_TOKEN_HEAD}
+
+
+def step_bytes_per_pair(variant: str, backward: bool) -> int:
+    f, b = {"gla": (FWD_BYTES_PER_TOKEN_HEAD, BWD_BYTES_PER_TOKEN_HEAD),
+            "gdn": (GDN_FWD_BYTES_PER_TOKEN_HEAD, GDN_BWD_BYTES_PER_TOKEN_HEAD),
+            "retnet": (RETNET_FWD_BYTES_PER_TOKEN_HEAD, RETNET_BWD_BYTES_PER_TOKEN_HEAD)}[variant]
+    return f + (b if backward else 0)
 
 
 def measured_peaks():
@@ -135,7 +146,7 @@ def cpu_oracle_sample(cfg, x, steps=1, warmup=0):
     """fp64 oracle, forward (+ backward where the workload has one), on the first CPU_ROWS batch rows of the workload
     (all T tokens, all heads)."""
     from oracle import sla_oracle as orc
-    s = lambda t: t[0:CPU_ROWS]
+    s = lambda t: t if t.dim() == 1 else t[0:CPU_ROWS]      # (RetNet's log-decay is per head, not per batch row)
     args = (s(x["q"]), s(x["k"]), s(x["v"]), s(x["log_decay"]), s(x["gq_logits"]), s(x["gk_logits"]))
     # widen once outside the timed region, as the GPU arm holds its inputs resident
     args = tuple(a.double().numpy() for a in args)
@@ -188,9 +199,10 @@ def main():
     ap.add_argument("--recompute", action="store_true",
                     help="plan without SLA_FLAG_SAVE_FOR_BACKWARD: the backward pass recomputes the chunk states "
                          "instead of reading what the forward pass of the same step left in the workspace")
-    ap.add_argument("--workload", default="C2", choices=["C1", "C2", "C3", "C4"],
+    ap.add_argument("--workload", default="C2", choices=["C1", "C2", "C3", "C4", "R2"],
                     help="C2 is the benchmark; the other configurations (C1, C3: forward only; C4: gated delta rule, "
-                         "forward + backward) are timed the same way for the per-configuration figures and profiles")
+                         "forward + backward; R2: Softmax-RetNet at the shapes of C2) are timed the same way for the "
+                         "per-configuration figures and profiles")
     ap.add_argument("--batch", type=int, default=0,
                     help="profiling aid: shrink the batch of the workload (0 = the full configuration; "
                          "a reduced batch is not the benchmark and is labelled in config)")
@@ -248,7 +260,7 @@ def main():
     grads = None
     if cfg.backward:
         grads = dict(dq=torch.empty_like(dev["q"]), dk=torch.empty_like(dev["k"]), dv=torch.empty_like(dev["v"]),
-                     dlog_decay=torch.empty_like(dev["log_decay"]),
+                     dlog_decay=None if cfg.variant == "retnet" else torch.empty_like(dev["log_decay"]),
                      dbeta=None if dev["beta"] is None else torch.empty_like(dev["beta"]),
                      dgq_logits=torch.empty_like(dev["gq_logits"]), dgk_logits=torch.empty_like(dev["gk_logits"]),
                      dh0=None)
@@ -460,7 +472,7 @@ def main():
         top = max(ktimes, key=lambda k: ktimes[k][1])
         cnt, tot = ktimes[top]
         avg_ms = tot / cnt
-        per_unit = KERNEL_BYTES.get(top)
+        per_unit = (KERNEL_BYTES_RETNET if cfg.variant == "retnet" else KERNEL_BYTES).get(top)
         share = {k: round(v[1] / sum(t[1] for t in ktimes.values()), 4) for k, v in ktimes.items()}
         if per_unit is not None:
             alg = per_unit * cfg.B * cfg.T * cfg.H
@@ -473,16 +485,14 @@ def main():
                     "peak_kind": f"of {peak_kind}", "traffic": None, "avg_launch_ms": avg_ms,
                     "kernel_time_share": share}
     # whole-step figure against the same peak: all compulsory bytes of forward + backward / step time
-    gdn = cfg.variant == "gdn"
-    step_bytes = ((GDN_FWD_BYTES_PER_TOKEN_HEAD if gdn else FWD_BYTES_PER_TOKEN_HEAD) +
-                  ((GDN_BWD_BYTES_PER_TOKEN_HEAD if gdn else BWD_BYTES_PER_TOKEN_HEAD) if cfg.backward else 0)) * cfg.B * cfg.T * cfg.H
+    step_bytes = step_bytes_per_pair(cfg.variant, cfg.backward) * cfg.B * cfg.T * cfg.H
     step_gbs = step_bytes / (ms / args.steps * 1e-3) / 1e9
 
     # the tensor-core side of the metric: algorithmic MMA FLOP of a step / step time against the dense bf16 peaks.
     # The step is HBM-bound (66 FLOP/B against a ridge near 256), so the fraction it could reach at the HBM roofline
     # is stated beside it.
     tensor = None
-    if cfg.variant == "gla" and cfg.d_k == 128 and cfg.d_v == 128 and not args.generic:
+    if cfg.variant in ("gla", "retnet") and cfg.d_k == 128 and cfg.d_v == 128 and not args.generic:
         pairs = cfg.B * cfg.T * cfg.H
         alg = GLA_FLOP["fwd_algorithmic"] + (GLA_FLOP["bwd_algorithmic"] if cfg.backward else 0)
         exe = GLA_FLOP["fwd_executed"] + ((GLA_FLOP["bwd_executed"] + (0 if saving else GLA_FLOP["state_recompute_executed"]))

@@ -57,6 +57,7 @@ struct FwdParams {
     int T, H, NT;
     int P, L;                       // segments per sequence and chunks per segment (P = 1: L = NT)
     float scale;
+    const float *log_gamma;         // Softmax-RetNet: [H] constant log-decays (no log-decay tensor is read); else nullptr
 };
 
 // One CTA per (batch, head) sequence, five roles that only meet on mbarriers:
@@ -247,18 +248,21 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             mbar_expect_tx(bar(FULL_G), TILE_G);
             tma_load_4d(base + OFF_G, &tm_g, 0, h, (n0 + n) * C, b, bar(FULL_G));
         };
-        if (ptid == 0) load_g(0);
+        const bool retnet = p.log_gamma != nullptr;
+        const float lgam = retnet ? p.log_gamma[h] : 0.f;
+        if (ptid == 0 && !retnet) load_g(0);
         for (int n = 0; n < NT; ++n) {
             wait(GREADY + (n & 3), (n >> 2) & 1);
-            wait(FULL_G, n & 1);
+            if (!retnet) wait(FULL_G, n & 1);
             wait(FULL_QK + n % 3, (n / 3) & 1);
             if (failed) break;
             uint8_t *qk = sm + OFF_QK + (n % 3) * QK_BYTES;
             const float *g = gate_s + (n & 3) * 2 * C;
             // eblast has four slots: these warps are never more than three chunks ahead of the rescale that reads one
-            chunk_prologue<true, false>(qk, qk + TILE_BF16, reinterpret_cast<const float *>(sm + OFF_G), tot, g, g + C,
+            chunk_prologue<true, false>(qk, qk + TILE_BF16, retnet ? nullptr : reinterpret_cast<const float *>(sm + OFF_G), tot, g, g + C,
                                         eblast + (n & 3) * D, nullptr, p.status, ptid, 2,
-                                        [&]() { if (ptid == 0 && n + 1 < NT) load_g(n + 1); });
+                                        [&]() { if (ptid == 0 && n + 1 < NT && !retnet) load_g(n + 1); },
+                                        ScalarDecay{lgam, min(C, p.T - (n0 + n) * C)});
             fence_proxy_async();
             mbar_arrive(bar(OPR + n % 3));
             mbar_arrive(bar(GFREE + (n & 3)));
@@ -451,8 +455,10 @@ void choose_segments(const Dims &d, int &P, int &L) {
 }
 }  // namespace
 
+// Softmax-GLA (Eq. 12-13) and Softmax-RetNet (Eq. 10-11: the same recurrence with a constant decay per head, which the
+// kernels generate instead of reading a [B,T,H,d_k] tensor).
 bool gla_tc_supported(const Dims &d) {
-    return d.variant == SLA_GLA && d.io_bf16 && d.dk == 128 && d.dv == 128 && d.C == 64;
+    return (d.variant == SLA_GLA || d.variant == SLA_RETNET) && d.io_bf16 && d.dk == 128 && d.dv == 128 && d.C == 64;
 }
 
 int gla_tc_configure() {
@@ -476,10 +482,12 @@ bool gla_tc_forward_can_save(const Dims &d) {
 
 int gla_tc_forward(const Dims &d, const FwdArgs &a, uint8_t *simg, int *status, cudaStream_t st, Tracer &tr) {
     CUtensorMap mq, mk, mv, mg, mo;
+    const bool retnet = d.variant == SLA_RETNET;
     if (!make_tile_map(&mq, a.q, d.B, d.T, d.H) || !make_tile_map(&mk, a.k, d.B, d.T, d.H) ||
-        !make_tile_map(&mv, a.v, d.B, d.T, d.H) || !make_map(&mg, a.log_decay, d.B, d.T, d.H, d.dk, true, 128) ||
-        !make_tile_map(&mo, a.o, d.B, d.T, d.H))
+        !make_tile_map(&mv, a.v, d.B, d.T, d.H) || !make_tile_map(&mo, a.o, d.B, d.T, d.H))
         return -1;
+    if (retnet) mg = mq;   // (never used: the decay is generated in the kernel)
+    else if (!make_map(&mg, a.log_decay, d.B, d.T, d.H, d.dk, true, 128)) return -1;
     int P, L, launches = 1;
     choose_segments(d, P, L);
     float *fin = nullptr, *gam = nullptr;
@@ -491,7 +499,7 @@ int gla_tc_forward(const Dims &d, const FwdArgs &a, uint8_t *simg, int *status, 
         launches = 2;
         simg = nullptr;
     }
-    FwdParams p{a.lq, a.lk, a.h0, fin, gam, (__nv_bfloat16 *)a.o, a.ht, simg, status, d.T, d.H, d.NT, P, L, d.scale};
+    FwdParams p{a.lq, a.lk, a.h0, fin, gam, (__nv_bfloat16 *)a.o, a.ht, simg, status, d.T, d.H, d.NT, P, L, d.scale, retnet ? a.log_decay : nullptr};
     k_gla_fwd_tc<<<d.B * d.H * P, NTHREADS, SMEM_BYTES, st>>>(mq, mk, mv, mg, mo, p);
     tr.mark("gla_fwd_tc");
     return cudaGetLastError() == cudaSuccess ? launches : -1;

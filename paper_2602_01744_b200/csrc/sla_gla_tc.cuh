@@ -103,7 +103,8 @@ __device__ __forceinline__ float ex2f(float x) {
 constexpr uint32_t NCOMPUTE = 256;      // compute threads (warps 0..7); they meet on named barrier 1
 constexpr float LOG2E = 1.4426950408889634f;
 
-// Chunk prologue, run by 256 threads (tid 0..255, meeting on named barrier bar_id) on one landed stage (Eq. 12's decay made chunk-local):
+// Chunk prologue, run by 256 threads (tid 0..255, meeting on named barrier bar_id) on one landed stage (the decay of Eq. 12, or of
+// Eq. 10 when gs is null, made chunk-local):
 //   b_i = inclusive cumulative log-decay (kept in log2 units), two-level: per-8-row sums, then a running sum
 //   qh_i = gq_i * q_i * 2^{b_i}   (gq_i = scale*Gq_i)      kh_i = gk_i * k_i * 2^{-b_i}
 // written over q and k in place (the swizzled tiles are the MMA operands); eblast[d] = 2^{b_last,d}.
@@ -114,11 +115,14 @@ constexpr float LOG2E = 1.4426950408889634f;
 // beyond the representable range raises STATUS_RANGE there).
 constexpr uint32_t TOT_BYTES = 8 * D * 4;
 struct NoHook { __device__ __forceinline__ void operator()() const {} };
+// Softmax-RetNet runs on the same kernels: with gs == nullptr the chunk's log-decay tile is not read but generated,
+// log_gamma on each of the chunk's cn tokens (all key dimensions alike).
+struct ScalarDecay { float log_gamma = 0.f; int cn = 0; };
 template <bool WITH_Q, bool WITH_E, class Hook = NoHook>
 __device__ __forceinline__ void chunk_prologue(uint8_t *q_tile, uint8_t *k_tile, const float *gs, float *tot,
                                                const float *gq_s, const float *gk_s, float *eblast,
                                                uint8_t *e2_tile, int *status, int tid, int bar_id = 1,
-                                               Hook tile_read = Hook()) {
+                                               Hook tile_read = Hook(), ScalarDecay sc = ScalarDecay()) {
     using namespace ptx;
     const int rg = tid >> 5, cj = tid & 31;
     float4 gl[8];                               // this thread's log-decay rows: read once, kept for the second pass
@@ -126,7 +130,12 @@ __device__ __forceinline__ void chunk_prologue(uint8_t *q_tile, uint8_t *k_tile,
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
         for (int rr = 0; rr < 8; ++rr) {
-            gl[rr] = *reinterpret_cast<const float4 *>(gs + (8 * rg + rr) * D + 4 * cj);
+            if (gs) {
+                gl[rr] = *reinterpret_cast<const float4 *>(gs + (8 * rg + rr) * D + 4 * cj);
+            } else {                            // Eq. 10: one constant log-decay per head, none past the sequence end
+                const float v = 8 * rg + rr < sc.cn ? sc.log_gamma : 0.f;
+                gl[rr] = make_float4(v, v, v, v);
+            }
             acc.x += gl[rr].x; acc.y += gl[rr].y; acc.z += gl[rr].z; acc.w += gl[rr].w;
         }
         *reinterpret_cast<float4 *>(tot + rg * D + 4 * cj) = acc;

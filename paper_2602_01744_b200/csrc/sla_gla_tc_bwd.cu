@@ -56,6 +56,7 @@ struct StatesParams {
     int *status;
     int T, H, NT;
     int P, L;               // segments per sequence and chunks per segment (image mode: P = 1, L = NT)
+    const float *log_gamma; // Softmax-RetNet: [H] constant log-decays (no log-decay tensor is read); else nullptr
 };
 
 // thread (row, colhalf) holds 32 consecutive state values of its row: bf16 them into the operand image
@@ -159,11 +160,12 @@ k_gla_states_tc(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
                 mbar_expect_tx(bf, TILE_BF16);
                 tma_load_5d(base + OFF_V + (n & 1) * TILE_BF16, &tm_v, 0, (n0 + n) * C, 0, h, b, bf);
             };
-            for (int n = 0; n < 2 && n < NT; ++n) load_g(n);
+            const bool retnet = p.log_gamma != nullptr;
+            for (int n = 0; n < 2 && n < NT && !retnet; ++n) load_g(n);
             for (int n = 0; n < 3 && n < NT; ++n) load_k(n);
             for (int n = 0; n < 2 && n < NT; ++n) load_v(n);
             for (int n = 0; n < NT && !failed; ++n) {
-                if (n + 2 < NT) {                    // log-decay buffer: free once the prologue of chunk n is done
+                if (n + 2 < NT && !retnet) {         // log-decay buffer: free once the prologue of chunk n is done
                     wait(OPR + n % 3, (n / 3) & 1);
                     if (failed) break;
                     load_g(n + 2);
@@ -223,13 +225,16 @@ k_gla_states_tc(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
         tc_fence_before();
         mbar_arrive(bar(SREADY));
 
+        const bool retnet = p.log_gamma != nullptr;
+        const float lgam = retnet ? p.log_gamma[h] : 0.f;
         auto prologue = [&](int n) {
             wait(GREADY + (n & 3), (n >> 2) & 1);
-            wait(FULL_G + (n & 1), (n >> 1) & 1);
+            if (!retnet) wait(FULL_G + (n & 1), (n >> 1) & 1);
             wait(FULL_K + n % 3, (n / 3) & 1);
             chunk_prologue<false, false>(nullptr, sm + OFF_K + (n % 3) * TILE_BF16,
-                                         reinterpret_cast<const float *>(sm + OFF_G + (n & 1) * TILE_G), tot, nullptr,
-                                         gate_s + (n & 3) * C, eblast + (n & 1) * D, nullptr, p.status, tid);
+                                         retnet ? nullptr : reinterpret_cast<const float *>(sm + OFF_G + (n & 1) * TILE_G), tot, nullptr,
+                                         gate_s + (n & 3) * C, eblast + (n & 1) * D, nullptr, p.status, tid, 1, NoHook(),
+                                         ScalarDecay{lgam, min(C, p.T - (n0 + n) * C)});
             fence_proxy_async();
             mbar_arrive(bar(OPR + n % 3));
             mbar_arrive(bar(GFREE + (n & 3)));
@@ -315,6 +320,7 @@ struct BwdParams {
     int *status;
     int T, H, NT;
     float scale;
+    const float *log_gamma;         // Softmax-RetNet: [H] constant log-decays (no log-decay read, no log-decay gradient)
 };
 
 // Sum v[j] over the 32 lanes for every j: afterwards lane l holds the total of v[l] in v[0].
@@ -497,11 +503,12 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
                 mbar_expect_tx(bar(FULL_S), STATE_BF16);
                 bulk_load(base + OFF_S, img0 + (size_t)n * STATE_BF16, STATE_BF16, bar(FULL_S));
             };
+            const bool retnet = p.log_gamma != nullptr;
             if (p.dht) {                               // S_NT, for rowsum(dht * S_NT)
                 mbar_expect_tx(bar(INIT_FULL), STATE_BF16);
                 bulk_load(base + OFF_S, img0 + (size_t)NT * STATE_BF16, STATE_BF16, bar(INIT_FULL));
             }
-            load_g(NT - 1);
+            if (!retnet) load_g(NT - 1);
             load_qk(NT - 1, 0);
             load_vdo(NT - 1, 0);
             if (p.dht) wait(INIT_DONE, 0);             // the compute warps are done with S_NT
@@ -519,7 +526,7 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
                     bulk_prefetch_l2(img0 + (size_t)(n - 1) * STATE_BF16, STATE_BF16);
                     wait(OPR, par);                    // prologue done: the log-decay buffer is free
                     if (failed) break;
-                    load_g(n - 1);
+                    if (!retnet) load_g(n - 1);
                     wait(DOFREE, par);                 // every MMA of the chunk is done: its (v, dO) buffer takes the next q, k
                     if (failed) break;
                     load_qk(n - 1, k + 1);
@@ -539,7 +546,7 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
                 wait_relaxed(OUT2, par);               // dv, dlog_decay staged
                 if (failed) break;
                 tma_store_5d(&tm_dv, base + OFF_A, 0, n * C, 0, h, b);
-                tma_store_4d(&tm_dg, base + OFF_DZ, 0, h, n * C, b);
+                if (!retnet) tma_store_4d(&tm_dg, base + OFF_DZ, 0, h, n * C, b);
                 bulk_commit();
                 bulk_wait_read0();
                 mbar_arrive(bar(DGFREE));
@@ -569,6 +576,8 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
         const uint32_t lane_base = (uint32_t)(32 * (warp & 3)) << 16;
         const int wh = warp >> 2;                       // column half (state passes) / token half (gradient tiles)
         const int row = 32 * (warp & 3) + lane;         // TMEM lane = key (value) dimension owned by this thread
+        const bool retnet = p.log_gamma != nullptr;
+        const float lgam = retnet ? p.log_gamma[h] : 0.f;
 
         // rowsum(dS * S) over this thread's 64 columns, with dS in registers part by part
         auto rowdot_part = [&](const float (&v)[32], int part) {
@@ -610,12 +619,13 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             uint8_t *qk = sm + ((k & 1) ? OFF_Y : OFF_X);          // this chunk's q, k tiles
             // ---- prologue: cumulative decay, qh, kh in place, the (gq 2^b, gk 2^-b) tile ----
             wait(GREADY + (k & 3), (k >> 2) & 1);
-            wait(FULL_G, par);
+            if (!retnet) wait(FULL_G, par);
             wait(FULL_QK, par);
             {
                 const float *g = gate_s + (k & 3) * 2 * C;
-                chunk_prologue<true, true>(qk, qk + TILE_BF16, reinterpret_cast<const float *>(sm + OFF_G), tot, g, g + C,
-                                           eblast, sm + OFF_E2, p.status, tid);
+                chunk_prologue<true, true>(qk, qk + TILE_BF16, retnet ? nullptr : reinterpret_cast<const float *>(sm + OFF_G), tot, g, g + C,
+                                           eblast, sm + OFF_E2, p.status, tid, 1, NoHook(),
+                                           ScalarDecay{lgam, min(C, p.T - t0)});
             }
             fence_proxy_async();
             mbar_arrive(bar(OPR));
@@ -854,10 +864,11 @@ size_t gla_tc_backward_workspace_bytes(const Dims &d) {
 int gla_tc_segment_summaries(const Dims &d, const FwdArgs &a, int P, int L, float *fin, float *gam, int *status,
                              cudaStream_t st, Tracer &tr) {
     CUtensorMap mk, mv, mg;
-    if (!make_tile_map(&mk, a.k, d.B, d.T, d.H) || !make_tile_map(&mv, a.v, d.B, d.T, d.H) ||
-        !make_map(&mg, a.log_decay, d.B, d.T, d.H, d.dk, true, 128))
-        return -1;
-    StatesParams sp{a.lq, a.lk, nullptr, nullptr, fin, gam, status, d.T, d.H, d.NT, P, L};
+    const bool retnet = d.variant == SLA_RETNET;
+    if (!make_tile_map(&mk, a.k, d.B, d.T, d.H) || !make_tile_map(&mv, a.v, d.B, d.T, d.H)) return -1;
+    if (retnet) mg = mk;   // (never used: the decay is generated in the kernel)
+    else if (!make_map(&mg, a.log_decay, d.B, d.T, d.H, d.dk, true, 128)) return -1;
+    StatesParams sp{a.lq, a.lk, nullptr, nullptr, fin, gam, status, d.T, d.H, d.NT, P, L, retnet ? a.log_decay : nullptr};
     k_gla_states_tc<<<d.B * d.H * P, st1::NTHREADS, st1::SMEM_BYTES, st>>>(mk, mv, mg, sp);
     tr.mark("gla_segment_states_tc");
     return cudaGetLastError() == cudaSuccess ? 1 : -1;
@@ -867,11 +878,15 @@ uint8_t *gla_tc_state_images(float *ws) { return reinterpret_cast<uint8_t *>(ws)
 
 int gla_tc_backward(const Dims &d, const BwdArgs &a, bool have_states, int *status, cudaStream_t st, Tracer &tr) {
     CUtensorMap mq, mk, mv, mdo, mg, mdq, mdk, mdv, mdg;
+    const bool retnet = d.variant == SLA_RETNET;      // constant decay: no log-decay tensor to read, no gradient for it
     if (!make_tile_map(&mq, a.q, d.B, d.T, d.H) || !make_tile_map(&mk, a.k, d.B, d.T, d.H) ||
         !make_tile_map(&mv, a.v, d.B, d.T, d.H) || !make_tile_map(&mdo, a.dO, d.B, d.T, d.H) ||
-        !make_map(&mg, a.log_decay, d.B, d.T, d.H, d.dk, true, 128) ||
         !make_tile_map(&mdq, a.dq, d.B, d.T, d.H) || !make_tile_map(&mdk, a.dk, d.B, d.T, d.H) ||
-        !make_tile_map(&mdv, a.dv, d.B, d.T, d.H) || !make_map(&mdg, a.dlog_decay, d.B, d.T, d.H, d.dk, true, 128))
+        !make_tile_map(&mdv, a.dv, d.B, d.T, d.H))
+        return -1;
+    if (retnet) { mg = mq; mdg = mdq; }               // (never used)
+    else if (!make_map(&mg, a.log_decay, d.B, d.T, d.H, d.dk, true, 128) ||
+             !make_map(&mdg, a.dlog_decay, d.B, d.T, d.H, d.dk, true, 128))
         return -1;
     // workspace: state images, then the two [B,T,H] gate products
     const size_t bth = (size_t)d.B * d.T * d.H;
@@ -881,11 +896,11 @@ int gla_tc_backward(const Dims &d, const BwdArgs &a, bool have_states, int *stat
     float *pk = pq + ((bth + 63) & ~(size_t)63);
 
     if (!have_states) {   // (otherwise the forward pass of the same inputs has left the images in this workspace)
-        StatesParams sp{a.lq, a.lk, a.h0, simg, nullptr, nullptr, status, d.T, d.H, d.NT, 1, d.NT};
+        StatesParams sp{a.lq, a.lk, a.h0, simg, nullptr, nullptr, status, d.T, d.H, d.NT, 1, d.NT, retnet ? a.log_decay : nullptr};
         k_gla_states_tc<<<d.B * d.H, st1::NTHREADS, st1::SMEM_BYTES, st>>>(mk, mv, mg, sp);
         tr.mark("gla_states_tc");
     }
-    BwdParams bp{a.lq, a.lk, a.dht, simg, pq, pk, a.dh0, status, d.T, d.H, d.NT, d.scale};
+    BwdParams bp{a.lq, a.lk, a.dht, simg, pq, pk, a.dh0, status, d.T, d.H, d.NT, d.scale, retnet ? a.log_decay : nullptr};
     k_gla_bwd_tc<<<d.B * d.H, st2::NTHREADS, st2::SMEM_BYTES, st>>>(mq, mk, mv, mdo, mg, mdq, mdk, mdv, mdg, bp);
     tr.mark("gla_bwd_tc");
     if (gate_bwd_prod(a.lq, a.lk, pq, pk, a.dlq, a.dlk, (long)d.B * d.T, d.H, st) < 0) return -1;

@@ -33,6 +33,9 @@ CONFIGS = {
     "C2": SLAConfig("C2", "gla", 8, 4096, 16, 128, 128, "bf16", 64, 2, True),
     "C3": SLAConfig("C3", "gla", 1, 65536, 16, 128, 128, "bf16", 64, 3, False),
     "C4": SLAConfig("C4", "gdn", 4, 4096, 16, 128, 128, "bf16", 64, 4, True),
+    # Softmax-RetNet at the shapes of C2 (the variant of Eq. 10-11 on the tensor-core kernels; not one of the five
+    # benchmark configurations, timed by `bench.py --workload R2`)
+    "R2": SLAConfig("R2", "retnet", 8, 4096, 16, 128, 128, "bf16", 64, 5, True),
 }
 C3_DECODE_BATCH = 64
 C3_DECODE_STEPS = 256

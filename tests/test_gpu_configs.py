@@ -63,6 +63,10 @@ def test_c4_gdn_forward_backward_full_size_every_row():
     _all_rows(CONFIGS["C4"], 2)
 
 
+def test_r2_retnet_forward_backward_full_size_every_row():
+    _all_rows(CONFIGS["R2"], 2)
+
+
 def test_c3_long_context_prefill_then_decode():
     cfg = CONFIGS["C3"]
     tol = gu.TOL[cfg.dtype]

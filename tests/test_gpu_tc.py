@@ -250,3 +250,36 @@ def test_training_step_is_reproducible_bit_for_bit(base, B, T, H):
         else:
             for a, b in zip(first, cur):
                 assert torch.equal(a, b)
+
+
+# ---- Softmax-RetNet (Eq. 10-11) on the tensor-core kernels: the GLA kernels with the decay generated in the kernel ----
+@pytest.mark.parametrize("B,T,H,with_h0", [(1, 64, 1, False), (2, 200, 3, True), (1, 1000, 16, True), (3, 65, 4, True),
+                                           (1, 5, 2, False), (1, 2048, 4, False)])       # the last one runs segmented
+def test_retnet_forward_and_backward_tc(B, T, H, with_h0):
+    cfg = small(CONFIGS["R2"], B=B, T=T, H=H, seed=1000 + T)
+    assert max(gu.check_forward(small(cfg, backward=False), with_h0=with_h0).values()) <= 1e-2
+    assert max(gu.check_backward(cfg, with_h0=with_h0).values()) <= 1e-2
+
+
+def test_retnet_takes_the_tensor_core_path_and_agrees_with_generic():
+    cfg = small(CONFIGS["R2"], B=2, T=300, H=4, seed=1010, scale=0.5)
+    x = gu.to_dev(make_inputs(cfg, with_dO=True, with_h0=True))
+    o1, ht1, plan = gu.gpu_forward(cfg, x, h0=x["h0"])
+    assert plan.last_launch_count == 1 and plan.forward_workspace_bytes == 0
+    o2, ht2, plan2 = gu.gpu_forward(cfg, x, h0=x["h0"], flags=api.SLA_FLAG_FORCE_GENERIC)
+    assert plan2.last_launch_count > 1
+    assert gu.rel_l2(o1, o2.double().cpu().numpy()) <= 1e-2 and gu.rel_l2(ht1, ht2.double().cpu().numpy()) <= 1e-2
+    g1, plan = gu.gpu_backward(cfg, x, h0=x["h0"], dht=x["dht"], want_dh0=True)
+    assert plan.last_launch_count == 3
+    g2, plan2 = gu.gpu_backward(cfg, x, h0=x["h0"], dht=x["dht"], want_dh0=True, flags=api.SLA_FLAG_FORCE_GENERIC)
+    for name in ("dq", "dk", "dv", "dgq_logits", "dgk_logits", "dh0"):
+        assert gu.rel_l2(g1[name], g2[name].double().cpu().numpy()) <= 1e-2, name
+    assert g1["dlog_decay"] is None
+
+
+@pytest.mark.parametrize("B,T,H,with_h0", [(2, 200, 3, True), (1, 960, 8, False)])
+def test_retnet_training_step_reads_what_the_forward_left(B, T, H, with_h0):
+    cfg = small(CONFIGS["R2"], B=B, T=T, H=H, seed=1020 + T)
+    errs, lf, lb = gu.check_training_step(cfg, with_h0=with_h0)
+    assert (lf, lb) == (1, 2)
+    assert max(errs.values()) <= 1e-2
