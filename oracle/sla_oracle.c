@@ -45,6 +45,37 @@ void sla_oracle_head_softmax(const double *logits, long n_tok, int H, double *ga
     }
 }
 
+/*
+ * Eq. 4, the score projections that feed the head softmax.  Reading taken: W_G in R^{d x H} with d the per-head
+ * width (the paper's parameter count, about 0.05M for 24 layers of two such matrices at hidden 1024 with 4 heads,
+ * only fits d = 256 = 1024 / 4), and the score of head h comes from that head's own vector through column h:
+ *     s[b,t,h] = sum_c x[b,t,h,c] * W[c,h]        (x = q with W_GQ, x = k with W_GK)
+ * x: [n_tok, H, d], W: [d, H], s: [n_tok, H].
+ */
+void sla_oracle_gate_scores(long n_tok, int H, int d, const double *x, const double *W, double *s) {
+    for (long t = 0; t < n_tok; ++t)
+        for (int h = 0; h < H; ++h) {
+            double acc = 0.0;
+            for (int c = 0; c < d; ++c) acc += x[(t * H + h) * d + c] * W[(long)c * H + h];
+            s[t * H + h] = acc;
+        }
+}
+
+/* Reverse of sla_oracle_gate_scores: dx[b,t,h,c] += ds[b,t,h] W[c,h] (ADDED to what dx holds: x also feeds the
+ * recurrence), dW[c,h] = sum_t ds[t,h] x[t,h,c] (overwritten). */
+void sla_oracle_gate_scores_backward(long n_tok, int H, int d, const double *x, const double *W,
+                                     const double *ds, double *dx, double *dW) {
+    for (long i = 0; i < (long)d * H; ++i) dW[i] = 0.0;
+    for (long t = 0; t < n_tok; ++t)
+        for (int h = 0; h < H; ++h) {
+            double g = ds[t * H + h];
+            for (int c = 0; c < d; ++c) {
+                dx[(t * H + h) * d + c] += g * W[(long)c * H + h];
+                dW[(long)c * H + h] += g * x[(t * H + h) * d + c];
+            }
+        }
+}
+
 /* Per-step decay factors a[0..d_k) for sequence (b,h) at token t. */
 static void decay_factors(int variant, const double *log_decay, long bt, int H, int h, int d_k,
                           double *a) {

@@ -66,6 +66,14 @@ int sla_oracle_decode_step(int variant, int Bdec, int H, int d_k, int d_v, doubl
                            const double *lq_t, const double *lk_t,
                            double *state, double *o_t);
 
+/* Eq. 4, score projections: s[t,h] = sum_c x[t,h,c] W[c,h]; x [n_tok,H,d], W [d,H], s [n_tok,H].
+ * Pinned by: an einsum of the same contraction, H = 1 (a plain matrix-vector product), lambda*W sharpening the gates
+ * to one-hot (Thm 3.2), finite differences of the whole layer with respect to W and through x. */
+void sla_oracle_gate_scores(long n_tok, int H, int d, const double *x, const double *W, double *s);
+/* dx += ds W^T per head (accumulated), dW = sum_t ds x (overwritten). */
+void sla_oracle_gate_scores_backward(long n_tok, int H, int d, const double *x, const double *W,
+                                     const double *ds, double *dx, double *dW);
+
 /* n_tok consecutive recurrent steps per sequence on a caller-held state (multi-token decode).
  * q, k [Bdec,n_tok,H,d_k]; v, o [Bdec,n_tok,H,d_v]; log_decay RETNET [H], GLA [Bdec,n_tok,H,d_k],
  * GDN [Bdec,n_tok,H]; beta, lq, lk [Bdec,n_tok,H]; state [Bdec,H,d_k,d_v] updated in place.

@@ -53,6 +53,10 @@ def _load():
         lib.sla_oracle_decode_step.restype = i
         lib.sla_oracle_decode_steps.argtypes = [i] * 6 + [d] + [dp] * 9
         lib.sla_oracle_decode_steps.restype = i
+        lib.sla_oracle_gate_scores.argtypes = [ctypes.c_long, i, i, dp, dp, dp]
+        lib.sla_oracle_gate_scores.restype = None
+        lib.sla_oracle_gate_scores_backward.argtypes = [ctypes.c_long, i, i, dp, dp, dp, dp, dp]
+        lib.sla_oracle_gate_scores_backward.restype = None
         _lib = lib
     return _lib
 
@@ -165,3 +169,23 @@ def decode_steps(variant, q, k, v, log_decay, lq, lk, state, beta=None, scale=1.
     if rc != 0:
         raise ValueError("sla_oracle_decode_steps rejected its arguments")
     return o
+
+
+def gate_scores(x, W):
+    """Eq. 4's score projection: x [..., H, d], W [d, H] -> s [..., H] with s[.., h] = x[.., h, :] @ W[:, h]."""
+    x, W = _f64(x), _f64(W)
+    H, d = x.shape[-2], x.shape[-1]
+    assert W.shape == (d, H)
+    s = np.zeros(x.shape[:-1])
+    _load().sla_oracle_gate_scores(x.size // (H * d), H, d, _p(x), _p(W), _p(s))
+    return s
+
+
+def gate_scores_backward(x, W, ds, dx):
+    """Adds ds W^T (per head) into the fp64 array dx (in place) and returns dW [d, H]."""
+    x, W, ds = _f64(x), _f64(W), _f64(ds)
+    H, d = x.shape[-2], x.shape[-1]
+    assert isinstance(dx, np.ndarray) and dx.dtype == np.float64 and dx.flags.c_contiguous and dx.shape == x.shape
+    dW = np.zeros((d, H))
+    _load().sla_oracle_gate_scores_backward(x.size // (H * d), H, d, _p(x), _p(W), _p(ds), _p(dx), _p(dW))
+    return dW
