@@ -369,6 +369,37 @@ def main():
     barrier()
     e2e_value, ms_e2e = whole_job_throughput(tokens_step, e2e_steps, e0.elapsed_time(e1), dist, "cuda")
 
+    # ---- the gate score projections of Eq. 4 (logits from q, k and W_GQ, W_GK) and their reverse: what it costs a step
+    # whose logits are not handed in but computed inside the boundary ----
+    scores = None
+    if rank == 0 and cfg.backward and not args.generic:
+        from paper_2602_01744_b200.inputs import make_gate_weights
+        wq, wk = (w.cuda() for w in make_gate_weights(cfg, seed=99))
+        sws = torch.empty(64 << 20, dtype=torch.uint8, device="cuda")
+        lq_, lk_ = torch.empty_like(dev["gq_logits"]), torch.empty_like(dev["gk_logits"])
+        tms = {}
+        for name, fn in (("forward", lambda: api.sla_gate_scores_forward(plan, dev["q"], dev["k"], wq, wk, lq_, lk_)),
+                         ("backward", lambda: api.sla_gate_scores_backward(plan, dev["q"], dev["k"], wq, wk, grads["dgq_logits"],
+                                                                           grads["dgk_logits"], grads["dq"], grads["dk"], workspace=sws))):
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize()
+            e0.record()
+            for _ in range(20):
+                fn()
+            e1.record()
+            torch.cuda.synchronize()
+            tms[name] = e0.elapsed_time(e1) / 20
+        pairs_ = cfg.B * cfg.T * cfg.H
+        es = 2 if cfg.dtype == "bf16" else 4
+        fb, bb = (2 * cfg.d_k * es + 8) * pairs_, (6 * cfg.d_k * es + 8) * pairs_
+        hb, _ = measured_peaks()
+        scores = {"what": "sla_gate_scores_forward / _backward on the workload's q, k (logits = per-head q, k through W [d_k,H])",
+                  "forward_ms": tms["forward"], "backward_ms": tms["backward"],
+                  "forward_hbm_frac": fb / (tms["forward"] * 1e-3) / 1e9 / hb, "backward_hbm_frac": bb / (tms["backward"] * 1e-3) / 1e9 / hb,
+                  "algorithmic_bytes": {"forward": fb, "backward": bb},
+                  "share_of_step": (tms["forward"] + tms["backward"]) / (ms / args.steps)}
+
     # ---- the decode step of the long-context configuration (C3): batch 64, fp32 state of 64 MiB, updated in place ----
     decode = None
     if rank == 0 and args.batch <= 0 and WORKLOAD == "C2":
@@ -539,6 +570,7 @@ def main():
             "tensor": tensor,
             "ms_per_step_with_kernel_events": ms_traced / args.steps,
             "step_hbm": {"algorithmic_bytes_per_step": step_bytes, "achieved_gbs": step_gbs, "frac": step_gbs / peak},
+            "gate_scores": scores,
             "decode_step": decode,
             "cpu_baseline": cpu,
         }

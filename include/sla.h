@@ -182,6 +182,33 @@ sla_status sla_decode_step(sla_plan *plan, int32_t Bdec,
                            float *state, void *o_t, void *cuda_stream);
 
 /*
+ * Gate score projections (Eq. 4: G^Q = softmax(Q W_GQ), G^K = softmax(K W_GK), W in R^{d x H} with d the per-head
+ * width).  The paper leaves open what a d-wide projection is applied to in a multi-head layer; its parameter count
+ * (about 0.05M for 24 layers at hidden 1024 with 4 heads, i.e. d = 256) fixes d as the per-head width, and the reading
+ * taken here is that head h scores itself through column h:
+ *     gq_logits[b,t,h] = sum_c q[b,t,h,c] w_gq[c,h]          gk_logits[b,t,h] = sum_c k[b,t,h,c] w_gk[c,h]
+ * q, k are the tensors handed to sla_forward (d = d_k); w_gq, w_gk fp32 [d_k,H] row-major; the logits feed sla_forward
+ * unchanged.  One streaming pass over q and k; needs no workspace.
+ */
+sla_status sla_gate_scores_forward(sla_plan *plan, const void *q, const void *k,
+                                   const float *w_gq, const float *w_gk,
+                                   float *gq_logits, float *gk_logits, void *cuda_stream);
+/*
+ * Reverse of sla_gate_scores_forward (chain rule of Eq. 4), run AFTER sla_backward on its outputs: dgq_logits,
+ * dgk_logits are sla_backward's logit gradients; dq, dk are sla_backward's dq, dk and are updated in place,
+ *     dq[b,t,h,:] += dgq_logits[b,t,h] w_gq[:,h]             dk[b,t,h,:] += dgk_logits[b,t,h] w_gk[:,h]
+ * (q and k reach the loss on two routes); dw_gq, dw_gk fp32 [d_k,H] are written in full,
+ *     dw_gq[c,h] = sum_{b,t} dgq_logits[b,t,h] q[b,t,h,c]    (same for k),
+ * summed in a fixed order (identical bits on every run).  Workspace: sla_plan_gate_scores_workspace_bytes.
+ */
+sla_status sla_plan_gate_scores_workspace_bytes(const sla_plan *plan, size_t *bytes);
+sla_status sla_gate_scores_backward(sla_plan *plan, const void *q, const void *k,
+                                    const float *w_gq, const float *w_gk,
+                                    const float *dgq_logits, const float *dgk_logits,
+                                    void *dq, void *dk, float *dw_gq, float *dw_gk,
+                                    void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
  * Multi-token decode: n_tokens consecutive recurrent steps (Eq. 5-6 / 10-16) per sequence in one call - what a
  * serving loop needs when several tokens of a sequence are known at once (chunked prefill of a short prompt tail,
  * verification of speculated tokens).  Token t of sequence b reads the state token t-1 left; the state travels

@@ -24,7 +24,8 @@ EXPORTS = (
     "sla_plan_create", "sla_plan_destroy", "sla_plan_workspace_bytes", "sla_plan_poll",
     "sla_plan_last_launch_count", "sla_plan_set_kernel_timing", "sla_plan_kernel_timing_collect",
     "sla_plan_kernel_timing_get", "sla_status_string", "sla_forward", "sla_backward", "sla_decode_step",
-    "sla_forward_noalloc", "sla_plan_selftest_timeout", "sla_decode_steps",
+    "sla_forward_noalloc", "sla_plan_selftest_timeout", "sla_decode_steps", "sla_gate_scores_forward",
+    "sla_gate_scores_backward", "sla_plan_gate_scores_workspace_bytes",
 )
 SLA_NOALLOC_SCRATCH_BYTES = 32 << 20
 
@@ -85,6 +86,12 @@ def lib():
         L.sla_decode_step.argtypes = [vp, i32] + [vp] * 10
         L.sla_decode_steps.argtypes = [vp, i32, i32] + [vp] * 10
         L.sla_decode_steps.restype = ctypes.c_int
+        L.sla_gate_scores_forward.argtypes = [vp] * 8
+        L.sla_gate_scores_forward.restype = ctypes.c_int
+        L.sla_gate_scores_backward.argtypes = [vp] * 11 + [vp, sz, vp]
+        L.sla_gate_scores_backward.restype = ctypes.c_int
+        L.sla_plan_gate_scores_workspace_bytes.argtypes = [vp, ctypes.POINTER(sz)]
+        L.sla_plan_gate_scores_workspace_bytes.restype = ctypes.c_int
         for name in ("sla_plan_create", "sla_plan_destroy", "sla_plan_workspace_bytes", "sla_plan_poll",
                      "sla_plan_set_kernel_timing", "sla_plan_kernel_timing_collect",
                      "sla_plan_kernel_timing_get", "sla_forward", "sla_backward", "sla_decode_step"):
@@ -242,3 +249,28 @@ def sla_decode_steps(plan: Plan, q, k, v, log_decay, gq_logits, gk_logits, state
         plan.handle, Bdec, n, _ptr(q), _ptr(k), _ptr(v), _ptr(log_decay), _ptr(beta), _ptr(gq_logits),
         _ptr(gk_logits), _ptr(state), _ptr(o), _stream()))
     return o
+
+
+def sla_gate_scores_forward(plan: Plan, q, k, w_gq, w_gk, gq_logits=None, gk_logits=None):
+    """Eq. 4's score projections: returns (gq_logits, gk_logits), fp32 [B,T,H], from q, k and w_gq, w_gk [d_k,H]."""
+    d = plan.desc
+    if gq_logits is None:
+        gq_logits = torch.empty((d.B, d.T, d.H), dtype=torch.float32, device=q.device)
+    if gk_logits is None:
+        gk_logits = torch.empty((d.B, d.T, d.H), dtype=torch.float32, device=q.device)
+    _check("sla_gate_scores_forward", lib().sla_gate_scores_forward(
+        plan.handle, _ptr(q), _ptr(k), _ptr(w_gq), _ptr(w_gk), _ptr(gq_logits), _ptr(gk_logits), _stream()))
+    return gq_logits, gk_logits
+
+
+def sla_gate_scores_backward(plan: Plan, q, k, w_gq, w_gk, dgq_logits, dgk_logits, dq, dk, workspace=None):
+    """Reverse of the score projections: adds the logit route into dq, dk (in place) and returns (dw_gq, dw_gk)."""
+    n = ctypes.c_size_t()
+    _check("sla_plan_gate_scores_workspace_bytes", lib().sla_plan_gate_scores_workspace_bytes(plan.handle, ctypes.byref(n)))
+    if workspace is None:
+        workspace = torch.empty(max(n.value, 16), dtype=torch.uint8, device=q.device)
+    dw_gq, dw_gk = torch.empty_like(w_gq), torch.empty_like(w_gk)
+    _check("sla_gate_scores_backward", lib().sla_gate_scores_backward(
+        plan.handle, _ptr(q), _ptr(k), _ptr(w_gq), _ptr(w_gk), _ptr(dgq_logits), _ptr(dgk_logits), _ptr(dq), _ptr(dk),
+        _ptr(dw_gq), _ptr(dw_gk), _ptr(workspace), workspace.numel(), _stream()))
+    return dw_gq, dw_gk

@@ -306,6 +306,57 @@ sla_status sla_backward(sla_plan *plan, const void *q, const void *k, const void
     return SLA_OK;
 }
 
+sla_status sla_plan_gate_scores_workspace_bytes(const sla_plan *plan, size_t *bytes) {
+    if (!plan || !bytes) return SLA_ERR_INVALID_ARG;
+    *bytes = sla::gate_scores_workspace_bytes(plan->dims);
+    return SLA_OK;
+}
+
+sla_status sla_gate_scores_forward(sla_plan *plan, const void *q, const void *k, const float *w_gq, const float *w_gk,
+                                   float *gq_logits, float *gk_logits, void *cuda_stream) {
+    if (!plan) return SLA_ERR_INVALID_ARG;
+    const sla::Dims &d = plan->dims;
+    plan->last_launches = 0;
+    if (d.B == 0 || d.T == 0) return SLA_OK;
+    if (!q || !k || !w_gq || !w_gk || !gq_logits || !gk_logits) return SLA_ERR_INVALID_ARG;
+    const void *ptrs[] = {q, k, w_gq, w_gk, gq_logits, gk_logits};
+    for (const void *p : ptrs)
+        if (!aligned16(p)) return SLA_ERR_INVALID_ARG;
+    plan->tracer.start((cudaStream_t)cuda_stream);
+    int n = sla::gate_scores_forward(d, q, k, w_gq, w_gk, gq_logits, gk_logits, (cudaStream_t)cuda_stream, plan->tracer);
+    if (n < 0) return SLA_ERR_CUDA;
+    plan->last_launches = n;
+    return SLA_OK;
+}
+
+sla_status sla_gate_scores_backward(sla_plan *plan, const void *q, const void *k, const float *w_gq, const float *w_gk,
+                                    const float *dgq_logits, const float *dgk_logits, void *dq, void *dk,
+                                    float *dw_gq, float *dw_gk, void *workspace, size_t workspace_bytes,
+                                    void *cuda_stream) {
+    if (!plan) return SLA_ERR_INVALID_ARG;
+    const sla::Dims &d = plan->dims;
+    plan->last_launches = 0;
+    if (!dw_gq || !dw_gk || !aligned16(dw_gq) || !aligned16(dw_gk)) return SLA_ERR_INVALID_ARG;
+    if (d.B == 0 || d.T == 0) {          // no tokens: the weight gradients are zero
+        const size_t wb = (size_t)d.dk * d.H * sizeof(float);
+        if (cudaMemsetAsync(dw_gq, 0, wb, (cudaStream_t)cuda_stream) != cudaSuccess ||
+            cudaMemsetAsync(dw_gk, 0, wb, (cudaStream_t)cuda_stream) != cudaSuccess)
+            return SLA_ERR_CUDA;
+        return SLA_OK;
+    }
+    if (!q || !k || !w_gq || !w_gk || !dgq_logits || !dgk_logits || !dq || !dk) return SLA_ERR_INVALID_ARG;
+    const void *ptrs[] = {q, k, w_gq, w_gk, dgq_logits, dgk_logits, dq, dk, workspace};
+    for (const void *p : ptrs)
+        if (!aligned16(p)) return SLA_ERR_INVALID_ARG;
+    if (!workspace || workspace_bytes < sla::gate_scores_workspace_bytes(d)) return SLA_ERR_WORKSPACE;
+    plan->tracer.start((cudaStream_t)cuda_stream);
+    int n = sla::gate_scores_backward(d, q, k, w_gq, w_gk, dgq_logits, dgk_logits, dq, dk, dw_gq, dw_gk,
+                                      (float *)workspace, (cudaStream_t)cuda_stream, plan->tracer);
+    if (n < 0) return SLA_ERR_CUDA;
+    plan->last_launches = n;
+    return SLA_OK;
+}
+
 sla_status sla_decode_steps(sla_plan *plan, int32_t Bdec, int32_t n_tokens, const void *q, const void *k,
                             const void *v, const float *log_decay, const float *beta,
                             const float *gq_logits, const float *gk_logits, float *state, void *o,

@@ -134,6 +134,14 @@ int gdn_tc_backward(const Dims &d, const BwdArgs &a, bool have_records, int *sta
 int gate_bwd_prod(const float *lq, const float *lk, const float *pq, const float *pk, float *dlq, float *dlk, long n_tok,
                   int H, cudaStream_t st);
 
+// ---- gate score projections of Eq. 4 and their reverse: sla_gate_scores.cu ----
+size_t gate_scores_workspace_bytes(const Dims &d);
+int gate_scores_forward(const Dims &d, const void *q, const void *k, const float *Wq, const float *Wk, float *lq,
+                        float *lk, cudaStream_t st, Tracer &tr);
+int gate_scores_backward(const Dims &d, const void *q, const void *k, const float *Wq, const float *Wk, const float *dlq,
+                         const float *dlk, void *dq, void *dk, float *dWq, float *dWk, float *ws, cudaStream_t st,
+                         Tracer &tr);
+
 // GDN per-tile gradient kernels (after the recompute pass and the state-gradient scan).
 int gdn_backward_tiles(const Dims &d, const Workspace &w, const BwdArgs &a, cudaStream_t st, Tracer &tr);
 

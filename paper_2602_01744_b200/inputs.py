@@ -118,3 +118,11 @@ def make_decode_inputs(cfg: SLAConfig, batch: int, steps: int, seed: int) -> dic
         k = k / k.norm(dim=-1, keepdim=True)
     return dict(q=q.to(io), k=k.to(io), v=v.to(io), log_decay=log_decay, beta=beta,
                 gq_logits=randn(steps, batch, H), gk_logits=randn(steps, batch, H))
+
+
+def make_gate_weights(cfg: SLAConfig, seed: int):
+    """Gate score projection matrices W_GQ, W_GK (fp32 [d_k, H]) drawn N(0,1): with q, k ~ N(0,1)/sqrt(d_k) the scores
+    q W come out ~ N(0,1) per (token, head), the distribution the configurations state for the gate logits."""
+    gen = torch.Generator(device="cpu").manual_seed(seed)
+    return (torch.randn(cfg.d_k, cfg.H, generator=gen, dtype=torch.float32),
+            torch.randn(cfg.d_k, cfg.H, generator=gen, dtype=torch.float32))
