@@ -76,6 +76,91 @@ void sla_oracle_gate_scores_backward(long n_tok, int H, int d, const double *x, 
         }
 }
 
+/*
+ * Feature map of the Gated-DeltaNet instantiation ("short-convolution module" followed by SiLU, Experimental setup),
+ * as published for Gated DeltaNet: a depthwise causal convolution of K taps over time, channel by channel, then
+ * SiLU, then (for q and k) L2 normalisation over the d features of each head.
+ *     y[b,t,c] = sum_{j<K} w[c,j] x[b,t-(K-1)+j,c]      (tokens before the sequence start read as zero)
+ *     z = y * sigmoid(y)
+ *     out[b,t,h,:] = z[b,t,h,:] / sqrt(sum_d z[b,t,h,d]^2 + eps)      when normalize != 0, else out = z
+ * x, out: [B,T,C] with C = H*d channels; w: [C,K].
+ */
+static double silu(double y) { return y / (1.0 + exp(-y)); }
+static double silu_grad(double y) { double s = 1.0 / (1.0 + exp(-y)); return s * (1.0 + y * (1.0 - s)); }
+
+void sla_oracle_shortconv(int B, int T, int H, int d, int K, int normalize, double eps,
+                          const double *x, const double *w, double *out) {
+    long C = (long)H * d;
+    for (int b = 0; b < B; ++b)
+        for (int t = 0; t < T; ++t) {
+            double *o = out + ((long)b * T + t) * C;
+            for (long c = 0; c < C; ++c) {
+                double y = 0.0;
+                for (int j = 0; j < K; ++j) {
+                    int tt = t - (K - 1) + j;
+                    if (tt >= 0) y += w[c * K + j] * x[((long)b * T + tt) * C + c];
+                }
+                o[c] = silu(y);
+            }
+            if (normalize)
+                for (int h = 0; h < H; ++h) {
+                    double ss = 0.0;
+                    for (int c = 0; c < d; ++c) ss += o[(long)h * d + c] * o[(long)h * d + c];
+                    double r = sqrt(ss + eps);
+                    for (int c = 0; c < d; ++c) o[(long)h * d + c] /= r;
+                }
+        }
+}
+
+/* Reverse of sla_oracle_shortconv: dx [B,T,C] and dw [C,K], both overwritten. */
+void sla_oracle_shortconv_backward(int B, int T, int H, int d, int K, int normalize, double eps,
+                                   const double *x, const double *w, const double *dout,
+                                   double *dx, double *dw) {
+    long C = (long)H * d;
+    double *y = (double *)malloc(sizeof(double) * C);
+    double *z = (double *)malloc(sizeof(double) * C);
+    double *dz = (double *)malloc(sizeof(double) * C);
+    for (long i = 0; i < (long)B * T * C; ++i) dx[i] = 0.0;
+    for (long i = 0; i < C * K; ++i) dw[i] = 0.0;
+    for (int b = 0; b < B; ++b)
+        for (int t = 0; t < T; ++t) {
+            const double *go = dout + ((long)b * T + t) * C;
+            for (long c = 0; c < C; ++c) {
+                double acc = 0.0;
+                for (int j = 0; j < K; ++j) {
+                    int tt = t - (K - 1) + j;
+                    if (tt >= 0) acc += w[c * K + j] * x[((long)b * T + tt) * C + c];
+                }
+                y[c] = acc;
+                z[c] = silu(acc);
+                dz[c] = go[c];
+            }
+            if (normalize)
+                for (int h = 0; h < H; ++h) {
+                    double ss = 0.0, dot = 0.0;
+                    for (int c = 0; c < d; ++c) {
+                        ss += z[(long)h * d + c] * z[(long)h * d + c];
+                        dot += z[(long)h * d + c] * go[(long)h * d + c];
+                    }
+                    double r = sqrt(ss + eps);
+                    /* out = z / r, r = sqrt(|z|^2 + eps):  dz = dout / r - z (z . dout) / r^3 */
+                    for (int c = 0; c < d; ++c)
+                        dz[(long)h * d + c] = go[(long)h * d + c] / r - z[(long)h * d + c] * dot / (r * r * r);
+                }
+            for (long c = 0; c < C; ++c) {
+                double dy = dz[c] * silu_grad(y[c]);
+                for (int j = 0; j < K; ++j) {
+                    int tt = t - (K - 1) + j;
+                    if (tt >= 0) {
+                        dx[((long)b * T + tt) * C + c] += w[c * K + j] * dy;
+                        dw[c * K + j] += dy * x[((long)b * T + tt) * C + c];
+                    }
+                }
+            }
+        }
+    free(y); free(z); free(dz);
+}
+
 /* Per-step decay factors a[0..d_k) for sequence (b,h) at token t. */
 static void decay_factors(int variant, const double *log_decay, long bt, int H, int h, int d_k,
                           double *a) {

@@ -74,6 +74,16 @@ void sla_oracle_gate_scores(long n_tok, int H, int d, const double *x, const dou
 void sla_oracle_gate_scores_backward(long n_tok, int H, int d, const double *x, const double *W,
                                      const double *ds, double *dx, double *dW);
 
+/* Feature map of the Gated-DeltaNet instantiation: depthwise causal convolution over time (K taps, w [C,K], C = H*d
+ * channels), SiLU, and with normalize != 0 L2 normalisation over the d features of each head (eps inside the root).
+ * x, out [B,T,C].  Pinned by: a library convolution per channel, K = 1 with unit weight = SiLU itself, unit row norms,
+ * causality, finite differences of the reverse sweep. */
+void sla_oracle_shortconv(int B, int T, int H, int d, int K, int normalize, double eps,
+                          const double *x, const double *w, double *out);
+void sla_oracle_shortconv_backward(int B, int T, int H, int d, int K, int normalize, double eps,
+                                   const double *x, const double *w, const double *dout,
+                                   double *dx, double *dw);
+
 /* n_tok consecutive recurrent steps per sequence on a caller-held state (multi-token decode).
  * q, k [Bdec,n_tok,H,d_k]; v, o [Bdec,n_tok,H,d_v]; log_decay RETNET [H], GLA [Bdec,n_tok,H,d_k],
  * GDN [Bdec,n_tok,H]; beta, lq, lk [Bdec,n_tok,H]; state [Bdec,H,d_k,d_v] updated in place.

@@ -53,6 +53,10 @@ def _load():
         lib.sla_oracle_decode_step.restype = i
         lib.sla_oracle_decode_steps.argtypes = [i] * 6 + [d] + [dp] * 9
         lib.sla_oracle_decode_steps.restype = i
+        lib.sla_oracle_shortconv.argtypes = [i] * 6 + [d] + [dp] * 3
+        lib.sla_oracle_shortconv.restype = None
+        lib.sla_oracle_shortconv_backward.argtypes = [i] * 6 + [d] + [dp] * 5
+        lib.sla_oracle_shortconv_backward.restype = None
         lib.sla_oracle_gate_scores.argtypes = [ctypes.c_long, i, i, dp, dp, dp]
         lib.sla_oracle_gate_scores.restype = None
         lib.sla_oracle_gate_scores_backward.argtypes = [ctypes.c_long, i, i, dp, dp, dp, dp, dp]
@@ -189,3 +193,26 @@ def gate_scores_backward(x, W, ds, dx):
     dW = np.zeros((d, H))
     _load().sla_oracle_gate_scores_backward(x.size // (H * d), H, d, _p(x), _p(W), _p(ds), _p(dx), _p(dW))
     return dW
+
+
+SHORTCONV_EPS = 1e-6
+
+
+def shortconv(x, w, normalize, eps=SHORTCONV_EPS):
+    """Depthwise causal convolution + SiLU (+ per-head L2 normalisation): x [B,T,H,d], w [H*d,K] -> [B,T,H,d]."""
+    x, w = _f64(x), _f64(w)
+    B, T, H, d = x.shape
+    assert w.shape[0] == H * d
+    out = np.zeros_like(x)
+    _load().sla_oracle_shortconv(B, T, H, d, w.shape[1], int(bool(normalize)), float(eps), _p(x), _p(w), _p(out))
+    return out
+
+
+def shortconv_backward(x, w, dout, normalize, eps=SHORTCONV_EPS):
+    """Returns (dx [B,T,H,d], dw [H*d,K])."""
+    x, w, dout = _f64(x), _f64(w), _f64(dout)
+    B, T, H, d = x.shape
+    dx, dw = np.zeros_like(x), np.zeros_like(w)
+    _load().sla_oracle_shortconv_backward(B, T, H, d, w.shape[1], int(bool(normalize)), float(eps), _p(x), _p(w),
+                                          _p(dout), _p(dx), _p(dw))
+    return dx, dw
