@@ -400,6 +400,34 @@ def main():
                   "algorithmic_bytes": {"forward": fb, "backward": bb},
                   "share_of_step": (tms["forward"] + tms["backward"]) / (ms / args.steps)}
 
+    # ---- the feature map of the Gated-DeltaNet instantiation (short convolution, SiLU, L2 norm) and its reverse ----
+    frontend = None
+    if rank == 0 and cfg.variant == "gdn" and not args.generic:
+        from paper_2602_01744_b200.inputs import make_frontend_inputs
+        fe = {n: t.cuda() for n, t in make_frontend_inputs(cfg, 4, seed=98).items()}
+        fws = torch.empty(64 << 20, dtype=torch.uint8, device="cuda")
+        fout = torch.empty_like(fe["x_q"])
+        tms = {}
+        for name, fn in (("forward", lambda: api.sla_shortconv_forward(plan, fe["x_q"], fe["w_q"], True, out=fout)),
+                         ("backward", lambda: api.sla_shortconv_backward(plan, fe["x_q"], fe["w_q"], fe["dout"], True, workspace=fws))):
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize()
+            e0.record()
+            for _ in range(20):
+                fn()
+            e1.record()
+            torch.cuda.synchronize()
+            tms[name] = e0.elapsed_time(e1) / 20
+        nb = fe["x_q"].numel() * fe["x_q"].element_size()
+        hb, _ = measured_peaks()
+        frontend = {"what": "sla_shortconv_forward / _backward on one [B,T,H,d_k] tensor (K = 4, with L2 normalisation); a layer "
+                            "applies it to q, k and v",
+                    "forward_ms": tms["forward"], "backward_ms": tms["backward"],
+                    "forward_hbm_frac": 2 * nb / (tms["forward"] * 1e-3) / 1e9 / hb,
+                    "backward_hbm_frac": 3 * nb / (tms["backward"] * 1e-3) / 1e9 / hb,
+                    "algorithmic_bytes": {"forward": 2 * nb, "backward": 3 * nb}}
+
     # ---- the decode step of the long-context configuration (C3): batch 64, fp32 state of 64 MiB, updated in place ----
     decode = None
     if rank == 0 and args.batch <= 0 and WORKLOAD == "C2":
@@ -571,6 +599,7 @@ def main():
             "ms_per_step_with_kernel_events": ms_traced / args.steps,
             "step_hbm": {"algorithmic_bytes_per_step": step_bytes, "achieved_gbs": step_gbs, "frac": step_gbs / peak},
             "gate_scores": scores,
+            "gdn_feature_map": frontend,
             "decode_step": decode,
             "cpu_baseline": cpu,
         }

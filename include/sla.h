@@ -209,6 +209,31 @@ sla_status sla_gate_scores_backward(sla_plan *plan, const void *q, const void *k
                                     void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * Feature map of the Gated-DeltaNet instantiation (Experimental setup: GDN uses "the short-convolution module" and SiLU
+ * as activation; RetNet and GLA use the identity and need none of this).  The paper names the module and cites Gated
+ * DeltaNet for it; what is computed here is that published design: per channel a causal convolution over time,
+ * SiLU, and - for q and k - L2 normalisation over the d features of each head:
+ *     y[b,t,c] = sum_{j<K} w[c,j] x[b,t-(K-1)+j,c]   (tokens before the sequence start read as zero; no bias)
+ *     z = y * sigmoid(y)
+ *     out[b,t,h,:] = z[b,t,h,:] / sqrt(sum_d z[b,t,h,d]^2 + SLA_SHORTCONV_EPS)   if normalize != 0, else out = z
+ * x, out [B,T,H,d] in the plan's io dtype (d = the per-head width of THIS tensor, a multiple of 16 up to 128: d_k for
+ * q and k, d_v for v); w fp32 [H*d, K], 1 <= K <= 4.  One call per tensor: q and k with normalize = 1, v with 0; the
+ * outputs are what sla_forward takes.  out may not alias x.  Uses the plan's B, T, H and io dtype.
+ */
+#define SLA_SHORTCONV_EPS 1e-6f
+sla_status sla_shortconv_forward(sla_plan *plan, const void *x, const float *w, int32_t d, int32_t K,
+                                 int32_t normalize, void *out, void *cuda_stream);
+/*
+ * Reverse of sla_shortconv_forward: from dout (gradient with respect to out, e.g. sla_backward's dq) to
+ * dx [B,T,H,d] (io dtype) and dw fp32 [H*d, K], both written in full; y is recomputed from x, nothing is kept from
+ * the forward call.  dw is summed in a fixed order.  Workspace: sla_plan_shortconv_workspace_bytes(plan, d).
+ */
+sla_status sla_plan_shortconv_workspace_bytes(const sla_plan *plan, int32_t d, size_t *bytes);
+sla_status sla_shortconv_backward(sla_plan *plan, const void *x, const float *w, int32_t d, int32_t K,
+                                  int32_t normalize, const void *dout, void *dx, float *dw,
+                                  void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
  * Multi-token decode: n_tokens consecutive recurrent steps (Eq. 5-6 / 10-16) per sequence in one call - what a
  * serving loop needs when several tokens of a sequence are known at once (chunked prefill of a short prompt tail,
  * verification of speculated tokens).  Token t of sequence b reads the state token t-1 left; the state travels

@@ -25,7 +25,8 @@ EXPORTS = (
     "sla_plan_last_launch_count", "sla_plan_set_kernel_timing", "sla_plan_kernel_timing_collect",
     "sla_plan_kernel_timing_get", "sla_status_string", "sla_forward", "sla_backward", "sla_decode_step",
     "sla_forward_noalloc", "sla_plan_selftest_timeout", "sla_decode_steps", "sla_gate_scores_forward",
-    "sla_gate_scores_backward", "sla_plan_gate_scores_workspace_bytes",
+    "sla_gate_scores_backward", "sla_plan_gate_scores_workspace_bytes", "sla_shortconv_forward",
+    "sla_shortconv_backward", "sla_plan_shortconv_workspace_bytes",
 )
 SLA_NOALLOC_SCRATCH_BYTES = 32 << 20
 
@@ -86,6 +87,12 @@ def lib():
         L.sla_decode_step.argtypes = [vp, i32] + [vp] * 10
         L.sla_decode_steps.argtypes = [vp, i32, i32] + [vp] * 10
         L.sla_decode_steps.restype = ctypes.c_int
+        L.sla_shortconv_forward.argtypes = [vp, vp, vp, i32, i32, i32, vp, vp]
+        L.sla_shortconv_forward.restype = ctypes.c_int
+        L.sla_shortconv_backward.argtypes = [vp, vp, vp, i32, i32, i32, vp, vp, vp, vp, sz, vp]
+        L.sla_shortconv_backward.restype = ctypes.c_int
+        L.sla_plan_shortconv_workspace_bytes.argtypes = [vp, i32, ctypes.POINTER(sz)]
+        L.sla_plan_shortconv_workspace_bytes.restype = ctypes.c_int
         L.sla_gate_scores_forward.argtypes = [vp] * 8
         L.sla_gate_scores_forward.restype = ctypes.c_int
         L.sla_gate_scores_backward.argtypes = [vp] * 11 + [vp, sz, vp]
@@ -274,3 +281,26 @@ def sla_gate_scores_backward(plan: Plan, q, k, w_gq, w_gk, dgq_logits, dgk_logit
         plan.handle, _ptr(q), _ptr(k), _ptr(w_gq), _ptr(w_gk), _ptr(dgq_logits), _ptr(dgk_logits), _ptr(dq), _ptr(dk),
         _ptr(dw_gq), _ptr(dw_gk), _ptr(workspace), workspace.numel(), _stream()))
     return dw_gq, dw_gk
+
+
+def sla_shortconv_forward(plan: Plan, x, w, normalize, out=None):
+    """Gated-DeltaNet feature map: causal depthwise convolution (w [H*d,K]) + SiLU (+ per-head L2 norm): x -> out [B,T,H,d]."""
+    if out is None:
+        out = torch.empty_like(x)
+    _check("sla_shortconv_forward", lib().sla_shortconv_forward(
+        plan.handle, _ptr(x), _ptr(w), x.shape[-1], w.shape[1], int(bool(normalize)), _ptr(out), _stream()))
+    return out
+
+
+def sla_shortconv_backward(plan: Plan, x, w, dout, normalize, workspace=None):
+    """Returns (dx, dw) of sla_shortconv_forward."""
+    n = ctypes.c_size_t()
+    _check("sla_plan_shortconv_workspace_bytes",
+           lib().sla_plan_shortconv_workspace_bytes(plan.handle, x.shape[-1], ctypes.byref(n)))
+    if workspace is None:
+        workspace = torch.empty(max(n.value, 16), dtype=torch.uint8, device=x.device)
+    dx, dw = torch.empty_like(x), torch.empty_like(w)
+    _check("sla_shortconv_backward", lib().sla_shortconv_backward(
+        plan.handle, _ptr(x), _ptr(w), x.shape[-1], w.shape[1], int(bool(normalize)), _ptr(dout), _ptr(dx), _ptr(dw),
+        _ptr(workspace), workspace.numel(), _stream()))
+    return dx, dw

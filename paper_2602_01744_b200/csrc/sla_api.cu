@@ -306,6 +306,55 @@ sla_status sla_backward(sla_plan *plan, const void *q, const void *k, const void
     return SLA_OK;
 }
 
+static bool conv_args_ok(int32_t d, int32_t K) { return d >= 16 && d <= 128 && d % 16 == 0 && K >= 1 && K <= 4; }
+
+sla_status sla_plan_shortconv_workspace_bytes(const sla_plan *plan, int32_t d, size_t *bytes) {
+    if (!plan || !bytes) return SLA_ERR_INVALID_ARG;
+    if (!conv_args_ok(d, 1)) return SLA_ERR_UNSUPPORTED;
+    *bytes = sla::shortconv_workspace_bytes(plan->dims, d);
+    return SLA_OK;
+}
+
+sla_status sla_shortconv_forward(sla_plan *plan, const void *x, const float *w, int32_t d, int32_t K, int32_t normalize,
+                                 void *out, void *cuda_stream) {
+    if (!plan) return SLA_ERR_INVALID_ARG;
+    if (!conv_args_ok(d, K)) return SLA_ERR_UNSUPPORTED;
+    const sla::Dims &dm = plan->dims;
+    plan->last_launches = 0;
+    if (dm.B == 0 || dm.T == 0) return SLA_OK;
+    if (!x || !w || !out || !aligned16(x) || !aligned16(w) || !aligned16(out)) return SLA_ERR_INVALID_ARG;
+    plan->tracer.start((cudaStream_t)cuda_stream);
+    int n = sla::shortconv_forward(dm, d, K, normalize != 0, SLA_SHORTCONV_EPS, x, w, out, (cudaStream_t)cuda_stream,
+                                   plan->tracer);
+    if (n < 0) return SLA_ERR_CUDA;
+    plan->last_launches = n;
+    return SLA_OK;
+}
+
+sla_status sla_shortconv_backward(sla_plan *plan, const void *x, const float *w, int32_t d, int32_t K, int32_t normalize,
+                                  const void *dout, void *dx, float *dw, void *workspace, size_t workspace_bytes,
+                                  void *cuda_stream) {
+    if (!plan) return SLA_ERR_INVALID_ARG;
+    if (!conv_args_ok(d, K)) return SLA_ERR_UNSUPPORTED;
+    const sla::Dims &dm = plan->dims;
+    plan->last_launches = 0;
+    if (!dw || !aligned16(dw)) return SLA_ERR_INVALID_ARG;
+    if (dm.B == 0 || dm.T == 0)
+        return cudaMemsetAsync(dw, 0, (size_t)dm.H * d * K * sizeof(float), (cudaStream_t)cuda_stream) == cudaSuccess
+                   ? SLA_OK : SLA_ERR_CUDA;
+    if (!x || !w || !dout || !dx) return SLA_ERR_INVALID_ARG;
+    const void *ptrs[] = {x, w, dout, dx, workspace};
+    for (const void *p : ptrs)
+        if (!aligned16(p)) return SLA_ERR_INVALID_ARG;
+    if (!workspace || workspace_bytes < sla::shortconv_workspace_bytes(dm, d)) return SLA_ERR_WORKSPACE;
+    plan->tracer.start((cudaStream_t)cuda_stream);
+    int n = sla::shortconv_backward(dm, d, K, normalize != 0, SLA_SHORTCONV_EPS, x, w, dout, dx, dw, (float *)workspace,
+                                    (cudaStream_t)cuda_stream, plan->tracer);
+    if (n < 0) return SLA_ERR_CUDA;
+    plan->last_launches = n;
+    return SLA_OK;
+}
+
 sla_status sla_plan_gate_scores_workspace_bytes(const sla_plan *plan, size_t *bytes) {
     if (!plan || !bytes) return SLA_ERR_INVALID_ARG;
     *bytes = sla::gate_scores_workspace_bytes(plan->dims);

@@ -142,6 +142,13 @@ int gate_scores_backward(const Dims &d, const void *q, const void *k, const floa
                          const float *dlk, void *dq, void *dk, float *dWq, float *dWk, float *ws, cudaStream_t st,
                          Tracer &tr);
 
+// ---- feature map of the Gated-DeltaNet instantiation (short causal convolution, SiLU, per-head L2 norm): sla_shortconv.cu ----
+size_t shortconv_workspace_bytes(const Dims &d, int width);
+int shortconv_forward(const Dims &d, int width, int K, bool normalize, float eps, const void *x, const float *w, void *out,
+                      cudaStream_t st, Tracer &tr);
+int shortconv_backward(const Dims &d, int width, int K, bool normalize, float eps, const void *x, const float *w,
+                       const void *dout, void *dx, float *dw, float *ws, cudaStream_t st, Tracer &tr);
+
 // GDN per-tile gradient kernels (after the recompute pass and the state-gradient scan).
 int gdn_backward_tiles(const Dims &d, const Workspace &w, const BwdArgs &a, cudaStream_t st, Tracer &tr);
 

@@ -1,0 +1,302 @@
+// Feature map of the Gated-DeltaNet instantiation (Experimental setup: "short-convolution module" and SiLU), inside the
+// boundary so that its gradient is too: per channel a causal convolution of K <= 4 taps over time, SiLU, and for q and k
+// L2 normalisation over the d features of each head,
+//     y[b,t,c] = sum_j w[c,j] x[b,t-(K-1)+j,c]      z = y sigmoid(y)      out = z / sqrt(sum_d z^2 + eps)  (or out = z).
+// Streaming kernels (HBM-bound): a thread owns one 16-byte vector of the token row [H*d] for the whole launch, its taps
+// in registers, and walks the tokens of its CTA's slice of one sequence with a sliding window over time.  The per-head
+// sums of the normalisation go through shared memory, a few tokens per barrier.  The reverse pass walks the slice
+// backwards (dx of a token needs dy of the next K-1 tokens: a sliding window again, warmed up on the tokens after the
+// slice) and recomputes y instead of storing it; weight gradients are summed per thread, written per CTA and reduced
+// over the CTAs in a fixed order.
+#include "sla_internal.h"
+
+#include <algorithm>
+
+namespace sla {
+namespace {
+
+constexpr int KMAX = 4;
+constexpr int TOKS = 4;          // tokens between two barriers, forward
+constexpr int TOKB = 2;          // ... and backward (more live values per token)
+
+template <typename TIO> struct V;
+template <> struct V<float> {
+    static constexpr int N = 4;
+    static __device__ __forceinline__ void load(const float *p, float (&x)[4]) {
+        const float4 v = *reinterpret_cast<const float4 *>(p);
+        x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w;
+    }
+    static __device__ __forceinline__ void store(float *p, const float (&x)[4]) {
+        *reinterpret_cast<float4 *>(p) = make_float4(x[0], x[1], x[2], x[3]);
+    }
+};
+template <> struct V<__nv_bfloat16> {
+    static constexpr int N = 8;
+    static __device__ __forceinline__ void load(const __nv_bfloat16 *p, float (&x)[8]) {
+        const uint4 v = *reinterpret_cast<const uint4 *>(p);
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&w[e]));
+            x[2 * e] = f.x; x[2 * e + 1] = f.y;
+        }
+    }
+    static __device__ __forceinline__ void store(__nv_bfloat16 *p, const float (&x)[8]) {
+        uint32_t w[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            __nv_bfloat162 v = __floats2bfloat162_rn(x[2 * e], x[2 * e + 1]);
+            w[e] = *reinterpret_cast<uint32_t *>(&v);
+        }
+        *reinterpret_cast<uint4 *>(p) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+};
+
+struct ConvDims { int T, H, d, K, per, hpc; float eps; };   // per: tokens of one sequence per CTA; hpc: heads per CTA (grid.z covers H)
+
+// taps of this thread's channels, padded at the front to KMAX: y_t = sum_j wt[j] x[t-3+j]
+template <int N>
+__device__ __forceinline__ void load_taps(const float *w, int c0, int K, bool live, float (&wt)[KMAX][N]) {
+#pragma unroll
+    for (int j = 0; j < KMAX; ++j)
+#pragma unroll
+        for (int e = 0; e < N; ++e) wt[j][e] = (live && j >= KMAX - K) ? __ldg(w + (size_t)(c0 + e) * K + j - (KMAX - K)) : 0.f;
+}
+// x[b, t, this thread's vector], zero before the sequence start
+template <typename TIO, int N>
+__device__ __forceinline__ void load_x(const TIO *row0, int t, size_t stride, bool live, float (&x)[N]) {
+    if (live && t >= 0) {
+        V<TIO>::load(row0 + (size_t)t * stride, x);
+    } else {
+#pragma unroll
+        for (int e = 0; e < N; ++e) x[e] = 0.f;
+    }
+}
+
+template <typename TIO, bool NORM>
+__global__ void __launch_bounds__(256)
+k_shortconv_fwd(ConvDims cd, const TIO *__restrict__ x, const float *__restrict__ w, TIO *__restrict__ out) {
+    constexpr int N = V<TIO>::N;
+    extern __shared__ float sm[];                       // part [TOKS][threads], rinv [TOKS][H]
+    float *part = sm, *rinv = sm + TOKS * blockDim.x;
+    const int C = cd.H * cd.d, vpr = cd.d / N, tid = threadIdx.x;
+    const int hb = blockIdx.z * cd.hpc, nh = min(cd.hpc, cd.H - hb);       // this CTA's heads: hb .. hb + nh - 1
+    const bool live = tid < nh * vpr;
+    const int h = live ? tid / vpr : 0;                                     // (local head)
+    const int gv = hb * vpr + tid;                                          // vector index inside the token row
+    float wt[KMAX][N];
+    load_taps<N>(w, gv * N, cd.K, live, wt);
+    const int b = blockIdx.y, t0 = blockIdx.x * cd.per, t1 = min(cd.T, t0 + cd.per);
+    const TIO *xr = x + ((size_t)b * cd.T) * C + (size_t)gv * N;
+    TIO *orow = out + ((size_t)b * cd.T) * C + (size_t)gv * N;
+    float xm3[N], xm2[N], xm1[N];
+    load_x<TIO, N>(xr, t0 - 3, C, live, xm3);
+    load_x<TIO, N>(xr, t0 - 2, C, live, xm2);
+    load_x<TIO, N>(xr, t0 - 1, C, live, xm1);
+    for (int t = t0; t < t1; t += TOKS) {
+        float z[TOKS][N];
+#pragma unroll
+        for (int s = 0; s < TOKS; ++s) {
+            float ss = 0.f;
+            if (t + s < t1) {
+                float xc[N];
+                load_x<TIO, N>(xr, t + s, C, live, xc);
+#pragma unroll
+                for (int e = 0; e < N; ++e) {
+                    const float y = fmaf(wt[0][e], xm3[e], fmaf(wt[1][e], xm2[e], fmaf(wt[2][e], xm1[e], wt[3][e] * xc[e])));
+                    z[s][e] = y / (1.f + __expf(-y));
+                    ss = fmaf(z[s][e], z[s][e], ss);
+                    xm3[e] = xm2[e]; xm2[e] = xm1[e]; xm1[e] = xc[e];
+                }
+                if (!NORM && live) V<TIO>::store(orow + (size_t)(t + s) * C, z[s]);
+            }
+            if (NORM) part[s * blockDim.x + tid] = ss;
+        }
+        if (NORM) {
+            __syncthreads();
+            if (tid < TOKS * nh) {                      // one thread per (token slot, head)
+                const int s = tid / nh, hh = tid % nh;
+                float acc = 0.f;
+                for (int j = 0; j < vpr; ++j) acc += part[s * blockDim.x + hh * vpr + j];
+                rinv[s * cd.hpc + hh] = 1.f / sqrtf(acc + cd.eps);
+            }
+            __syncthreads();
+#pragma unroll
+            for (int s = 0; s < TOKS; ++s)
+                if (live && t + s < t1) {
+                    const float r = rinv[s * cd.hpc + h];
+#pragma unroll
+                    for (int e = 0; e < N; ++e) z[s][e] *= r;
+                    V<TIO>::store(orow + (size_t)(t + s) * C, z[s]);
+                }
+        }
+    }
+}
+
+// Reverse pass.  partial: [CTAs][H*d][KMAX] per-CTA sums of the tap gradients.
+template <typename TIO, bool NORM>
+__global__ void __launch_bounds__(256)
+k_shortconv_bwd(ConvDims cd, const TIO *__restrict__ x, const float *__restrict__ w, const TIO *__restrict__ dout,
+                TIO *__restrict__ dx, float *__restrict__ partial) {
+    constexpr int N = V<TIO>::N;
+    extern __shared__ float sm[];                       // pss, pdot [TOKB][threads]; ca, cb [TOKB][H]
+    float *pss = sm, *pdot = sm + TOKB * blockDim.x, *ca = sm + 2 * TOKB * blockDim.x, *cb = ca + TOKB * cd.hpc;
+    const int C = cd.H * cd.d, vpr = cd.d / N, tid = threadIdx.x;
+    const int hb = blockIdx.z * cd.hpc, nh = min(cd.hpc, cd.H - hb);
+    const bool live = tid < nh * vpr;
+    const int h = live ? tid / vpr : 0;
+    const int gv = hb * vpr + tid;
+    float wt[KMAX][N];
+    load_taps<N>(w, gv * N, cd.K, live, wt);
+    const int b = blockIdx.y, t0 = blockIdx.x * cd.per, t1 = min(cd.T, t0 + cd.per);
+    const int ue = min(cd.T, t1 + KMAX - 1) - 1;        // last token whose dy this CTA needs
+    const size_t rowoff = ((size_t)b * cd.T) * C + (size_t)gv * N;
+    const TIO *xr = x + rowoff, *gr = dout + rowoff;
+    TIO *dxr = dx + rowoff;
+    float dy1[N], dy2[N], dy3[N], acc[KMAX][N];         // dy of tokens u+1, u+2, u+3
+#pragma unroll
+    for (int e = 0; e < N; ++e) {
+        dy1[e] = dy2[e] = dy3[e] = 0.f;
+#pragma unroll
+        for (int j = 0; j < KMAX; ++j) acc[j][e] = 0.f;
+    }
+    for (int top = ue; top >= t0; top -= TOKB) {
+        float zs[TOKB][N], gs[TOKB][N], dz[TOKB][N];
+#pragma unroll
+        for (int s = 0; s < TOKB; ++s) {
+            const int u = top - s;
+            float ss = 0.f, dot = 0.f;
+            if (u >= t0) {
+                float x0[N], x1[N], x2[N], x3[N];
+                load_x<TIO, N>(xr, u - 3, C, live, x0);
+                load_x<TIO, N>(xr, u - 2, C, live, x1);
+                load_x<TIO, N>(xr, u - 1, C, live, x2);
+                load_x<TIO, N>(xr, u, C, live, x3);
+                load_x<TIO, N>(gr, u, C, live, dz[s]);
+#pragma unroll
+                for (int e = 0; e < N; ++e) {
+                    const float y = fmaf(wt[0][e], x0[e], fmaf(wt[1][e], x1[e], fmaf(wt[2][e], x2[e], wt[3][e] * x3[e])));
+                    const float sg = 1.f / (1.f + __expf(-y));
+                    zs[s][e] = y * sg;
+                    gs[s][e] = sg * (1.f + y * (1.f - sg));         // d silu / dy
+                    ss = fmaf(zs[s][e], zs[s][e], ss);
+                    dot = fmaf(zs[s][e], dz[s][e], dot);
+                }
+            }
+            if (NORM) {
+                pss[s * blockDim.x + tid] = ss;
+                pdot[s * blockDim.x + tid] = dot;
+            }
+        }
+        if (NORM) {
+            __syncthreads();
+            if (tid < TOKB * nh) {
+                const int s = tid / nh, hh = tid % nh;
+                float a = 0.f, d2 = 0.f;
+                for (int j = 0; j < vpr; ++j) {
+                    a += pss[s * blockDim.x + hh * vpr + j];
+                    d2 += pdot[s * blockDim.x + hh * vpr + j];
+                }
+                const float r = sqrtf(a + cd.eps);
+                ca[s * cd.hpc + hh] = 1.f / r;                      // out = z / r:  dz = dout / r - z (z . dout) / r^3
+                cb[s * cd.hpc + hh] = d2 / (r * r * r);
+            }
+            __syncthreads();
+        }
+#pragma unroll
+        for (int s = 0; s < TOKB; ++s) {
+            const int u = top - s;
+            if (u < t0) continue;
+            float dy[N], dxu[N];
+            const float fa = NORM ? ca[s * cd.hpc + h] : 1.f, fb = NORM ? cb[s * cd.hpc + h] : 0.f;
+#pragma unroll
+            for (int e = 0; e < N; ++e) {
+                dy[e] = (dz[s][e] * fa - zs[s][e] * fb) * gs[s][e];
+                dxu[e] = fmaf(wt[3][e], dy[e], fmaf(wt[2][e], dy1[e], fmaf(wt[1][e], dy2[e], wt[0][e] * dy3[e])));
+            }
+            if (u < t1 && live) {                                   // this CTA's own tokens: dx out, tap gradients in
+                V<TIO>::store(dxr + (size_t)u * C, dxu);
+#pragma unroll
+                for (int j = 0; j < KMAX; ++j) {
+                    float xv[N];
+                    load_x<TIO, N>(xr, u - (KMAX - 1) + j, C, true, xv);
+#pragma unroll
+                    for (int e = 0; e < N; ++e) acc[j][e] = fmaf(dy[e], xv[e], acc[j][e]);
+                }
+            }
+#pragma unroll
+            for (int e = 0; e < N; ++e) { dy3[e] = dy2[e]; dy2[e] = dy1[e]; dy1[e] = dy[e]; }
+        }
+    }
+    if (live) {
+        float *dst = partial + (((size_t)blockIdx.y * gridDim.x + blockIdx.x) * C + (size_t)gv * N) * KMAX;
+#pragma unroll
+        for (int e = 0; e < N; ++e)
+#pragma unroll
+            for (int j = 0; j < KMAX; ++j) dst[e * KMAX + j] = acc[j][e];
+    }
+}
+
+// dw[c, j] = sum over the CTAs' partial sums, in CTA order
+__global__ void k_shortconv_dw(int n_cta, int C, int K, const float *__restrict__ partial, float *__restrict__ dw) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= C * K) return;
+    const int c = i / K, j = i % K + (KMAX - K);
+    float acc = 0.f;
+    for (int n = 0; n < n_cta; ++n) acc += partial[((size_t)n * C + c) * KMAX + j];
+    dw[i] = acc;
+}
+
+int tokens_per_cta(const Dims &d) {       // about four CTAs per SM, slices of at least 64 tokens
+    int dev = 0, sms = 148;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const long total = (long)d.B * d.T, want = 4L * sms;
+    long per = (total + want - 1) / want;
+    if (per < 64) per = 64;
+    return (int)per;
+}
+
+}  // namespace
+
+size_t shortconv_workspace_bytes(const Dims &d, int width) {
+    const int per = tokens_per_cta(d);
+    const size_t ctas = (size_t)((d.T + per - 1) / per) * d.B;
+    return ctas * d.H * width * KMAX * sizeof(float);
+}
+
+int shortconv_forward(const Dims &d, int width, int K, bool normalize, float eps, const void *x, const float *w, void *out,
+                      cudaStream_t st, Tracer &tr) {
+    const int N = d.io_bf16 ? 8 : 4, vpr = width / N;
+    const int hpc = std::max(1, std::min(d.H, 256 / vpr)), threads = (hpc * vpr + 31) / 32 * 32;
+    ConvDims cd{d.T, d.H, width, K, tokens_per_cta(d), hpc, eps};
+    dim3 grid((d.T + cd.per - 1) / cd.per, d.B, (d.H + hpc - 1) / hpc);
+    const size_t smem = (size_t)(TOKS * threads + TOKS * hpc) * sizeof(float);
+#define SLA_LAUNCH_FWD(TIO, NORM) \
+    k_shortconv_fwd<TIO, NORM><<<grid, threads, smem, st>>>(cd, (const TIO *)x, w, (TIO *)out)
+    if (d.io_bf16) { if (normalize) SLA_LAUNCH_FWD(__nv_bfloat16, true); else SLA_LAUNCH_FWD(__nv_bfloat16, false); }
+    else { if (normalize) SLA_LAUNCH_FWD(float, true); else SLA_LAUNCH_FWD(float, false); }
+#undef SLA_LAUNCH_FWD
+    tr.mark("shortconv_fwd");
+    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+}
+
+int shortconv_backward(const Dims &d, int width, int K, bool normalize, float eps, const void *x, const float *w,
+                       const void *dout, void *dx, float *dw, float *ws, cudaStream_t st, Tracer &tr) {
+    const int N = d.io_bf16 ? 8 : 4, vpr = width / N;
+    const int hpc = std::max(1, std::min(d.H, 256 / vpr)), threads = (hpc * vpr + 31) / 32 * 32;
+    ConvDims cd{d.T, d.H, width, K, tokens_per_cta(d), hpc, eps};
+    dim3 grid((d.T + cd.per - 1) / cd.per, d.B, (d.H + hpc - 1) / hpc);
+    const size_t smem = (size_t)(2 * TOKB * threads + 2 * TOKB * hpc) * sizeof(float);
+#define SLA_LAUNCH_BWD(TIO, NORM) \
+    k_shortconv_bwd<TIO, NORM><<<grid, threads, smem, st>>>(cd, (const TIO *)x, w, (const TIO *)dout, (TIO *)dx, ws)
+    if (d.io_bf16) { if (normalize) SLA_LAUNCH_BWD(__nv_bfloat16, true); else SLA_LAUNCH_BWD(__nv_bfloat16, false); }
+    else { if (normalize) SLA_LAUNCH_BWD(float, true); else SLA_LAUNCH_BWD(float, false); }
+#undef SLA_LAUNCH_BWD
+    tr.mark("shortconv_bwd");
+    const int C = d.H * width;
+    k_shortconv_dw<<<(C * K + 255) / 256, 256, 0, st>>>((int)(grid.x * grid.y), C, K, ws, dw);
+    tr.mark("shortconv_dw");
+    return cudaGetLastError() == cudaSuccess ? 2 : -1;
+}
+
+}  // namespace sla

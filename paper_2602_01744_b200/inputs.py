@@ -126,3 +126,18 @@ def make_gate_weights(cfg: SLAConfig, seed: int):
     gen = torch.Generator(device="cpu").manual_seed(seed)
     return (torch.randn(cfg.d_k, cfg.H, generator=gen, dtype=torch.float32),
             torch.randn(cfg.d_k, cfg.H, generator=gen, dtype=torch.float32))
+
+
+def make_frontend_inputs(cfg: SLAConfig, K: int, seed: int) -> dict:
+    """Raw inputs of the Gated-DeltaNet feature map: x_q, x_k, x_v ~ N(0,1) [B,T,H,d] in the I/O dtype (the layer's
+    linear projections are upstream and leave unit-scale activations), taps w_* ~ N(0,1)/sqrt(K) fp32 [H*d,K], and an
+    upstream gradient dout ~ N(0,1)."""
+    gen = torch.Generator(device="cpu").manual_seed(seed)
+    io = torch_dtype(cfg.dtype)
+    B, T, H = cfg.B, cfg.T, cfg.H
+    out = {}
+    for n, d in (("q", cfg.d_k), ("k", cfg.d_k), ("v", cfg.d_v)):
+        out[f"x_{n}"] = torch.randn(B, T, H, d, generator=gen, dtype=torch.float32).to(io)
+        out[f"w_{n}"] = torch.randn(H * d, K, generator=gen, dtype=torch.float32) / (K ** 0.5)
+    out["dout"] = torch.randn(B, T, H, cfg.d_k, generator=gen, dtype=torch.float32).to(io)
+    return out
