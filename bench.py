@@ -203,6 +203,10 @@ def main():
                     help="C2 is the benchmark; the other configurations (C1, C3: forward only; C4: gated delta rule, "
                          "forward + backward; R2: Softmax-RetNet at the shapes of C2) are timed the same way for the "
                          "per-configuration figures and profiles")
+    ap.add_argument("--packed", action="store_true",
+                    help="the workload's B*T tokens as ONE packed row of variable-length sequences (a seeded mix of "
+                         "lengths from 64 to 8192 tokens; sla_plan_set_sequences) instead of B rows of T: not the "
+                         "benchmark, labelled in config")
     ap.add_argument("--batch", type=int, default=0,
                     help="profiling aid: shrink the batch of the workload (0 = the full configuration; "
                          "a reduced batch is not the benchmark and is labelled in config)")
@@ -219,6 +223,17 @@ def main():
     if args.batch > 0:
         from paper_2602_01744_b200.inputs import small
         cfg = small(cfg, B=args.batch)
+    packed_cu = None
+    if args.packed:
+        import random
+        from paper_2602_01744_b200.inputs import small
+        total = cfg.B * cfg.T
+        rng, cu = random.Random(7), [0]
+        while cu[-1] < total:
+            cu.append(min(total, cu[-1] + rng.choice([64, 200, 512, 1000, 2048, 4096, 8192])))
+        packed_cu = cu
+        cfg = small(cfg, B=1, T=total)
+        METRIC += f" [packed: {len(cu) - 1} sequences of 64..8192 tokens in one row of {total}]"
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
@@ -255,6 +270,8 @@ def main():
         flags |= api.SLA_FLAG_SAVE_FOR_BACKWARD
     plan = api.sla_plan_create(cfg.variant, cfg.dtype, cfg.B, cfg.T, cfg.H, cfg.d_k, cfg.d_v, cfg.chunk,
                                cfg.scale, flags)
+    if packed_cu is not None:
+        plan.set_sequences(packed_cu)
     ws = plan.workspace(backward=cfg.backward)
     o = torch.empty_like(dev["v"])
     grads = None
@@ -585,6 +602,7 @@ def main():
                        "d_k": cfg.d_k, "d_v": cfg.d_v, "chunk": cfg.chunk, "pass": passes,
                        "io": "bf16 q,k,v,o and gradients; fp32 decay, logits, state; fp32 accumulation",
                        "l2": f"inputs ({h2d / 1e9:.2f} GB per step) exceed the 126 MB L2; no flush needed",
+                       "packed_sequences": None if packed_cu is None else len(packed_cu) - 1,
                        "parallelism": "replicas only" if world > 1 else "single GPU",
                        "kernels": "generic fp32 CUDA-core" if args.generic else "default",
                        "chunk_states": ("written by the forward pass of each step into the workspace, read by the backward "

@@ -94,6 +94,21 @@ typedef struct {
 sla_status sla_plan_create(sla_plan **out, const sla_desc *desc);
 sla_status sla_plan_destroy(sla_plan *plan);
 
+/*
+ * Packed variable-length batches (training data packed to a fixed token budget; the paper trains at a maximum sequence
+ * length of 4096 on such data).  For a plan with B == 1 the T tokens are n_seq sequences laid one after another:
+ * sequence s covers tokens cu_seqlens[s] .. cu_seqlens[s+1]-1 (cu_seqlens: HOST array of n_seq + 1 ascending offsets,
+ * first 0, last T; no empty sequence).  After this call sla_forward / sla_backward on the plan run the recurrence of
+ * Eq. 5-6 per sequence: the state starts from h0[s] (or zero) at each sequence's first token, chunks are cut from each
+ * sequence's own start and never straddle a boundary, and h0, ht, dht, dh0 have the shape [n_seq,H,d_k,d_v].
+ * sla_plan_workspace_bytes changes with the table: query it again.  n_seq == 0 returns the plan to a regular batch.
+ * The plan copies the table (and owns a few small device arrays for it until it is destroyed or the table replaced);
+ * this is a set-up call, not to be made between a forward and its backward pass.  Only plans that select the
+ * tensor-core kernels (bf16, d_k = d_v = 128, chunk 64) take a table: SLA_ERR_UNSUPPORTED otherwise.  Calls on one
+ * plan must be ordered on one stream (the per-sequence tensor maps are uploaded in stream order).
+ */
+sla_status sla_plan_set_sequences(sla_plan *plan, const int32_t *cu_seqlens, int32_t n_seq);
+
 /* Bytes of caller-provided scratch that sla_forward / sla_backward need for this plan (it depends on the kernels the
  * plan selects; 0 means none is needed and the workspace pointer may then be NULL). */
 sla_status sla_plan_workspace_bytes(const sla_plan *plan, size_t *forward_bytes, size_t *backward_bytes);

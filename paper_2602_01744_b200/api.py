@@ -26,7 +26,7 @@ EXPORTS = (
     "sla_plan_kernel_timing_get", "sla_status_string", "sla_forward", "sla_backward", "sla_decode_step",
     "sla_forward_noalloc", "sla_plan_selftest_timeout", "sla_decode_steps", "sla_gate_scores_forward",
     "sla_gate_scores_backward", "sla_plan_gate_scores_workspace_bytes", "sla_shortconv_forward",
-    "sla_shortconv_backward", "sla_plan_shortconv_workspace_bytes",
+    "sla_shortconv_backward", "sla_plan_shortconv_workspace_bytes", "sla_plan_set_sequences",
 )
 SLA_NOALLOC_SCRATCH_BYTES = 32 << 20
 
@@ -87,6 +87,8 @@ def lib():
         L.sla_decode_step.argtypes = [vp, i32] + [vp] * 10
         L.sla_decode_steps.argtypes = [vp, i32, i32] + [vp] * 10
         L.sla_decode_steps.restype = ctypes.c_int
+        L.sla_plan_set_sequences.argtypes = [vp, ctypes.POINTER(i32), i32]
+        L.sla_plan_set_sequences.restype = ctypes.c_int
         L.sla_shortconv_forward.argtypes = [vp, vp, vp, i32, i32, i32, vp, vp]
         L.sla_shortconv_forward.restype = ctypes.c_int
         L.sla_shortconv_backward.argtypes = [vp, vp, vp, i32, i32, i32, vp, vp, vp, vp, sz, vp]
@@ -147,6 +149,18 @@ class Plan:
             self.handle.value = None
 
     __del__ = close
+
+    def set_sequences(self, cu_seqlens):
+        """Packed variable-length batch (see sla_plan_set_sequences): cu_seqlens = n_seq + 1 ascending token offsets
+        (a host sequence of ints), or None / [] for a regular batch.  Workspace sizes are queried again."""
+        cu = list(cu_seqlens) if cu_seqlens is not None else []
+        n = max(len(cu) - 1, 0)
+        arr = (ctypes.c_int32 * max(len(cu), 1))(*cu)
+        _check("sla_plan_set_sequences", lib().sla_plan_set_sequences(self.handle, arr, n))
+        f, b = ctypes.c_size_t(), ctypes.c_size_t()
+        _check("sla_plan_workspace_bytes", lib().sla_plan_workspace_bytes(self.handle, ctypes.byref(f), ctypes.byref(b)))
+        self.forward_workspace_bytes, self.backward_workspace_bytes = f.value, b.value
+        self.n_seq = n
 
     def poll(self):
         _check("sla_plan_poll", lib().sla_plan_poll(self.handle))
@@ -220,7 +234,7 @@ def sla_backward(plan: Plan, q, k, v, log_decay, gq_logits, gk_logits, dO, beta=
             dlog_decay=None if d.variant == SLA_RETNET else torch.empty_like(log_decay),
             dbeta=torch.empty_like(beta) if d.variant == SLA_GDN else None,
             dgq_logits=torch.empty_like(gq_logits), dgk_logits=torch.empty_like(gk_logits),
-            dh0=torch.empty((d.B, d.H, d.d_k, d.d_v), dtype=torch.float32, device=dev) if want_dh0 else None,
+            dh0=torch.empty((getattr(plan, "n_seq", 0) or d.B, d.H, d.d_k, d.d_v), dtype=torch.float32, device=dev) if want_dh0 else None,
         )
     if workspace is None:
         workspace = plan.workspace(True, dev)

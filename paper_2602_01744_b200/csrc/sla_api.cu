@@ -60,8 +60,37 @@ __global__ void k_selftest_bounded_wait(int *status, unsigned long long limit_ns
 // paths do, and Softmax-GLA only where the forward runs each sequence in one piece.
 static bool forward_can_save(const sla_plan &p) {
     if (p.flags & SLA_FLAG_FORCE_GENERIC) return false;
-    if (sla::gla_tc_supported(p.dims)) return sla::gla_tc_forward_can_save(p.dims);
+    if (sla::gla_tc_supported(p.dims)) return sla::gla_tc_forward_can_save(p.dims, &p.varlen);
     return sla::gdn_tc_supported(p.dims);
+}
+
+// What the kernels this plan selects need as workspace (regular batch, or the packed batch of sla_plan_set_sequences).
+static void plan_workspace_sizes(sla_plan *p) {
+    const sla::Dims &d = p->dims;
+    const bool generic = p->flags & SLA_FLAG_FORCE_GENERIC;
+    p->fwd_bytes = p->ws.fwd_floats * sizeof(float);
+    p->bwd_bytes = p->ws.bwd_floats * sizeof(float);
+    if (sla::gla_tc_supported(d) && !generic) {
+        p->fwd_bytes = sla::gla_tc_forward_workspace_bytes(d, &p->varlen);
+        p->bwd_bytes = sla::gla_tc_backward_workspace_bytes(d, &p->varlen);
+    }
+    if (sla::gdn_tc_supported(d) && !generic) {
+        p->fwd_bytes = 0;
+        p->bwd_bytes = sla::gdn_tc_backward_workspace_bytes(d, &p->varlen);
+    }
+    if ((p->flags & SLA_FLAG_SAVE_FOR_BACKWARD) && forward_can_save(*p) && p->bwd_bytes > p->fwd_bytes)
+        p->fwd_bytes = p->bwd_bytes;     // the forward writes into the backward pass's workspace layout
+}
+
+static void varlen_release(sla::Varlen &v) {
+    if (v.d_seqs) cudaFree(v.d_seqs);
+    for (auto &g : v.reg) {
+        if (g.dev) cudaFree(g.dev);
+        if (g.host) cudaFreeHost(g.host);
+        if (g.uploaded) cudaEventDestroy(g.uploaded);
+        g = sla::Varlen::Region();
+    }
+    v = sla::Varlen();
 }
 
 extern "C" {
@@ -115,18 +144,7 @@ sla_status sla_plan_create(sla_plan **out, const sla_desc *desc) {
     d.scale = desc->scale;
     p->ws = sla::plan_workspace(d);
     p->flags = desc->flags;
-    p->fwd_bytes = p->ws.fwd_floats * sizeof(float);
-    p->bwd_bytes = p->ws.bwd_floats * sizeof(float);
-    if (sla::gla_tc_supported(d) && !(desc->flags & SLA_FLAG_FORCE_GENERIC)) {
-        p->fwd_bytes = sla::gla_tc_forward_workspace_bytes(d);
-        p->bwd_bytes = sla::gla_tc_backward_workspace_bytes(d);
-    }
-    if (sla::gdn_tc_supported(d) && !(desc->flags & SLA_FLAG_FORCE_GENERIC)) {
-        p->fwd_bytes = 0;
-        p->bwd_bytes = sla::gdn_tc_backward_workspace_bytes(d);
-    }
-    if ((desc->flags & SLA_FLAG_SAVE_FOR_BACKWARD) && forward_can_save(*p) && p->bwd_bytes > p->fwd_bytes)
-        p->fwd_bytes = p->bwd_bytes;     // the forward writes into the backward pass's workspace layout
+    plan_workspace_sizes(p);
     p->device = dev;
     p->last_launches = 0;
     p->d_status = nullptr;
@@ -143,8 +161,48 @@ sla_status sla_plan_create(sla_plan **out, const sla_desc *desc) {
 sla_status sla_plan_destroy(sla_plan *plan) {
     if (!plan) return SLA_OK;
     if (plan->d_status) cudaFree(plan->d_status);
+    varlen_release(plan->varlen);
     plan->tracer.destroy();
     delete plan;
+    return SLA_OK;
+}
+
+sla_status sla_plan_set_sequences(sla_plan *plan, const int32_t *cu_seqlens, int32_t n_seq) {
+    if (!plan || n_seq < 0 || (n_seq > 0 && !cu_seqlens)) return SLA_ERR_INVALID_ARG;
+    const sla::Dims &d = plan->dims;
+    plan->saved.valid = false;
+    varlen_release(plan->varlen);
+    if (n_seq == 0) {
+        plan_workspace_sizes(plan);
+        return SLA_OK;
+    }
+    // the tensor-core kernels only (they address a sequence through tensor maps of its own)
+    if ((plan->flags & SLA_FLAG_FORCE_GENERIC) || !(sla::gla_tc_supported(d) || sla::gdn_tc_supported(d))) return SLA_ERR_UNSUPPORTED;
+    if (d.B != 1 || cu_seqlens[0] != 0 || cu_seqlens[n_seq] != d.T) return SLA_ERR_INVALID_ARG;
+    if ((uint64_t)n_seq * d.H > 0x7fffffffu) return SLA_ERR_UNSUPPORTED;
+    sla::Varlen &v = plan->varlen;
+    long slots = 0;
+    for (int s = 0; s < n_seq; ++s) {
+        const int len = cu_seqlens[s + 1] - cu_seqlens[s];
+        if (len <= 0) { v.seqs.clear(); return SLA_ERR_INVALID_ARG; }      // (empty sequences are not allowed)
+        const int nt = (len + d.C - 1) / d.C;
+        v.seqs.push_back({cu_seqlens[s], len, nt, (int)slots});
+        slots += nt + 1;
+    }
+    v.slots = slots;
+    v.n_seq = n_seq;
+    bool ok = cudaMalloc((void **)&v.d_seqs, sizeof(sla::SeqInfo) * n_seq) == cudaSuccess &&
+              cudaMemcpy(v.d_seqs, v.seqs.data(), sizeof(sla::SeqInfo) * n_seq, cudaMemcpyHostToDevice) == cudaSuccess;
+    const size_t mb = (size_t)n_seq * sla::Varlen::MAPS_PER_SEQ * sizeof(CUtensorMap);
+    for (auto &g : v.reg)
+        ok = ok && cudaMalloc((void **)&g.dev, mb) == cudaSuccess && cudaMallocHost((void **)&g.host, mb) == cudaSuccess &&
+             cudaEventCreateWithFlags(&g.uploaded, cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) {
+        varlen_release(v);
+        plan_workspace_sizes(plan);
+        return SLA_ERR_CUDA;
+    }
+    plan_workspace_sizes(plan);
     return SLA_OK;
 }
 
@@ -230,7 +288,8 @@ sla_status sla_forward(sla_plan *plan, const void *q, const void *k, const void 
     for (const void *p : ptrs)
         if (!aligned16(p)) return SLA_ERR_INVALID_ARG;
     if (plan->fwd_bytes > 0 && (!workspace || workspace_bytes < plan->fwd_bytes)) return SLA_ERR_WORKSPACE;
-    sla::FwdArgs a{q, k, v, log_decay, beta, gq_logits, gk_logits, h0, o, ht, (float *)workspace, plan->d_status};
+    sla::FwdArgs a{q, k, v, log_decay, beta, gq_logits, gk_logits, h0, o, ht, (float *)workspace, plan->d_status,
+                   plan->varlen.n_seq ? &plan->varlen : nullptr};
     plan->tracer.start((cudaStream_t)cuda_stream);
     const bool generic = plan->flags & SLA_FLAG_FORCE_GENERIC;
     const bool save = (plan->flags & SLA_FLAG_SAVE_FOR_BACKWARD) && forward_can_save(*plan);
@@ -284,7 +343,8 @@ sla_status sla_backward(sla_plan *plan, const void *q, const void *k, const void
         if (!aligned16(p)) return SLA_ERR_INVALID_ARG;
     if (plan->bwd_bytes > 0 && (!workspace || workspace_bytes < plan->bwd_bytes)) return SLA_ERR_WORKSPACE;
     sla::BwdArgs a{q, k, v, log_decay, beta, gq_logits, gk_logits, h0, dO, dht, dq, dk, dv,
-                   dlog_decay, dbeta, dgq_logits, dgk_logits, dh0, (float *)workspace, plan->d_status};
+                   dlog_decay, dbeta, dgq_logits, dgk_logits, dh0, (float *)workspace, plan->d_status,
+                   plan->varlen.n_seq ? &plan->varlen : nullptr};
     plan->tracer.start((cudaStream_t)cuda_stream);
     const bool generic = plan->flags & SLA_FLAG_FORCE_GENERIC;
     // the states (GLA) or per-chunk records (GDN) are taken from the workspace only if the last sla_forward of this plan

@@ -59,18 +59,34 @@ struct GdnParams {
     int *status;
     int T, H, NT;
     float scale;
+    const SeqInfo *seqs;    // packed variable-length batch: per-sequence table and tensor maps (q, k, v, o), else nullptr
+    const CUtensorMap *vmaps;
 };
 
 __global__ void __launch_bounds__(gd::NTHREADS, 1)
-k_gdn_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-             const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o, GdnParams p) {
+k_gdn_fwd_tc(const __grid_constant__ CUtensorMap gm_q, const __grid_constant__ CUtensorMap gm_k,
+             const __grid_constant__ CUtensorMap gm_v, const __grid_constant__ CUtensorMap gm_o, GdnParams p) {
     using namespace gd;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t *sm = smem_raw + (base - raw);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int bh = blockIdx.x, b = bh / p.H, h = bh % p.H;
+    const int bh = blockIdx.x, h = bh % p.H;
+    int b = bh / p.H;
+    // A packed batch: this CTA's sequence has its own length, chunk count, first token, record slots and tensor maps
+    // (based at its first token, so token coordinates stay relative and the batch coordinate is 0).
+    size_t tokb = (size_t)b * p.T, slot = (size_t)bh * (p.NT + 1);
+    const CUtensorMap *vm = nullptr;
+    if (p.seqs) {
+        const SeqInfo si = p.seqs[b];
+        vm = p.vmaps + (size_t)b * Varlen::MAPS_PER_SEQ;
+        p.T = si.T; p.NT = si.NT;
+        tokb = (size_t)si.t0;
+        slot = (size_t)si.slot0 * p.H + (size_t)h * (si.NT + 1);
+        b = 0;
+    }
+    const CUtensorMap &tm_q = vm ? vm[0] : gm_q, &tm_k = vm ? vm[1] : gm_k, &tm_v = vm ? vm[2] : gm_v, &tm_o = vm ? vm[3] : gm_o;
     const int NT = p.NT;
     auto bar = [&](int i) { return base + OFF_BAR + 8u * i; };
     float *Ls = reinterpret_cast<float *>(sm + OFF_LS);
@@ -104,7 +120,6 @@ k_gdn_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *reinterpret_cast<volatile uint32_t *>(sm + OFF_TMEM);
-    const size_t tokb = (size_t)b * p.T;
 
     if (warp == 8) {
         // ---------------- MMA issue (one lane) ----------------
@@ -186,7 +201,7 @@ k_gdn_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
                     bulk_commit();
                 }
                 if (p.save) {   // the chunk's record: T, U and S_{n+1} stand in shared memory in exactly the record's layout
-                    uint8_t *rec = p.save + ((size_t)bh * (NT + 1) + n) * REC_BYTES;
+                    uint8_t *rec = p.save + (slot + n) * REC_BYTES;
                     bulk_store(rec + REC_T, base + OFF_T, HALF_BF16);
                     bulk_store(rec + REC_U, base + (n & 1) * STAGE + OFF_K, TILE_BF16);
                     bulk_store(rec + REC_BYTES + REC_S, base + OFF_S, STATE_BF16);
@@ -228,7 +243,7 @@ k_gdn_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
         const int row = 32 * (warp & 3) + lane;                          // state row (M = 128 tiles)
         const int ti = 16 * (warp & 3) + lane;                           // token row (M = 64 tiles, lanes 0..15)
 
-        uint8_t *rec0 = p.save ? p.save + (size_t)bh * (NT + 1) * REC_BYTES : nullptr;   // this sequence's records
+        uint8_t *rec0 = p.save ? p.save + slot * REC_BYTES : nullptr;   // this sequence's records
         {   // initial state: fp32 into TMEM, bf16 copy into shared memory (row = key dimension)
             const float *src = p.h0 ? p.h0 + ((size_t)bh * D + row) * D + 64 * colhalf : nullptr;
 #pragma unroll
@@ -558,14 +573,32 @@ int gdn_tc_configure() {
                    cudaSuccess ? 0 : -1;
 }
 
+// per-sequence tensor maps of a packed batch (q, k, v and, when given, o) into region `r`
+static const CUtensorMap *gdn_varlen_maps(const Dims &d, const FwdArgs &a, int r, cudaStream_t st) {
+    const void *key[] = {a.q, a.k, a.v, a.o};
+    return varlen_maps(*a.vl, r, key, 4, st, [&](const SeqInfo &si, CUtensorMap *m) {
+        const size_t off = (size_t)si.t0 * d.H * D;
+        if (!make_tile_map(m + 0, (const __nv_bfloat16 *)a.q + off, 1, si.T, d.H) ||
+            !make_tile_map(m + 1, (const __nv_bfloat16 *)a.k + off, 1, si.T, d.H) ||
+            !make_tile_map(m + 2, (const __nv_bfloat16 *)a.v + off, 1, si.T, d.H))
+            return false;
+        if (!a.o) { m[3] = m[0]; return true; }
+        return make_tile_map(m + 3, (__nv_bfloat16 *)a.o + off, 1, si.T, d.H);
+    });
+}
+
 // Forward sweep in save mode, for the gradient sweep: writes the per-chunk records (S_n, U, T), stores no output.
 int gdn_tc_forward_save(const Dims &d, const FwdArgs &a, uint8_t *save, int *status, cudaStream_t st, Tracer &tr) {
     CUtensorMap mq, mk, mv;
     if (!make_tile_map(&mq, a.q, d.B, d.T, d.H) || !make_tile_map(&mk, a.k, d.B, d.T, d.H) ||
         !make_tile_map(&mv, a.v, d.B, d.T, d.H))
         return -1;
-    GdnParams p{a.lq, a.lk, a.log_decay, a.beta, a.h0, nullptr, save, 0, status, d.T, d.H, d.NT, d.scale};
-    k_gdn_fwd_tc<<<d.B * d.H, gd::NTHREADS, gd::SMEM_BYTES, st>>>(mq, mk, mv, mq /* unused: nothing is stored */, p);
+    const bool vl = a.vl && a.vl->n_seq;
+    const CUtensorMap *vm = vl ? gdn_varlen_maps(d, a, 1, st) : nullptr;
+    if (vl && !vm) return -1;
+    GdnParams p{a.lq, a.lk, a.log_decay, a.beta, a.h0, nullptr, save, 0, status, d.T, d.H, d.NT, d.scale,
+                vl ? a.vl->d_seqs : nullptr, vm};
+    k_gdn_fwd_tc<<<vl ? a.vl->n_seq * d.H : d.B * d.H, gd::NTHREADS, gd::SMEM_BYTES, st>>>(mq, mk, mv, mq /* unused: nothing is stored */, p);
     tr.mark("gdn_states_tc");
     return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
@@ -576,8 +609,12 @@ int gdn_tc_forward(const Dims &d, const FwdArgs &a, uint8_t *save, int *status, 
     if (!make_tile_map(&mq, a.q, d.B, d.T, d.H) || !make_tile_map(&mk, a.k, d.B, d.T, d.H) ||
         !make_tile_map(&mv, a.v, d.B, d.T, d.H) || !make_tile_map(&mo, a.o, d.B, d.T, d.H))
         return -1;
-    GdnParams p{a.lq, a.lk, a.log_decay, a.beta, a.h0, a.ht, save, 1, status, d.T, d.H, d.NT, d.scale};
-    k_gdn_fwd_tc<<<d.B * d.H, gd::NTHREADS, gd::SMEM_BYTES, st>>>(mq, mk, mv, mo, p);
+    const bool vl = a.vl && a.vl->n_seq;
+    const CUtensorMap *vm = vl ? gdn_varlen_maps(d, a, 0, st) : nullptr;
+    if (vl && !vm) return -1;
+    GdnParams p{a.lq, a.lk, a.log_decay, a.beta, a.h0, a.ht, save, 1, status, d.T, d.H, d.NT, d.scale,
+                vl ? a.vl->d_seqs : nullptr, vm};
+    k_gdn_fwd_tc<<<vl ? a.vl->n_seq * d.H : d.B * d.H, gd::NTHREADS, gd::SMEM_BYTES, st>>>(mq, mk, mv, mo, p);
     tr.mark("gdn_fwd_tc");
     return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }

@@ -68,20 +68,35 @@ struct GdnBwdParams {
     int *status;
     int T, H, NT;
     float scale;
+    const SeqInfo *seqs;            // packed variable-length batch: per-sequence table and tensor maps (the seven below), else nullptr
+    const CUtensorMap *vmaps;
 };
 
 __global__ void __launch_bounds__(gb::NTHREADS, 1)
-k_gdn_bwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-             const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
-             const __grid_constant__ CUtensorMap tm_dq, const __grid_constant__ CUtensorMap tm_dk,
-             const __grid_constant__ CUtensorMap tm_dv, GdnBwdParams p) {
+k_gdn_bwd_tc(const __grid_constant__ CUtensorMap gm_q, const __grid_constant__ CUtensorMap gm_k,
+             const __grid_constant__ CUtensorMap gm_v, const __grid_constant__ CUtensorMap gm_do,
+             const __grid_constant__ CUtensorMap gm_dq, const __grid_constant__ CUtensorMap gm_dk,
+             const __grid_constant__ CUtensorMap gm_dv, GdnBwdParams p) {
     using namespace gb;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t *sm = smem_raw + (base - raw);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int bh = blockIdx.x, b = bh / p.H, h = bh % p.H;
+    const int bh = blockIdx.x, h = bh % p.H;
+    int b = bh / p.H;
+    size_t tokb = (size_t)b * p.T, slot = (size_t)bh * (p.NT + 1);
+    const CUtensorMap *vm = nullptr;
+    if (p.seqs) {                                           // packed batch: see k_gdn_fwd_tc
+        const SeqInfo si = p.seqs[b];
+        vm = p.vmaps + (size_t)b * Varlen::MAPS_PER_SEQ;
+        p.T = si.T; p.NT = si.NT;
+        tokb = (size_t)si.t0;
+        slot = (size_t)si.slot0 * p.H + (size_t)h * (si.NT + 1);
+        b = 0;
+    }
+    const CUtensorMap &tm_q = vm ? vm[0] : gm_q, &tm_k = vm ? vm[1] : gm_k, &tm_v = vm ? vm[2] : gm_v, &tm_do = vm ? vm[3] : gm_do,
+                      &tm_dq = vm ? vm[4] : gm_dq, &tm_dk = vm ? vm[5] : gm_dk, &tm_dv = vm ? vm[6] : gm_dv;
     const int NT = p.NT;
     auto bar = [&](int i) { return base + OFF_BAR + 8u * i; };
     float *sc = reinterpret_cast<float *>(sm + OFF_SC);
@@ -116,8 +131,7 @@ k_gdn_bwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *reinterpret_cast<volatile uint32_t *>(sm + OFF_TMEM);
-    const size_t tokb = (size_t)b * p.T;
-    const uint8_t *rec0 = p.save + (size_t)bh * (NT + 1) * REC_BYTES;
+    const uint8_t *rec0 = p.save + slot * REC_BYTES;
     // chunks are visited in the order n = NT-1 ... 0; k = NT-1-n is the visit number that drives every barrier parity
 
     if (warp == 8) {
@@ -751,9 +765,14 @@ int gdn_tc_bwd_configure() {
                    cudaSuccess ? 0 : -1;
 }
 
-size_t gdn_tc_backward_workspace_bytes(const Dims &d) {
+// record slots (one per chunk plus one per sequence) over all (sequence, head) pairs
+static size_t record_slots(const Dims &d, const Varlen *vl) {
+    return (vl && vl->n_seq) ? (size_t)vl->slots * d.H : (size_t)d.B * d.H * (d.NT + 1);
+}
+
+size_t gdn_tc_backward_workspace_bytes(const Dims &d, const Varlen *vl) {
     const size_t bth = (size_t)d.B * d.T * d.H;
-    return (size_t)d.B * d.H * (d.NT + 1) * REC_BYTES + 2 * ((bth + 63) & ~(size_t)63) * sizeof(float);
+    return record_slots(d, vl) * REC_BYTES + 2 * ((bth + 63) & ~(size_t)63) * sizeof(float);
 }
 
 uint8_t *gdn_tc_records(float *ws) { return reinterpret_cast<uint8_t *>(ws); }
@@ -765,16 +784,29 @@ int gdn_tc_backward(const Dims &d, const BwdArgs &a, bool have_records, int *sta
         !make_tile_map(&mdq, a.dq, d.B, d.T, d.H) || !make_tile_map(&mdk, a.dk, d.B, d.T, d.H) ||
         !make_tile_map(&mdv, a.dv, d.B, d.T, d.H))
         return -1;
+    Varlen *vl = (a.vl && a.vl->n_seq) ? a.vl : nullptr;
     const size_t bth = (size_t)d.B * d.T * d.H;
     uint8_t *save = reinterpret_cast<uint8_t *>(a.ws);
-    float *pq = reinterpret_cast<float *>(save + (size_t)d.B * d.H * (d.NT + 1) * REC_BYTES);
+    float *pq = reinterpret_cast<float *>(save + record_slots(d, vl) * REC_BYTES);
     float *pk = pq + ((bth + 63) & ~(size_t)63);
-    FwdArgs f{a.q, a.k, a.v, a.log_decay, a.beta, a.lq, a.lk, a.h0, nullptr, nullptr, a.ws, a.status};
+    FwdArgs f{a.q, a.k, a.v, a.log_decay, a.beta, a.lq, a.lk, a.h0, nullptr, nullptr, a.ws, a.status, vl};
     // (with have_records the forward pass of the same inputs has left the records in this workspace)
     if (!have_records && gdn_tc_forward_save(d, f, save, status, st, tr) < 0) return -1;
+    const CUtensorMap *vm = nullptr;
+    if (vl) {
+        const void *key[] = {a.q, a.k, a.v, a.dO, a.dq, a.dk, a.dv};
+        vm = varlen_maps(*vl, 2, key, 7, st, [&](const SeqInfo &si, CUtensorMap *m) {
+            const size_t off = (size_t)si.t0 * d.H * D;
+            const void *src[7] = {a.q, a.k, a.v, a.dO, a.dq, a.dk, a.dv};
+            for (int i = 0; i < 7; ++i)
+                if (!make_tile_map(m + i, (const __nv_bfloat16 *)src[i] + off, 1, si.T, d.H)) return false;
+            return true;
+        });
+        if (!vm) return -1;
+    }
     GdnBwdParams bp{a.lq, a.lk, a.log_decay, a.beta, a.dht, save, a.dlog_decay, a.dbeta, pq, pk, a.dh0, status,
-                    d.T, d.H, d.NT, d.scale};
-    k_gdn_bwd_tc<<<d.B * d.H, gb::NTHREADS, gb::SMEM_BYTES, st>>>(mq, mk, mv, mdo, mdq, mdk, mdv, bp);
+                    d.T, d.H, d.NT, d.scale, vl ? vl->d_seqs : nullptr, vm};
+    k_gdn_bwd_tc<<<vl ? vl->n_seq * d.H : d.B * d.H, gb::NTHREADS, gb::SMEM_BYTES, st>>>(mq, mk, mv, mdo, mdq, mdk, mdv, bp);
     tr.mark("gdn_bwd_tc");
     if (gate_bwd_prod(a.lq, a.lk, pq, pk, a.dlq, a.dlk, (long)d.B * d.T, d.H, st) < 0) return -1;
     tr.mark("gate_bwd");

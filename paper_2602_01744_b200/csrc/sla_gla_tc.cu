@@ -58,6 +58,8 @@ struct FwdParams {
     int P, L;                       // segments per sequence and chunks per segment (P = 1: L = NT)
     float scale;
     const float *log_gamma;         // Softmax-RetNet: [H] constant log-decays (no log-decay tensor is read); else nullptr
+    const SeqInfo *seqs;            // packed variable-length batch: per-sequence table and tensor maps (q, k, v, g, o), else nullptr
+    const CUtensorMap *vmaps;
 };
 
 // One CTA per (batch, head) sequence, five roles that only meet on mbarriers:
@@ -69,16 +71,31 @@ struct FwdParams {
 // The prologue of chunk n+1.. runs beside the mask / rescale / store work of chunk n, so the shared-memory,
 // special-function and FMA phases of the two groups overlap instead of following one another.
 __global__ void __launch_bounds__(NTHREADS, 1)
-k_gla_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-             const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_g,
-             const __grid_constant__ CUtensorMap tm_o, FwdParams p) {
+k_gla_fwd_tc(const __grid_constant__ CUtensorMap gm_q, const __grid_constant__ CUtensorMap gm_k,
+             const __grid_constant__ CUtensorMap gm_v, const __grid_constant__ CUtensorMap gm_g,
+             const __grid_constant__ CUtensorMap gm_o, FwdParams p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t *sm = smem_raw + (base - raw);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     // a sequence may be cut into p.P segments of p.L chunks, one CTA each, every segment starting from its own state
-    const int bh = blockIdx.x / p.P, seg = blockIdx.x % p.P, b = bh / p.H, h = bh % p.H;
+    const int bh = blockIdx.x / p.P, seg = blockIdx.x % p.P, h = bh % p.H;
+    int b = bh / p.H;
+    // A packed batch: this CTA's sequence has its own length, chunk count, first token, state slots and tensor maps
+    // (based at its first token, so token coordinates stay relative and the batch coordinate is 0).
+    size_t tokb = (size_t)b * p.T, slot = (size_t)bh * (p.NT + 1);
+    const CUtensorMap *vm = nullptr;
+    if (p.seqs) {
+        const SeqInfo si = p.seqs[b];
+        vm = p.vmaps + (size_t)b * Varlen::MAPS_PER_SEQ;
+        p.T = si.T; p.NT = si.NT; p.L = si.NT;
+        tokb = (size_t)si.t0;
+        slot = (size_t)si.slot0 * p.H + (size_t)h * (si.NT + 1);
+        b = 0;
+    }
+    const CUtensorMap &tm_q = vm ? vm[0] : gm_q, &tm_k = vm ? vm[1] : gm_k, &tm_v = vm ? vm[2] : gm_v,
+                      &tm_g = vm ? vm[3] : gm_g, &tm_o = vm ? vm[4] : gm_o;
     const int n0 = seg * p.L, NT = min(p.L, p.NT - n0);     // this CTA's chunks: n0 .. n0+NT-1
     auto bar = [&](int i) { return base + OFF_BAR + 8u * i; };
     float *tot = reinterpret_cast<float *>(sm + OFF_TOT);
@@ -113,7 +130,6 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *reinterpret_cast<volatile uint32_t *>(sm + OFF_TMEM);
-    const size_t tokb = (size_t)b * p.T;
 
     if (warp == W_MMA) {
         // ---------------- MMA issue (one lane) ----------------
@@ -181,7 +197,7 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
                 tma_load_5d(dst, &tm_v, 0, (n0 + n) * C, 0, h, b, bf);
             };
             // save mode: S_m (the bf16 operand copy, as it stands in shared memory) -> image slot m, for the backward pass
-            uint8_t *img0 = p.simg ? p.simg + (size_t)bh * (p.NT + 1) * STATE_BF16 : nullptr;
+            uint8_t *img0 = p.simg ? p.simg + slot * STATE_BF16 : nullptr;
             for (int n = 0; n < 3 && n < NT; ++n) load_qk(n);
             for (int n = 0; n < 2 && n < NT; ++n) load_v(n);
             // From here on the lane serves whichever buffer falls free or fills first (no fixed order: the prologue warps
@@ -467,14 +483,15 @@ int gla_tc_configure() {
                    cudaSuccess ? 0 : -1;
 }
 
-size_t gla_tc_forward_workspace_bytes(const Dims &d) {
+size_t gla_tc_forward_workspace_bytes(const Dims &d, const Varlen *vl) {
     int P, L;
     choose_segments(d, P, L);
-    if (P == 1) return 0;
+    if (P == 1 || (vl && vl->n_seq)) return 0;
     return (size_t)d.B * d.H * P * (D * D + D) * sizeof(float);
 }
 
-bool gla_tc_forward_can_save(const Dims &d) {
+bool gla_tc_forward_can_save(const Dims &d, const Varlen *vl) {
+    if (vl && vl->n_seq) return true;     // (a packed batch always runs one CTA per sequence)
     int P, L;
     choose_segments(d, P, L);
     return P == 1;
@@ -483,6 +500,24 @@ bool gla_tc_forward_can_save(const Dims &d) {
 int gla_tc_forward(const Dims &d, const FwdArgs &a, uint8_t *simg, int *status, cudaStream_t st, Tracer &tr) {
     CUtensorMap mq, mk, mv, mg, mo;
     const bool retnet = d.variant == SLA_RETNET;
+    if (a.vl && a.vl->n_seq) {          // packed batch: one CTA per (sequence, head), per-sequence tensor maps
+        const void *key[] = {a.q, a.k, a.v, a.log_decay, a.o};
+        const CUtensorMap *vm = varlen_maps(*a.vl, 0, key, 5, st, [&](const SeqInfo &si, CUtensorMap *m) {
+            const size_t off = (size_t)si.t0 * d.H * D;
+            const __nv_bfloat16 *q = (const __nv_bfloat16 *)a.q, *k = (const __nv_bfloat16 *)a.k, *v = (const __nv_bfloat16 *)a.v;
+            if (!make_tile_map(m + 0, q + off, 1, si.T, d.H) || !make_tile_map(m + 1, k + off, 1, si.T, d.H) ||
+                !make_tile_map(m + 2, v + off, 1, si.T, d.H) || !make_tile_map(m + 4, (__nv_bfloat16 *)a.o + off, 1, si.T, d.H))
+                return false;
+            if (retnet) { m[3] = m[0]; return true; }
+            return make_map(m + 3, a.log_decay + off, 1, si.T, d.H, d.dk, true, 128);
+        });
+        if (!vm || !make_tile_map(&mq, a.q, d.B, d.T, d.H)) return -1;
+        FwdParams p{a.lq, a.lk, a.h0, nullptr, nullptr, (__nv_bfloat16 *)a.o, a.ht, simg, status, d.T, d.H, d.NT, 1, d.NT, d.scale,
+                    retnet ? a.log_decay : nullptr, a.vl->d_seqs, vm};
+        k_gla_fwd_tc<<<a.vl->n_seq * d.H, NTHREADS, SMEM_BYTES, st>>>(mq, mq, mq, mq, mq, p);
+        tr.mark("gla_fwd_tc");
+        return cudaGetLastError() == cudaSuccess ? 1 : -1;
+    }
     if (!make_tile_map(&mq, a.q, d.B, d.T, d.H) || !make_tile_map(&mk, a.k, d.B, d.T, d.H) ||
         !make_tile_map(&mv, a.v, d.B, d.T, d.H) || !make_tile_map(&mo, a.o, d.B, d.T, d.H))
         return -1;
@@ -499,7 +534,7 @@ int gla_tc_forward(const Dims &d, const FwdArgs &a, uint8_t *simg, int *status, 
         launches = 2;
         simg = nullptr;
     }
-    FwdParams p{a.lq, a.lk, a.h0, fin, gam, (__nv_bfloat16 *)a.o, a.ht, simg, status, d.T, d.H, d.NT, P, L, d.scale, retnet ? a.log_decay : nullptr};
+    FwdParams p{a.lq, a.lk, a.h0, fin, gam, (__nv_bfloat16 *)a.o, a.ht, simg, status, d.T, d.H, d.NT, P, L, d.scale, retnet ? a.log_decay : nullptr, nullptr, nullptr};
     k_gla_fwd_tc<<<d.B * d.H * P, NTHREADS, SMEM_BYTES, st>>>(mq, mk, mv, mg, mo, p);
     tr.mark("gla_fwd_tc");
     return cudaGetLastError() == cudaSuccess ? launches : -1;

@@ -85,6 +85,27 @@ inline bool make_tile_map(CUtensorMap *m, const void *ptr, int B, int T, int H) 
     return r == CUDA_SUCCESS;
 }
 
+// Device array of the per-sequence tensor maps of region r of a packed batch: `make(seq, maps)` encodes one sequence's
+// maps.  They are encoded and uploaded (stream-ordered, from a pinned mirror) only when `key`, the tensors they point
+// at, differs from the last call's; a training loop that reuses its buffers encodes once.  nullptr on failure.
+template <class Make>
+inline const CUtensorMap *varlen_maps(Varlen &vl, int r, const void *const *key, int nkey, cudaStream_t st, Make make) {
+    Varlen::Region &g = vl.reg[r];
+    bool same = g.valid;
+    for (int i = 0; i < nkey && same; ++i) same = g.key[i] == key[i];
+    if (same) return g.dev;
+    g.valid = false;
+    if (cudaEventSynchronize(g.uploaded) != cudaSuccess) return nullptr;      // the mirror's last upload has been read
+    for (int s = 0; s < vl.n_seq; ++s)
+        if (!make(vl.seqs[s], g.host + (size_t)s * Varlen::MAPS_PER_SEQ)) return nullptr;
+    const size_t bytes = (size_t)vl.n_seq * Varlen::MAPS_PER_SEQ * sizeof(CUtensorMap);
+    if (cudaMemcpyAsync(g.dev, g.host, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return nullptr;
+    if (cudaEventRecord(g.uploaded, st) != cudaSuccess) return nullptr;
+    for (int i = 0; i < nkey; ++i) g.key[i] = key[i];
+    g.valid = true;
+    return g.dev;
+}
+
 // Head-softmax gates (Eq. 4) of one token for head h: returns (Gq_h, Gk_h).
 __device__ __forceinline__ float2 head_gates(const float *lq, const float *lk, int H, int h) {
     float m1 = -INFINITY, m2 = -INFINITY;

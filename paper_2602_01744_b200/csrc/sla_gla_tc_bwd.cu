@@ -57,6 +57,8 @@ struct StatesParams {
     int T, H, NT;
     int P, L;               // segments per sequence and chunks per segment (image mode: P = 1, L = NT)
     const float *log_gamma; // Softmax-RetNet: [H] constant log-decays (no log-decay tensor is read); else nullptr
+    const SeqInfo *seqs;    // packed variable-length batch: per-sequence table and tensor maps (k, v, g), else nullptr
+    const CUtensorMap *vmaps;
 };
 
 // thread (row, colhalf) holds 32 consecutive state values of its row: bf16 them into the operand image
@@ -78,15 +80,27 @@ __device__ __forceinline__ void store_state_part(uint8_t *img, int row, int colh
 // sequence from a zero state and leaves only where it ended and the segment's total decay; a scan over the segments
 // then gives every segment its true starting state.
 __global__ void __launch_bounds__(st1::NTHREADS, 1)
-k_gla_states_tc(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
-                const __grid_constant__ CUtensorMap tm_g, StatesParams p) {
+k_gla_states_tc(const __grid_constant__ CUtensorMap gm_k, const __grid_constant__ CUtensorMap gm_v,
+                const __grid_constant__ CUtensorMap gm_g, StatesParams p) {
     using namespace st1;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t *sm = smem_raw + (base - raw);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int bh = blockIdx.x / p.P, seg = blockIdx.x % p.P, b = bh / p.H, h = bh % p.H;
+    const int bh = blockIdx.x / p.P, seg = blockIdx.x % p.P, h = bh % p.H;
+    int b = bh / p.H;
+    size_t tokb = (size_t)b * p.T, slot = (size_t)bh * (p.NT + 1);
+    const CUtensorMap *vm = nullptr;
+    if (p.seqs) {                                           // packed batch: see k_gla_fwd_tc
+        const SeqInfo si = p.seqs[b];
+        vm = p.vmaps + (size_t)b * Varlen::MAPS_PER_SEQ;
+        p.T = si.T; p.NT = si.NT; p.L = si.NT;
+        tokb = (size_t)si.t0;
+        slot = (size_t)si.slot0 * p.H + (size_t)h * (si.NT + 1);
+        b = 0;
+    }
+    const CUtensorMap &tm_k = vm ? vm[0] : gm_k, &tm_v = vm ? vm[1] : gm_v, &tm_g = vm ? vm[2] : gm_g;
     const int n0 = seg * p.L, NT = min(p.L, p.NT - n0);     // this CTA's chunks: n0 .. n0+NT-1
     const bool images = p.simg != nullptr;
     auto bar = [&](int i) { return base + OFF_BAR + 8u * i; };
@@ -118,8 +132,7 @@ k_gla_states_tc(const __grid_constant__ CUtensorMap tm_k, const __grid_constant_
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *reinterpret_cast<volatile uint32_t *>(sm + OFF_TMEM);
-    const size_t tokb = (size_t)b * p.T;
-    uint8_t *img0 = p.simg + (size_t)bh * (NT + 1) * STATE_BF16;      // (image mode: one segment, NT = p.NT)
+    uint8_t *img0 = p.simg + slot * STATE_BF16;                       // (image mode: one segment, NT = p.NT)
 
     if (warp == 8) {
         // ---------------- MMA issue (one lane) ----------------
@@ -321,6 +334,8 @@ struct BwdParams {
     int T, H, NT;
     float scale;
     const float *log_gamma;         // Softmax-RetNet: [H] constant log-decays (no log-decay read, no log-decay gradient)
+    const SeqInfo *seqs;            // packed variable-length batch: per-sequence table and tensor maps (the nine below), else nullptr
+    const CUtensorMap *vmaps;
 };
 
 // Sum v[j] over the 32 lanes for every j: afterwards lane l holds the total of v[l] in v[0].
@@ -344,18 +359,32 @@ __device__ __forceinline__ float warp_transpose_sum(float (&v)[32], int lane) {
 // with the masked tiles wait for the mask.  All four gradient tensors leave through staged TMA stores (rows past T
 // are clipped by the tensor map).
 __global__ void __launch_bounds__(st2::NTHREADS, 1)
-k_gla_bwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-             const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
-             const __grid_constant__ CUtensorMap tm_g, const __grid_constant__ CUtensorMap tm_dq,
-             const __grid_constant__ CUtensorMap tm_dk, const __grid_constant__ CUtensorMap tm_dv,
-             const __grid_constant__ CUtensorMap tm_dg, BwdParams p) {
+k_gla_bwd_tc(const __grid_constant__ CUtensorMap gm_q, const __grid_constant__ CUtensorMap gm_k,
+             const __grid_constant__ CUtensorMap gm_v, const __grid_constant__ CUtensorMap gm_do,
+             const __grid_constant__ CUtensorMap gm_g, const __grid_constant__ CUtensorMap gm_dq,
+             const __grid_constant__ CUtensorMap gm_dk, const __grid_constant__ CUtensorMap gm_dv,
+             const __grid_constant__ CUtensorMap gm_dg, BwdParams p) {
     using namespace st2;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t *sm = smem_raw + (base - raw);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int bh = blockIdx.x, b = bh / p.H, h = bh % p.H;
+    const int bh = blockIdx.x, h = bh % p.H;
+    int b = bh / p.H;
+    size_t tokb = (size_t)b * p.T, slot = (size_t)bh * (p.NT + 1);
+    const CUtensorMap *vm = nullptr;
+    if (p.seqs) {                                           // packed batch: see k_gla_fwd_tc
+        const SeqInfo si = p.seqs[b];
+        vm = p.vmaps + (size_t)b * Varlen::MAPS_PER_SEQ;
+        p.T = si.T; p.NT = si.NT;
+        tokb = (size_t)si.t0;
+        slot = (size_t)si.slot0 * p.H + (size_t)h * (si.NT + 1);
+        b = 0;
+    }
+    const CUtensorMap &tm_q = vm ? vm[0] : gm_q, &tm_k = vm ? vm[1] : gm_k, &tm_v = vm ? vm[2] : gm_v,
+                      &tm_do = vm ? vm[3] : gm_do, &tm_g = vm ? vm[4] : gm_g, &tm_dq = vm ? vm[5] : gm_dq,
+                      &tm_dk = vm ? vm[6] : gm_dk, &tm_dv = vm ? vm[7] : gm_dv, &tm_dg = vm ? vm[8] : gm_dg;
     auto bar = [&](int i) { return base + OFF_BAR + 8u * i; };
     float *tot = reinterpret_cast<float *>(sm + OFF_TOT);
     float *eblast = reinterpret_cast<float *>(sm + OFF_EB);
@@ -394,8 +423,7 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *reinterpret_cast<volatile uint32_t *>(sm + OFF_TMEM);
-    const size_t tokb = (size_t)b * p.T;
-    const uint8_t *img0 = p.simg + (size_t)bh * (p.NT + 1) * STATE_BF16;
+    const uint8_t *img0 = p.simg + slot * STATE_BF16;
     const int NT = p.NT;
     // chunks are visited in the order n = NT-1 ... 0; k = NT-1-n is the visit number that drives every barrier parity
 
@@ -856,9 +884,14 @@ int gate_bwd_prod(const float *lq, const float *lk, const float *pq, const float
     return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 
-size_t gla_tc_backward_workspace_bytes(const Dims &d) {
+// state slots (one per chunk plus one per sequence) over all (sequence, head) pairs
+static size_t state_slots(const Dims &d, const Varlen *vl) {
+    return (vl && vl->n_seq) ? (size_t)vl->slots * d.H : (size_t)d.B * d.H * (d.NT + 1);
+}
+
+size_t gla_tc_backward_workspace_bytes(const Dims &d, const Varlen *vl) {
     const size_t bth = (size_t)d.B * d.T * d.H;
-    return (size_t)d.B * d.H * (d.NT + 1) * STATE_BF16 + 2 * ((bth + 63) & ~(size_t)63) * sizeof(float);
+    return state_slots(d, vl) * STATE_BF16 + 2 * ((bth + 63) & ~(size_t)63) * sizeof(float);
 }
 
 int gla_tc_segment_summaries(const Dims &d, const FwdArgs &a, int P, int L, float *fin, float *gam, int *status,
@@ -868,7 +901,8 @@ int gla_tc_segment_summaries(const Dims &d, const FwdArgs &a, int P, int L, floa
     if (!make_tile_map(&mk, a.k, d.B, d.T, d.H) || !make_tile_map(&mv, a.v, d.B, d.T, d.H)) return -1;
     if (retnet) mg = mk;   // (never used: the decay is generated in the kernel)
     else if (!make_map(&mg, a.log_decay, d.B, d.T, d.H, d.dk, true, 128)) return -1;
-    StatesParams sp{a.lq, a.lk, nullptr, nullptr, fin, gam, status, d.T, d.H, d.NT, P, L, retnet ? a.log_decay : nullptr};
+    StatesParams sp{a.lq, a.lk, nullptr, nullptr, fin, gam, status, d.T, d.H, d.NT, P, L, retnet ? a.log_decay : nullptr,
+                    nullptr, nullptr};
     k_gla_states_tc<<<d.B * d.H * P, st1::NTHREADS, st1::SMEM_BYTES, st>>>(mk, mv, mg, sp);
     tr.mark("gla_segment_states_tc");
     return cudaGetLastError() == cudaSuccess ? 1 : -1;
@@ -889,19 +923,53 @@ int gla_tc_backward(const Dims &d, const BwdArgs &a, bool have_states, int *stat
              !make_map(&mdg, a.dlog_decay, d.B, d.T, d.H, d.dk, true, 128))
         return -1;
     // workspace: state images, then the two [B,T,H] gate products
+    Varlen *vl = (a.vl && a.vl->n_seq) ? a.vl : nullptr;
     const size_t bth = (size_t)d.B * d.T * d.H;
-    const size_t img_floats = (size_t)d.B * d.H * (d.NT + 1) * (STATE_BF16 / 4);
+    const size_t img_floats = state_slots(d, vl) * (STATE_BF16 / 4);
     uint8_t *simg = reinterpret_cast<uint8_t *>(a.ws);
     float *pq = a.ws + img_floats;
     float *pk = pq + ((bth + 63) & ~(size_t)63);
+    const int ctas = vl ? vl->n_seq * d.H : d.B * d.H;
+    const SeqInfo *dseqs = vl ? vl->d_seqs : nullptr;
+    const __nv_bfloat16 *q = (const __nv_bfloat16 *)a.q, *k = (const __nv_bfloat16 *)a.k, *v = (const __nv_bfloat16 *)a.v,
+                        *dO = (const __nv_bfloat16 *)a.dO;
 
     if (!have_states) {   // (otherwise the forward pass of the same inputs has left the images in this workspace)
-        StatesParams sp{a.lq, a.lk, a.h0, simg, nullptr, nullptr, status, d.T, d.H, d.NT, 1, d.NT, retnet ? a.log_decay : nullptr};
-        k_gla_states_tc<<<d.B * d.H, st1::NTHREADS, st1::SMEM_BYTES, st>>>(mk, mv, mg, sp);
+        const CUtensorMap *vm = nullptr;
+        if (vl) {
+            const void *key[] = {a.k, a.v, a.log_decay};
+            vm = varlen_maps(*vl, 1, key, 3, st, [&](const SeqInfo &si, CUtensorMap *m) {
+                const size_t off = (size_t)si.t0 * d.H * D;
+                if (!make_tile_map(m + 0, k + off, 1, si.T, d.H) || !make_tile_map(m + 1, v + off, 1, si.T, d.H)) return false;
+                if (retnet) { m[2] = m[0]; return true; }
+                return make_map(m + 2, a.log_decay + off, 1, si.T, d.H, d.dk, true, 128);
+            });
+            if (!vm) return -1;
+        }
+        StatesParams sp{a.lq, a.lk, a.h0, simg, nullptr, nullptr, status, d.T, d.H, d.NT, 1, d.NT, retnet ? a.log_decay : nullptr,
+                        dseqs, vm};
+        k_gla_states_tc<<<ctas, st1::NTHREADS, st1::SMEM_BYTES, st>>>(mk, mv, mg, sp);
         tr.mark("gla_states_tc");
     }
-    BwdParams bp{a.lq, a.lk, a.dht, simg, pq, pk, a.dh0, status, d.T, d.H, d.NT, d.scale, retnet ? a.log_decay : nullptr};
-    k_gla_bwd_tc<<<d.B * d.H, st2::NTHREADS, st2::SMEM_BYTES, st>>>(mq, mk, mv, mdo, mg, mdq, mdk, mdv, mdg, bp);
+    const CUtensorMap *vm = nullptr;
+    if (vl) {
+        const void *key[] = {a.q, a.k, a.v, a.dO, a.log_decay, a.dq, a.dk, a.dv, a.dlog_decay};
+        vm = varlen_maps(*vl, 2, key, 9, st, [&](const SeqInfo &si, CUtensorMap *m) {
+            const size_t off = (size_t)si.t0 * d.H * D;
+            if (!make_tile_map(m + 0, q + off, 1, si.T, d.H) || !make_tile_map(m + 1, k + off, 1, si.T, d.H) ||
+                !make_tile_map(m + 2, v + off, 1, si.T, d.H) || !make_tile_map(m + 3, dO + off, 1, si.T, d.H) ||
+                !make_tile_map(m + 5, (__nv_bfloat16 *)a.dq + off, 1, si.T, d.H) ||
+                !make_tile_map(m + 6, (__nv_bfloat16 *)a.dk + off, 1, si.T, d.H) ||
+                !make_tile_map(m + 7, (__nv_bfloat16 *)a.dv + off, 1, si.T, d.H))
+                return false;
+            if (retnet) { m[4] = m[0]; m[8] = m[5]; return true; }
+            return make_map(m + 4, a.log_decay + off, 1, si.T, d.H, d.dk, true, 128) &&
+                   make_map(m + 8, a.dlog_decay + off, 1, si.T, d.H, d.dk, true, 128);
+        });
+        if (!vm) return -1;
+    }
+    BwdParams bp{a.lq, a.lk, a.dht, simg, pq, pk, a.dh0, status, d.T, d.H, d.NT, d.scale, retnet ? a.log_decay : nullptr, dseqs, vm};
+    k_gla_bwd_tc<<<ctas, st2::NTHREADS, st2::SMEM_BYTES, st>>>(mq, mk, mv, mdo, mg, mdq, mdk, mdv, mdg, bp);
     tr.mark("gla_bwd_tc");
     if (gate_bwd_prod(a.lq, a.lk, pq, pk, a.dlq, a.dlk, (long)d.B * d.T, d.H, st) < 0) return -1;
     tr.mark("gate_bwd");

@@ -1,5 +1,6 @@
 // Internal declarations shared by the host API and the kernel translation units.
 #pragma once
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
 #include <stdint.h>
@@ -20,6 +21,28 @@ struct Dims {
     int io_bf16;      // 1: q,k,v,o are bf16, 0: fp32
     int B, T, H, dk, dv, C, NT;
     float scale;
+};
+
+// Packed variable-length batches (B = 1: sequences one after another along T, the state reset at every boundary,
+// chunks cut from each sequence's own start).  Per sequence: first token, length, chunks, and the index of its first
+// state slot (the sum of chunks + 1 over the sequences before it).
+struct SeqInfo { int t0, T, NT, slot0; };
+// Host side of a plan's sequence table.  The tensor-core kernels address a sequence through tensor maps of its own
+// (based at its first token, T = its length: loads past its end read zeros, stores are clipped there, exactly as at the
+// end of a batch row); those live in device arrays, one region per kernel kind, encoded again only when the tensors
+// they point at change.
+struct Varlen {
+    int n_seq = 0;
+    long slots = 0;                     // sum over the sequences of (chunks + 1)
+    std::vector<SeqInfo> seqs;
+    SeqInfo *d_seqs = nullptr;
+    struct Region {
+        CUtensorMap *dev = nullptr, *host = nullptr;    // [n_seq][MAPS_PER_SEQ]; host: pinned mirror
+        const void *key[10] = {};
+        bool valid = false;
+        cudaEvent_t uploaded = nullptr;
+    } reg[3];                           // 0: forward, 1: state / record sweep, 2: gradient sweep
+    static constexpr int MAPS_PER_SEQ = 9;
 };
 
 // Carve-up of the caller's workspace (all fp32, offsets in floats, each 64-float aligned).
@@ -46,6 +69,7 @@ struct FwdArgs {
     float *ht;
     float *ws;
     int *status;            // the plan's device status word
+    Varlen *vl = nullptr;   // packed variable-length batch (tensor-core kernels only), else nullptr
 };
 struct BwdArgs {
     const void *q, *k, *v;
@@ -56,6 +80,7 @@ struct BwdArgs {
     float *dlog_decay, *dbeta, *dlq, *dlk, *dh0;
     float *ws;
     int *status;
+    Varlen *vl = nullptr;
 };
 struct DecArgs {
     const void *q, *k, *v;
@@ -106,7 +131,7 @@ bool gla_tc_supported(const Dims &d);
 int gla_tc_configure();
 // With `simg` not null (and gla_tc_forward_can_save) the forward also leaves the bf16 image of the state before every
 // chunk there, in the layout the gradient sweep reads: the backward pass of the same inputs then needs no state sweep.
-bool gla_tc_forward_can_save(const Dims &d);
+bool gla_tc_forward_can_save(const Dims &d, const Varlen *vl = nullptr);
 uint8_t *gla_tc_state_images(float *ws);   // where in the backward workspace the images sit
 int gla_tc_forward(const Dims &d, const FwdArgs &a, uint8_t *simg, int *status, cudaStream_t st, Tracer &tr);
 // Backward: chunk-state sweep, gradient sweep, gate softmax backward.  Needs the first
@@ -117,8 +142,8 @@ int gla_tc_bwd_configure();
 int gla_tc_segment_summaries(const Dims &d, const FwdArgs &a, int P, int L, float *fin, float *gam, int *status,
                              cudaStream_t st, Tracer &tr);
 // Bytes of workspace the tensor-core forward / backward need (the generic kernels need more).
-size_t gla_tc_forward_workspace_bytes(const Dims &d);
-size_t gla_tc_backward_workspace_bytes(const Dims &d);
+size_t gla_tc_forward_workspace_bytes(const Dims &d, const Varlen *vl = nullptr);
+size_t gla_tc_backward_workspace_bytes(const Dims &d, const Varlen *vl = nullptr);
 int gla_tc_backward(const Dims &d, const BwdArgs &a, bool have_states, int *status, cudaStream_t st, Tracer &tr);
 
 // ---- tensor-core Softmax-GatedDeltaNet forward (WY form): sla_gdn_tc.cu.  Needs no workspace. ----
@@ -129,7 +154,7 @@ uint8_t *gdn_tc_records(float *ws);        // where in the backward workspace th
 int gdn_tc_forward_save(const Dims &d, const FwdArgs &a, uint8_t *save, int *status, cudaStream_t st, Tracer &tr);
 // backward: forward sweep in save mode (per-chunk S_n, U, T records), reverse gradient sweep, gate softmax backward
 int gdn_tc_bwd_configure();
-size_t gdn_tc_backward_workspace_bytes(const Dims &d);
+size_t gdn_tc_backward_workspace_bytes(const Dims &d, const Varlen *vl = nullptr);
 int gdn_tc_backward(const Dims &d, const BwdArgs &a, bool have_records, int *status, cudaStream_t st, Tracer &tr);
 int gate_bwd_prod(const float *lq, const float *lk, const float *pq, const float *pk, float *dlq, float *dlk, long n_tok,
                   int H, cudaStream_t st);
@@ -170,6 +195,7 @@ struct sla_plan {
                    *lk = nullptr, *h0 = nullptr;
         void *stream = nullptr;
     } saved;
+    sla::Varlen varlen;     // sla_plan_set_sequences: packed variable-length batch (n_seq == 0: regular batch)
     sla::Tracer tracer;
     std::vector<std::pair<const char *, std::pair<int, float>>> agg;   // name -> (launches, total ms)
 };
