@@ -588,7 +588,7 @@ def main():
 
     if rank == 0:
         cpu = None
-        if world == 1 and not args.no_cpu_baseline:
+        if world == 1 and not args.no_cpu_baseline and packed_cu is None:
             tokens, times, cores = cpu_oracle_sample(cfg, x, steps=1)
             cpu = {"value": tokens / times[0], "unit": UNIT, "cores": cores, "kind": "oracle",
                    "sample": f"first {min(CPU_ROWS, cfg.B)} batch rows of {WORKLOAD} (T={cfg.T}, H={cfg.H}), {passes}, "

@@ -55,13 +55,16 @@ template <> struct Vec<__nv_bfloat16> {
 
 constexpr int TOKS = 4;          // tokens a CTA handles between two barriers of the forward pass
 
-// Forward.  grid (CTAs, 2 sides); blockDim = H*d/N threads rounded up to whole warps.
-template <typename TIO>
+// Forward.  grid (CTAs, 2 sides); blockDim = H*d/N threads rounded up to whole warps.  A head's d/N partial dots sit in
+// d/N consecutive threads: when that is a power of two (<= 32) they are folded with shuffles and every warp streams on
+// its own, SHFL tokens in flight; otherwise they meet in shared memory, TOKS tokens per barrier pair.
+template <typename TIO, bool SHFL>
 __global__ void k_gate_scores_fwd(long n_tok, int H, int d, const TIO *__restrict__ q, const TIO *__restrict__ k,
                                   const float *__restrict__ Wq, const float *__restrict__ Wk,
                                   float *__restrict__ lq, float *__restrict__ lk) {
     constexpr int N = Vec<TIO>::N;
-    extern __shared__ float part[];                  // [TOKS][blockDim.x] partial dots
+    constexpr int NT = TOKS;                         // tokens per block of loads
+    extern __shared__ float part[];                  // [TOKS][blockDim.x] partial dots (not used with SHFL)
     const TIO *x = blockIdx.y ? k : q;
     const float *W = blockIdx.y ? Wk : Wq;
     float *out = blockIdx.y ? lk : lq;
@@ -74,28 +77,37 @@ __global__ void k_gate_scores_fwd(long n_tok, int H, int d, const TIO *__restric
     for (int e = 0; e < N; ++e) w[e] = live ? __ldg(W + (size_t)(c0 + e) * H + h) : 0.f;
     const long per = (n_tok + gridDim.x - 1) / gridDim.x;
     const long t0 = (long)blockIdx.x * per, t1 = min(n_tok, t0 + per);
-    for (long t = t0; t < t1; t += TOKS) {
+    for (long t = t0; t < t1; t += NT) {
+        float xv[NT][N];
 #pragma unroll
-        for (int s = 0; s < TOKS; ++s) {
+        for (int s = 0; s < NT; ++s)                 // all loads of the block in flight at once
+            if (live && t + s < t1) Vec<TIO>::load(x + ((size_t)(t + s) * H) * d + (size_t)tid * N, xv[s]);
+#pragma unroll
+        for (int s = 0; s < NT; ++s) {
             float acc = 0.f;
             if (live && t + s < t1) {
-                float xv[N];
-                Vec<TIO>::load(x + ((size_t)(t + s) * H) * d + (size_t)tid * N, xv);
 #pragma unroll
-                for (int e = 0; e < N; ++e) acc = fmaf(xv[e], w[e], acc);
+                for (int e = 0; e < N; ++e) acc = fmaf(xv[s][e], w[e], acc);
             }
-            part[s * blockDim.x + tid] = acc;
-        }
-        __syncthreads();
-        if (tid < TOKS * H) {                        // one thread per (token slot, head): the head's vpr partial dots
-            const int s = tid / H, hh = tid % H;
-            if (t + s < t1) {
-                float acc = 0.f;
-                for (int j = 0; j < vpr; ++j) acc += part[s * blockDim.x + hh * vpr + j];
-                out[(t + s) * H + hh] = acc;
+            if (SHFL) {
+                for (int o = vpr >> 1; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+                if (live && t + s < t1 && tid % vpr == 0) out[(t + s) * H + h] = acc;
+            } else {
+                part[s * blockDim.x + tid] = acc;
             }
         }
-        __syncthreads();
+        if (!SHFL) {
+            __syncthreads();
+            if (tid < NT * H) {                      // one thread per (token slot, head): the head's vpr partial dots
+                const int s = tid / H, hh = tid % H;
+                if (t + s < t1) {
+                    float acc = 0.f;
+                    for (int j = 0; j < vpr; ++j) acc += part[s * blockDim.x + hh * vpr + j];
+                    out[(t + s) * H + hh] = acc;
+                }
+            }
+            __syncthreads();
+        }
     }
 }
 
@@ -122,35 +134,46 @@ __global__ void k_gate_scores_bwd(long n_tok, int H, int d, const TIO *__restric
     }
     const long per = (n_tok + gridDim.x - 1) / gridDim.x;
     const long t0 = (long)blockIdx.x * per, t1 = min(n_tok, t0 + per);
-#pragma unroll 4
-    for (long t = t0; t < t1; ++t) {
-        const size_t off = ((size_t)t * H) * d + (size_t)tid * N;
-        float xv[N], gv[N];
-        Vec<TIO>::load(x + off, xv);
-        Vec<TIO>::load_rw(dx + off, gv);
-        const float g = __ldg(dl + t * H + h);
+    constexpr int UNR = 4;       // tokens whose loads are all in flight before the first store (the compiler may not
+                                 // move a load of dx above a store to dx on its own)
+    for (long t = t0; t < t1; t += UNR) {
+        float xv[UNR][N], gv[UNR][N], g[UNR];
 #pragma unroll
-        for (int e = 0; e < N; ++e) {
-            acc[e] = fmaf(g, xv[e], acc[e]);
-            gv[e] = fmaf(g, w[e], gv[e]);
-        }
-        Vec<TIO>::store(dx + off, gv);
+        for (int s = 0; s < UNR; ++s)
+            if (t + s < t1) {
+                const size_t off = ((size_t)(t + s) * H) * d + (size_t)tid * N;
+                Vec<TIO>::load(x + off, xv[s]);
+                Vec<TIO>::load_rw(dx + off, gv[s]);
+                g[s] = __ldg(dl + (t + s) * H + h);
+            }
+#pragma unroll
+        for (int s = 0; s < UNR; ++s)
+            if (t + s < t1) {
+#pragma unroll
+                for (int e = 0; e < N; ++e) {
+                    acc[e] = fmaf(g[s], xv[s][e], acc[e]);
+                    gv[s][e] = fmaf(g[s], w[e], gv[s][e]);
+                }
+                Vec<TIO>::store(dx + ((size_t)(t + s) * H) * d + (size_t)tid * N, gv[s]);
+            }
     }
     float *dst = partial + ((size_t)blockIdx.y * gridDim.x + blockIdx.x) * nvec * N + (size_t)tid * N;
 #pragma unroll
     for (int e = 0; e < N; ++e) dst[e] = acc[e];
 }
 
-// dW[c,h] = sum over the CTAs' partial sums (stored [h][c]), in CTA order.  grid (ceil(H*d/256), 2 sides).
+// dW[c,h] = sum over the CTAs' partial sums (stored [h][c]): one warp per element, lane l adds the partials of CTAs
+// l, l+32, .. in order, then the lanes are folded in a fixed tree - the same bits on every run.  grid (H*d/8, 2 sides).
 __global__ void k_gate_scores_dw(int n_cta, int H, int d, const float *__restrict__ partial, float *__restrict__ dWq,
                                  float *__restrict__ dWk) {
-    const int i = blockIdx.x * blockDim.x + threadIdx.x, n = H * d;
+    const int i = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31, n = H * d;
     if (i >= n) return;
     const float *src = partial + (size_t)blockIdx.y * n_cta * n + i;
     float acc = 0.f;
-    for (int c = 0; c < n_cta; ++c) acc += src[(size_t)c * n];
-    const int h = i / d, cc = i % d;
-    (blockIdx.y ? dWk : dWq)[(size_t)cc * H + h] = acc;
+    for (int c = lane; c < n_cta; c += 32) acc += src[(size_t)c * n];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if (lane == 0) (blockIdx.y ? dWk : dWq)[(size_t)(i % d) * H + i / d] = acc;
 }
 
 int score_ctas(long n_tok) {
@@ -172,12 +195,13 @@ int gate_scores_forward(const Dims &d, const void *q, const void *k, const float
     const int N = d.io_bf16 ? 8 : 4, threads = ((d.H * d.dk / N) + 31) / 32 * 32;
     dim3 grid(score_ctas(n_tok), 2);
     const size_t smem = (size_t)TOKS * threads * sizeof(float);
-    if (d.io_bf16)
-        k_gate_scores_fwd<__nv_bfloat16><<<grid, threads, smem, st>>>(n_tok, d.H, d.dk, (const __nv_bfloat16 *)q,
-                                                                      (const __nv_bfloat16 *)k, Wq, Wk, lq, lk);
-    else
-        k_gate_scores_fwd<float><<<grid, threads, smem, st>>>(n_tok, d.H, d.dk, (const float *)q, (const float *)k, Wq, Wk,
-                                                              lq, lk);
+    const int vpr = d.dk / N;
+    const bool shfl = vpr <= 32 && (vpr & (vpr - 1)) == 0;
+#define SLA_SCORES_FWD(TIO, SH) \
+    k_gate_scores_fwd<TIO, SH><<<grid, threads, SH ? 0 : smem, st>>>(n_tok, d.H, d.dk, (const TIO *)q, (const TIO *)k, Wq, Wk, lq, lk)
+    if (d.io_bf16) { if (shfl) SLA_SCORES_FWD(__nv_bfloat16, true); else SLA_SCORES_FWD(__nv_bfloat16, false); }
+    else { if (shfl) SLA_SCORES_FWD(float, true); else SLA_SCORES_FWD(float, false); }
+#undef SLA_SCORES_FWD
     tr.mark("gate_scores_fwd");
     return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
@@ -197,7 +221,7 @@ int gate_scores_backward(const Dims &d, const void *q, const void *k, const floa
         k_gate_scores_bwd<float><<<grid, threads, 0, st>>>(n_tok, d.H, d.dk, (const float *)q, (const float *)k, Wq, Wk, dlq,
                                                            dlk, (float *)dq, (float *)dk, ws);
     tr.mark("gate_scores_bwd");
-    dim3 g2((d.H * d.dk + 255) / 256, 2);
+    dim3 g2((d.H * d.dk + 7) / 8, 2);
     k_gate_scores_dw<<<g2, 256, 0, st>>>(ctas, d.H, d.dk, ws, dWq, dWk);
     tr.mark("gate_scores_dw");
     return cudaGetLastError() == cudaSuccess ? 2 : -1;

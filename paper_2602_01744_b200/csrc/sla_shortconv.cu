@@ -73,8 +73,10 @@ __device__ __forceinline__ void load_x(const TIO *row0, int t, size_t stride, bo
     }
 }
 
-template <typename TIO, bool NORM>
-__global__ void __launch_bounds__(256)
+// SHFL: a head's d/N vectors sit in d/N consecutive lanes of one warp (a power of two <= 32), so the per-head sums of
+// the normalisation are folded with shuffles and the warps run free of each other; otherwise through shared memory.
+template <typename TIO, bool NORM, bool SHFL>
+__global__ void __launch_bounds__(256, 2)
 k_shortconv_fwd(ConvDims cd, const TIO *__restrict__ x, const float *__restrict__ w, TIO *__restrict__ out) {
     constexpr int N = V<TIO>::N;
     extern __shared__ float sm[];                       // part [TOKS][threads], rinv [TOKS][H]
@@ -96,23 +98,35 @@ k_shortconv_fwd(ConvDims cd, const TIO *__restrict__ x, const float *__restrict_
     for (int t = t0; t < t1; t += TOKS) {
         float z[TOKS][N];
 #pragma unroll
+        for (int s = 0; s < TOKS; ++s)                  // all loads of the block in flight at once
+            if (t + s < t1) load_x<TIO, N>(xr, t + s, C, live, z[s]);
+#pragma unroll
         for (int s = 0; s < TOKS; ++s) {
             float ss = 0.f;
             if (t + s < t1) {
-                float xc[N];
-                load_x<TIO, N>(xr, t + s, C, live, xc);
 #pragma unroll
                 for (int e = 0; e < N; ++e) {
-                    const float y = fmaf(wt[0][e], xm3[e], fmaf(wt[1][e], xm2[e], fmaf(wt[2][e], xm1[e], wt[3][e] * xc[e])));
-                    z[s][e] = y / (1.f + __expf(-y));
+                    const float xc = z[s][e];
+                    const float y = fmaf(wt[0][e], xm3[e], fmaf(wt[1][e], xm2[e], fmaf(wt[2][e], xm1[e], wt[3][e] * xc)));
+                    z[s][e] = __fdividef(y, 1.f + __expf(-y));
                     ss = fmaf(z[s][e], z[s][e], ss);
-                    xm3[e] = xm2[e]; xm2[e] = xm1[e]; xm1[e] = xc[e];
+                    xm3[e] = xm2[e]; xm2[e] = xm1[e]; xm1[e] = xc;
                 }
                 if (!NORM && live) V<TIO>::store(orow + (size_t)(t + s) * C, z[s]);
             }
-            if (NORM) part[s * blockDim.x + tid] = ss;
+            if (NORM && SHFL) {
+                for (int o = vpr >> 1; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+                if (live && t + s < t1) {
+                    const float r = 1.f / sqrtf(ss + cd.eps);
+#pragma unroll
+                    for (int e = 0; e < N; ++e) z[s][e] *= r;
+                    V<TIO>::store(orow + (size_t)(t + s) * C, z[s]);
+                }
+            } else if (NORM) {
+                part[s * blockDim.x + tid] = ss;
+            }
         }
-        if (NORM) {
+        if (NORM && !SHFL) {
             __syncthreads();
             if (tid < TOKS * nh) {                      // one thread per (token slot, head)
                 const int s = tid / nh, hh = tid % nh;
@@ -134,8 +148,8 @@ k_shortconv_fwd(ConvDims cd, const TIO *__restrict__ x, const float *__restrict_
 }
 
 // Reverse pass.  partial: [CTAs][H*d][KMAX] per-CTA sums of the tap gradients.
-template <typename TIO, bool NORM>
-__global__ void __launch_bounds__(256)
+template <typename TIO, bool NORM, bool SHFL>
+__global__ void __launch_bounds__(256, 2)
 k_shortconv_bwd(ConvDims cd, const TIO *__restrict__ x, const float *__restrict__ w, const TIO *__restrict__ dout,
                 TIO *__restrict__ dx, float *__restrict__ partial) {
     constexpr int N = V<TIO>::N;
@@ -161,11 +175,13 @@ k_shortconv_bwd(ConvDims cd, const TIO *__restrict__ x, const float *__restrict_
         for (int j = 0; j < KMAX; ++j) acc[j][e] = 0.f;
     }
     for (int top = ue; top >= t0; top -= TOKB) {
-        float zs[TOKB][N], gs[TOKB][N], dz[TOKB][N];
+        float zs[TOKB][N], gs[TOKB][N], dz[TOKB][N], fa_r[TOKB], fb_r[TOKB];
 #pragma unroll
         for (int s = 0; s < TOKB; ++s) {
             const int u = top - s;
             float ss = 0.f, dot = 0.f;
+            fa_r[s] = 1.f;
+            fb_r[s] = 0.f;
             if (u >= t0) {
                 float x0[N], x1[N], x2[N], x3[N];
                 load_x<TIO, N>(xr, u - 3, C, live, x0);
@@ -176,19 +192,27 @@ k_shortconv_bwd(ConvDims cd, const TIO *__restrict__ x, const float *__restrict_
 #pragma unroll
                 for (int e = 0; e < N; ++e) {
                     const float y = fmaf(wt[0][e], x0[e], fmaf(wt[1][e], x1[e], fmaf(wt[2][e], x2[e], wt[3][e] * x3[e])));
-                    const float sg = 1.f / (1.f + __expf(-y));
+                    const float sg = __fdividef(1.f, 1.f + __expf(-y));
                     zs[s][e] = y * sg;
                     gs[s][e] = sg * (1.f + y * (1.f - sg));         // d silu / dy
                     ss = fmaf(zs[s][e], zs[s][e], ss);
                     dot = fmaf(zs[s][e], dz[s][e], dot);
                 }
             }
-            if (NORM) {
+            if (NORM && SHFL) {         // out = z / r:  dz = dout / r - z (z . dout) / r^3, the head sums by shuffles
+                for (int o = vpr >> 1; o > 0; o >>= 1) {
+                    ss += __shfl_xor_sync(0xffffffffu, ss, o);
+                    dot += __shfl_xor_sync(0xffffffffu, dot, o);
+                }
+                const float r = sqrtf(ss + cd.eps);
+                fa_r[s] = 1.f / r;
+                fb_r[s] = dot / (r * r * r);
+            } else if (NORM) {
                 pss[s * blockDim.x + tid] = ss;
                 pdot[s * blockDim.x + tid] = dot;
             }
         }
-        if (NORM) {
+        if (NORM && !SHFL) {
             __syncthreads();
             if (tid < TOKB * nh) {
                 const int s = tid / nh, hh = tid % nh;
@@ -208,7 +232,7 @@ k_shortconv_bwd(ConvDims cd, const TIO *__restrict__ x, const float *__restrict_
             const int u = top - s;
             if (u < t0) continue;
             float dy[N], dxu[N];
-            const float fa = NORM ? ca[s * cd.hpc + h] : 1.f, fb = NORM ? cb[s * cd.hpc + h] : 0.f;
+            const float fa = !NORM ? 1.f : SHFL ? fa_r[s] : ca[s * cd.hpc + h], fb = !NORM ? 0.f : SHFL ? fb_r[s] : cb[s * cd.hpc + h];
 #pragma unroll
             for (int e = 0; e < N; ++e) {
                 dy[e] = (dz[s][e] * fa - zs[s][e] * fb) * gs[s][e];
@@ -237,22 +261,25 @@ k_shortconv_bwd(ConvDims cd, const TIO *__restrict__ x, const float *__restrict_
     }
 }
 
-// dw[c, j] = sum over the CTAs' partial sums, in CTA order
+// dw[c, j] = sum over the CTAs' partial sums: one warp per element, lane l adds the partials of CTAs l, l+32, .. in
+// order, then the lanes are folded in a fixed tree (same bits on every run)
 __global__ void k_shortconv_dw(int n_cta, int C, int K, const float *__restrict__ partial, float *__restrict__ dw) {
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    const int i = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
     if (i >= C * K) return;
     const int c = i / K, j = i % K + (KMAX - K);
     float acc = 0.f;
-    for (int n = 0; n < n_cta; ++n) acc += partial[((size_t)n * C + c) * KMAX + j];
-    dw[i] = acc;
+    for (int n = lane; n < n_cta; n += 32) acc += partial[((size_t)n * C + c) * KMAX + j];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if (lane == 0) dw[i] = acc;
 }
 
-int tokens_per_cta(const Dims &d) {       // about four CTAs per SM, slices of at least 64 tokens
+int tokens_per_cta(const Dims &d) {       // about four CTAs per SM, slices of at least 32 tokens
     int dev = 0, sms = 148;
     if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const long total = (long)d.B * d.T, want = 4L * sms;
     long per = (total + want - 1) / want;
-    if (per < 64) per = 64;
+    if (per < 32) per = 32;           // (the reverse pass recomputes three tokens beyond its slice)
     return (int)per;
 }
 
@@ -271,10 +298,18 @@ int shortconv_forward(const Dims &d, int width, int K, bool normalize, float eps
     ConvDims cd{d.T, d.H, width, K, tokens_per_cta(d), hpc, eps};
     dim3 grid((d.T + cd.per - 1) / cd.per, d.B, (d.H + hpc - 1) / hpc);
     const size_t smem = (size_t)(TOKS * threads + TOKS * hpc) * sizeof(float);
-#define SLA_LAUNCH_FWD(TIO, NORM) \
-    k_shortconv_fwd<TIO, NORM><<<grid, threads, smem, st>>>(cd, (const TIO *)x, w, (TIO *)out)
-    if (d.io_bf16) { if (normalize) SLA_LAUNCH_FWD(__nv_bfloat16, true); else SLA_LAUNCH_FWD(__nv_bfloat16, false); }
-    else { if (normalize) SLA_LAUNCH_FWD(float, true); else SLA_LAUNCH_FWD(float, false); }
+    const bool shfl = vpr <= 32 && (vpr & (vpr - 1)) == 0;
+#define SLA_LAUNCH_FWD(TIO, NORM, SH) \
+    k_shortconv_fwd<TIO, NORM, SH><<<grid, threads, smem, st>>>(cd, (const TIO *)x, w, (TIO *)out)
+    if (d.io_bf16) {
+        if (!normalize) SLA_LAUNCH_FWD(__nv_bfloat16, false, true);
+        else if (shfl) SLA_LAUNCH_FWD(__nv_bfloat16, true, true);
+        else SLA_LAUNCH_FWD(__nv_bfloat16, true, false);
+    } else {
+        if (!normalize) SLA_LAUNCH_FWD(float, false, true);
+        else if (shfl) SLA_LAUNCH_FWD(float, true, true);
+        else SLA_LAUNCH_FWD(float, true, false);
+    }
 #undef SLA_LAUNCH_FWD
     tr.mark("shortconv_fwd");
     return cudaGetLastError() == cudaSuccess ? 1 : -1;
@@ -287,14 +322,22 @@ int shortconv_backward(const Dims &d, int width, int K, bool normalize, float ep
     ConvDims cd{d.T, d.H, width, K, tokens_per_cta(d), hpc, eps};
     dim3 grid((d.T + cd.per - 1) / cd.per, d.B, (d.H + hpc - 1) / hpc);
     const size_t smem = (size_t)(2 * TOKB * threads + 2 * TOKB * hpc) * sizeof(float);
-#define SLA_LAUNCH_BWD(TIO, NORM) \
-    k_shortconv_bwd<TIO, NORM><<<grid, threads, smem, st>>>(cd, (const TIO *)x, w, (const TIO *)dout, (TIO *)dx, ws)
-    if (d.io_bf16) { if (normalize) SLA_LAUNCH_BWD(__nv_bfloat16, true); else SLA_LAUNCH_BWD(__nv_bfloat16, false); }
-    else { if (normalize) SLA_LAUNCH_BWD(float, true); else SLA_LAUNCH_BWD(float, false); }
+    const bool shfl = vpr <= 32 && (vpr & (vpr - 1)) == 0;
+#define SLA_LAUNCH_BWD(TIO, NORM, SH) \
+    k_shortconv_bwd<TIO, NORM, SH><<<grid, threads, smem, st>>>(cd, (const TIO *)x, w, (const TIO *)dout, (TIO *)dx, ws)
+    if (d.io_bf16) {
+        if (!normalize) SLA_LAUNCH_BWD(__nv_bfloat16, false, true);
+        else if (shfl) SLA_LAUNCH_BWD(__nv_bfloat16, true, true);
+        else SLA_LAUNCH_BWD(__nv_bfloat16, true, false);
+    } else {
+        if (!normalize) SLA_LAUNCH_BWD(float, false, true);
+        else if (shfl) SLA_LAUNCH_BWD(float, true, true);
+        else SLA_LAUNCH_BWD(float, true, false);
+    }
 #undef SLA_LAUNCH_BWD
     tr.mark("shortconv_bwd");
     const int C = d.H * width;
-    k_shortconv_dw<<<(C * K + 255) / 256, 256, 0, st>>>((int)(grid.x * grid.y), C, K, ws, dw);
+    k_shortconv_dw<<<(C * K + 7) / 8, 256, 0, st>>>((int)(grid.x * grid.y), C, K, ws, dw);
     tr.mark("shortconv_dw");
     return cudaGetLastError() == cudaSuccess ? 2 : -1;
 }
