@@ -321,7 +321,7 @@ constexpr uint32_t SMEM_BYTES = OFF_TMEM + 16 + 1024;
 constexpr uint32_t COL_DS = 0, COL_A = 128, COL_DA = 192, COL_DQ = 256, COL_DK = 320, COL_DV = 384, TMEM_COLS = 512;
 constexpr int NTHREADS = NCOMPUTE + 32 + NGATE + 32;    // warps 0..7 compute, 8 MMA issue, 9..12 gates, 13 TMA
 enum Bar { FULL_G = 0, FULL_QK, FULL_V, FULL_DO, FULL_S, OPR, GREADY /*[4]*/, GFREE = GREADY + 4 /*[4]*/, ZREADY = GFREE + 4,
-           AREADY, OUT1, OUT2, SNFREE, INIT_DONE, DGFREE, BAR_A, BAR_M1, BAR_M2, DOFREE, INIT_FULL, DRAIN, NBAR };
+           AREADY, OUT1, OUT2, SNFREE, INIT_DONE, DGFREE, BAR_A, BAR_M1, BAR_M2, DOFREE, INIT_FULL, DRAIN, BAR_DS, NBAR };
 static_assert(SMEM_BYTES <= 232448, "shared memory budget");
 static_assert(NBAR <= 32, "barrier slots");
 }  // namespace st2
@@ -488,6 +488,7 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap gm_q, const __grid_constant__ C
                     tc_mma_bf16(tmem + COL_DV, mDZ + kstep_mnmajor(kk), kK + kstep_kmajor(kk, HALF_BF16), ID_MK, kk > 0);            // dV^T = dZ^T kh^T ...
                     if (kk < 4) tc_mma_bf16(tmem + COL_DS, mQ + kstep_mnmajor(kk), mDO + kstep_mnmajor(kk), ID_S, 1);                // dS_n = dZ + qh^T dO
                 }
+                tc_commit(bar(BAR_DS));                // dS_n is complete (and S_n dO^T has read S_n)
                 wait(AREADY, par);                     // masked A, dA in shared memory
                 if (failed) break;
                 tc_fence_after();
@@ -559,6 +560,11 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap gm_q, const __grid_constant__ C
                     if (failed) break;
                     load_qk(n - 1, k + 1);
                 }
+                if (n > 0) {
+                    wait_relaxed(SNFREE, par);         // rowsum(dS_n * S_n) done (and S_n dO^T issued long ago): S_n no longer needed
+                    if (failed) break;
+                    load_s(n - 1);
+                }
                 wait_relaxed(OUT1, par);               // dq, dk staged over qh, kh
                 if (failed) break;
                 tma_store_5d(&tm_dq, sQK, 0, n * C, 0, h, b);
@@ -566,11 +572,6 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap gm_q, const __grid_constant__ C
                 bulk_commit();
                 bulk_wait_read0();
                 if (n > 0) load_vdo(n - 1, k + 1);     // ... and this buffer takes the next v, dO
-                if (n > 0) {
-                    wait_relaxed(SNFREE, par);         // rowsum(dS_n * S_n) done: S_n no longer needed
-                    if (failed) break;
-                    load_s(n - 1);
-                }
                 wait_relaxed(OUT2, par);               // dv, dlog_decay staged
                 if (failed) break;
                 tma_store_5d(&tm_dv, base + OFF_A, 0, n * C, 0, h, b);
@@ -720,6 +721,18 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap gm_q, const __grid_constant__ C
             tc_fence_before();
             mbar_arrive(bar(AREADY));
 
+            // ---- R_{n-1} = rowsum(dS_n * S_n), while the tensor core works on the products with the masked tiles ----
+            wait(BAR_DS, par);
+            tc_fence_after();
+            {
+                float v0[32], v1[32];
+                tmem_ld32(tmem + lane_base + COL_DS + 64 * wh, v0);
+                tmem_ld32(tmem + lane_base + COL_DS + 64 * wh + 32, v1);
+                tmem_wait_ld();
+                Rs[((n & 1) ^ 1) * 2 * D + wh * D + row] = rowdot_part(v0, 0) + rowdot_part(v1, 1);
+            }
+            mbar_arrive(bar(SNFREE));                   // S_n is no longer needed: the next image may land
+
             // ---- dqh^T, dkh^T: this thread owns key dimension `row` and tokens 32*wh .. 32*wh+31 ----
             wait(BAR_M1, par);
             tc_fence_after();
@@ -757,7 +770,7 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap gm_q, const __grid_constant__ C
             tc_fence_before();
             mbar_arrive(bar(OUT1));
 
-            // ---- dV^T -> dv tile; R_{n-1} = rowsum(dS_n * S_n); dlog_decay tile; gate products ----
+            // ---- dV^T -> dv tile; dlog_decay tile; gate products ----
             wait(BAR_M2, par);
             tc_fence_after();
             {
@@ -770,14 +783,6 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap gm_q, const __grid_constant__ C
                     *reinterpret_cast<__nv_bfloat16 *>(sm + OFF_A + dhalf + swz(32 * wh + ii, dchunk) + dbyte) =
                         __float2bfloat16_rn(dvt[ii]);
             }
-            {
-                float v0[32], v1[32];
-                tmem_ld32(tmem + lane_base + COL_DS + 64 * wh, v0);
-                tmem_ld32(tmem + lane_base + COL_DS + 64 * wh + 32, v1);
-                tmem_wait_ld();
-                Rs[((n & 1) ^ 1) * 2 * D + wh * D + row] = rowdot_part(v0, 0) + rowdot_part(v1, 1);
-            }
-            mbar_arrive(bar(SNFREE));
             named_bar_sync(1, NCOMPUTE);                // up, red and the R partials are complete
             {   // log-decay gradient: in-chunk suffix sum + what flows in from the right of the chunk
                 const float offs = wh == 1 ? Rcur[row] + Rcur[D + row] : up[row];
