@@ -22,6 +22,9 @@ constexpr int TOKB = 2;          // ... and backward (more live values per token
 template <typename TIO> struct V;
 template <> struct V<float> {
     static constexpr int N = 4;
+    static __device__ __forceinline__ void widen(const uint4 v, float (&x)[4]) {
+        x[0] = __uint_as_float(v.x); x[1] = __uint_as_float(v.y); x[2] = __uint_as_float(v.z); x[3] = __uint_as_float(v.w);
+    }
     static __device__ __forceinline__ void load(const float *p, float (&x)[4]) {
         const float4 v = *reinterpret_cast<const float4 *>(p);
         x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w;
@@ -32,14 +35,16 @@ template <> struct V<float> {
 };
 template <> struct V<__nv_bfloat16> {
     static constexpr int N = 8;
-    static __device__ __forceinline__ void load(const __nv_bfloat16 *p, float (&x)[8]) {
-        const uint4 v = *reinterpret_cast<const uint4 *>(p);
+    static __device__ __forceinline__ void widen(const uint4 v, float (&x)[8]) {
         const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
             const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&w[e]));
             x[2 * e] = f.x; x[2 * e + 1] = f.y;
         }
+    }
+    static __device__ __forceinline__ void load(const __nv_bfloat16 *p, float (&x)[8]) {
+        widen(*reinterpret_cast<const uint4 *>(p), x);
     }
     static __device__ __forceinline__ void store(__nv_bfloat16 *p, const float (&x)[8]) {
         uint32_t w[4];
@@ -143,6 +148,58 @@ k_shortconv_fwd(ConvDims cd, const TIO *__restrict__ x, const float *__restrict_
                     for (int e = 0; e < N; ++e) z[s][e] *= r;
                     V<TIO>::store(orow + (size_t)(t + s) * C, z[s]);
                 }
+        }
+    }
+}
+
+// Forward without state carried from token to token, for heads that are a power-of-two run of lanes: blocks of TB
+// tokens of a sequence are dealt round robin to the CTAs; a thread fetches its vector of the block's TB + 3 token rows as
+// packed 16-byte values, all in flight together (the three rows before the block come from L2, its neighbour has just
+// read them), and widens them one by one as the window moves.  Head sums by shuffles, no shared memory, no barrier.
+template <typename TIO, bool NORM>
+__global__ void __launch_bounds__(256, 2)
+k_shortconv_fwd_blocks(ConvDims cd, int B, const TIO *__restrict__ x, const float *__restrict__ w, TIO *__restrict__ out) {
+    constexpr int N = V<TIO>::N;
+    constexpr int TB = 8;
+    const int C = cd.H * cd.d, vpr = cd.d / N, tid = threadIdx.x;
+    const int hb = blockIdx.z * cd.hpc, nh = min(cd.hpc, cd.H - hb);
+    const bool live = tid < nh * vpr;
+    const int gv = hb * vpr + tid;
+    float wt[KMAX][N];
+    load_taps<N>(w, gv * N, cd.K, live, wt);
+    const int nblk = (cd.T + TB - 1) / TB;
+    for (long item = blockIdx.x; item < (long)B * nblk; item += gridDim.x) {
+        const int b = (int)(item / nblk), t = (int)(item % nblk) * TB;
+        const TIO *xr = x + ((size_t)b * cd.T) * C + (size_t)gv * N;
+        TIO *orow = out + ((size_t)b * cd.T) * C + (size_t)gv * N;
+        uint4 raw[TB + 3];
+#pragma unroll
+        for (int s = 0; s < TB + 3; ++s) {
+            const int tt = t - 3 + s;
+            raw[s] = (live && tt >= 0 && tt < cd.T) ? __ldg(reinterpret_cast<const uint4 *>(xr + (size_t)tt * C)) : make_uint4(0u, 0u, 0u, 0u);
+        }
+        float xm3[N], xm2[N], xm1[N];
+        V<TIO>::widen(raw[0], xm3);
+        V<TIO>::widen(raw[1], xm2);
+        V<TIO>::widen(raw[2], xm1);
+#pragma unroll
+        for (int s = 0; s < TB; ++s) {
+            float xc[N], z[N], ss = 0.f;
+            V<TIO>::widen(raw[s + 3], xc);
+#pragma unroll
+            for (int e = 0; e < N; ++e) {
+                const float y = fmaf(wt[0][e], xm3[e], fmaf(wt[1][e], xm2[e], fmaf(wt[2][e], xm1[e], wt[3][e] * xc[e])));
+                z[e] = __fdividef(y, 1.f + __expf(-y));
+                ss = fmaf(z[e], z[e], ss);
+                xm3[e] = xm2[e]; xm2[e] = xm1[e]; xm1[e] = xc[e];
+            }
+            if (NORM) {
+                for (int o = vpr >> 1; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+                const float r = 1.f / sqrtf(ss + cd.eps);
+#pragma unroll
+                for (int e = 0; e < N; ++e) z[e] *= r;
+            }
+            if (live && t + s < cd.T) V<TIO>::store(orow + (size_t)(t + s) * C, z);
         }
     }
 }
@@ -299,6 +356,21 @@ int shortconv_forward(const Dims &d, int width, int K, bool normalize, float eps
     dim3 grid((d.T + cd.per - 1) / cd.per, d.B, (d.H + hpc - 1) / hpc);
     const size_t smem = (size_t)(TOKS * threads + TOKS * hpc) * sizeof(float);
     const bool shfl = vpr <= 32 && (vpr & (vpr - 1)) == 0;
+    if (shfl || !normalize) {
+        int dev = 0, sms = 148;
+        if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        const long items = (long)d.B * ((d.T + 7) / 8);
+        dim3 g((unsigned)std::min<long>(items, 2L * sms), 1, (d.H + hpc - 1) / hpc);
+        if (d.io_bf16) {
+            if (normalize) k_shortconv_fwd_blocks<__nv_bfloat16, true><<<g, threads, 0, st>>>(cd, d.B, (const __nv_bfloat16 *)x, w, (__nv_bfloat16 *)out);
+            else k_shortconv_fwd_blocks<__nv_bfloat16, false><<<g, threads, 0, st>>>(cd, d.B, (const __nv_bfloat16 *)x, w, (__nv_bfloat16 *)out);
+        } else {
+            if (normalize) k_shortconv_fwd_blocks<float, true><<<g, threads, 0, st>>>(cd, d.B, (const float *)x, w, (float *)out);
+            else k_shortconv_fwd_blocks<float, false><<<g, threads, 0, st>>>(cd, d.B, (const float *)x, w, (float *)out);
+        }
+        tr.mark("shortconv_fwd");
+        return cudaGetLastError() == cudaSuccess ? 1 : -1;
+    }
 #define SLA_LAUNCH_FWD(TIO, NORM, SH) \
     k_shortconv_fwd<TIO, NORM, SH><<<grid, threads, smem, st>>>(cd, (const TIO *)x, w, (TIO *)out)
     if (d.io_bf16) {
