@@ -77,6 +77,45 @@ void sla_oracle_gate_scores_backward(long n_tok, int H, int d, const double *x, 
 }
 
 /*
+ * Eq. 7, the output projection: the heads' outputs of a token, concatenated, times W^O:
+ *     y[t,n] = sum_c o[t,c] * W[c,n]        (c runs over the H*d_v concatenated features)
+ * o: [n_tok, K], W: [K, N], y: [n_tok, N].  Tokens are independent (the loop over them runs in parallel).
+ */
+void sla_oracle_out_proj(long n_tok, int K, int N, const double *o, const double *W, double *y) {
+#pragma omp parallel for schedule(static)
+    for (long t = 0; t < n_tok; ++t) {
+        double *yt = y + t * N;
+        for (int n = 0; n < N; ++n) yt[n] = 0.0;
+        for (int c = 0; c < K; ++c) {
+            double a = o[t * K + c];
+            const double *Wc = W + (long)c * N;
+            for (int n = 0; n < N; ++n) yt[n] += a * Wc[n];
+        }
+    }
+}
+
+/* Reverse of sla_oracle_out_proj: d_o[t,c] = sum_n dy[t,n] W[c,n];  dW[c,n] = sum_t o[t,c] dy[t,n] (tokens in order). */
+void sla_oracle_out_proj_backward(long n_tok, int K, int N, const double *o, const double *W, const double *dy,
+                                  double *d_o, double *dW) {
+#pragma omp parallel for schedule(static)
+    for (long t = 0; t < n_tok; ++t)
+        for (int c = 0; c < K; ++c) {
+            double acc = 0.0;
+            for (int n = 0; n < N; ++n) acc += dy[t * N + n] * W[(long)c * N + n];
+            d_o[t * K + c] = acc;
+        }
+#pragma omp parallel for schedule(static)
+    for (int c = 0; c < K; ++c) {
+        double *dWc = dW + (long)c * N;
+        for (int n = 0; n < N; ++n) dWc[n] = 0.0;
+        for (long t = 0; t < n_tok; ++t) {
+            double a = o[t * K + c];
+            for (int n = 0; n < N; ++n) dWc[n] += a * dy[t * N + n];
+        }
+    }
+}
+
+/*
  * Feature map of the Gated-DeltaNet instantiation ("short-convolution module" followed by SiLU, Experimental setup),
  * as published for Gated DeltaNet: a depthwise causal convolution of K taps over time, channel by channel, then
  * SiLU, then (for q and k) L2 normalisation over the d features of each head.

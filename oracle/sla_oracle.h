@@ -73,6 +73,10 @@ void sla_oracle_gate_scores(long n_tok, int H, int d, const double *x, const dou
 /* dx += ds W^T per head (accumulated), dW = sum_t ds x (overwritten). */
 void sla_oracle_gate_scores_backward(long n_tok, int H, int d, const double *x, const double *W,
                                      const double *ds, double *dx, double *dW);
+/* Eq. 7: y = o W^O over the concatenated head outputs; o [n_tok,K], W [K,N], y [n_tok,N]; and its reverse. */
+void sla_oracle_out_proj(long n_tok, int K, int N, const double *o, const double *W, double *y);
+void sla_oracle_out_proj_backward(long n_tok, int K, int N, const double *o, const double *W, const double *dy,
+                                  double *d_o, double *dW);
 
 /* Feature map of the Gated-DeltaNet instantiation: depthwise causal convolution over time (K taps, w [C,K], C = H*d
  * channels), SiLU, and with normalize != 0 L2 normalisation over the d features of each head (eps inside the root).

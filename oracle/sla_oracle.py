@@ -61,6 +61,10 @@ def _load():
         lib.sla_oracle_gate_scores.restype = None
         lib.sla_oracle_gate_scores_backward.argtypes = [ctypes.c_long, i, i, dp, dp, dp, dp, dp]
         lib.sla_oracle_gate_scores_backward.restype = None
+        lib.sla_oracle_out_proj.argtypes = [ctypes.c_long, i, i, dp, dp, dp]
+        lib.sla_oracle_out_proj.restype = None
+        lib.sla_oracle_out_proj_backward.argtypes = [ctypes.c_long, i, i, dp, dp, dp, dp, dp]
+        lib.sla_oracle_out_proj_backward.restype = None
         _lib = lib
     return _lib
 
@@ -193,6 +197,26 @@ def gate_scores_backward(x, W, ds, dx):
     dW = np.zeros((d, H))
     _load().sla_oracle_gate_scores_backward(x.size // (H * d), H, d, _p(x), _p(W), _p(ds), _p(dx), _p(dW))
     return dW
+
+
+def out_proj(o, W):
+    """Eq. 7's output projection: o [..., K] (the heads' outputs concatenated), W [K, N] -> y [..., N]."""
+    o, W = _f64(o), _f64(W)
+    K, N = W.shape
+    assert o.shape[-1] == K
+    y = np.zeros(o.shape[:-1] + (N,))
+    _load().sla_oracle_out_proj(o.size // K, K, N, _p(o), _p(W), _p(y))
+    return y
+
+
+def out_proj_backward(o, W, dy):
+    """Reverse of out_proj: returns (d_o [..., K], dW [K, N])."""
+    o, W, dy = _f64(o), _f64(W), _f64(dy)
+    K, N = W.shape
+    assert o.shape[-1] == K and dy.shape == o.shape[:-1] + (N,)
+    d_o, dW = np.zeros(o.shape), np.zeros((K, N))
+    _load().sla_oracle_out_proj_backward(o.size // K, K, N, _p(o), _p(W), _p(dy), _p(d_o), _p(dW))
+    return d_o, dW
 
 
 SHORTCONV_EPS = 1e-6
