@@ -224,6 +224,23 @@ sla_status sla_gate_scores_backward(sla_plan *plan, const void *q, const void *k
                                     void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * Output projection (Eq. 7: y_t = Concat_h(o_{t,h}) W^O).  o [B,T,H*d_v] is sla_forward's output (the heads of a
+ * token are already side by side), w_o [H*d_v, d_model] row-major, y [B,T,d_model]; all bf16 (the plan's io dtype
+ * must be SLA_BF16: the products run on the bf16 tensor cores with fp32 accumulation; fp32 plans get
+ * SLA_ERR_UNSUPPORTED), d_model and H*d_v multiples of 8.  A dense contraction: one persistent tcgen05 kernel.
+ * Needs no workspace.  y may not alias o.
+ */
+sla_status sla_out_proj_forward(sla_plan *plan, const void *o, const void *w_o, int32_t d_model, void *y,
+                                void *cuda_stream);
+/*
+ * Reverse of sla_out_proj_forward: d_o [B,T,H*d_v] (bf16; it is the dO that sla_backward takes) = dy W^O^T and
+ * dw_o fp32 [H*d_v, d_model] = sum over tokens of o_t^T dy_t, both written in full; the token sum of dw_o runs in a
+ * fixed order inside one accumulator per element (identical bits on every run).  Two launches, no workspace.
+ */
+sla_status sla_out_proj_backward(sla_plan *plan, const void *o, const void *w_o, const void *dy, int32_t d_model,
+                                 void *d_o, float *dw_o, void *cuda_stream);
+
+/*
  * Feature map of the Gated-DeltaNet instantiation (Experimental setup: GDN uses "the short-convolution module" and SiLU
  * as activation; RetNet and GLA use the identity and need none of this).  The paper names the module and cites Gated
  * DeltaNet for it; what is computed here is that published design: per channel a causal convolution over time,

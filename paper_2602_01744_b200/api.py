@@ -27,6 +27,7 @@ EXPORTS = (
     "sla_forward_noalloc", "sla_plan_selftest_timeout", "sla_decode_steps", "sla_gate_scores_forward",
     "sla_gate_scores_backward", "sla_plan_gate_scores_workspace_bytes", "sla_shortconv_forward",
     "sla_shortconv_backward", "sla_plan_shortconv_workspace_bytes", "sla_plan_set_sequences",
+    "sla_out_proj_forward", "sla_out_proj_backward",
 )
 SLA_NOALLOC_SCRATCH_BYTES = 32 << 20
 
@@ -93,6 +94,10 @@ def lib():
         L.sla_shortconv_forward.restype = ctypes.c_int
         L.sla_shortconv_backward.argtypes = [vp, vp, vp, i32, i32, i32, vp, vp, vp, vp, sz, vp]
         L.sla_shortconv_backward.restype = ctypes.c_int
+        L.sla_out_proj_forward.argtypes = [vp, vp, vp, i32, vp, vp]
+        L.sla_out_proj_forward.restype = ctypes.c_int
+        L.sla_out_proj_backward.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp]
+        L.sla_out_proj_backward.restype = ctypes.c_int
         L.sla_plan_shortconv_workspace_bytes.argtypes = [vp, i32, ctypes.POINTER(sz)]
         L.sla_plan_shortconv_workspace_bytes.restype = ctypes.c_int
         L.sla_gate_scores_forward.argtypes = [vp] * 8
@@ -295,6 +300,24 @@ def sla_gate_scores_backward(plan: Plan, q, k, w_gq, w_gk, dgq_logits, dgk_logit
         plan.handle, _ptr(q), _ptr(k), _ptr(w_gq), _ptr(w_gk), _ptr(dgq_logits), _ptr(dgk_logits), _ptr(dq), _ptr(dk),
         _ptr(dw_gq), _ptr(dw_gk), _ptr(workspace), workspace.numel(), _stream()))
     return dw_gq, dw_gk
+
+
+def sla_out_proj_forward(plan: Plan, o, w_o, y=None):
+    """Eq. 7's output projection: o [B,T,H,d_v] (or [B,T,H*d_v]) bf16, w_o [H*d_v, d_model] bf16 -> y [B,T,d_model] bf16."""
+    if y is None:
+        y = torch.empty(o.shape[0], o.shape[1], w_o.shape[1], dtype=o.dtype, device=o.device)
+    _check("sla_out_proj_forward", lib().sla_out_proj_forward(
+        plan.handle, _ptr(o), _ptr(w_o), w_o.shape[1], _ptr(y), _stream()))
+    return y
+
+
+def sla_out_proj_backward(plan: Plan, o, w_o, dy):
+    """Returns (d_o like o, dw_o fp32 [H*d_v, d_model]) of sla_out_proj_forward."""
+    d_o = torch.empty_like(o)
+    dw = torch.empty(w_o.shape, dtype=torch.float32, device=o.device)
+    _check("sla_out_proj_backward", lib().sla_out_proj_backward(
+        plan.handle, _ptr(o), _ptr(w_o), _ptr(dy), w_o.shape[1], _ptr(d_o), _ptr(dw), _stream()))
+    return d_o, dw
 
 
 def sla_shortconv_forward(plan: Plan, x, w, normalize, out=None):

@@ -130,7 +130,7 @@ sla_status sla_plan_create(sla_plan **out, const sla_desc *desc) {
     if (prop.major != 10) return SLA_ERR_ARCH;
     if (sla::generic_configure() != 0 || sla::gdn_configure() != 0 || sla::gla_tc_configure() != 0 ||
         sla::gla_tc_bwd_configure() != 0 || sla::gdn_tc_configure() != 0 ||
-        sla::gdn_tc_bwd_configure() != 0 || sla::decode_configure() != 0)
+        sla::gdn_tc_bwd_configure() != 0 || sla::decode_configure() != 0 || sla::out_proj_configure() != 0)
         return SLA_ERR_CUDA;
 
     sla_plan *p = new (std::nothrow) sla_plan();
@@ -410,6 +410,45 @@ sla_status sla_shortconv_backward(sla_plan *plan, const void *x, const float *w,
     plan->tracer.start((cudaStream_t)cuda_stream);
     int n = sla::shortconv_backward(dm, d, K, normalize != 0, SLA_SHORTCONV_EPS, x, w, dout, dx, dw, (float *)workspace,
                                     (cudaStream_t)cuda_stream, plan->tracer);
+    if (n < 0) return SLA_ERR_CUDA;
+    plan->last_launches = n;
+    return SLA_OK;
+}
+
+static bool out_proj_args_ok(const sla::Dims &d, int32_t d_model) {
+    return d.io_bf16 && d_model >= 8 && d_model % 8 == 0 && (d.H * d.dv) % 8 == 0;
+}
+
+sla_status sla_out_proj_forward(sla_plan *plan, const void *o, const void *w_o, int32_t d_model, void *y, void *cuda_stream) {
+    if (!plan) return SLA_ERR_INVALID_ARG;
+    const sla::Dims &d = plan->dims;
+    if (!out_proj_args_ok(d, d_model)) return SLA_ERR_UNSUPPORTED;
+    plan->last_launches = 0;
+    if (d.B == 0 || d.T == 0) return SLA_OK;
+    if (!o || !w_o || !y || !aligned16(o) || !aligned16(w_o) || !aligned16(y)) return SLA_ERR_INVALID_ARG;
+    plan->tracer.start((cudaStream_t)cuda_stream);
+    int n = sla::out_proj_forward((long)d.B * d.T, d.H * d.dv, d_model, o, w_o, y, plan->d_status, (cudaStream_t)cuda_stream,
+                                  plan->tracer);
+    if (n < 0) return SLA_ERR_CUDA;
+    plan->last_launches = n;
+    return SLA_OK;
+}
+
+sla_status sla_out_proj_backward(sla_plan *plan, const void *o, const void *w_o, const void *dy, int32_t d_model, void *d_o,
+                                 float *dw_o, void *cuda_stream) {
+    if (!plan) return SLA_ERR_INVALID_ARG;
+    const sla::Dims &d = plan->dims;
+    if (!out_proj_args_ok(d, d_model)) return SLA_ERR_UNSUPPORTED;
+    plan->last_launches = 0;
+    if (!dw_o || !aligned16(dw_o)) return SLA_ERR_INVALID_ARG;
+    if (d.B == 0 || d.T == 0)           // no tokens: the weight gradient is zero
+        return cudaMemsetAsync(dw_o, 0, (size_t)d.H * d.dv * d_model * sizeof(float), (cudaStream_t)cuda_stream) == cudaSuccess
+                   ? SLA_OK : SLA_ERR_CUDA;
+    if (!o || !w_o || !dy || !d_o || !aligned16(o) || !aligned16(w_o) || !aligned16(dy) || !aligned16(d_o))
+        return SLA_ERR_INVALID_ARG;
+    plan->tracer.start((cudaStream_t)cuda_stream);
+    int n = sla::out_proj_backward((long)d.B * d.T, d.H * d.dv, d_model, o, w_o, dy, d_o, dw_o, plan->d_status,
+                                   (cudaStream_t)cuda_stream, plan->tracer);
     if (n < 0) return SLA_ERR_CUDA;
     plan->last_launches = n;
     return SLA_OK;

@@ -53,17 +53,7 @@ template <> __device__ __forceinline__ void st_io4<__nv_bfloat16>(__nv_bfloat16 
     *reinterpret_cast<uint2 *>(p + i) = make_uint2(pack_bf16(v.x, v.y), pack_bf16(v.z, v.w));
 }
 
-// 2-D tiled TMA load / store of one state (coordinates: column, row of the [Bdec*H*d_k, d_v] view)
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int c0, int c1, uint32_t bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"((uint64_t)map), "r"(c0), "r"(c1), "r"(bar) : "memory");
-}
-__device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, uint32_t src, int c0, int c1) {
-    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
-                 ::"l"((uint64_t)map), "r"(src), "r"(c0), "r"(c1) : "memory");
-}
-
+// (states move by 2-D tiled TMA: coordinates are column, row of the [Bdec*H*d_k, d_v] view)
 struct DecParams {
     const void *q, *k, *v;
     const float *log_decay, *beta, *lq, *lk;

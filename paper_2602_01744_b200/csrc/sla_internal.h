@@ -174,6 +174,12 @@ int shortconv_forward(const Dims &d, int width, int K, bool normalize, float eps
 int shortconv_backward(const Dims &d, int width, int K, bool normalize, float eps, const void *x, const float *w,
                        const void *dout, void *dx, float *dw, float *ws, cudaStream_t st, Tracer &tr);
 
+// Output projection (Eq. 7) and its reverse: dense bf16 contractions on the tensor cores (sla_out_proj.cu).
+int out_proj_configure();
+int out_proj_forward(long n_tok, int K, int Dm, const void *o, const void *w, void *y, int *status, cudaStream_t st, Tracer &tr);
+int out_proj_backward(long n_tok, int K, int Dm, const void *o, const void *w, const void *dy, void *d_o, float *dw, int *status,
+                      cudaStream_t st, Tracer &tr);
+
 // GDN per-tile gradient kernels (after the recompute pass and the state-gradient scan).
 int gdn_backward_tiles(const Dims &d, const Workspace &w, const BwdArgs &a, cudaStream_t st, Tracer &tr);
 

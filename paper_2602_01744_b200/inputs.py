@@ -128,6 +128,19 @@ def make_gate_weights(cfg: SLAConfig, seed: int):
             torch.randn(cfg.d_k, cfg.H, generator=gen, dtype=torch.float32))
 
 
+def make_out_proj_inputs(cfg: SLAConfig, d_model: int, seed: int):
+    """Inputs of the output projection (Eq. 7): head outputs o ~ N(0,1) [B,T,H,d_v] (the scale the layer's outputs
+    have behind an output norm), W^O ~ N(0,1)/sqrt(H d_v) [H*d_v, d_model] (unit-scale y) and an upstream gradient
+    dy ~ N(0,1) [B,T,d_model]; all in the I/O dtype."""
+    gen = torch.Generator(device="cpu").manual_seed(seed)
+    io = torch_dtype(cfg.dtype)
+    K = cfg.H * cfg.d_v
+    o = torch.randn(cfg.B, cfg.T, cfg.H, cfg.d_v, generator=gen, dtype=torch.float32).to(io)
+    w = (torch.randn(K, d_model, generator=gen, dtype=torch.float32) / (K ** 0.5)).to(io)
+    dy = torch.randn(cfg.B, cfg.T, d_model, generator=gen, dtype=torch.float32).to(io)
+    return o, w, dy
+
+
 def make_frontend_inputs(cfg: SLAConfig, K: int, seed: int) -> dict:
     """Raw inputs of the Gated-DeltaNet feature map: x_q, x_k, x_v ~ N(0,1) [B,T,H,d] in the I/O dtype (the layer's
     linear projections are upstream and leave unit-scale activations), taps w_* ~ N(0,1)/sqrt(K) fp32 [H*d,K], and an
