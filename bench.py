@@ -417,6 +417,36 @@ def main():
                   "algorithmic_bytes": {"forward": fb, "backward": bb},
                   "share_of_step": (tms["forward"] + tms["backward"]) / (ms / args.steps)}
 
+    # ---- the output projection of Eq. 7 (y = Concat_h(o_h) W^O, d_model = H d_v) and its reverse: dense contractions, so
+    # their roofline is the tensor core's ----
+    out_proj = None
+    if rank == 0 and cfg.dtype == "bf16" and not args.generic and not args.packed:
+        from paper_2602_01744_b200.inputs import make_out_proj_inputs
+        dm = cfg.H * cfg.d_v
+        po, pw, pdy = (t.cuda() for t in make_out_proj_inputs(cfg, dm, seed=97))
+        py = torch.empty_like(pdy)
+        tms = {}
+        for name, fn in (("forward", lambda: api.sla_out_proj_forward(plan, po, pw, y=py)),
+                         ("backward", lambda: api.sla_out_proj_backward(plan, po, pw, pdy))):
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize()
+            e0.record()
+            for _ in range(20):
+                fn()
+            e1.record()
+            torch.cuda.synchronize()
+            tms[name] = e0.elapsed_time(e1) / 20
+        flop = 2.0 * cfg.B * cfg.T * dm * dm                      # per product; the reverse pass runs two
+        tb, tsus, tkind = measured_tensor_peaks()
+        out_proj = {"what": "sla_out_proj_forward / _backward: [B*T, H*d_v] x [H*d_v, d_model] with d_model = H*d_v, bf16, fp32 accumulation",
+                    "bound": "tensor", "forward_ms": tms["forward"], "backward_ms": tms["backward"],
+                    "forward_tflops": flop / (tms["forward"] * 1e-3) / 1e12, "backward_tflops": 2 * flop / (tms["backward"] * 1e-3) / 1e12,
+                    "peak": tb, "unit": "TFLOP/s", "peak_kind": f"bf16 burst, of {tkind}",
+                    "forward_frac": flop / (tms["forward"] * 1e-3) / 1e12 / tb,
+                    "backward_frac": 2 * flop / (tms["backward"] * 1e-3) / 1e12 / tb,
+                    "flop": {"forward": flop, "backward": 2 * flop}}
+
     # ---- the feature map of the Gated-DeltaNet instantiation (short convolution, SiLU, L2 norm) and its reverse ----
     frontend = None
     if rank == 0 and cfg.variant == "gdn" and not args.generic:
@@ -617,6 +647,7 @@ def main():
             "ms_per_step_with_kernel_events": ms_traced / args.steps,
             "step_hbm": {"algorithmic_bytes_per_step": step_bytes, "achieved_gbs": step_gbs, "frac": step_gbs / peak},
             "gate_scores": scores,
+            "out_proj": out_proj,
             "gdn_feature_map": frontend,
             "decode_step": decode,
             "cpu_baseline": cpu,
