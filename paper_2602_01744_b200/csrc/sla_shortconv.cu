@@ -318,6 +318,114 @@ k_shortconv_bwd(ConvDims cd, const TIO *__restrict__ x, const float *__restrict_
     }
 }
 
+// Reverse pass without state carried from block to block (bf16, heads that are a power-of-two run of lanes): blocks of
+// TB tokens are dealt round robin to the CTAs; a thread owns FOUR channels and fetches, packed and all in flight together,
+// the TB + 6 rows of x and the TB + 3 rows of dout its block needs (dx of a token needs dy of the three tokens after it,
+// each of which needs the three rows of x before it; the overlap with the neighbouring blocks comes from L2).  It then
+// walks the block backwards with the window in registers: every row is widened once and serves y, dx and the tap
+// gradients.  Head sums by shuffles, no shared memory, no barrier.  Tap gradients are summed per thread over its blocks
+// and written per CTA.
+template <bool NORM>
+__global__ void __launch_bounds__(256, 2)
+k_shortconv_bwd_blocks(ConvDims cd, int B, const __nv_bfloat16 *__restrict__ x, const float *__restrict__ w,
+                       const __nv_bfloat16 *__restrict__ dout, __nv_bfloat16 *__restrict__ dx, float *__restrict__ partial) {
+    constexpr int N = 4, TB = 8;
+    const int C = cd.H * cd.d, vpr = cd.d / N, tid = threadIdx.x;
+    const int hb = blockIdx.z * cd.hpc, nh = min(cd.hpc, cd.H - hb);
+    const bool live = tid < nh * vpr;
+    const int gv = hb * vpr + tid;
+    float wt[KMAX][N], acc[KMAX][N];
+    load_taps<N>(w, gv * N, cd.K, live, wt);
+#pragma unroll
+    for (int j = 0; j < KMAX; ++j)
+#pragma unroll
+        for (int e = 0; e < N; ++e) acc[j][e] = 0.f;
+    auto widen = [](const uint2 v, float (&f)[N]) {
+        const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&v.x));
+        const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&v.y));
+        f[0] = a.x; f[1] = a.y; f[2] = b.x; f[3] = b.y;
+    };
+    const int nblk = (cd.T + TB - 1) / TB;
+    for (long item = blockIdx.x; item < (long)B * nblk; item += gridDim.x) {
+        const int b = (int)(item / nblk), t = (int)(item % nblk) * TB;
+        const size_t rowoff = ((size_t)b * cd.T) * C + (size_t)gv * N;
+        const __nv_bfloat16 *xr = x + rowoff, *gr = dout + rowoff;
+        uint2 rx[TB + 6], rg[TB + 3];                   // x rows t-3 .. t+TB+2, dout rows t .. t+TB+2 (zero outside the sequence)
+#pragma unroll
+        for (int s = 0; s < TB + 6; ++s) {
+            const int tt = t - 3 + s;
+            rx[s] = (live && tt >= 0 && tt < cd.T) ? __ldg(reinterpret_cast<const uint2 *>(xr + (size_t)tt * C)) : make_uint2(0u, 0u);
+        }
+#pragma unroll
+        for (int s = 0; s < TB + 3; ++s) {
+            const int tt = t + s;
+            rg[s] = (live && tt < cd.T) ? __ldg(reinterpret_cast<const uint2 *>(gr + (size_t)tt * C)) : make_uint2(0u, 0u);
+        }
+        float x1[N], x2[N], x3[N], dy1[N], dy2[N], dy3[N];      // x of tokens u-2, u-1, u; dy of tokens u+1, u+2, u+3
+        widen(rx[TB + 3], x1);
+        widen(rx[TB + 4], x2);
+        widen(rx[TB + 5], x3);
+#pragma unroll
+        for (int e = 0; e < N; ++e) dy1[e] = dy2[e] = dy3[e] = 0.f;
+#pragma unroll
+        for (int s = TB + 2; s >= 0; --s) {             // token u = t + s; past the sequence end dout = 0 makes dy = 0
+            float x0[N], g[N], z[N], gs[N], dy[N], ss = 0.f, dot = 0.f;
+            widen(rx[s], x0);                           // x of token u-3
+            widen(rg[s], g);
+#pragma unroll
+            for (int e = 0; e < N; ++e) {
+                const float y = fmaf(wt[0][e], x0[e], fmaf(wt[1][e], x1[e], fmaf(wt[2][e], x2[e], wt[3][e] * x3[e])));
+                const float sg = __fdividef(1.f, 1.f + __expf(-y));
+                z[e] = y * sg;
+                gs[e] = sg * (1.f + y * (1.f - sg));            // d silu / dy
+                ss = fmaf(z[e], z[e], ss);
+                dot = fmaf(z[e], g[e], dot);
+            }
+            float fa = 1.f, fb = 0.f;
+            if (NORM) {                                 // out = z / r:  dz = dout / r - z (z . dout) / r^3
+                for (int o = vpr >> 1; o > 0; o >>= 1) {
+                    ss += __shfl_xor_sync(0xffffffffu, ss, o);
+                    dot += __shfl_xor_sync(0xffffffffu, dot, o);
+                }
+                const float ri = rsqrtf(ss + cd.eps);
+                fa = ri;
+                fb = dot * ri * ri * ri;
+            }
+#pragma unroll
+            for (int e = 0; e < N; ++e) dy[e] = (g[e] * fa - z[e] * fb) * gs[e];
+            if (s < TB) {                               // this block's own tokens: dx out, tap gradients in
+                __nv_bfloat162 lo = __floats2bfloat162_rn(
+                    fmaf(wt[3][0], dy[0], fmaf(wt[2][0], dy1[0], fmaf(wt[1][0], dy2[0], wt[0][0] * dy3[0]))),
+                    fmaf(wt[3][1], dy[1], fmaf(wt[2][1], dy1[1], fmaf(wt[1][1], dy2[1], wt[0][1] * dy3[1]))));
+                __nv_bfloat162 hi = __floats2bfloat162_rn(
+                    fmaf(wt[3][2], dy[2], fmaf(wt[2][2], dy1[2], fmaf(wt[1][2], dy2[2], wt[0][2] * dy3[2]))),
+                    fmaf(wt[3][3], dy[3], fmaf(wt[2][3], dy1[3], fmaf(wt[1][3], dy2[3], wt[0][3] * dy3[3]))));
+                if (live && t + s < cd.T)
+                    *reinterpret_cast<uint2 *>(dx + rowoff + (size_t)(t + s) * C) =
+                        make_uint2(*reinterpret_cast<uint32_t *>(&lo), *reinterpret_cast<uint32_t *>(&hi));
+#pragma unroll
+                for (int e = 0; e < N; ++e) {
+                    acc[0][e] = fmaf(dy[e], x0[e], acc[0][e]);
+                    acc[1][e] = fmaf(dy[e], x1[e], acc[1][e]);
+                    acc[2][e] = fmaf(dy[e], x2[e], acc[2][e]);
+                    acc[3][e] = fmaf(dy[e], x3[e], acc[3][e]);
+                }
+            }
+#pragma unroll
+            for (int e = 0; e < N; ++e) {
+                dy3[e] = dy2[e]; dy2[e] = dy1[e]; dy1[e] = dy[e];
+                x3[e] = x2[e]; x2[e] = x1[e]; x1[e] = x0[e];
+            }
+        }
+    }
+    if (live) {
+        float *dst = partial + ((size_t)blockIdx.x * C + (size_t)gv * N) * KMAX;
+#pragma unroll
+        for (int e = 0; e < N; ++e)
+            *reinterpret_cast<float4 *>(dst + e * KMAX) = make_float4(acc[0][e], acc[1][e], acc[2][e], acc[3][e]);
+    }
+}
+
 // dw[c, j] = sum over the CTAs' partial sums: one warp per element, lane l adds the partials of CTAs l, l+32, .. in
 // order, then the lanes are folded in a fixed tree (same bits on every run)
 __global__ void k_shortconv_dw(int n_cta, int C, int K, const float *__restrict__ partial, float *__restrict__ dw) {
@@ -395,6 +503,23 @@ int shortconv_backward(const Dims &d, int width, int K, bool normalize, float ep
     dim3 grid((d.T + cd.per - 1) / cd.per, d.B, (d.H + hpc - 1) / hpc);
     const size_t smem = (size_t)(2 * TOKB * threads + 2 * TOKB * hpc) * sizeof(float);
     const bool shfl = vpr <= 32 && (vpr & (vpr - 1)) == 0;
+    const int C = d.H * width;
+    const int vpr4 = width / 4;
+    if (d.io_bf16 && vpr4 <= 32 && (vpr4 & (vpr4 - 1)) == 0) {
+        int dev = 0, sms = 148;
+        if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        const int hpc4 = std::max(1, std::min(d.H, 256 / vpr4)), threads4 = (hpc4 * vpr4 + 31) / 32 * 32;
+        ConvDims cd4{d.T, d.H, width, K, cd.per, hpc4, eps};
+        // (no more CTAs than the workspace has partial-sum slots for)
+        const long slots = (long)grid.x * grid.y;
+        dim3 g((unsigned)std::min<long>(slots, 2L * sms), 1, (d.H + hpc4 - 1) / hpc4);
+        if (normalize) k_shortconv_bwd_blocks<true><<<g, threads4, 0, st>>>(cd4, d.B, (const __nv_bfloat16 *)x, w, (const __nv_bfloat16 *)dout, (__nv_bfloat16 *)dx, ws);
+        else k_shortconv_bwd_blocks<false><<<g, threads4, 0, st>>>(cd4, d.B, (const __nv_bfloat16 *)x, w, (const __nv_bfloat16 *)dout, (__nv_bfloat16 *)dx, ws);
+        tr.mark("shortconv_bwd");
+        k_shortconv_dw<<<(C * K + 7) / 8, 256, 0, st>>>((int)g.x, C, K, ws, dw);
+        tr.mark("shortconv_dw");
+        return cudaGetLastError() == cudaSuccess ? 2 : -1;
+    }
 #define SLA_LAUNCH_BWD(TIO, NORM, SH) \
     k_shortconv_bwd<TIO, NORM, SH><<<grid, threads, smem, st>>>(cd, (const TIO *)x, w, (const TIO *)dout, (TIO *)dx, ws)
     if (d.io_bf16) {
@@ -408,7 +533,6 @@ int shortconv_backward(const Dims &d, int width, int K, bool normalize, float ep
     }
 #undef SLA_LAUNCH_BWD
     tr.mark("shortconv_bwd");
-    const int C = d.H * width;
     k_shortconv_dw<<<(C * K + 7) / 8, 256, 0, st>>>((int)(grid.x * grid.y), C, K, ws, dw);
     tr.mark("shortconv_dw");
     return cudaGetLastError() == cudaSuccess ? 2 : -1;
