@@ -78,23 +78,27 @@ def measured_tensor_peaks():
     return 1590.0, 1400.0, "fallback"
 
 
+def sources_sha256(files) -> str:
+    """Hash of the named files of the kernel source folder (the sources a profiled kernel is built from)."""
+    import hashlib
+    h = hashlib.sha256()
+    for f in sorted(files):
+        h.update((ROOT / "paper_2602_01744_b200" / "csrc" / f).read_bytes())
+    return h.hexdigest()
+
+
 def recorded_counters(workload: str, kernel: str, key: str = "bytes_per_launch_full_size"):
     """A figure from the committed ncu summary (DRAM bytes per launch, tensor-pipe activity), if one covers this kernel
-    on this workload (full size, plan flags as in the default run).  The record carries a hash of the kernel sources
-    it was taken on: once they have changed, the figure is stale and None is reported."""
-    import hashlib
+    on this workload (full size, plan flags as in the default run).  Each record names the source files its kernel is
+    built from and carries their hash: once one of them has changed, the figure is stale and None is reported."""
     p = ROOT / "profiles" / "dram_traffic.json"
     if not p.exists():
         return None
     try:
-        rec = json.loads(p.read_text())
-        h = hashlib.sha256()
-        for f in sorted((ROOT / "paper_2602_01744_b200" / "csrc").glob("*")):
-            h.update(f.read_bytes())
-        if rec.get("source_sha256") != h.hexdigest():
+        e = json.loads(p.read_text()).get(workload, {}).get(kernel)
+        if e is None or e.get("source_sha256") != sources_sha256(e["sources"]):
             return None
-        e = rec.get(workload, {}).get(kernel)
-        return None if e is None else e.get(key)
+        return e.get(key)
     except Exception:
         return None
 

@@ -85,3 +85,37 @@ def test_refusals():
     plan = api.sla_plan_create("gla", "bf16", 1, 64, 2, 64, 64, 64)
     with pytest.raises(api.SLAError):                       # d_model must be a multiple of 8
         api.sla_out_proj_forward(plan, o.bfloat16(), torch.zeros(128, 12, device="cuda", dtype=torch.bfloat16))
+
+
+@pytest.mark.parametrize("base,T,H", [("C2", 200, 4), ("C4", 130, 3)])
+def test_layer_followed_by_the_projection(base, T, H):
+    """sla_forward -> output projection, and back: dy -> d_o -> sla_backward.  The oracle runs the same chain in fp64
+    (on the GPU's bf16 o, and its bf16 d_o, where the GPU rounds them: those are tensors of the interface)."""
+    from paper_2602_01744_b200.inputs import make_inputs
+    cfg = small(CONFIGS[base], B=2, T=T, H=H, seed=1360 + T)
+    xh = make_inputs(cfg, with_dO=False)
+    dm = 264
+    _, w, dy = make_out_proj_inputs(cfg, dm, seed=1361)
+    x = gu.to_dev(xh)
+    plan = api.sla_plan_create(cfg.variant, cfg.dtype, cfg.B, cfg.T, cfg.H, cfg.d_k, cfg.d_v, cfg.chunk, cfg.scale)
+    o, _ = api.sla_forward(plan, x["q"], x["k"], x["v"], x["log_decay"], x["gq_logits"], x["gk_logits"], beta=x["beta"])
+    y = api.sla_out_proj_forward(plan, o, w.cuda())
+    d_o, dw = api.sla_out_proj_backward(plan, o, w.cuda(), dy.cuda())
+    g = api.sla_backward(plan, x["q"], x["k"], x["v"], x["log_decay"], x["gq_logits"], x["gk_logits"], d_o, beta=x["beta"])
+    torch.cuda.synchronize()
+    plan.poll()
+    K = cfg.H * cfg.d_v
+    o_ref, _ = orc.forward(cfg.variant, xh["q"], xh["k"], xh["v"], xh["log_decay"], xh["gq_logits"], xh["gk_logits"],
+                           beta=xh["beta"], scale=cfg.scale)
+    y_ref = orc.out_proj(o_ref.reshape(cfg.B, cfg.T, K), w)
+    do_ref, dw_ref = orc.out_proj_backward(o_ref.reshape(cfg.B, cfg.T, K), w, dy)
+    g_ref = orc.backward(cfg.variant, xh["q"], xh["k"], xh["v"], xh["log_decay"], xh["gq_logits"], xh["gk_logits"],
+                         do_ref.reshape(cfg.B, cfg.T, cfg.H, cfg.d_v), beta=xh["beta"], scale=cfg.scale)
+    names = {"dq": "dq", "dk": "dk", "dv": "dv"}
+    errs = {"y": gu.rel_l2(y, y_ref), "d_o": gu.rel_l2(d_o.reshape(cfg.B, cfg.T, K), do_ref)}
+    rows = {"y": gu.row_err(y, y_ref), "d_o": gu.row_err(d_o.reshape(cfg.B, cfg.T, K), do_ref)}
+    for n, r in names.items():
+        errs[n], rows[n] = gu.rel_l2(g[n], g_ref[r]), gu.row_err(g[n], g_ref[r])
+    gu.assert_close(errs, rows, "bf16", (base, T, H))
+    # dw_o is fed by the GPU's o (bf16-rounded, itself within 1e-2 of the oracle's): the chain carries that error
+    assert gu.rel_l2(dw, dw_ref) <= gu.TOL["bf16"]
