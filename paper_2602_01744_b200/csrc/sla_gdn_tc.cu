@@ -1,4 +1,4 @@
-// Softmax-GatedDeltaNet forward on the 5th-generation tensor cores (bf16 I/O, d_k = d_v = 128, chunk 64):
+// Softmax-GatedDeltaNet forward on the 5th-generation tensor cores (bf16 I/O, d_k = d_v = 128 - or 64, run as 128 with zero padding supplied by the tensor maps -, chunk 64):
 // Eq. 14-16 with a scalar decay per (token, head), evaluated chunkwise in WY form.
 //
 // Per chunk (local token i, b_i = cumulative log-decay, Gam_i = e^{b_i}, S = state at the chunk start):
@@ -61,6 +61,7 @@ struct GdnParams {
     float scale;
     const SeqInfo *seqs;    // packed variable-length batch: per-sequence table and tensor maps (q, k, v, o), else nullptr
     const CUtensorMap *vmaps;
+    int d;                  // head width d_k = d_v: 128, or 64 (the upper half of every 128-wide tile is then zero padding)
 };
 
 __global__ void __launch_bounds__(gd::NTHREADS, 1)
@@ -245,7 +246,7 @@ k_gdn_fwd_tc(const __grid_constant__ CUtensorMap gm_q, const __grid_constant__ C
 
         uint8_t *rec0 = p.save ? p.save + slot * REC_BYTES : nullptr;   // this sequence's records
         {   // initial state: fp32 into TMEM, bf16 copy into shared memory (row = key dimension)
-            const float *src = p.h0 ? p.h0 + ((size_t)bh * D + row) * D + 64 * colhalf : nullptr;
+            const float *src = state_row(p.h0, bh, row, colhalf, p.d);
 #pragma unroll
             for (int part = 0; part < 2; ++part) {
                 float v[32];
@@ -543,7 +544,7 @@ k_gdn_fwd_tc(const __grid_constant__ CUtensorMap gm_q, const __grid_constant__ C
         }
 
         if (p.ht) {   // final state, fp32 (each thread reads back what it wrote in the last rescale)
-            float *dst = p.ht + ((size_t)bh * D + row) * D + 64 * colhalf;
+            float *dst = state_row(p.ht, bh, row, colhalf, p.d);
 #pragma unroll
             for (int part = 0; part < 2; ++part) {
                 float v[32];
@@ -551,7 +552,7 @@ k_gdn_fwd_tc(const __grid_constant__ CUtensorMap gm_q, const __grid_constant__ C
                 tmem_wait_ld();
 #pragma unroll
                 for (int j = 0; j < 32; j += 4)
-                    *reinterpret_cast<float4 *>(dst + 32 * part + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                    if (dst) *reinterpret_cast<float4 *>(dst + 32 * part + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
             }
         }
     }
@@ -564,7 +565,7 @@ k_gdn_fwd_tc(const __grid_constant__ CUtensorMap gm_q, const __grid_constant__ C
 }  // namespace
 
 bool gdn_tc_supported(const Dims &d) {
-    return d.variant == SLA_GDN && d.io_bf16 && d.dk == 128 && d.dv == 128 && d.C == 64;
+    return d.variant == SLA_GDN && d.io_bf16 && d.dk == d.dv && (d.dk == 128 || d.dk == 64) && d.C == 64;
 }
 
 int gdn_tc_configure() {
@@ -577,27 +578,27 @@ int gdn_tc_configure() {
 static const CUtensorMap *gdn_varlen_maps(const Dims &d, const FwdArgs &a, int r, cudaStream_t st) {
     const void *key[] = {a.q, a.k, a.v, a.o};
     return varlen_maps(*a.vl, r, key, 4, st, [&](const SeqInfo &si, CUtensorMap *m) {
-        const size_t off = (size_t)si.t0 * d.H * D;
-        if (!make_tile_map(m + 0, (const __nv_bfloat16 *)a.q + off, 1, si.T, d.H) ||
-            !make_tile_map(m + 1, (const __nv_bfloat16 *)a.k + off, 1, si.T, d.H) ||
-            !make_tile_map(m + 2, (const __nv_bfloat16 *)a.v + off, 1, si.T, d.H))
+        const size_t off = (size_t)si.t0 * d.H * d.dk;
+        if (!make_tile_map(m + 0, (const __nv_bfloat16 *)a.q + off, 1, si.T, d.H, d.dk) ||
+            !make_tile_map(m + 1, (const __nv_bfloat16 *)a.k + off, 1, si.T, d.H, d.dk) ||
+            !make_tile_map(m + 2, (const __nv_bfloat16 *)a.v + off, 1, si.T, d.H, d.dk))
             return false;
         if (!a.o) { m[3] = m[0]; return true; }
-        return make_tile_map(m + 3, (__nv_bfloat16 *)a.o + off, 1, si.T, d.H);
+        return make_tile_map(m + 3, (__nv_bfloat16 *)a.o + off, 1, si.T, d.H, d.dk);
     });
 }
 
 // Forward sweep in save mode, for the gradient sweep: writes the per-chunk records (S_n, U, T), stores no output.
 int gdn_tc_forward_save(const Dims &d, const FwdArgs &a, uint8_t *save, int *status, cudaStream_t st, Tracer &tr) {
     CUtensorMap mq, mk, mv;
-    if (!make_tile_map(&mq, a.q, d.B, d.T, d.H) || !make_tile_map(&mk, a.k, d.B, d.T, d.H) ||
-        !make_tile_map(&mv, a.v, d.B, d.T, d.H))
+    if (!make_tile_map(&mq, a.q, d.B, d.T, d.H, d.dk) || !make_tile_map(&mk, a.k, d.B, d.T, d.H, d.dk) ||
+        !make_tile_map(&mv, a.v, d.B, d.T, d.H, d.dk))
         return -1;
     const bool vl = a.vl && a.vl->n_seq;
     const CUtensorMap *vm = vl ? gdn_varlen_maps(d, a, 1, st) : nullptr;
     if (vl && !vm) return -1;
     GdnParams p{a.lq, a.lk, a.log_decay, a.beta, a.h0, nullptr, save, 0, status, d.T, d.H, d.NT, d.scale,
-                vl ? a.vl->d_seqs : nullptr, vm};
+                vl ? a.vl->d_seqs : nullptr, vm, d.dk};
     k_gdn_fwd_tc<<<vl ? a.vl->n_seq * d.H : d.B * d.H, gd::NTHREADS, gd::SMEM_BYTES, st>>>(mq, mk, mv, mq /* unused: nothing is stored */, p);
     tr.mark("gdn_states_tc");
     return cudaGetLastError() == cudaSuccess ? 1 : -1;
@@ -606,14 +607,14 @@ int gdn_tc_forward_save(const Dims &d, const FwdArgs &a, uint8_t *save, int *sta
 // Forward; with `save` not null it also leaves the per-chunk records for a later gradient sweep over the same inputs.
 int gdn_tc_forward(const Dims &d, const FwdArgs &a, uint8_t *save, int *status, cudaStream_t st, Tracer &tr) {
     CUtensorMap mq, mk, mv, mo;
-    if (!make_tile_map(&mq, a.q, d.B, d.T, d.H) || !make_tile_map(&mk, a.k, d.B, d.T, d.H) ||
-        !make_tile_map(&mv, a.v, d.B, d.T, d.H) || !make_tile_map(&mo, a.o, d.B, d.T, d.H))
+    if (!make_tile_map(&mq, a.q, d.B, d.T, d.H, d.dk) || !make_tile_map(&mk, a.k, d.B, d.T, d.H, d.dk) ||
+        !make_tile_map(&mv, a.v, d.B, d.T, d.H, d.dk) || !make_tile_map(&mo, a.o, d.B, d.T, d.H, d.dk))
         return -1;
     const bool vl = a.vl && a.vl->n_seq;
     const CUtensorMap *vm = vl ? gdn_varlen_maps(d, a, 0, st) : nullptr;
     if (vl && !vm) return -1;
     GdnParams p{a.lq, a.lk, a.log_decay, a.beta, a.h0, a.ht, save, 1, status, d.T, d.H, d.NT, d.scale,
-                vl ? a.vl->d_seqs : nullptr, vm};
+                vl ? a.vl->d_seqs : nullptr, vm, d.dk};
     k_gdn_fwd_tc<<<vl ? a.vl->n_seq * d.H : d.B * d.H, gd::NTHREADS, gd::SMEM_BYTES, st>>>(mq, mk, mv, mo, p);
     tr.mark("gdn_fwd_tc");
     return cudaGetLastError() == cudaSuccess ? 1 : -1;

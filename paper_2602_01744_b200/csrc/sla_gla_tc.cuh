@@ -1,5 +1,5 @@
 // Constants and host helpers shared by the tensor-core (tcgen05 / TMEM / TMA) Softmax-GLA kernels:
-// bf16 I/O, d_k = d_v = 128, 64-token chunks.  Shared-memory tiles are rows of 128 bytes (64 bf16) in the
+// bf16 I/O, d_k = d_v = 128 (64-wide heads run padded), 64-token chunks.  Shared-memory tiles are rows of 128 bytes (64 bf16) in the
 // 128-byte swizzle; a 128-wide tile is two such halves side by side.
 #pragma once
 #include <type_traits>
@@ -68,21 +68,31 @@ inline bool make_map(CUtensorMap *m, const void *ptr, int B, int T, int H, int d
     return r == CUDA_SUCCESS;
 }
 
-// Tensor map over a bf16 [B,T,H,128] tensor that moves a whole 64-token x 128-feature tile of one head in ONE copy:
-// the feature axis is split as (64 within a half, 2 halves) and the halves are made the slowest box dimension, so the
-// tile lands as two 128-byte-swizzled [64 rows][128 B] halves, 8 KiB apart - the layout the MMA descriptors expect.
+// Tensor map over a bf16 [B,T,H,d] tensor (d = 128 or 64) that moves a whole 64-token x 128-feature tile of one head in
+// ONE copy: the feature axis is split as (64 within a half, d/64 halves) and the halves are made the slowest box
+// dimension, so the tile lands as two 128-byte-swizzled [64 rows][128 B] halves, 8 KiB apart - the layout the MMA
+// descriptors expect.  With d = 64 the second half lies outside the tensor: it loads as zeros and is dropped by stores,
+// so a 64-wide head runs through the 128-wide kernels as if padded with zero features, at no cost in memory traffic.
 // Coordinates: (0, token, 0, head, batch).
-inline bool make_tile_map(CUtensorMap *m, const void *ptr, int B, int T, int H) {
+inline bool make_tile_map(CUtensorMap *m, const void *ptr, int B, int T, int H, int d = D) {
     EncodeFn fn = encode_fn();
     if (!fn) return false;
-    cuuint64_t dims[5] = {64, (cuuint64_t)T, 2, (cuuint64_t)H, (cuuint64_t)B};
-    cuuint64_t strides[4] = {(cuuint64_t)H * D * 2, 128, (cuuint64_t)D * 2, (cuuint64_t)T * H * D * 2};
+    cuuint64_t dims[5] = {64, (cuuint64_t)T, (cuuint64_t)(d / 64), (cuuint64_t)H, (cuuint64_t)B};
+    cuuint64_t strides[4] = {(cuuint64_t)H * d * 2, 128, (cuuint64_t)d * 2, (cuuint64_t)T * H * d * 2};
     cuuint32_t box[5] = {64, (cuuint32_t)C, 2, 1, 1};
     cuuint32_t estr[5] = {1, 1, 1, 1, 1};
     CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void *>(ptr), dims, strides, box, estr,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
+}
+
+// Row `row`, columns 64*half .. 64*half+63 of the fp32 [d, d] state of sequence-head bh inside a [.., d, d] tensor, as
+// seen by the thread that owns that part of the kernels' 128 x 128 state; nullptr where a 64-wide head has no such
+// part (the padded rows and columns stay zero) or the tensor is absent.
+template <typename T>
+__device__ __forceinline__ T *state_row(T *t, size_t bh, int row, int half, int d) {
+    return (t && row < d && 64 * half < d) ? t + (bh * d + row) * d + 64 * half : nullptr;
 }
 
 // Device array of the per-sequence tensor maps of region r of a packed batch: `make(seq, maps)` encodes one sequence's

@@ -1,4 +1,4 @@
-// Softmax-GLA backward on the 5th-generation tensor cores (bf16 I/O, d_k = d_v = 128, chunk 64).
+// Softmax-GLA backward on the 5th-generation tensor cores (bf16 I/O, d_k = d_v = 128 - or 64, run as 128 with zero padding supplied by the tensor maps -, chunk 64).
 //
 // The paper states no gradients; these are the chain rule applied to Eq. 4, 12-13, evaluated chunkwise.
 // Two sweeps per (batch, head) sequence, one CTA each, chunk after chunk:
@@ -59,6 +59,7 @@ struct StatesParams {
     const float *log_gamma; // Softmax-RetNet: [H] constant log-decays (no log-decay tensor is read); else nullptr
     const SeqInfo *seqs;    // packed variable-length batch: per-sequence table and tensor maps (k, v, g), else nullptr
     const CUtensorMap *vmaps;
+    int d;                  // head width d_k = d_v: 128, or 64 (the upper half of every 128-wide tile is then zero padding)
 };
 
 // thread (row, colhalf) holds 32 consecutive state values of its row: bf16 them into the operand image
@@ -224,7 +225,7 @@ k_gla_states_tc(const __grid_constant__ CUtensorMap gm_k, const __grid_constant_
         const int colhalf = warp >> 2;
         const int row = 32 * (warp & 3) + lane;
         {   // S_0: fp32 into TMEM, bf16 image into slot 0
-            const float *src = (p.h0 && images) ? p.h0 + ((size_t)bh * D + row) * D + 64 * colhalf : nullptr;
+            const float *src = images ? state_row(p.h0, bh, row, colhalf, p.d) : nullptr;
 #pragma unroll
             for (int part = 0; part < 2; ++part) {
                 float v[32];
@@ -336,6 +337,7 @@ struct BwdParams {
     const float *log_gamma;         // Softmax-RetNet: [H] constant log-decays (no log-decay read, no log-decay gradient)
     const SeqInfo *seqs;            // packed variable-length batch: per-sequence table and tensor maps (the nine below), else nullptr
     const CUtensorMap *vmaps;
+    int d;                  // head width d_k = d_v: 128, or 64 (the upper half of every 128-wide tile is then zero padding)
 };
 
 // Sum v[j] over the 32 lanes for every j: afterwards lane l holds the total of v[l] in v[0].
@@ -628,7 +630,7 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap gm_q, const __grid_constant__ C
         {   // dS_NT = dht (or zero) into TMEM; R_{NT-1} = rowsum(dht * S_NT)
             float rpart = 0.f;
             if (p.dht) wait(INIT_FULL, 0);
-            const float *src = p.dht ? p.dht + ((size_t)bh * D + row) * D + 64 * wh : nullptr;
+            const float *src = state_row(p.dht, bh, row, wh, p.d);
 #pragma unroll
             for (int part = 0; part < 2; ++part) {
                 float v[32];
@@ -810,7 +812,7 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap gm_q, const __grid_constant__ C
         }
 
         if (p.dh0) {   // dS_0, fp32 (the last chunk's MMAs were waited for above)
-            float *dst = p.dh0 + ((size_t)bh * D + row) * D + 64 * wh;
+            float *dst = state_row(p.dh0, bh, row, wh, p.d);
 #pragma unroll
             for (int part = 0; part < 2; ++part) {
                 float v[32];
@@ -818,7 +820,7 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap gm_q, const __grid_constant__ C
                 tmem_wait_ld();
 #pragma unroll
                 for (int j = 0; j < 32; j += 4)
-                    *reinterpret_cast<float4 *>(dst + 32 * part + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                    if (dst) *reinterpret_cast<float4 *>(dst + 32 * part + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
             }
         }
     }
@@ -903,11 +905,11 @@ int gla_tc_segment_summaries(const Dims &d, const FwdArgs &a, int P, int L, floa
                              cudaStream_t st, Tracer &tr) {
     CUtensorMap mk, mv, mg;
     const bool retnet = d.variant == SLA_RETNET;
-    if (!make_tile_map(&mk, a.k, d.B, d.T, d.H) || !make_tile_map(&mv, a.v, d.B, d.T, d.H)) return -1;
+    if (!make_tile_map(&mk, a.k, d.B, d.T, d.H, d.dk) || !make_tile_map(&mv, a.v, d.B, d.T, d.H, d.dk)) return -1;
     if (retnet) mg = mk;   // (never used: the decay is generated in the kernel)
     else if (!make_map(&mg, a.log_decay, d.B, d.T, d.H, d.dk, true, 128)) return -1;
     StatesParams sp{a.lq, a.lk, nullptr, nullptr, fin, gam, status, d.T, d.H, d.NT, P, L, retnet ? a.log_decay : nullptr,
-                    nullptr, nullptr};
+                    nullptr, nullptr, d.dk};
     k_gla_states_tc<<<d.B * d.H * P, st1::NTHREADS, st1::SMEM_BYTES, st>>>(mk, mv, mg, sp);
     tr.mark("gla_segment_states_tc");
     return cudaGetLastError() == cudaSuccess ? 1 : -1;
@@ -918,10 +920,10 @@ uint8_t *gla_tc_state_images(float *ws) { return reinterpret_cast<uint8_t *>(ws)
 int gla_tc_backward(const Dims &d, const BwdArgs &a, bool have_states, int *status, cudaStream_t st, Tracer &tr) {
     CUtensorMap mq, mk, mv, mdo, mg, mdq, mdk, mdv, mdg;
     const bool retnet = d.variant == SLA_RETNET;      // constant decay: no log-decay tensor to read, no gradient for it
-    if (!make_tile_map(&mq, a.q, d.B, d.T, d.H) || !make_tile_map(&mk, a.k, d.B, d.T, d.H) ||
-        !make_tile_map(&mv, a.v, d.B, d.T, d.H) || !make_tile_map(&mdo, a.dO, d.B, d.T, d.H) ||
-        !make_tile_map(&mdq, a.dq, d.B, d.T, d.H) || !make_tile_map(&mdk, a.dk, d.B, d.T, d.H) ||
-        !make_tile_map(&mdv, a.dv, d.B, d.T, d.H))
+    if (!make_tile_map(&mq, a.q, d.B, d.T, d.H, d.dk) || !make_tile_map(&mk, a.k, d.B, d.T, d.H, d.dk) ||
+        !make_tile_map(&mv, a.v, d.B, d.T, d.H, d.dk) || !make_tile_map(&mdo, a.dO, d.B, d.T, d.H, d.dk) ||
+        !make_tile_map(&mdq, a.dq, d.B, d.T, d.H, d.dk) || !make_tile_map(&mdk, a.dk, d.B, d.T, d.H, d.dk) ||
+        !make_tile_map(&mdv, a.dv, d.B, d.T, d.H, d.dk))
         return -1;
     if (retnet) { mg = mq; mdg = mdq; }               // (never used)
     else if (!make_map(&mg, a.log_decay, d.B, d.T, d.H, d.dk, true, 128) ||
@@ -944,15 +946,15 @@ int gla_tc_backward(const Dims &d, const BwdArgs &a, bool have_states, int *stat
         if (vl) {
             const void *key[] = {a.k, a.v, a.log_decay};
             vm = varlen_maps(*vl, 1, key, 3, st, [&](const SeqInfo &si, CUtensorMap *m) {
-                const size_t off = (size_t)si.t0 * d.H * D;
-                if (!make_tile_map(m + 0, k + off, 1, si.T, d.H) || !make_tile_map(m + 1, v + off, 1, si.T, d.H)) return false;
+                const size_t off = (size_t)si.t0 * d.H * d.dk;
+                if (!make_tile_map(m + 0, k + off, 1, si.T, d.H, d.dk) || !make_tile_map(m + 1, v + off, 1, si.T, d.H, d.dk)) return false;
                 if (retnet) { m[2] = m[0]; return true; }
                 return make_map(m + 2, a.log_decay + off, 1, si.T, d.H, d.dk, true, 128);
             });
             if (!vm) return -1;
         }
         StatesParams sp{a.lq, a.lk, a.h0, simg, nullptr, nullptr, status, d.T, d.H, d.NT, 1, d.NT, retnet ? a.log_decay : nullptr,
-                        dseqs, vm};
+                        dseqs, vm, d.dk};
         k_gla_states_tc<<<ctas, st1::NTHREADS, st1::SMEM_BYTES, st>>>(mk, mv, mg, sp);
         tr.mark("gla_states_tc");
     }
@@ -960,12 +962,12 @@ int gla_tc_backward(const Dims &d, const BwdArgs &a, bool have_states, int *stat
     if (vl) {
         const void *key[] = {a.q, a.k, a.v, a.dO, a.log_decay, a.dq, a.dk, a.dv, a.dlog_decay};
         vm = varlen_maps(*vl, 2, key, 9, st, [&](const SeqInfo &si, CUtensorMap *m) {
-            const size_t off = (size_t)si.t0 * d.H * D;
-            if (!make_tile_map(m + 0, q + off, 1, si.T, d.H) || !make_tile_map(m + 1, k + off, 1, si.T, d.H) ||
-                !make_tile_map(m + 2, v + off, 1, si.T, d.H) || !make_tile_map(m + 3, dO + off, 1, si.T, d.H) ||
-                !make_tile_map(m + 5, (__nv_bfloat16 *)a.dq + off, 1, si.T, d.H) ||
-                !make_tile_map(m + 6, (__nv_bfloat16 *)a.dk + off, 1, si.T, d.H) ||
-                !make_tile_map(m + 7, (__nv_bfloat16 *)a.dv + off, 1, si.T, d.H))
+            const size_t off = (size_t)si.t0 * d.H * d.dk;
+            if (!make_tile_map(m + 0, q + off, 1, si.T, d.H, d.dk) || !make_tile_map(m + 1, k + off, 1, si.T, d.H, d.dk) ||
+                !make_tile_map(m + 2, v + off, 1, si.T, d.H, d.dk) || !make_tile_map(m + 3, dO + off, 1, si.T, d.H, d.dk) ||
+                !make_tile_map(m + 5, (__nv_bfloat16 *)a.dq + off, 1, si.T, d.H, d.dk) ||
+                !make_tile_map(m + 6, (__nv_bfloat16 *)a.dk + off, 1, si.T, d.H, d.dk) ||
+                !make_tile_map(m + 7, (__nv_bfloat16 *)a.dv + off, 1, si.T, d.H, d.dk))
                 return false;
             if (retnet) { m[4] = m[0]; m[8] = m[5]; return true; }
             return make_map(m + 4, a.log_decay + off, 1, si.T, d.H, d.dk, true, 128) &&
@@ -973,7 +975,7 @@ int gla_tc_backward(const Dims &d, const BwdArgs &a, bool have_states, int *stat
         });
         if (!vm) return -1;
     }
-    BwdParams bp{a.lq, a.lk, a.dht, simg, pq, pk, a.dh0, status, d.T, d.H, d.NT, d.scale, retnet ? a.log_decay : nullptr, dseqs, vm};
+    BwdParams bp{a.lq, a.lk, a.dht, simg, pq, pk, a.dh0, status, d.T, d.H, d.NT, d.scale, retnet ? a.log_decay : nullptr, dseqs, vm, d.dk};
     k_gla_bwd_tc<<<ctas, st2::NTHREADS, st2::SMEM_BYTES, st>>>(mq, mk, mv, mdo, mg, mdq, mdk, mdv, mdg, bp);
     tr.mark("gla_bwd_tc");
     if (gate_bwd_prod(a.lq, a.lk, pq, pk, a.dlq, a.dlk, (long)d.B * d.T, d.H, st) < 0) return -1;

@@ -1,4 +1,4 @@
-"""GPU parity of the tcgen05/TMEM/TMA Softmax-GLA and Softmax-GatedDeltaNet kernels (bf16, d_k = d_v = 128, chunk 64) against
+"""GPU parity of the tcgen05/TMEM/TMA Softmax-GLA and Softmax-GatedDeltaNet kernels (bf16, d_k = d_v = 128 or 64, chunk 64) against
 the fp64 oracle, through the C ABI with default kernel selection."""
 import pytest
 import torch
@@ -170,12 +170,13 @@ def test_saved_states_are_not_reused_once_another_backward_has_overwritten_them(
             assert torch.equal(t, g_a2[n]) and torch.equal(g_b[n], g_b2[n]), n
 
 
-@pytest.mark.parametrize("base,T", [("C2", 200), ("C2", 64), ("C4", 200), ("C4", 65)])
-def test_nothing_is_written_outside_the_buffers_handed_in(base, T):
+@pytest.mark.parametrize("base,T,d", [("C2", 200, 128), ("C2", 64, 128), ("C4", 200, 128), ("C4", 65, 128),
+                                      ("C2", 200, 64), ("C2", 65, 64), ("C4", 200, 64)])
+def test_nothing_is_written_outside_the_buffers_handed_in(base, T, d):
     """In place of a memory checker: outputs and workspace are carved out of one pattern-filled arena with guard bands
     around each; after a training step and a recomputing backward no guard byte may differ, every output element must
     have been written (they start as NaN) and the results must still match the oracle."""
-    cfg = small(CONFIGS[base], B=2, T=T, H=3, seed=940 + T)
+    cfg = small(CONFIGS[base], B=2, T=T, H=3, d_k=d, d_v=d, seed=940 + T)     # (d = 64: heads padded inside the kernels)
     xh = make_inputs(cfg, with_dO=True, with_h0=True)
     x = gu.to_dev(xh)
     plan = api.sla_plan_create(cfg.variant, cfg.dtype, cfg.B, cfg.T, cfg.H, cfg.d_k, cfg.d_v, cfg.chunk, cfg.scale,
@@ -283,3 +284,36 @@ def test_retnet_training_step_reads_what_the_forward_left(B, T, H, with_h0):
     errs, lf, lb = gu.check_training_step(cfg, with_h0=with_h0)
     assert (lf, lb) == (1, 2)
     assert max(errs.values()) <= 1e-2
+
+
+# ---- 64-wide heads: the same kernels, the upper half of every 128-wide tile being zero padding that the tensor maps
+# supply on loads and drop on stores (no padded copies in memory)
+@pytest.mark.parametrize("base", ["C2", "R2", "C4"])
+@pytest.mark.parametrize("B,T,H,with_h0", [(2, 200, 3, True), (1, 1000, 16, True), (3, 65, 4, False), (2, 5, 2, True)])
+def test_heads_of_width_64_take_the_tensor_core_kernels(base, B, T, H, with_h0):
+    cfg = small(CONFIGS[base], B=B, T=T, H=H, d_k=64, d_v=64, seed=1400 + T)
+    x = make_inputs(cfg, with_dO=True, with_h0=with_h0)
+    xd = gu.to_dev(x)
+    o, ht, g, plan, ws, lf, lb = gu.gpu_training_step(cfg, xd, h0=xd.get("h0"), dht=xd.get("dht"), want_dh0=with_h0)
+    # fused forward and a backward that reads the states it left; or, for few long sequences, a forward in segments
+    # (which leaves none) and a backward that recomputes them
+    assert (lf, lb) in ((1, 2), (2, 3)), (lf, lb)
+    oref, htref = gu.oracle_forward(cfg, x, h0=x.get("h0"))
+    ref = gu.oracle_backward(cfg, x, h0=x.get("h0"), dht=x.get("dht"))
+    pairs = {"o": (o, oref), "ht": (ht, htref)}
+    pairs.update({n: (g[n], ref[r]) for n, r in gu.GRAD_NAMES.items() if g.get(n) is not None})
+    gu.assert_close({n: gu.rel_l2(a, r) for n, (a, r) in pairs.items()},
+                    {n: gu.row_err(a, r) for n, (a, r) in pairs.items()}, cfg.dtype, cfg)
+    # the recomputing backward gives the same bits
+    g2, plan2 = gu.gpu_backward(cfg, xd, h0=xd.get("h0"), dht=xd.get("dht"), want_dh0=with_h0)
+    assert plan2.last_launch_count == 3
+    for n, t in g.items():
+        if t is not None:
+            assert torch.equal(t, g2[n]), n
+
+
+def test_mixed_widths_stay_on_the_generic_kernels():
+    cfg = small(CONFIGS["C2"], B=1, T=130, H=2, d_k=64, d_v=128, seed=1410)
+    x = gu.to_dev(make_inputs(cfg))
+    o, ht, plan = gu.gpu_forward(cfg, x)
+    assert plan.last_launch_count > 1

@@ -13,9 +13,9 @@ pytestmark = pytest.mark.gpu
 LENGTHS = (1, 63, 64, 65, 900, 130)      # (under 16 chunks each: run alone, such a sequence is not cut into segments)
 
 
-def _packed(base, lengths, H, seed, with_h0):
+def _packed(base, lengths, H, seed, with_h0, d=128):
     T = sum(lengths)
-    cfg = small(CONFIGS[base], B=1, T=T, H=H, seed=seed)
+    cfg = small(CONFIGS[base], B=1, T=T, H=H, d_k=d, d_v=d, seed=seed)
     x = make_inputs(cfg, with_dO=True)
     n = len(lengths)
     if with_h0:
@@ -41,11 +41,11 @@ def _slice(x, s, a, b):
     return out
 
 
-@pytest.mark.parametrize("base", ["C2", "R2", "C4"])
+@pytest.mark.parametrize("base,d", [("C2", 128), ("R2", 128), ("C4", 128), ("C2", 64), ("C4", 64)])
 @pytest.mark.parametrize("with_h0", [False, True])
-def test_packed_batch_matches_the_oracle_and_the_single_sequence_runs(base, with_h0):
+def test_packed_batch_matches_the_oracle_and_the_single_sequence_runs(base, d, with_h0):
     H = 3
-    cfg, xh, cu = _packed(base, LENGTHS, H, 1300, with_h0)
+    cfg, xh, cu = _packed(base, LENGTHS, H, 1300, with_h0, d)
     x = gu.to_dev(xh)
     n = len(LENGTHS)
     plan = api.sla_plan_create(cfg.variant, cfg.dtype, 1, cfg.T, H, cfg.d_k, cfg.d_v, cfg.chunk, cfg.scale,
