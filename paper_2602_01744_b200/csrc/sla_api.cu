@@ -72,7 +72,8 @@ static void plan_workspace_sizes(sla_plan *p) {
     p->bwd_bytes = p->ws.bwd_floats * sizeof(float);
     if (sla::gla_tc_supported(d) && !generic) {
         p->fwd_bytes = sla::gla_tc_forward_workspace_bytes(d, &p->varlen);
-        p->bwd_bytes = sla::gla_tc_backward_workspace_bytes(d, &p->varlen);
+        p->bwd_bytes = (!p->varlen.n_seq && p->segs.n_seq) ? sla::gla_tc_backward_segmented_workspace_bytes(d, p->segs)
+                                                           : sla::gla_tc_backward_workspace_bytes(d, &p->varlen);
     }
     if (sla::gdn_tc_supported(d) && !generic) {
         p->fwd_bytes = 0;
@@ -91,6 +92,18 @@ static void varlen_release(sla::Varlen &v) {
         g = sla::Varlen::Region();
     }
     v = sla::Varlen();
+}
+
+// Device side of a filled sequence table: the table itself and, per kernel kind, room for the sequences' tensor maps.
+static bool varlen_to_device(sla::Varlen &v) {
+    const int n_seq = v.n_seq;
+    bool ok = cudaMalloc((void **)&v.d_seqs, sizeof(sla::SeqInfo) * n_seq) == cudaSuccess &&
+              cudaMemcpy(v.d_seqs, v.seqs.data(), sizeof(sla::SeqInfo) * n_seq, cudaMemcpyHostToDevice) == cudaSuccess;
+    const size_t mb = (size_t)n_seq * sla::Varlen::MAPS_PER_SEQ * sizeof(CUtensorMap);
+    for (auto &g : v.reg)
+        ok = ok && cudaMalloc((void **)&g.dev, mb) == cudaSuccess && cudaMallocHost((void **)&g.host, mb) == cudaSuccess &&
+             cudaEventCreateWithFlags(&g.uploaded, cudaEventDisableTiming) == cudaSuccess;
+    return ok;
 }
 
 extern "C" {
@@ -144,6 +157,19 @@ sla_status sla_plan_create(sla_plan **out, const sla_desc *desc) {
     d.scale = desc->scale;
     p->ws = sla::plan_workspace(d);
     p->flags = desc->flags;
+    // few long sequences on the tensor-core GLA / RetNet kernels: the table of segments the backward runs in
+    if (sla::gla_tc_supported(d) && !(p->flags & SLA_FLAG_FORCE_GENERIC) && d.B > 0 && d.T > 0) {
+        int P, L;
+        sla::gla_tc_backward_choose_segments(d, P, L);
+        if (P > 1) {
+            sla::gla_tc_backward_segment_table(d, P, L, p->segs);
+            if (!varlen_to_device(p->segs)) {
+                varlen_release(p->segs);
+                delete p;
+                return SLA_ERR_CUDA;
+            }
+        }
+    }
     plan_workspace_sizes(p);
     p->device = dev;
     p->last_launches = 0;
@@ -162,6 +188,7 @@ sla_status sla_plan_destroy(sla_plan *plan) {
     if (!plan) return SLA_OK;
     if (plan->d_status) cudaFree(plan->d_status);
     varlen_release(plan->varlen);
+    varlen_release(plan->segs);
     plan->tracer.destroy();
     delete plan;
     return SLA_OK;
@@ -191,13 +218,7 @@ sla_status sla_plan_set_sequences(sla_plan *plan, const int32_t *cu_seqlens, int
     }
     v.slots = slots;
     v.n_seq = n_seq;
-    bool ok = cudaMalloc((void **)&v.d_seqs, sizeof(sla::SeqInfo) * n_seq) == cudaSuccess &&
-              cudaMemcpy(v.d_seqs, v.seqs.data(), sizeof(sla::SeqInfo) * n_seq, cudaMemcpyHostToDevice) == cudaSuccess;
-    const size_t mb = (size_t)n_seq * sla::Varlen::MAPS_PER_SEQ * sizeof(CUtensorMap);
-    for (auto &g : v.reg)
-        ok = ok && cudaMalloc((void **)&g.dev, mb) == cudaSuccess && cudaMallocHost((void **)&g.host, mb) == cudaSuccess &&
-             cudaEventCreateWithFlags(&g.uploaded, cudaEventDisableTiming) == cudaSuccess;
-    if (!ok) {
+    if (!varlen_to_device(v)) {
         varlen_release(v);
         plan_workspace_sizes(plan);
         return SLA_ERR_CUDA;
@@ -355,7 +376,9 @@ sla_status sla_backward(sla_plan *plan, const void *q, const void *k, const void
     // a backward pass that recomputes writes its own states into `workspace`: whatever an earlier forward left there
     // (for other inputs) is gone, and must not be taken for valid by a later call
     if (!have && sv.ws == workspace) sv.valid = false;
-    int n = (!generic && sla::gla_tc_supported(d))
+    int n = (!generic && sla::gla_tc_supported(d) && !a.vl && plan->segs.n_seq)
+                ? sla::gla_tc_backward_segmented(d, a, plan->segs, plan->d_status, (cudaStream_t)cuda_stream, plan->tracer)
+            : (!generic && sla::gla_tc_supported(d))
                 ? sla::gla_tc_backward(d, a, have, plan->d_status, (cudaStream_t)cuda_stream, plan->tracer)
             : (!generic && sla::gdn_tc_supported(d))
                 ? sla::gdn_tc_backward(d, a, have, plan->d_status, (cudaStream_t)cuda_stream, plan->tracer)

@@ -484,6 +484,13 @@ int gla_tc_configure() {
                    cudaSuccess ? 0 : -1;
 }
 
+// The backward runs the gradient sweep twice when it is cut into segments (once for the state gradients that leave
+// each segment, once for the results), so cutting pays only from three segments per sequence on.
+void gla_tc_backward_choose_segments(const Dims &d, int &P, int &L) {
+    choose_segments(d, P, L);
+    if (P < 3) { P = 1; L = d.NT; }
+}
+
 size_t gla_tc_forward_workspace_bytes(const Dims &d, const Varlen *vl) {
     int P, L;
     choose_segments(d, P, L);

@@ -18,6 +18,9 @@
 //                     qh*dqh - kh*dkh plus rowsum(dS_{n+1} * S_{n+1}) carried from the chunk to the right.
 //                     Gate gradients leave as the products Gq*dGq = sum_d qh*dqh, Gk*dGk = sum_d kh*dkh per
 //                     (token, head); the softmax backward over heads runs afterwards on [B,T,H].
+// Few long sequences (at least three segments per sequence fit the SMs): gla_tc_backward_segmented runs both sweeps
+// on segments of every sequence as the sequences of a packed batch, twice, with the states at the cuts and the state
+// gradients across them folded from per-segment summaries (see there).
 // Both kernels use the forward kernel's roles: one MMA-issuing lane, one TMA lane, gate warps running ahead and
 // eight compute warps; every wait is bounded and abortable.
 #include "sla_gla_tc.cuh"
@@ -865,6 +868,33 @@ void launch_gate_bwd_prod(const float *lq, const float *lk, const float *Pq, con
     k_gate_bwd_prod<HP><<<grid, 256, 0, st>>>(lq, lk, Pq, Pk, dlq, dlk, n_tok, H);
 }
 
+// Segmented backward, between the passes.  A batch row's P segments are sequences b*P .. b*P+P-1 of the packed batch;
+// summaries are indexed by (b*H + h)*P + p as the summary kernel leaves them, states by ((b*P + p)*H + h) as the
+// packed kernels read them.  One thread per state element, a short loop over the segments.
+// Start states: S_0 = h0 (or zero), S_{p+1} = diag(gam_p) S_p + fin_p.
+__global__ void k_fold_segment_states(int H, int P, int d, const float *__restrict__ h0, const float *__restrict__ fin,
+                                      const float *__restrict__ gam, float *__restrict__ h0seg) {
+    const int bh = blockIdx.x, b = bh / H, h = bh % H, row = blockIdx.y, col = threadIdx.x;
+    float sv = h0 ? h0[((size_t)bh * d + row) * d + col] : 0.f;
+    for (int p = 0; p < P; ++p) {
+        h0seg[((((size_t)b * P + p) * H + h) * d + row) * d + col] = sv;
+        const size_t c = (size_t)bh * P + p;
+        sv = fmaf(gam[c * D + row], sv, fin[(c * D + row) * D + col]);
+    }
+}
+// State gradients entering each segment from its right: R_{P-1} = dht (or zero), R_p = diag(gam_{p+1}) R_{p+1} + F_{p+1},
+// F_p being what segment p alone sends out of its left edge (its dh0 when run with a zero dht).
+__global__ void k_fold_segment_dstates(int H, int P, int d, const float *__restrict__ dht, const float *__restrict__ gam,
+                                       const float *__restrict__ dsfin, float *__restrict__ dhtseg) {
+    const int bh = blockIdx.x, b = bh / H, h = bh % H, row = blockIdx.y, col = threadIdx.x;
+    float r = dht ? dht[((size_t)bh * d + row) * d + col] : 0.f;
+    for (int p = P - 1; p >= 0; --p) {
+        const size_t i = ((((size_t)b * P + p) * H + h) * d + row) * d + col;
+        dhtseg[i] = r;
+        r = fmaf(gam[((size_t)bh * P + p) * D + row], r, dsfin[i]);
+    }
+}
+
 }  // namespace
 
 int gla_tc_bwd_configure() {
@@ -981,6 +1011,66 @@ int gla_tc_backward(const Dims &d, const BwdArgs &a, bool have_states, int *stat
     if (gate_bwd_prod(a.lq, a.lk, pq, pk, a.dlq, a.dlk, (long)d.B * d.T, d.H, st) < 0) return -1;
     tr.mark("gate_bwd");
     return cudaGetLastError() == cudaSuccess ? (have_states ? 2 : 3) : -1;
+}
+
+
+void gla_tc_backward_segment_table(const Dims &d, int P, int L, Varlen &segs) {
+    segs.seqs.clear();
+    long slots = 0;
+    for (int b = 0; b < d.B; ++b)
+        for (int p = 0; p < P; ++p) {
+            const int t0 = p * L * C, len = std::min(L * C, d.T - t0), nt = (len + C - 1) / C;
+            segs.seqs.push_back({b * d.T + t0, len, nt, (int)slots});
+            slots += nt + 1;
+        }
+    segs.slots = slots;
+    segs.n_seq = d.B * P;
+    segs.seg_P = P;
+    segs.seg_L = L;
+}
+
+// floats: [images of the segments' slots | pq | pk] as gla_tc_backward lays them out, then fin, gam, h0seg, dhtseg, dsfin
+static size_t segmented_base_floats(const Dims &d, const Varlen &segs) {
+    const size_t bth = (size_t)d.B * d.T * d.H;
+    return state_slots(d, &segs) * (STATE_BF16 / 4) + 2 * ((bth + 63) & ~(size_t)63);
+}
+size_t gla_tc_backward_segmented_workspace_bytes(const Dims &d, const Varlen &segs) {
+    const size_t nseg = (size_t)d.B * d.H * segs.seg_P, st = (size_t)segs.n_seq * d.H * d.dk * d.dv;
+    return (segmented_base_floats(d, segs) + nseg * (D * D + D) + 3 * st) * sizeof(float);
+}
+
+int gla_tc_backward_segmented(const Dims &d, const BwdArgs &a, Varlen &segs, int *status, cudaStream_t st, Tracer &tr) {
+    const int P = segs.seg_P, L = segs.seg_L;
+    const size_t nseg = (size_t)d.B * d.H * P, stf = (size_t)segs.n_seq * d.H * d.dk * d.dv;
+    float *fin = a.ws + segmented_base_floats(d, segs), *gam = fin + nseg * D * D;
+    float *h0seg = gam + nseg * D, *dhtseg = h0seg + stf, *dsfin = dhtseg + stf;
+    // the state every segment starts from
+    FwdArgs f{a.q, a.k, a.v, a.log_decay, a.beta, a.lq, a.lk, a.h0, nullptr, nullptr, a.ws, a.status, nullptr};
+    if (gla_tc_segment_summaries(d, f, P, L, fin, gam, status, st, tr) < 0) return -1;
+    const dim3 grid(d.B * d.H, d.dk);
+    k_fold_segment_states<<<grid, d.dv, 0, st>>>(d.H, P, d.dk, a.h0, fin, gam, h0seg);
+    tr.mark("fold_segment_states");
+    // first pass over the segments as a packed batch, no state gradient entering: what each sends out of its left edge
+    BwdArgs a1 = a;
+    a1.h0 = h0seg;
+    a1.dht = nullptr;
+    a1.dh0 = dsfin;
+    a1.vl = &segs;
+    const int n1 = gla_tc_backward(d, a1, false, status, st, tr);
+    if (n1 < 0) return -1;
+    k_fold_segment_dstates<<<grid, d.dv, 0, st>>>(d.H, P, d.dk, a.dht, gam, dsfin, dhtseg);
+    tr.mark("fold_segment_dstates");
+    // second pass with the true state gradient entering every segment (the state images of the first pass are in place)
+    BwdArgs a2 = a1;
+    a2.dht = dhtseg;
+    a2.dh0 = a.dh0 ? dsfin : nullptr;
+    const int n2 = gla_tc_backward(d, a2, true, status, st, tr);
+    if (n2 < 0) return -1;
+    if (a.dh0) {    // dS_0 of a batch row = what its first segment sends out
+        const size_t row = (size_t)d.H * d.dk * d.dv * sizeof(float);
+        if (cudaMemcpy2DAsync(a.dh0, row, dsfin, row * P, row, d.B, cudaMemcpyDeviceToDevice, st) != cudaSuccess) return -1;
+    }
+    return cudaGetLastError() == cudaSuccess ? 3 + n1 + n2 : -1;
 }
 
 }  // namespace sla

@@ -43,6 +43,7 @@ struct Varlen {
         cudaEvent_t uploaded = nullptr;
     } reg[3];                           // 0: forward, 1: state / record sweep, 2: gradient sweep
     static constexpr int MAPS_PER_SEQ = 9;
+    int seg_P = 0, seg_L = 0;           // > 0: an internal table that cuts each of the B batch rows into seg_P segments of seg_L chunks
 };
 
 // Carve-up of the caller's workspace (all fp32, offsets in floats, each 64-float aligned).
@@ -145,6 +146,13 @@ int gla_tc_segment_summaries(const Dims &d, const FwdArgs &a, int P, int L, floa
 size_t gla_tc_forward_workspace_bytes(const Dims &d, const Varlen *vl = nullptr);
 size_t gla_tc_backward_workspace_bytes(const Dims &d, const Varlen *vl = nullptr);
 int gla_tc_backward(const Dims &d, const BwdArgs &a, bool have_states, int *status, cudaStream_t st, Tracer &tr);
+// Few long sequences: the backward in segments.  Every batch row is cut into P segments of L chunks that run as the
+// sequences of a packed batch (`segs`, filled by gla_tc_backward_segment_table); the states at the segment starts and
+// the state gradients at the segment ends come from summaries folded along each row.  P == 1: not worth it.
+void gla_tc_backward_choose_segments(const Dims &d, int &P, int &L);
+void gla_tc_backward_segment_table(const Dims &d, int P, int L, Varlen &segs);
+size_t gla_tc_backward_segmented_workspace_bytes(const Dims &d, const Varlen &segs);
+int gla_tc_backward_segmented(const Dims &d, const BwdArgs &a, Varlen &segs, int *status, cudaStream_t st, Tracer &tr);
 
 // ---- tensor-core Softmax-GatedDeltaNet forward (WY form): sla_gdn_tc.cu.  Needs no workspace. ----
 bool gdn_tc_supported(const Dims &d);
@@ -202,6 +210,7 @@ struct sla_plan {
         void *stream = nullptr;
     } saved;
     sla::Varlen varlen;     // sla_plan_set_sequences: packed variable-length batch (n_seq == 0: regular batch)
+    sla::Varlen segs;       // tensor-core GLA / RetNet plans with few long sequences: the segments the backward runs in
     sla::Tracer tracer;
     std::vector<std::pair<const char *, std::pair<int, float>>> agg;   // name -> (launches, total ms)
 };

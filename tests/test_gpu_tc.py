@@ -230,10 +230,35 @@ def test_nothing_is_written_outside_the_buffers_handed_in(base, T, d):
 
 
 def test_segmented_forward_leaves_nothing_and_the_backward_recomputes():
-    cfg = small(CONFIGS["C2"], B=1, T=2048, H=4, seed=920)     # few long sequences: the forward runs in segments
+    cfg = small(CONFIGS["C2"], B=2, T=1024, H=16, seed=920)    # few long sequences: the forward runs in two segments
     errs, lf, lb = gu.check_training_step(cfg)
     assert lf == 2 and lb == 3                       # (segment summaries + forward; state sweep + gradient sweep + gates)
     assert max(errs.values()) <= 1e-2
+
+
+@pytest.mark.parametrize("base,B,T,H,d,with_h0", [("C2", 1, 2048, 4, 128, True), ("C2", 2, 1990, 3, 128, False),
+                                                   ("R2", 1, 4096, 2, 128, True), ("C2", 1, 2048, 4, 64, True)])
+def test_backward_in_segments_for_few_long_sequences(base, B, T, H, d, with_h0):
+    """From three segments per sequence on, the backward runs every sequence in segments too (as the sequences of a
+    packed batch, twice: once for the state gradients that leave each segment, once for the results), with the
+    initial state, the final-state gradient and dh0 carried across the cuts."""
+    cfg = small(CONFIGS[base], B=B, T=T, H=H, d_k=d, d_v=d, seed=925 + T)
+    x = make_inputs(cfg, with_dO=True, with_h0=with_h0)
+    xd = gu.to_dev(x)
+    o, ht, g, plan, ws, lf, lb = gu.gpu_training_step(cfg, xd, h0=xd.get("h0"), dht=xd.get("dht"), want_dh0=with_h0)
+    assert lf == 2 and lb == 8, (lf, lb)    # summaries, fold, (states, sweep, gates), fold, (sweep, gates)
+    oref, htref = gu.oracle_forward(cfg, x, h0=x.get("h0"))
+    ref = gu.oracle_backward(cfg, x, h0=x.get("h0"), dht=x.get("dht"))
+    pairs = {"o": (o, oref), "ht": (ht, htref)}
+    pairs.update({n: (g[n], ref[r]) for n, r in gu.GRAD_NAMES.items() if g.get(n) is not None})
+    gu.assert_close({n: gu.rel_l2(a, r) for n, (a, r) in pairs.items()},
+                    {n: gu.row_err(a, r) for n, (a, r) in pairs.items()}, cfg.dtype, cfg)
+    g2 = api.sla_backward(plan, xd["q"], xd["k"], xd["v"], xd["log_decay"], xd["gq_logits"], xd["gk_logits"], xd["dO"],
+                          h0=xd.get("h0"), dht=xd.get("dht"), want_dh0=with_h0, workspace=ws)
+    torch.cuda.synchronize()
+    for n, t in g.items():
+        if t is not None:
+            assert torch.equal(t, g2[n]), n          # same bits on every run
 
 
 @pytest.mark.parametrize("base,B,T,H", [("C2", 8, 1024, 16), ("C2", 1, 4096, 4), ("C4", 4, 1024, 16)])
