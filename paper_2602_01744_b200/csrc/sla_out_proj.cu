@@ -8,8 +8,8 @@
 //   dW [K,  Dm ] = o^T dy                      A M-major  (rows of o: K contiguous),  B N-major (rows of dy)
 // CTA tile 128 x 256, 64 contraction steps per stage (four MMAs of K = 16), four stages of 48 KiB, two 256-column
 // accumulators in TMEM so that the epilogue of one tile runs under the MMAs of the next.  Roles: warp 0 TMA, warp 1
-// MMA issue, warps 2..5 epilogue (TMEM -> registers -> global memory, 64 or 128 contiguous bytes per thread and
-// step).  Tiles are dealt round robin with the column tiles of a row panel next to each other, so that the CTAs
+// MMA issue, warps 2..5 epilogue (TMEM -> registers -> swizzled staging blocks -> TMA stores for bf16 results; fp32 results
+// go from registers to global memory, 128 contiguous bytes per thread and step).  Tiles are dealt round robin with the column tiles of a row panel next to each other, so that the CTAs
 // running at a time share A panels and all of B in L2.  Tails: rows, columns and contraction steps past the edge
 // read as zeros through the tensor maps, stores are predicated.  Every wait is bounded and abortable.
 #include <algorithm>
@@ -28,7 +28,9 @@ namespace gm {
 constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4;
 constexpr uint32_t A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr uint32_t BLOCK64 = 64 * 128;                  // a [64 rows][128 B] swizzled block
-constexpr uint32_t OFF_BAR = STAGES * STAGE_BYTES;
+constexpr uint32_t OFF_OUT = STAGES * STAGE_BYTES;       // bf16 output staging: [4 epilogue warps][2][32 rows][128 B], swizzled
+constexpr uint32_t OUT_BYTES = 32 * 128;
+constexpr uint32_t OFF_BAR = OFF_OUT + 4 * 2 * OUT_BYTES;
 enum Bar { FULL = 0 /*[4]*/, EMPTY = 4 /*[4]*/, TFULL = 8 /*[2]*/, TEMPTY = 10 /*[2]*/, NBAR = 12 };
 constexpr uint32_t OFF_TMEM = OFF_BAR + NBAR * 8;       // TMEM base address, then the abort flag
 constexpr uint32_t SMEM_BYTES = OFF_TMEM + 16 + 1024;
@@ -46,7 +48,8 @@ struct GemmParams {
 // A_MN / B_MN: the operand's M (N) index is the contiguous one in memory (else its contraction index).
 template <bool A_MN, bool B_MN, typename TOUT>
 __global__ void __launch_bounds__(gm::NTHREADS, 1)
-k_dense_tc(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b, GemmParams p) {
+k_dense_tc(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
+           const __grid_constant__ CUtensorMap tm_c, GemmParams p) {
     using namespace gm;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -65,6 +68,7 @@ k_dense_tc(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUt
         fence_mbar_init();
         tma_prefetch_desc(&tm_a);
         tma_prefetch_desc(&tm_b);
+        if (sizeof(TOUT) == 2) tma_prefetch_desc(&tm_c);
     }
     if (warp == 0) tmem_alloc(base + OFF_TMEM, TMEM_COLS);
     tc_fence_before();
@@ -132,28 +136,51 @@ k_dense_tc(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUt
         // ---------------- epilogue: TMEM lane = output row ----------------
         const uint32_t quad = warp & 3;                     // the TMEM lanes this warp may read: 32 quad .. 32 quad + 31
         const uint32_t lane_base = (32u * quad) << 16;
-        uint32_t it = 0;
+        uint32_t it = 0, nst = 0;                           // nst: staged blocks so far (bf16 output)
         for (int t = blockIdx.x; t < tiles; t += gridDim.x, ++it) {
             const uint32_t acc = it & 1;
-            const int m = (t / tiles_n) * BM + 32 * quad + lane, n0 = (t % tiles_n) * BN;
+            const int m0 = (t / tiles_n) * BM + 32 * quad, m = m0 + lane, n0 = (t % tiles_n) * BN;
             wait(TFULL + acc, (it >> 1) & 1);
             tc_fence_after();
-            TOUT *crow = reinterpret_cast<TOUT *>(p.c) + (size_t)m * p.Nc + n0;
-#pragma unroll 2
-            for (int j = 0; j < BN / 32; ++j) {
-                float v[32];
-                tmem_ld32(tmem + lane_base + acc * BN + 32 * j, v);
-                tmem_wait_ld();
-                if (failed || m >= p.Mr) continue;
+            if (sizeof(TOUT) == 2) {
+                // bf16: 64 columns of the warp's 32 rows at a time through a swizzled staging block and a TMA store
+                // (which clips rows and columns past the edge); two blocks per warp, so a store runs under the next read-out
+                for (int jj = 0; jj < BN / 64; ++jj, ++nst) {
+                    float v0[32], v1[32];
+                    tmem_ld32(tmem + lane_base + acc * BN + 64 * jj, v0);
+                    tmem_ld32(tmem + lane_base + acc * BN + 64 * jj + 32, v1);
+                    tmem_wait_ld();
+                    const uint32_t blk = OFF_OUT + (quad * 2 + (nst & 1)) * OUT_BYTES;
+                    if (lane == 0 && nst >= 2) bulk_wait_read1();   // the store that last used this block has read it
+                    __syncwarp();
 #pragma unroll
-                for (int c = 0; c < 32; c += 8) {           // columns come in groups of 8 (Nc is a multiple of 8)
-                    if (n0 + 32 * j + c >= p.Nc) break;
-                    if (sizeof(TOUT) == 2) {
+                    for (int c = 0; c < 4; ++c) {
                         uint4 w;
-                        w.x = pack_bf16(v[c + 0], v[c + 1]); w.y = pack_bf16(v[c + 2], v[c + 3]);
-                        w.z = pack_bf16(v[c + 4], v[c + 5]); w.w = pack_bf16(v[c + 6], v[c + 7]);
-                        *reinterpret_cast<uint4 *>(crow + 32 * j + c) = w;
-                    } else {
+                        w.x = pack_bf16(v0[8 * c + 0], v0[8 * c + 1]); w.y = pack_bf16(v0[8 * c + 2], v0[8 * c + 3]);
+                        w.z = pack_bf16(v0[8 * c + 4], v0[8 * c + 5]); w.w = pack_bf16(v0[8 * c + 6], v0[8 * c + 7]);
+                        *reinterpret_cast<uint4 *>(sm + blk + lane * 128 + ((c ^ (lane & 7)) << 4)) = w;
+                        w.x = pack_bf16(v1[8 * c + 0], v1[8 * c + 1]); w.y = pack_bf16(v1[8 * c + 2], v1[8 * c + 3]);
+                        w.z = pack_bf16(v1[8 * c + 4], v1[8 * c + 5]); w.w = pack_bf16(v1[8 * c + 6], v1[8 * c + 7]);
+                        *reinterpret_cast<uint4 *>(sm + blk + lane * 128 + (((4 + c) ^ (lane & 7)) << 4)) = w;
+                    }
+                    fence_proxy_async();
+                    __syncwarp();
+                    if (lane == 0 && !failed && m0 < p.Mr && n0 + 64 * jj < p.Nc) {
+                        tma_store_2d(&tm_c, base + blk, n0 + 64 * jj, m0);
+                        bulk_commit();
+                    }
+                }
+            } else {
+                float *crow = reinterpret_cast<float *>(p.c) + (size_t)m * p.Nc + n0;
+#pragma unroll 2
+                for (int j = 0; j < BN / 32; ++j) {
+                    float v[32];
+                    tmem_ld32(tmem + lane_base + acc * BN + 32 * j, v);
+                    tmem_wait_ld();
+                    if (failed || m >= p.Mr) continue;
+#pragma unroll
+                    for (int c = 0; c < 32; c += 8) {       // columns come in groups of 8 (Nc is a multiple of 8)
+                        if (n0 + 32 * j + c >= p.Nc) break;
                         float4 *dst = reinterpret_cast<float4 *>(crow + 32 * j + c);
                         dst[0] = make_float4(v[c + 0], v[c + 1], v[c + 2], v[c + 3]);
                         dst[1] = make_float4(v[c + 4], v[c + 5], v[c + 6], v[c + 7]);
@@ -163,6 +190,7 @@ k_dense_tc(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUt
             tc_fence_before();
             mbar_arrive(bar(TEMPTY + acc));
         }
+        if (sizeof(TOUT) == 2 && lane == 0) bulk_wait0();   // the last stores have left shared memory and landed
     }
     if (failed) atomicOr(p.status, STATUS_TIMEOUT);
     tc_fence_before();
@@ -196,12 +224,14 @@ int sm_count() {
 // and B as b (B_MN: b = B, [Kc, Nc]; else b = B^T, [Nc, Kc]).
 template <bool A_MN, bool B_MN, typename TOUT>
 int launch_dense(const void *a, const void *b, void *c, int Mr, int Nc, int Kc, int *status, cudaStream_t st) {
-    CUtensorMap ma, mb;
+    CUtensorMap ma, mb, mc;
+    if (sizeof(TOUT) == 2 ? !make_matrix_map(&mc, c, Mr, Nc, 32) : false) return -1;
+    if (sizeof(TOUT) != 2) mc = CUtensorMap();
     if (!(A_MN ? make_matrix_map(&ma, a, Kc, Mr, 64) : make_matrix_map(&ma, a, Mr, Kc, gm::BM))) return -1;
     if (!(B_MN ? make_matrix_map(&mb, b, Kc, Nc, 64) : make_matrix_map(&mb, b, Nc, Kc, gm::BN))) return -1;
     const int tiles = ((Mr + gm::BM - 1) / gm::BM) * ((Nc + gm::BN - 1) / gm::BN);
     GemmParams gp{c, Mr, Nc, Kc, status};
-    k_dense_tc<A_MN, B_MN, TOUT><<<std::min(tiles, sm_count()), gm::NTHREADS, gm::SMEM_BYTES, st>>>(ma, mb, gp);
+    k_dense_tc<A_MN, B_MN, TOUT><<<std::min(tiles, sm_count()), gm::NTHREADS, gm::SMEM_BYTES, st>>>(ma, mb, mc, gp);
     return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 
