@@ -104,7 +104,7 @@ sla_status sla_plan_destroy(sla_plan *plan);
  * sla_plan_workspace_bytes changes with the table: query it again.  n_seq == 0 returns the plan to a regular batch.
  * The plan copies the table (and owns a few small device arrays for it until it is destroyed or the table replaced);
  * this is a set-up call, not to be made between a forward and its backward pass.  Only plans that select the
- * tensor-core kernels (bf16, d_k = d_v = 128 or 64, chunk 64) take a table: SLA_ERR_UNSUPPORTED otherwise.  Calls on one
+ * tensor-core kernels (bf16, d_k and d_v 128 or 64, chunk 64) take a table: SLA_ERR_UNSUPPORTED otherwise.  Calls on one
  * plan must be ordered on one stream (the per-sequence tensor maps are uploaded in stream order).
  */
 sla_status sla_plan_set_sequences(sla_plan *plan, const int32_t *cu_seqlens, int32_t n_seq);

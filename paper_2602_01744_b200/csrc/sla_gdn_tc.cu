@@ -1,4 +1,4 @@
-// Softmax-GatedDeltaNet forward on the 5th-generation tensor cores (bf16 I/O, d_k = d_v = 128 - or 64, run as 128 with zero padding supplied by the tensor maps -, chunk 64):
+// Softmax-GatedDeltaNet forward on the 5th-generation tensor cores (bf16 I/O, d_k and d_v 128 - or 64, run as 128 with zero padding supplied by the tensor maps -, chunk 64):
 // Eq. 14-16 with a scalar decay per (token, head), evaluated chunkwise in WY form.
 //
 // Per chunk (local token i, b_i = cumulative log-decay, Gam_i = e^{b_i}, S = state at the chunk start):
@@ -61,7 +61,7 @@ struct GdnParams {
     float scale;
     const SeqInfo *seqs;    // packed variable-length batch: per-sequence table and tensor maps (q, k, v, o), else nullptr
     const CUtensorMap *vmaps;
-    int d;                  // head width d_k = d_v: 128, or 64 (the upper half of every 128-wide tile is then zero padding)
+    int dk, dv;             // head widths, each 128 or 64 (the upper half of a 128-wide tile is then zero padding)
 };
 
 __global__ void __launch_bounds__(gd::NTHREADS, 1)
@@ -246,7 +246,7 @@ k_gdn_fwd_tc(const __grid_constant__ CUtensorMap gm_q, const __grid_constant__ C
 
         uint8_t *rec0 = p.save ? p.save + slot * REC_BYTES : nullptr;   // this sequence's records
         {   // initial state: fp32 into TMEM, bf16 copy into shared memory (row = key dimension)
-            const float *src = state_row(p.h0, bh, row, colhalf, p.d);
+            const float *src = state_row(p.h0, bh, row, colhalf, p.dk, p.dv);
 #pragma unroll
             for (int part = 0; part < 2; ++part) {
                 float v[32];
@@ -544,7 +544,7 @@ k_gdn_fwd_tc(const __grid_constant__ CUtensorMap gm_q, const __grid_constant__ C
         }
 
         if (p.ht) {   // final state, fp32 (each thread reads back what it wrote in the last rescale)
-            float *dst = state_row(p.ht, bh, row, colhalf, p.d);
+            float *dst = state_row(p.ht, bh, row, colhalf, p.dk, p.dv);
 #pragma unroll
             for (int part = 0; part < 2; ++part) {
                 float v[32];
@@ -565,7 +565,7 @@ k_gdn_fwd_tc(const __grid_constant__ CUtensorMap gm_q, const __grid_constant__ C
 }  // namespace
 
 bool gdn_tc_supported(const Dims &d) {
-    return d.variant == SLA_GDN && d.io_bf16 && d.dk == d.dv && (d.dk == 128 || d.dk == 64) && d.C == 64;
+    return d.variant == SLA_GDN && d.io_bf16 && (d.dk == 128 || d.dk == 64) && (d.dv == 128 || d.dv == 64) && d.C == 64;
 }
 
 int gdn_tc_configure() {
@@ -578,13 +578,13 @@ int gdn_tc_configure() {
 static const CUtensorMap *gdn_varlen_maps(const Dims &d, const FwdArgs &a, int r, cudaStream_t st) {
     const void *key[] = {a.q, a.k, a.v, a.o};
     return varlen_maps(*a.vl, r, key, 4, st, [&](const SeqInfo &si, CUtensorMap *m) {
-        const size_t off = (size_t)si.t0 * d.H * d.dk;
-        if (!make_tile_map(m + 0, (const __nv_bfloat16 *)a.q + off, 1, si.T, d.H, d.dk) ||
-            !make_tile_map(m + 1, (const __nv_bfloat16 *)a.k + off, 1, si.T, d.H, d.dk) ||
-            !make_tile_map(m + 2, (const __nv_bfloat16 *)a.v + off, 1, si.T, d.H, d.dk))
+        const size_t tok = (size_t)si.t0 * d.H;      // (q, k are d_k wide, v, o and their gradients d_v)
+        if (!make_tile_map(m + 0, (const __nv_bfloat16 *)a.q + tok * d.dk, 1, si.T, d.H, d.dk) ||
+            !make_tile_map(m + 1, (const __nv_bfloat16 *)a.k + tok * d.dk, 1, si.T, d.H, d.dk) ||
+            !make_tile_map(m + 2, (const __nv_bfloat16 *)a.v + tok * d.dv, 1, si.T, d.H, d.dv))
             return false;
         if (!a.o) { m[3] = m[0]; return true; }
-        return make_tile_map(m + 3, (__nv_bfloat16 *)a.o + off, 1, si.T, d.H, d.dk);
+        return make_tile_map(m + 3, (__nv_bfloat16 *)a.o + tok * d.dv, 1, si.T, d.H, d.dv);
     });
 }
 
@@ -592,13 +592,13 @@ static const CUtensorMap *gdn_varlen_maps(const Dims &d, const FwdArgs &a, int r
 int gdn_tc_forward_save(const Dims &d, const FwdArgs &a, uint8_t *save, int *status, cudaStream_t st, Tracer &tr) {
     CUtensorMap mq, mk, mv;
     if (!make_tile_map(&mq, a.q, d.B, d.T, d.H, d.dk) || !make_tile_map(&mk, a.k, d.B, d.T, d.H, d.dk) ||
-        !make_tile_map(&mv, a.v, d.B, d.T, d.H, d.dk))
+        !make_tile_map(&mv, a.v, d.B, d.T, d.H, d.dv))
         return -1;
     const bool vl = a.vl && a.vl->n_seq;
     const CUtensorMap *vm = vl ? gdn_varlen_maps(d, a, 1, st) : nullptr;
     if (vl && !vm) return -1;
     GdnParams p{a.lq, a.lk, a.log_decay, a.beta, a.h0, nullptr, save, 0, status, d.T, d.H, d.NT, d.scale,
-                vl ? a.vl->d_seqs : nullptr, vm, d.dk};
+                vl ? a.vl->d_seqs : nullptr, vm, d.dk, d.dv};
     k_gdn_fwd_tc<<<vl ? a.vl->n_seq * d.H : d.B * d.H, gd::NTHREADS, gd::SMEM_BYTES, st>>>(mq, mk, mv, mq /* unused: nothing is stored */, p);
     tr.mark("gdn_states_tc");
     return cudaGetLastError() == cudaSuccess ? 1 : -1;
@@ -608,13 +608,13 @@ int gdn_tc_forward_save(const Dims &d, const FwdArgs &a, uint8_t *save, int *sta
 int gdn_tc_forward(const Dims &d, const FwdArgs &a, uint8_t *save, int *status, cudaStream_t st, Tracer &tr) {
     CUtensorMap mq, mk, mv, mo;
     if (!make_tile_map(&mq, a.q, d.B, d.T, d.H, d.dk) || !make_tile_map(&mk, a.k, d.B, d.T, d.H, d.dk) ||
-        !make_tile_map(&mv, a.v, d.B, d.T, d.H, d.dk) || !make_tile_map(&mo, a.o, d.B, d.T, d.H, d.dk))
+        !make_tile_map(&mv, a.v, d.B, d.T, d.H, d.dv) || !make_tile_map(&mo, a.o, d.B, d.T, d.H, d.dv))
         return -1;
     const bool vl = a.vl && a.vl->n_seq;
     const CUtensorMap *vm = vl ? gdn_varlen_maps(d, a, 0, st) : nullptr;
     if (vl && !vm) return -1;
     GdnParams p{a.lq, a.lk, a.log_decay, a.beta, a.h0, a.ht, save, 1, status, d.T, d.H, d.NT, d.scale,
-                vl ? a.vl->d_seqs : nullptr, vm, d.dk};
+                vl ? a.vl->d_seqs : nullptr, vm, d.dk, d.dv};
     k_gdn_fwd_tc<<<vl ? a.vl->n_seq * d.H : d.B * d.H, gd::NTHREADS, gd::SMEM_BYTES, st>>>(mq, mk, mv, mo, p);
     tr.mark("gdn_fwd_tc");
     return cudaGetLastError() == cudaSuccess ? 1 : -1;

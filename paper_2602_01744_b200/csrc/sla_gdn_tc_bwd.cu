@@ -1,4 +1,4 @@
-// Softmax-GatedDeltaNet backward on the 5th-generation tensor cores (bf16 I/O, d_k = d_v = 128 - or 64, run as 128 with zero padding supplied by the tensor maps -, chunk 64).
+// Softmax-GatedDeltaNet backward on the 5th-generation tensor cores (bf16 I/O, d_k and d_v 128 - or 64, run as 128 with zero padding supplied by the tensor maps -, chunk 64).
 //
 // The paper states no gradients; these are the chain rule applied to Eq. 4, 14-16 in the chunkwise WY form of the
 // forward kernel (sla_gdn_tc.cu), which in save mode leaves per chunk the bf16 state image S_n, U and T.
@@ -70,7 +70,7 @@ struct GdnBwdParams {
     float scale;
     const SeqInfo *seqs;            // packed variable-length batch: per-sequence table and tensor maps (the seven below), else nullptr
     const CUtensorMap *vmaps;
-    int d;                  // head width d_k = d_v: 128, or 64 (the upper half of every 128-wide tile is then zero padding)
+    int dk, dv;             // head widths, each 128 or 64 (the upper half of a 128-wide tile is then zero padding)
 };
 
 __global__ void __launch_bounds__(gb::NTHREADS, 1)
@@ -404,7 +404,7 @@ k_gdn_bwd_tc(const __grid_constant__ CUtensorMap gm_q, const __grid_constant__ C
         {   // dS_NT = dht (or zero) into TMEM; carried scalar <dht, S_NT>
             float v0[32], v1[32];
             if (p.dht) wait(INIT_FULL, 0);
-            const float *src = state_row(p.dht, bh, row, ch, p.d);
+            const float *src = state_row(p.dht, bh, row, ch, p.dk, p.dv);
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
                 v0[j] = src ? src[j] : 0.f;
@@ -741,7 +741,7 @@ k_gdn_bwd_tc(const __grid_constant__ CUtensorMap gm_q, const __grid_constant__ C
         }
 
         if (p.dh0) {   // dS_0, fp32 (complete since the last chunk's group 3)
-            float *dst = state_row(p.dh0, bh, row, ch, p.d);
+            float *dst = state_row(p.dh0, bh, row, ch, p.dk, p.dv);
 #pragma unroll
             for (int part = 0; part < 2; ++part) {
                 float v[32];
@@ -781,9 +781,9 @@ uint8_t *gdn_tc_records(float *ws) { return reinterpret_cast<uint8_t *>(ws); }
 int gdn_tc_backward(const Dims &d, const BwdArgs &a, bool have_records, int *status, cudaStream_t st, Tracer &tr) {
     CUtensorMap mq, mk, mv, mdo, mdq, mdk, mdv;
     if (!make_tile_map(&mq, a.q, d.B, d.T, d.H, d.dk) || !make_tile_map(&mk, a.k, d.B, d.T, d.H, d.dk) ||
-        !make_tile_map(&mv, a.v, d.B, d.T, d.H, d.dk) || !make_tile_map(&mdo, a.dO, d.B, d.T, d.H, d.dk) ||
+        !make_tile_map(&mv, a.v, d.B, d.T, d.H, d.dv) || !make_tile_map(&mdo, a.dO, d.B, d.T, d.H, d.dv) ||
         !make_tile_map(&mdq, a.dq, d.B, d.T, d.H, d.dk) || !make_tile_map(&mdk, a.dk, d.B, d.T, d.H, d.dk) ||
-        !make_tile_map(&mdv, a.dv, d.B, d.T, d.H, d.dk))
+        !make_tile_map(&mdv, a.dv, d.B, d.T, d.H, d.dv))
         return -1;
     Varlen *vl = (a.vl && a.vl->n_seq) ? a.vl : nullptr;
     const size_t bth = (size_t)d.B * d.T * d.H;
@@ -797,16 +797,16 @@ int gdn_tc_backward(const Dims &d, const BwdArgs &a, bool have_records, int *sta
     if (vl) {
         const void *key[] = {a.q, a.k, a.v, a.dO, a.dq, a.dk, a.dv};
         vm = varlen_maps(*vl, 2, key, 7, st, [&](const SeqInfo &si, CUtensorMap *m) {
-            const size_t off = (size_t)si.t0 * d.H * d.dk;
+            const size_t tok = (size_t)si.t0 * d.H;      // (q, k are d_k wide, v, o and their gradients d_v)
             const void *src[7] = {a.q, a.k, a.v, a.dO, a.dq, a.dk, a.dv};
             for (int i = 0; i < 7; ++i)
-                if (!make_tile_map(m + i, (const __nv_bfloat16 *)src[i] + off, 1, si.T, d.H, d.dk)) return false;
+                if (!make_tile_map(m + i, (const __nv_bfloat16 *)src[i] + tok * (i == 2 || i == 3 || i == 6 ? d.dv : d.dk), 1, si.T, d.H, (i == 2 || i == 3 || i == 6 ? d.dv : d.dk))) return false;
             return true;
         });
         if (!vm) return -1;
     }
     GdnBwdParams bp{a.lq, a.lk, a.log_decay, a.beta, a.dht, save, a.dlog_decay, a.dbeta, pq, pk, a.dh0, status,
-                    d.T, d.H, d.NT, d.scale, vl ? vl->d_seqs : nullptr, vm, d.dk};
+                    d.T, d.H, d.NT, d.scale, vl ? vl->d_seqs : nullptr, vm, d.dk, d.dv};
     k_gdn_bwd_tc<<<vl ? vl->n_seq * d.H : d.B * d.H, gb::NTHREADS, gb::SMEM_BYTES, st>>>(mq, mk, mv, mdo, mdq, mdk, mdv, bp);
     tr.mark("gdn_bwd_tc");
     if (gate_bwd_prod(a.lq, a.lk, pq, pk, a.dlq, a.dlk, (long)d.B * d.T, d.H, st) < 0) return -1;

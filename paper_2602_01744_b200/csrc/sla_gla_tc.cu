@@ -1,4 +1,4 @@
-// Softmax-GLA forward on the 5th-generation tensor cores (bf16 I/O, d_k = d_v = 128 - or 64, run as 128 with zero padding supplied by the tensor maps -, chunk 64).
+// Softmax-GLA forward on the 5th-generation tensor cores (bf16 I/O, d_k and d_v 128 - or 64, run as 128 with zero padding supplied by the tensor maps -, chunk 64).
 //
 // One CTA owns one (batch, head) sequence and walks its chunks in order, so q, k, v, log-decay are
 // read from HBM exactly once and o is written once; nothing else touches HBM.
@@ -60,7 +60,7 @@ struct FwdParams {
     const float *log_gamma;         // Softmax-RetNet: [H] constant log-decays (no log-decay tensor is read); else nullptr
     const SeqInfo *seqs;            // packed variable-length batch: per-sequence table and tensor maps (q, k, v, g, o), else nullptr
     const CUtensorMap *vmaps;
-    int d;                  // head width d_k = d_v: 128, or 64 (the upper half of every 128-wide tile is then zero padding)
+    int dk, dv;             // head widths, each 128 or 64 (the upper half of a 128-wide tile is then zero padding)
 };
 
 // One CTA per (batch, head) sequence, five roles that only meet on mbarriers:
@@ -293,7 +293,7 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap gm_q, const __grid_constant__ C
         {   // initial state: fp32 into TMEM, bf16 copy into shared memory (row = key dimension).  A segment that is not the
             // first starts from S <- diag(gam_s) S + fin_s taken over the segments s before it (a short scan over their
             // summaries, elementwise, done here rather than in a launch of its own).
-            const float *src = state_row(p.h0, bh, row, colhalf, p.d);
+            const float *src = state_row(p.h0, bh, row, colhalf, p.dk, p.dv);
 #pragma unroll
             for (int part = 0; part < 2; ++part) {
                 float v[32];
@@ -428,7 +428,7 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap gm_q, const __grid_constant__ C
         }
 
         if (p.ht && seg == p.P - 1) {   // final state, fp32 (each thread reads back what it wrote in the last rescale)
-            float *dst = state_row(p.ht, bh, row, colhalf, p.d);
+            float *dst = state_row(p.ht, bh, row, colhalf, p.dk, p.dv);
 #pragma unroll
             for (int part = 0; part < 2; ++part) {
                 float v[32];
@@ -475,7 +475,7 @@ void choose_segments(const Dims &d, int &P, int &L) {
 // Softmax-GLA (Eq. 12-13) and Softmax-RetNet (Eq. 10-11: the same recurrence with a constant decay per head, which the
 // kernels generate instead of reading a [B,T,H,d_k] tensor).
 bool gla_tc_supported(const Dims &d) {
-    return (d.variant == SLA_GLA || d.variant == SLA_RETNET) && d.io_bf16 && d.dk == d.dv && (d.dk == 128 || d.dk == 64) && d.C == 64;
+    return (d.variant == SLA_GLA || d.variant == SLA_RETNET) && d.io_bf16 && (d.dk == 128 || d.dk == 64) && (d.dv == 128 || d.dv == 64) && d.C == 64;
 }
 
 int gla_tc_configure() {
@@ -511,23 +511,23 @@ int gla_tc_forward(const Dims &d, const FwdArgs &a, uint8_t *simg, int *status, 
     if (a.vl && a.vl->n_seq) {          // packed batch: one CTA per (sequence, head), per-sequence tensor maps
         const void *key[] = {a.q, a.k, a.v, a.log_decay, a.o};
         const CUtensorMap *vm = varlen_maps(*a.vl, 0, key, 5, st, [&](const SeqInfo &si, CUtensorMap *m) {
-            const size_t off = (size_t)si.t0 * d.H * d.dk;
+            const size_t tok = (size_t)si.t0 * d.H;      // (q, k are d_k wide, v, o and their gradients d_v)
             const __nv_bfloat16 *q = (const __nv_bfloat16 *)a.q, *k = (const __nv_bfloat16 *)a.k, *v = (const __nv_bfloat16 *)a.v;
-            if (!make_tile_map(m + 0, q + off, 1, si.T, d.H, d.dk) || !make_tile_map(m + 1, k + off, 1, si.T, d.H, d.dk) ||
-                !make_tile_map(m + 2, v + off, 1, si.T, d.H, d.dk) || !make_tile_map(m + 4, (__nv_bfloat16 *)a.o + off, 1, si.T, d.H, d.dk))
+            if (!make_tile_map(m + 0, q + tok * d.dk, 1, si.T, d.H, d.dk) || !make_tile_map(m + 1, k + tok * d.dk, 1, si.T, d.H, d.dk) ||
+                !make_tile_map(m + 2, v + tok * d.dv, 1, si.T, d.H, d.dv) || !make_tile_map(m + 4, (__nv_bfloat16 *)a.o + tok * d.dv, 1, si.T, d.H, d.dv))
                 return false;
             if (retnet) { m[3] = m[0]; return true; }
-            return make_map(m + 3, a.log_decay + off, 1, si.T, d.H, d.dk, true, 128);
+            return make_map(m + 3, a.log_decay + tok * d.dk, 1, si.T, d.H, d.dk, true, 128);
         });
         if (!vm || !make_tile_map(&mq, a.q, d.B, d.T, d.H, d.dk)) return -1;
         FwdParams p{a.lq, a.lk, a.h0, nullptr, nullptr, (__nv_bfloat16 *)a.o, a.ht, simg, status, d.T, d.H, d.NT, 1, d.NT, d.scale,
-                    retnet ? a.log_decay : nullptr, a.vl->d_seqs, vm, d.dk};
+                    retnet ? a.log_decay : nullptr, a.vl->d_seqs, vm, d.dk, d.dv};
         k_gla_fwd_tc<<<a.vl->n_seq * d.H, NTHREADS, SMEM_BYTES, st>>>(mq, mq, mq, mq, mq, p);
         tr.mark("gla_fwd_tc");
         return cudaGetLastError() == cudaSuccess ? 1 : -1;
     }
     if (!make_tile_map(&mq, a.q, d.B, d.T, d.H, d.dk) || !make_tile_map(&mk, a.k, d.B, d.T, d.H, d.dk) ||
-        !make_tile_map(&mv, a.v, d.B, d.T, d.H, d.dk) || !make_tile_map(&mo, a.o, d.B, d.T, d.H, d.dk))
+        !make_tile_map(&mv, a.v, d.B, d.T, d.H, d.dv) || !make_tile_map(&mo, a.o, d.B, d.T, d.H, d.dv))
         return -1;
     if (retnet) mg = mq;   // (never used: the decay is generated in the kernel)
     else if (!make_map(&mg, a.log_decay, d.B, d.T, d.H, d.dk, true, 128)) return -1;
@@ -542,7 +542,7 @@ int gla_tc_forward(const Dims &d, const FwdArgs &a, uint8_t *simg, int *status, 
         launches = 2;
         simg = nullptr;
     }
-    FwdParams p{a.lq, a.lk, a.h0, fin, gam, (__nv_bfloat16 *)a.o, a.ht, simg, status, d.T, d.H, d.NT, P, L, d.scale, retnet ? a.log_decay : nullptr, nullptr, nullptr, d.dk};
+    FwdParams p{a.lq, a.lk, a.h0, fin, gam, (__nv_bfloat16 *)a.o, a.ht, simg, status, d.T, d.H, d.NT, P, L, d.scale, retnet ? a.log_decay : nullptr, nullptr, nullptr, d.dk, d.dv};
     k_gla_fwd_tc<<<d.B * d.H * P, NTHREADS, SMEM_BYTES, st>>>(mq, mk, mv, mg, mo, p);
     tr.mark("gla_fwd_tc");
     return cudaGetLastError() == cudaSuccess ? launches : -1;

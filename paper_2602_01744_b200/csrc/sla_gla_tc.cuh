@@ -87,12 +87,12 @@ inline bool make_tile_map(CUtensorMap *m, const void *ptr, int B, int T, int H, 
     return r == CUDA_SUCCESS;
 }
 
-// Row `row`, columns 64*half .. 64*half+63 of the fp32 [d, d] state of sequence-head bh inside a [.., d, d] tensor, as
-// seen by the thread that owns that part of the kernels' 128 x 128 state; nullptr where a 64-wide head has no such
-// part (the padded rows and columns stay zero) or the tensor is absent.
+// Row `row`, columns 64*half .. 64*half+63 of the fp32 [dk, dv] state of sequence-head bh inside a [.., dk, dv]
+// tensor, as seen by the thread that owns that part of the kernels' 128 x 128 state; nullptr where a 64-wide head has
+// no such part (the padded rows and columns stay zero) or the tensor is absent.
 template <typename T>
-__device__ __forceinline__ T *state_row(T *t, size_t bh, int row, int half, int d) {
-    return (t && row < d && 64 * half < d) ? t + (bh * d + row) * d + 64 * half : nullptr;
+__device__ __forceinline__ T *state_row(T *t, size_t bh, int row, int half, int dk, int dv) {
+    return (t && row < dk && 64 * half < dv) ? t + (bh * dk + row) * dv + 64 * half : nullptr;
 }
 
 // Device array of the per-sequence tensor maps of region r of a packed batch: `make(seq, maps)` encodes one sequence's

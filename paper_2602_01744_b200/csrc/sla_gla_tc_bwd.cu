@@ -1,4 +1,4 @@
-// Softmax-GLA backward on the 5th-generation tensor cores (bf16 I/O, d_k = d_v = 128 - or 64, run as 128 with zero padding supplied by the tensor maps -, chunk 64).
+// Softmax-GLA backward on the 5th-generation tensor cores (bf16 I/O, d_k and d_v 128 - or 64, run as 128 with zero padding supplied by the tensor maps -, chunk 64).
 //
 // The paper states no gradients; these are the chain rule applied to Eq. 4, 12-13, evaluated chunkwise.
 // Two sweeps per (batch, head) sequence, one CTA each, chunk after chunk:
@@ -62,7 +62,7 @@ struct StatesParams {
     const float *log_gamma; // Softmax-RetNet: [H] constant log-decays (no log-decay tensor is read); else nullptr
     const SeqInfo *seqs;    // packed variable-length batch: per-sequence table and tensor maps (k, v, g), else nullptr
     const CUtensorMap *vmaps;
-    int d;                  // head width d_k = d_v: 128, or 64 (the upper half of every 128-wide tile is then zero padding)
+    int dk, dv;             // head widths, each 128 or 64 (the upper half of a 128-wide tile is then zero padding)
 };
 
 // thread (row, colhalf) holds 32 consecutive state values of its row: bf16 them into the operand image
@@ -228,7 +228,7 @@ k_gla_states_tc(const __grid_constant__ CUtensorMap gm_k, const __grid_constant_
         const int colhalf = warp >> 2;
         const int row = 32 * (warp & 3) + lane;
         {   // S_0: fp32 into TMEM, bf16 image into slot 0
-            const float *src = images ? state_row(p.h0, bh, row, colhalf, p.d) : nullptr;
+            const float *src = images ? state_row(p.h0, bh, row, colhalf, p.dk, p.dv) : nullptr;
 #pragma unroll
             for (int part = 0; part < 2; ++part) {
                 float v[32];
@@ -340,7 +340,7 @@ struct BwdParams {
     const float *log_gamma;         // Softmax-RetNet: [H] constant log-decays (no log-decay read, no log-decay gradient)
     const SeqInfo *seqs;            // packed variable-length batch: per-sequence table and tensor maps (the nine below), else nullptr
     const CUtensorMap *vmaps;
-    int d;                  // head width d_k = d_v: 128, or 64 (the upper half of every 128-wide tile is then zero padding)
+    int dk, dv;             // head widths, each 128 or 64 (the upper half of a 128-wide tile is then zero padding)
 };
 
 // Sum v[j] over the 32 lanes for every j: afterwards lane l holds the total of v[l] in v[0].
@@ -633,7 +633,7 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap gm_q, const __grid_constant__ C
         {   // dS_NT = dht (or zero) into TMEM; R_{NT-1} = rowsum(dht * S_NT)
             float rpart = 0.f;
             if (p.dht) wait(INIT_FULL, 0);
-            const float *src = state_row(p.dht, bh, row, wh, p.d);
+            const float *src = state_row(p.dht, bh, row, wh, p.dk, p.dv);
 #pragma unroll
             for (int part = 0; part < 2; ++part) {
                 float v[32];
@@ -815,7 +815,7 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap gm_q, const __grid_constant__ C
         }
 
         if (p.dh0) {   // dS_0, fp32 (the last chunk's MMAs were waited for above)
-            float *dst = state_row(p.dh0, bh, row, wh, p.d);
+            float *dst = state_row(p.dh0, bh, row, wh, p.dk, p.dv);
 #pragma unroll
             for (int part = 0; part < 2; ++part) {
                 float v[32];
@@ -872,24 +872,24 @@ void launch_gate_bwd_prod(const float *lq, const float *lk, const float *Pq, con
 // summaries are indexed by (b*H + h)*P + p as the summary kernel leaves them, states by ((b*P + p)*H + h) as the
 // packed kernels read them.  One thread per state element, a short loop over the segments.
 // Start states: S_0 = h0 (or zero), S_{p+1} = diag(gam_p) S_p + fin_p.
-__global__ void k_fold_segment_states(int H, int P, int d, const float *__restrict__ h0, const float *__restrict__ fin,
+__global__ void k_fold_segment_states(int H, int P, int dk, int dv, const float *__restrict__ h0, const float *__restrict__ fin,
                                       const float *__restrict__ gam, float *__restrict__ h0seg) {
     const int bh = blockIdx.x, b = bh / H, h = bh % H, row = blockIdx.y, col = threadIdx.x;
-    float sv = h0 ? h0[((size_t)bh * d + row) * d + col] : 0.f;
+    float sv = h0 ? h0[((size_t)bh * dk + row) * dv + col] : 0.f;
     for (int p = 0; p < P; ++p) {
-        h0seg[((((size_t)b * P + p) * H + h) * d + row) * d + col] = sv;
+        h0seg[((((size_t)b * P + p) * H + h) * dk + row) * dv + col] = sv;
         const size_t c = (size_t)bh * P + p;
         sv = fmaf(gam[c * D + row], sv, fin[(c * D + row) * D + col]);
     }
 }
 // State gradients entering each segment from its right: R_{P-1} = dht (or zero), R_p = diag(gam_{p+1}) R_{p+1} + F_{p+1},
 // F_p being what segment p alone sends out of its left edge (its dh0 when run with a zero dht).
-__global__ void k_fold_segment_dstates(int H, int P, int d, const float *__restrict__ dht, const float *__restrict__ gam,
+__global__ void k_fold_segment_dstates(int H, int P, int dk, int dv, const float *__restrict__ dht, const float *__restrict__ gam,
                                        const float *__restrict__ dsfin, float *__restrict__ dhtseg) {
     const int bh = blockIdx.x, b = bh / H, h = bh % H, row = blockIdx.y, col = threadIdx.x;
-    float r = dht ? dht[((size_t)bh * d + row) * d + col] : 0.f;
+    float r = dht ? dht[((size_t)bh * dk + row) * dv + col] : 0.f;
     for (int p = P - 1; p >= 0; --p) {
-        const size_t i = ((((size_t)b * P + p) * H + h) * d + row) * d + col;
+        const size_t i = ((((size_t)b * P + p) * H + h) * dk + row) * dv + col;
         dhtseg[i] = r;
         r = fmaf(gam[((size_t)bh * P + p) * D + row], r, dsfin[i]);
     }
@@ -935,11 +935,11 @@ int gla_tc_segment_summaries(const Dims &d, const FwdArgs &a, int P, int L, floa
                              cudaStream_t st, Tracer &tr) {
     CUtensorMap mk, mv, mg;
     const bool retnet = d.variant == SLA_RETNET;
-    if (!make_tile_map(&mk, a.k, d.B, d.T, d.H, d.dk) || !make_tile_map(&mv, a.v, d.B, d.T, d.H, d.dk)) return -1;
+    if (!make_tile_map(&mk, a.k, d.B, d.T, d.H, d.dk) || !make_tile_map(&mv, a.v, d.B, d.T, d.H, d.dv)) return -1;
     if (retnet) mg = mk;   // (never used: the decay is generated in the kernel)
     else if (!make_map(&mg, a.log_decay, d.B, d.T, d.H, d.dk, true, 128)) return -1;
     StatesParams sp{a.lq, a.lk, nullptr, nullptr, fin, gam, status, d.T, d.H, d.NT, P, L, retnet ? a.log_decay : nullptr,
-                    nullptr, nullptr, d.dk};
+                    nullptr, nullptr, d.dk, d.dv};
     k_gla_states_tc<<<d.B * d.H * P, st1::NTHREADS, st1::SMEM_BYTES, st>>>(mk, mv, mg, sp);
     tr.mark("gla_segment_states_tc");
     return cudaGetLastError() == cudaSuccess ? 1 : -1;
@@ -951,9 +951,9 @@ int gla_tc_backward(const Dims &d, const BwdArgs &a, bool have_states, int *stat
     CUtensorMap mq, mk, mv, mdo, mg, mdq, mdk, mdv, mdg;
     const bool retnet = d.variant == SLA_RETNET;      // constant decay: no log-decay tensor to read, no gradient for it
     if (!make_tile_map(&mq, a.q, d.B, d.T, d.H, d.dk) || !make_tile_map(&mk, a.k, d.B, d.T, d.H, d.dk) ||
-        !make_tile_map(&mv, a.v, d.B, d.T, d.H, d.dk) || !make_tile_map(&mdo, a.dO, d.B, d.T, d.H, d.dk) ||
+        !make_tile_map(&mv, a.v, d.B, d.T, d.H, d.dv) || !make_tile_map(&mdo, a.dO, d.B, d.T, d.H, d.dv) ||
         !make_tile_map(&mdq, a.dq, d.B, d.T, d.H, d.dk) || !make_tile_map(&mdk, a.dk, d.B, d.T, d.H, d.dk) ||
-        !make_tile_map(&mdv, a.dv, d.B, d.T, d.H, d.dk))
+        !make_tile_map(&mdv, a.dv, d.B, d.T, d.H, d.dv))
         return -1;
     if (retnet) { mg = mq; mdg = mdq; }               // (never used)
     else if (!make_map(&mg, a.log_decay, d.B, d.T, d.H, d.dk, true, 128) ||
@@ -976,15 +976,15 @@ int gla_tc_backward(const Dims &d, const BwdArgs &a, bool have_states, int *stat
         if (vl) {
             const void *key[] = {a.k, a.v, a.log_decay};
             vm = varlen_maps(*vl, 1, key, 3, st, [&](const SeqInfo &si, CUtensorMap *m) {
-                const size_t off = (size_t)si.t0 * d.H * d.dk;
-                if (!make_tile_map(m + 0, k + off, 1, si.T, d.H, d.dk) || !make_tile_map(m + 1, v + off, 1, si.T, d.H, d.dk)) return false;
+                const size_t tok = (size_t)si.t0 * d.H;      // (q, k are d_k wide, v, o and their gradients d_v)
+                if (!make_tile_map(m + 0, k + tok * d.dk, 1, si.T, d.H, d.dk) || !make_tile_map(m + 1, v + tok * d.dv, 1, si.T, d.H, d.dv)) return false;
                 if (retnet) { m[2] = m[0]; return true; }
-                return make_map(m + 2, a.log_decay + off, 1, si.T, d.H, d.dk, true, 128);
+                return make_map(m + 2, a.log_decay + tok * d.dk, 1, si.T, d.H, d.dk, true, 128);
             });
             if (!vm) return -1;
         }
         StatesParams sp{a.lq, a.lk, a.h0, simg, nullptr, nullptr, status, d.T, d.H, d.NT, 1, d.NT, retnet ? a.log_decay : nullptr,
-                        dseqs, vm, d.dk};
+                        dseqs, vm, d.dk, d.dv};
         k_gla_states_tc<<<ctas, st1::NTHREADS, st1::SMEM_BYTES, st>>>(mk, mv, mg, sp);
         tr.mark("gla_states_tc");
     }
@@ -992,20 +992,20 @@ int gla_tc_backward(const Dims &d, const BwdArgs &a, bool have_states, int *stat
     if (vl) {
         const void *key[] = {a.q, a.k, a.v, a.dO, a.log_decay, a.dq, a.dk, a.dv, a.dlog_decay};
         vm = varlen_maps(*vl, 2, key, 9, st, [&](const SeqInfo &si, CUtensorMap *m) {
-            const size_t off = (size_t)si.t0 * d.H * d.dk;
-            if (!make_tile_map(m + 0, q + off, 1, si.T, d.H, d.dk) || !make_tile_map(m + 1, k + off, 1, si.T, d.H, d.dk) ||
-                !make_tile_map(m + 2, v + off, 1, si.T, d.H, d.dk) || !make_tile_map(m + 3, dO + off, 1, si.T, d.H, d.dk) ||
-                !make_tile_map(m + 5, (__nv_bfloat16 *)a.dq + off, 1, si.T, d.H, d.dk) ||
-                !make_tile_map(m + 6, (__nv_bfloat16 *)a.dk + off, 1, si.T, d.H, d.dk) ||
-                !make_tile_map(m + 7, (__nv_bfloat16 *)a.dv + off, 1, si.T, d.H, d.dk))
+            const size_t tok = (size_t)si.t0 * d.H;      // (q, k are d_k wide, v, o and their gradients d_v)
+            if (!make_tile_map(m + 0, q + tok * d.dk, 1, si.T, d.H, d.dk) || !make_tile_map(m + 1, k + tok * d.dk, 1, si.T, d.H, d.dk) ||
+                !make_tile_map(m + 2, v + tok * d.dv, 1, si.T, d.H, d.dv) || !make_tile_map(m + 3, dO + tok * d.dv, 1, si.T, d.H, d.dv) ||
+                !make_tile_map(m + 5, (__nv_bfloat16 *)a.dq + tok * d.dk, 1, si.T, d.H, d.dk) ||
+                !make_tile_map(m + 6, (__nv_bfloat16 *)a.dk + tok * d.dk, 1, si.T, d.H, d.dk) ||
+                !make_tile_map(m + 7, (__nv_bfloat16 *)a.dv + tok * d.dv, 1, si.T, d.H, d.dv))
                 return false;
             if (retnet) { m[4] = m[0]; m[8] = m[5]; return true; }
-            return make_map(m + 4, a.log_decay + off, 1, si.T, d.H, d.dk, true, 128) &&
-                   make_map(m + 8, a.dlog_decay + off, 1, si.T, d.H, d.dk, true, 128);
+            return make_map(m + 4, a.log_decay + tok * d.dk, 1, si.T, d.H, d.dk, true, 128) &&
+                   make_map(m + 8, a.dlog_decay + tok * d.dk, 1, si.T, d.H, d.dk, true, 128);
         });
         if (!vm) return -1;
     }
-    BwdParams bp{a.lq, a.lk, a.dht, simg, pq, pk, a.dh0, status, d.T, d.H, d.NT, d.scale, retnet ? a.log_decay : nullptr, dseqs, vm, d.dk};
+    BwdParams bp{a.lq, a.lk, a.dht, simg, pq, pk, a.dh0, status, d.T, d.H, d.NT, d.scale, retnet ? a.log_decay : nullptr, dseqs, vm, d.dk, d.dv};
     k_gla_bwd_tc<<<ctas, st2::NTHREADS, st2::SMEM_BYTES, st>>>(mq, mk, mv, mdo, mg, mdq, mdk, mdv, mdg, bp);
     tr.mark("gla_bwd_tc");
     if (gate_bwd_prod(a.lq, a.lk, pq, pk, a.dlq, a.dlk, (long)d.B * d.T, d.H, st) < 0) return -1;
@@ -1048,7 +1048,7 @@ int gla_tc_backward_segmented(const Dims &d, const BwdArgs &a, Varlen &segs, int
     FwdArgs f{a.q, a.k, a.v, a.log_decay, a.beta, a.lq, a.lk, a.h0, nullptr, nullptr, a.ws, a.status, nullptr};
     if (gla_tc_segment_summaries(d, f, P, L, fin, gam, status, st, tr) < 0) return -1;
     const dim3 grid(d.B * d.H, d.dk);
-    k_fold_segment_states<<<grid, d.dv, 0, st>>>(d.H, P, d.dk, a.h0, fin, gam, h0seg);
+    k_fold_segment_states<<<grid, d.dv, 0, st>>>(d.H, P, d.dk, d.dv, a.h0, fin, gam, h0seg);
     tr.mark("fold_segment_states");
     // first pass over the segments as a packed batch, no state gradient entering: what each sends out of its left edge
     BwdArgs a1 = a;
@@ -1058,7 +1058,7 @@ int gla_tc_backward_segmented(const Dims &d, const BwdArgs &a, Varlen &segs, int
     a1.vl = &segs;
     const int n1 = gla_tc_backward(d, a1, false, status, st, tr);
     if (n1 < 0) return -1;
-    k_fold_segment_dstates<<<grid, d.dv, 0, st>>>(d.H, P, d.dk, a.dht, gam, dsfin, dhtseg);
+    k_fold_segment_dstates<<<grid, d.dv, 0, st>>>(d.H, P, d.dk, d.dv, a.dht, gam, dsfin, dhtseg);
     tr.mark("fold_segment_dstates");
     // second pass with the true state gradient entering every segment (the state images of the first pass are in place)
     BwdArgs a2 = a1;

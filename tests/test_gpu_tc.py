@@ -314,9 +314,10 @@ def test_retnet_training_step_reads_what_the_forward_left(B, T, H, with_h0):
 # ---- 64-wide heads: the same kernels, the upper half of every 128-wide tile being zero padding that the tensor maps
 # supply on loads and drop on stores (no padded copies in memory)
 @pytest.mark.parametrize("base", ["C2", "R2", "C4"])
+@pytest.mark.parametrize("dk,dv", [(64, 64), (64, 128), (128, 64)])
 @pytest.mark.parametrize("B,T,H,with_h0", [(2, 200, 3, True), (1, 1000, 16, True), (3, 65, 4, False), (2, 5, 2, True)])
-def test_heads_of_width_64_take_the_tensor_core_kernels(base, B, T, H, with_h0):
-    cfg = small(CONFIGS[base], B=B, T=T, H=H, d_k=64, d_v=64, seed=1400 + T)
+def test_heads_of_width_64_take_the_tensor_core_kernels(base, dk, dv, B, T, H, with_h0):
+    cfg = small(CONFIGS[base], B=B, T=T, H=H, d_k=dk, d_v=dv, seed=1400 + T)
     x = make_inputs(cfg, with_dO=True, with_h0=with_h0)
     xd = gu.to_dev(x)
     o, ht, g, plan, ws, lf, lb = gu.gpu_training_step(cfg, xd, h0=xd.get("h0"), dht=xd.get("dht"), want_dh0=with_h0)
@@ -337,8 +338,8 @@ def test_heads_of_width_64_take_the_tensor_core_kernels(base, B, T, H, with_h0):
             assert torch.equal(t, g2[n]), n
 
 
-def test_mixed_widths_stay_on_the_generic_kernels():
-    cfg = small(CONFIGS["C2"], B=1, T=130, H=2, d_k=64, d_v=128, seed=1410)
+def test_other_widths_stay_on_the_generic_kernels():
+    cfg = small(CONFIGS["C2"], B=1, T=130, H=2, d_k=96, d_v=128, seed=1410)
     x = gu.to_dev(make_inputs(cfg))
     o, ht, plan = gu.gpu_forward(cfg, x)
     assert plan.last_launch_count > 1

@@ -15,7 +15,8 @@ LENGTHS = (1, 63, 64, 65, 900, 130)      # (under 16 chunks each: run alone, suc
 
 def _packed(base, lengths, H, seed, with_h0, d=128):
     T = sum(lengths)
-    cfg = small(CONFIGS[base], B=1, T=T, H=H, d_k=d, d_v=d, seed=seed)
+    dk, dv = d if isinstance(d, tuple) else (d, d)
+    cfg = small(CONFIGS[base], B=1, T=T, H=H, d_k=dk, d_v=dv, seed=seed)
     x = make_inputs(cfg, with_dO=True)
     n = len(lengths)
     if with_h0:
@@ -41,7 +42,7 @@ def _slice(x, s, a, b):
     return out
 
 
-@pytest.mark.parametrize("base,d", [("C2", 128), ("R2", 128), ("C4", 128), ("C2", 64), ("C4", 64)])
+@pytest.mark.parametrize("base,d", [("C2", 128), ("R2", 128), ("C4", 128), ("C2", 64), ("C4", 64), ("C2", (64, 128)), ("C4", (128, 64))])
 @pytest.mark.parametrize("with_h0", [False, True])
 def test_packed_batch_matches_the_oracle_and_the_single_sequence_runs(base, d, with_h0):
     H = 3
