@@ -209,7 +209,7 @@ def main():
                          "per-configuration figures and profiles")
     ap.add_argument("--packed", action="store_true",
                     help="the workload's B*T tokens as ONE packed row of variable-length sequences (a seeded mix of "
-                         "lengths from 64 to 8192 tokens; sla_plan_set_sequences) instead of B rows of T: not the "
+                         "lengths from 64 to 4096 tokens, the maximum training length of the paper; sla_plan_set_sequences) instead of B rows of T: not the "
                          "benchmark, labelled in config")
     ap.add_argument("--batch", type=int, default=0,
                     help="profiling aid: shrink the batch of the workload (0 = the full configuration; "
@@ -234,10 +234,10 @@ def main():
         total = cfg.B * cfg.T
         rng, cu = random.Random(7), [0]
         while cu[-1] < total:
-            cu.append(min(total, cu[-1] + rng.choice([64, 200, 512, 1000, 2048, 4096, 8192])))
+            cu.append(min(total, cu[-1] + rng.choice([64, 200, 512, 1000, 2048, 4096])))
         packed_cu = cu
         cfg = small(cfg, B=1, T=total)
-        METRIC += f" [packed: {len(cu) - 1} sequences of 64..8192 tokens in one row of {total}]"
+        METRIC += f" [packed: {len(cu) - 1} sequences of 64..4096 tokens in one row of {total}]"
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))

@@ -2,6 +2,7 @@
 #include "sla_internal.h"
 #include "sla_ptx.cuh"
 
+#include <algorithm>
 #include <new>
 #include <string.h>
 #include <utility>
@@ -213,8 +214,12 @@ sla_status sla_plan_set_sequences(sla_plan *plan, const int32_t *cu_seqlens, int
         const int len = cu_seqlens[s + 1] - cu_seqlens[s];
         if (len <= 0) { v.seqs.clear(); return SLA_ERR_INVALID_ARG; }      // (empty sequences are not allowed)
         const int nt = (len + d.C - 1) / d.C;
-        v.seqs.push_back({cu_seqlens[s], len, nt, (int)slots});
-        slots += nt + 1;
+        v.seqs.push_back({cu_seqlens[s], len, nt, 0, s});
+    }
+    std::stable_sort(v.seqs.begin(), v.seqs.end(), [](const sla::SeqInfo &a, const sla::SeqInfo &b) { return a.NT > b.NT; });
+    for (auto &si : v.seqs) {
+        si.slot0 = (int)slots;
+        slots += si.NT + 1;
     }
     v.slots = slots;
     v.n_seq = n_seq;

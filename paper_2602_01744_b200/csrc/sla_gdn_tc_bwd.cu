@@ -87,6 +87,7 @@ k_gdn_bwd_tc(const __grid_constant__ CUtensorMap gm_q, const __grid_constant__ C
     const int bh = blockIdx.x, h = bh % p.H;
     int b = bh / p.H;
     size_t tokb = (size_t)b * p.T, slot = (size_t)bh * (p.NT + 1);
+    size_t sbh = (size_t)bh;                                // (sequence, head) index into h0 / ht / dht / dh0
     const CUtensorMap *vm = nullptr;
     if (p.seqs) {                                           // packed batch: see k_gdn_fwd_tc
         const SeqInfo si = p.seqs[b];
@@ -94,6 +95,7 @@ k_gdn_bwd_tc(const __grid_constant__ CUtensorMap gm_q, const __grid_constant__ C
         p.T = si.T; p.NT = si.NT;
         tokb = (size_t)si.t0;
         slot = (size_t)si.slot0 * p.H + (size_t)h * (si.NT + 1);
+        sbh = (size_t)si.id * p.H + h;                      // (the table is ordered longest first, the state tensors as the caller gave them)
         b = 0;
     }
     const CUtensorMap &tm_q = vm ? vm[0] : gm_q, &tm_k = vm ? vm[1] : gm_k, &tm_v = vm ? vm[2] : gm_v, &tm_do = vm ? vm[3] : gm_do,
@@ -404,7 +406,7 @@ k_gdn_bwd_tc(const __grid_constant__ CUtensorMap gm_q, const __grid_constant__ C
         {   // dS_NT = dht (or zero) into TMEM; carried scalar <dht, S_NT>
             float v0[32], v1[32];
             if (p.dht) wait(INIT_FULL, 0);
-            const float *src = state_row(p.dht, bh, row, ch, p.dk, p.dv);
+            const float *src = state_row(p.dht, sbh, row, ch, p.dk, p.dv);
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
                 v0[j] = src ? src[j] : 0.f;
@@ -741,7 +743,7 @@ k_gdn_bwd_tc(const __grid_constant__ CUtensorMap gm_q, const __grid_constant__ C
         }
 
         if (p.dh0) {   // dS_0, fp32 (complete since the last chunk's group 3)
-            float *dst = state_row(p.dh0, bh, row, ch, p.dk, p.dv);
+            float *dst = state_row(p.dh0, sbh, row, ch, p.dk, p.dv);
 #pragma unroll
             for (int part = 0; part < 2; ++part) {
                 float v[32];

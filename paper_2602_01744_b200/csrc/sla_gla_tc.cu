@@ -86,6 +86,7 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap gm_q, const __grid_constant__ C
     // A packed batch: this CTA's sequence has its own length, chunk count, first token, state slots and tensor maps
     // (based at its first token, so token coordinates stay relative and the batch coordinate is 0).
     size_t tokb = (size_t)b * p.T, slot = (size_t)bh * (p.NT + 1);
+    size_t sbh = (size_t)bh;                                // (sequence, head) index into h0 / ht / dht / dh0
     const CUtensorMap *vm = nullptr;
     if (p.seqs) {
         const SeqInfo si = p.seqs[b];
@@ -93,6 +94,7 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap gm_q, const __grid_constant__ C
         p.T = si.T; p.NT = si.NT; p.L = si.NT;
         tokb = (size_t)si.t0;
         slot = (size_t)si.slot0 * p.H + (size_t)h * (si.NT + 1);
+        sbh = (size_t)si.id * p.H + h;                      // (the table is ordered longest first, the state tensors as the caller gave them)
         b = 0;
     }
     const CUtensorMap &tm_q = vm ? vm[0] : gm_q, &tm_k = vm ? vm[1] : gm_k, &tm_v = vm ? vm[2] : gm_v,
@@ -293,7 +295,7 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap gm_q, const __grid_constant__ C
         {   // initial state: fp32 into TMEM, bf16 copy into shared memory (row = key dimension).  A segment that is not the
             // first starts from S <- diag(gam_s) S + fin_s taken over the segments s before it (a short scan over their
             // summaries, elementwise, done here rather than in a launch of its own).
-            const float *src = state_row(p.h0, bh, row, colhalf, p.dk, p.dv);
+            const float *src = state_row(p.h0, sbh, row, colhalf, p.dk, p.dv);
 #pragma unroll
             for (int part = 0; part < 2; ++part) {
                 float v[32];
@@ -428,7 +430,7 @@ k_gla_fwd_tc(const __grid_constant__ CUtensorMap gm_q, const __grid_constant__ C
         }
 
         if (p.ht && seg == p.P - 1) {   // final state, fp32 (each thread reads back what it wrote in the last rescale)
-            float *dst = state_row(p.ht, bh, row, colhalf, p.dk, p.dv);
+            float *dst = state_row(p.ht, sbh, row, colhalf, p.dk, p.dv);
 #pragma unroll
             for (int part = 0; part < 2; ++part) {
                 float v[32];

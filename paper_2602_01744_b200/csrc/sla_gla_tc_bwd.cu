@@ -95,6 +95,7 @@ k_gla_states_tc(const __grid_constant__ CUtensorMap gm_k, const __grid_constant_
     const int bh = blockIdx.x / p.P, seg = blockIdx.x % p.P, h = bh % p.H;
     int b = bh / p.H;
     size_t tokb = (size_t)b * p.T, slot = (size_t)bh * (p.NT + 1);
+    size_t sbh = (size_t)bh;                                // (sequence, head) index into h0 / ht / dht / dh0
     const CUtensorMap *vm = nullptr;
     if (p.seqs) {                                           // packed batch: see k_gla_fwd_tc
         const SeqInfo si = p.seqs[b];
@@ -102,6 +103,7 @@ k_gla_states_tc(const __grid_constant__ CUtensorMap gm_k, const __grid_constant_
         p.T = si.T; p.NT = si.NT; p.L = si.NT;
         tokb = (size_t)si.t0;
         slot = (size_t)si.slot0 * p.H + (size_t)h * (si.NT + 1);
+        sbh = (size_t)si.id * p.H + h;                      // (the table is ordered longest first, the state tensors as the caller gave them)
         b = 0;
     }
     const CUtensorMap &tm_k = vm ? vm[0] : gm_k, &tm_v = vm ? vm[1] : gm_v, &tm_g = vm ? vm[2] : gm_g;
@@ -228,7 +230,7 @@ k_gla_states_tc(const __grid_constant__ CUtensorMap gm_k, const __grid_constant_
         const int colhalf = warp >> 2;
         const int row = 32 * (warp & 3) + lane;
         {   // S_0: fp32 into TMEM, bf16 image into slot 0
-            const float *src = images ? state_row(p.h0, bh, row, colhalf, p.dk, p.dv) : nullptr;
+            const float *src = images ? state_row(p.h0, sbh, row, colhalf, p.dk, p.dv) : nullptr;
 #pragma unroll
             for (int part = 0; part < 2; ++part) {
                 float v[32];
@@ -378,6 +380,7 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap gm_q, const __grid_constant__ C
     const int bh = blockIdx.x, h = bh % p.H;
     int b = bh / p.H;
     size_t tokb = (size_t)b * p.T, slot = (size_t)bh * (p.NT + 1);
+    size_t sbh = (size_t)bh;                                // (sequence, head) index into h0 / ht / dht / dh0
     const CUtensorMap *vm = nullptr;
     if (p.seqs) {                                           // packed batch: see k_gla_fwd_tc
         const SeqInfo si = p.seqs[b];
@@ -385,6 +388,7 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap gm_q, const __grid_constant__ C
         p.T = si.T; p.NT = si.NT;
         tokb = (size_t)si.t0;
         slot = (size_t)si.slot0 * p.H + (size_t)h * (si.NT + 1);
+        sbh = (size_t)si.id * p.H + h;                      // (the table is ordered longest first, the state tensors as the caller gave them)
         b = 0;
     }
     const CUtensorMap &tm_q = vm ? vm[0] : gm_q, &tm_k = vm ? vm[1] : gm_k, &tm_v = vm ? vm[2] : gm_v,
@@ -633,7 +637,7 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap gm_q, const __grid_constant__ C
         {   // dS_NT = dht (or zero) into TMEM; R_{NT-1} = rowsum(dht * S_NT)
             float rpart = 0.f;
             if (p.dht) wait(INIT_FULL, 0);
-            const float *src = state_row(p.dht, bh, row, wh, p.dk, p.dv);
+            const float *src = state_row(p.dht, sbh, row, wh, p.dk, p.dv);
 #pragma unroll
             for (int part = 0; part < 2; ++part) {
                 float v[32];
@@ -849,7 +853,7 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap gm_q, const __grid_constant__ C
         }
 
         if (p.dh0) {   // dS_0, fp32 (the last chunk's MMAs were waited for above)
-            float *dst = state_row(p.dh0, bh, row, wh, p.dk, p.dv);
+            float *dst = state_row(p.dh0, sbh, row, wh, p.dk, p.dv);
 #pragma unroll
             for (int part = 0; part < 2; ++part) {
                 float v[32];
@@ -1054,7 +1058,7 @@ void gla_tc_backward_segment_table(const Dims &d, int P, int L, Varlen &segs) {
     for (int b = 0; b < d.B; ++b)
         for (int p = 0; p < P; ++p) {
             const int t0 = p * L * C, len = std::min(L * C, d.T - t0), nt = (len + C - 1) / C;
-            segs.seqs.push_back({b * d.T + t0, len, nt, (int)slots});
+            segs.seqs.push_back({b * d.T + t0, len, nt, (int)slots, b * P + p});
             slots += nt + 1;
         }
     segs.slots = slots;

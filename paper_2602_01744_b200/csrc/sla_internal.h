@@ -25,8 +25,9 @@ struct Dims {
 
 // Packed variable-length batches (B = 1: sequences one after another along T, the state reset at every boundary,
 // chunks cut from each sequence's own start).  Per sequence: first token, length, chunks, and the index of its first
-// state slot (the sum of chunks + 1 over the sequences before it).
-struct SeqInfo { int t0, T, NT, slot0; };
+// state slot (the sum of chunks + 1 over the sequences before it).  The table is kept longest sequence first, so that the
+// CTAs of long sequences are dispatched first (one CTA per (sequence, head), in table order).
+struct SeqInfo { int t0, T, NT, slot0, id; };     // id: the sequence's number as the caller counts them
 // Host side of a plan's sequence table.  The tensor-core kernels address a sequence through tensor maps of its own
 // (based at its first token, T = its length: loads past its end read zeros, stores are clipped there, exactly as at the
 // end of a batch row); those live in device arrays, one region per kernel kind, encoded again only when the tensors
