@@ -752,50 +752,22 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap gm_q, const __grid_constant__ C
                 tmem_ld32(tmem + lane_base + COL_DQ + 32 * wh, dqh);
                 tmem_ld32(tmem + lane_base + COL_DK + 32 * wh, dkh);
                 tmem_wait_ld();
-                // A 2-byte shared-memory access costs as much as a 4-byte one, so neighbouring lanes (key dimensions row, row^1)
-                // share 4-byte words: of the token pair (j, j+4) of a group of eight the even lane moves the word of token
-                // j, the odd lane the word of token j+4 (their swizzled positions fall into different halves of the 128-byte
-                // row: no bank conflict) and a shuffle hands each lane the half it misses.
-                const uint32_t dhalf = (uint32_t)(row >> 6) * HALF_BF16, dchunk = (uint32_t)(row & 63) >> 3, wbyte = (row & 6) * 2;
-                const bool odd = lane & 1;
+                const uint32_t dhalf = (uint32_t)(row >> 6) * HALF_BF16, dchunk = (uint32_t)(row & 63) >> 3, dbyte = (row & 7) * 2;
                 float run = 0.f;
 #pragma unroll
-                for (int g = 3; g >= 0; --g) {
-                    const int i0 = 32 * wh + 8 * g;
-                    float qv[8], kv[8], oq[8], ok[8];
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const uint32_t off = dhalf + swz(i0 + j + (odd ? 4 : 0), dchunk) + wbyte;
-                        const uint32_t wq = *reinterpret_cast<const uint32_t *>(qk + off);
-                        const uint32_t wk = *reinterpret_cast<const uint32_t *>(qk + TILE_BF16 + off);
-                        const uint32_t xq = __shfl_xor_sync(0xffffffffu, wq, 1), xk = __shfl_xor_sync(0xffffffffu, wk, 1);
-                        // even lane: own token j in the low half of its word, token j+4 in the low half of the partner's;
-                        // odd lane: token j+4 in the high half of its word, token j in the high half of the partner's
-                        qv[j] = __uint_as_float(odd ? (xq & 0xffff0000u) : (wq << 16));
-                        qv[j + 4] = __uint_as_float(odd ? (wq & 0xffff0000u) : (xq << 16));
-                        kv[j] = __uint_as_float(odd ? (xk & 0xffff0000u) : (wk << 16));
-                        kv[j + 4] = __uint_as_float(odd ? (wk & 0xffff0000u) : (xk << 16));
-                    }
-#pragma unroll
-                    for (int j = 7; j >= 0; --j) {
-                        const int ii = 8 * g + j, i = i0 + j;
-                        const float2 ee = unpack_bf16(*reinterpret_cast<const uint32_t *>(sm + OFF_E2 + i * (D * 4) + row * 4));
-                        const float pq = qv[j] * dqh[ii], pk = kv[j] * dkh[ii];
-                        run += pq - pk;
-                        sfx[ii] = run;
-                        oq[j] = ee.x * dqh[ii];                      // dq = scale Gq 2^b dqh   (over qh, for the store)
-                        ok[j] = ee.y * dkh[ii];                      // dk = Gk 2^-b dkh
-                        dqh[ii] = pq;
-                        dkh[ii] = pk;
-                    }
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const float rq = __shfl_xor_sync(0xffffffffu, odd ? oq[j] : oq[j + 4], 1);
-                        const float rk = __shfl_xor_sync(0xffffffffu, odd ? ok[j] : ok[j + 4], 1);
-                        const uint32_t off = dhalf + swz(i0 + j + (odd ? 4 : 0), dchunk) + wbyte;
-                        *reinterpret_cast<uint32_t *>(qk + off) = odd ? pack_bf16(rq, oq[j + 4]) : pack_bf16(oq[j], rq);
-                        *reinterpret_cast<uint32_t *>(qk + TILE_BF16 + off) = odd ? pack_bf16(rk, ok[j + 4]) : pack_bf16(ok[j], rk);
-                    }
+                for (int ii = 31; ii >= 0; --ii) {
+                    const int i = 32 * wh + ii;
+                    const uint32_t off = dhalf + swz(i, dchunk) + dbyte;
+                    __nv_bfloat16 *qp = reinterpret_cast<__nv_bfloat16 *>(qk + off);
+                    __nv_bfloat16 *kp = reinterpret_cast<__nv_bfloat16 *>(qk + TILE_BF16 + off);
+                    const float2 ee = unpack_bf16(*reinterpret_cast<const uint32_t *>(sm + OFF_E2 + i * (D * 4) + row * 4));
+                    const float pq = __bfloat162float(*qp) * dqh[ii], pk = __bfloat162float(*kp) * dkh[ii];
+                    run += pq - pk;
+                    sfx[ii] = run;
+                    *qp = __float2bfloat16_rn(ee.x * dqh[ii]);       // dq = scale Gq 2^b dqh   (over qh, for the store)
+                    *kp = __float2bfloat16_rn(ee.y * dkh[ii]);       // dk = Gk 2^-b dkh
+                    dqh[ii] = pq;
+                    dkh[ii] = pk;
                 }
                 if (wh == 1) up[row] = run + Rcur[row] + Rcur[D + row];
                 const float sq = warp_transpose_sum(dqh, lane);
@@ -814,17 +786,11 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap gm_q, const __grid_constant__ C
                 float dvt[32];
                 tmem_ld32(tmem + lane_base + COL_DV + 32 * wh, dvt);
                 tmem_wait_ld();
-                const uint32_t dhalf = (uint32_t)(row >> 6) * HALF_BF16, dchunk = (uint32_t)(row & 63) >> 3, wbyte = (row & 6) * 2;
-                const bool odd = lane & 1;
+                const uint32_t dhalf = (uint32_t)(row >> 6) * HALF_BF16, dchunk = (uint32_t)(row & 63) >> 3, dbyte = (row & 7) * 2;
 #pragma unroll
-                for (int g = 0; g < 4; ++g)
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {       // (4-byte words shared by neighbouring lanes, as above)
-                        const int ii = 8 * g + j;
-                        const float r = __shfl_xor_sync(0xffffffffu, odd ? dvt[ii] : dvt[ii + 4], 1);
-                        *reinterpret_cast<uint32_t *>(sm + OFF_A + dhalf + swz(32 * wh + ii + (odd ? 4 : 0), dchunk) + wbyte) =
-                            odd ? pack_bf16(r, dvt[ii + 4]) : pack_bf16(dvt[ii], r);
-                    }
+                for (int ii = 0; ii < 32; ++ii)
+                    *reinterpret_cast<__nv_bfloat16 *>(sm + OFF_A + dhalf + swz(32 * wh + ii, dchunk) + dbyte) =
+                        __float2bfloat16_rn(dvt[ii]);
             }
             named_bar_sync(1, NCOMPUTE);                // up, red and the R partials are complete
             {   // log-decay gradient: in-chunk suffix sum + what flows in from the right of the chunk
