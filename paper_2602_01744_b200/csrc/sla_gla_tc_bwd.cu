@@ -570,18 +570,18 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap gm_q, const __grid_constant__ C
                     load_qk(n - 1, k + 1);
                 }
                 if (n > 0) {
-                    wait_relaxed(SNFREE, par);         // rowsum(dS_n * S_n) done (and S_n dO^T issued long ago): S_n no longer needed
+                    wait(SNFREE, par);                 // rowsum(dS_n * S_n) done (and S_n dO^T issued long ago): S_n no longer needed
                     if (failed) break;
                     load_s(n - 1);
                 }
-                wait_relaxed(OUT1, par);               // dq, dk staged over qh, kh
+                wait(OUT1, par);                       // dq, dk staged over qh, kh
                 if (failed) break;
                 tma_store_5d(&tm_dq, sQK, 0, n * C, 0, h, b);
                 tma_store_5d(&tm_dk, sQK + TILE_BF16, 0, n * C, 0, h, b);
                 bulk_commit();
                 bulk_wait_read0();
                 if (n > 0) load_vdo(n - 1, k + 1);     // ... and this buffer takes the next v, dO
-                wait_relaxed(OUT2, par);               // dv, dlog_decay staged
+                wait(OUT2, par);                       // dv, dlog_decay staged
                 if (failed) break;
                 tma_store_5d(&tm_dv, base + OFF_A, 0, n * C, 0, h, b);
                 if (!retnet) tma_store_4d(&tm_dg, base + OFF_DZ, 0, h, n * C, b);
@@ -731,9 +731,10 @@ k_gla_bwd_tc(const __grid_constant__ CUtensorMap gm_q, const __grid_constant__ C
             mbar_arrive(bar(AREADY));
 
             // ---- R_{n-1} = rowsum(dS_n * S_n), while the tensor core works on the products with the masked tiles ----
+            // (it feeds the log-decay gradient only: Softmax-RetNet, whose decay is a constant, has none and skips it)
             wait(BAR_DS, par);
             tc_fence_after();
-            {
+            if (!retnet) {
                 float v0[32], v1[32];
                 tmem_ld32(tmem + lane_base + COL_DS + 64 * wh, v0);
                 tmem_ld32(tmem + lane_base + COL_DS + 64 * wh + 32, v1);
